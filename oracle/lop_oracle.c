@@ -1,0 +1,132 @@
+/*
+ * CPU oracle for local-operator chains: TEST INFRASTRUCTURE, not part of the product.
+ *
+ * Plain direct-loop definitions of the block-wise local operators of Sec. IV-A of the
+ * paper (convolution and max pooling; "the block size is determined by the operator's
+ * parameters": kernel size, padding, dilation, and stride) with the element-wise local
+ * operators (ReLU, SiLU) and the residual addition applied per output element.
+ * Nothing here is blocked, fused or reordered; nothing here is shared with the CUDA
+ * library.  Only tests, the smoke check and the benchmark's CPU-baseline leg call it.
+ *
+ * Layout: activations NHWC, weights [cout][kh][kw][cin], all float32 in memory.  On the
+ * "bf16 path" every stored value is a float32 that is exactly representable in bfloat16:
+ * inputs arrive that way and each layer output is rounded (nearest, ties to even) when it
+ * is stored.
+ *
+ * Each routine computes the output rows oh in [oh_lo, oh_hi) of the FULL output tensor
+ * and leaves every other row untouched, so the same routine serves whole-tensor
+ * execution (oh_lo = 0, oh_hi = H_out) and band-wise execution.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <string.h>
+
+/* float -> nearest bfloat16-representable float, ties to even (NaN passed through). */
+float lop_oracle_bf16_rne(float v)
+{
+    uint32_t u;
+    memcpy(&u, &v, 4);
+    if ((u & 0x7F800000u) == 0x7F800000u && (u & 0x007FFFFFu)) {   /* NaN: keep it a NaN */
+        u |= 0x00400000u;
+        u &= 0xFFFF0000u;
+    } else {
+        uint32_t lsb = (u >> 16) & 1u;
+        u += 0x7FFFu + lsb;
+        u &= 0xFFFF0000u;
+    }
+    memcpy(&v, &u, 4);
+    return v;
+}
+
+static float activate(float t, int act)
+{
+    if (act == 1) return t > 0.0f ? t : 0.0f;                /* ReLU */
+    if (act == 2) return t / (1.0f + expf(-t));              /* SiLU */
+    return t;
+}
+
+/*
+ * y[n,oh,ow,co] = epilogue( sum_{kh,kw,ci} x[n, oh*sh-ph+kh*dh, ow*sw-pw+kw*dw, ci] * w[co,kh,kw,ci] )
+ * taps outside the input contribute zero.  Accumulation in double, in the order kh, kw, ci.
+ * epilogue: t = scale[co]*(float)acc + shift[co]; res_pos==1: t += res; t = act(t); res_pos==2: t += res.
+ * scale / shift / res may be NULL (1 / 0 / none).  res has the output's shape.
+ */
+void lop_oracle_conv2d(const float *x, int N, int H, int W, int Cin,
+                       const float *w, int Cout, int kh, int kw, int sh, int sw,
+                       int ph, int pw, int dh, int dw,
+                       const float *scale, const float *shift,
+                       const float *res, int res_pos, int act, int round_bf16,
+                       int oh_lo, int oh_hi, float *y)
+{
+    const int Ho = (H + 2 * ph - dh * (kh - 1) - 1) / sh + 1;
+    const int Wo = (W + 2 * pw - dw * (kw - 1) - 1) / sw + 1;
+    if (oh_lo < 0) oh_lo = 0;
+    if (oh_hi > Ho) oh_hi = Ho;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (int n = 0; n < N; ++n)
+        for (int oh = oh_lo; oh < oh_hi; ++oh)
+            for (int ow = 0; ow < Wo; ++ow)
+                for (int co = 0; co < Cout; ++co) {
+                    double acc = 0.0;
+                    for (int a = 0; a < kh; ++a) {
+                        const int ih = oh * sh - ph + a * dh;
+                        if (ih < 0 || ih >= H) continue;
+                        for (int b = 0; b < kw; ++b) {
+                            const int iw = ow * sw - pw + b * dw;
+                            if (iw < 0 || iw >= W) continue;
+                            const float *xp = x + (((size_t)n * H + ih) * W + iw) * Cin;
+                            const float *wp = w + (((size_t)co * kh + a) * kw + b) * Cin;
+                            for (int ci = 0; ci < Cin; ++ci) acc += (double)xp[ci] * (double)wp[ci];
+                        }
+                    }
+                    const size_t o = (((size_t)n * Ho + oh) * Wo + ow) * Cout + co;
+                    float t = (float)acc;
+                    t = (scale ? scale[co] : 1.0f) * t + (shift ? shift[co] : 0.0f);
+                    if (res && res_pos == 1) t += res[o];
+                    t = activate(t, act);
+                    if (res && res_pos == 2) t += res[o];
+                    y[o] = round_bf16 ? lop_oracle_bf16_rne(t) : t;
+                }
+}
+
+/*
+ * y[n,oh,ow,c] = max over the taps (kh,kw) that fall inside the input; padding never wins
+ * (it behaves as minus infinity).  A window with no in-bounds tap yields -inf.
+ */
+void lop_oracle_maxpool2d(const float *x, int N, int H, int W, int C,
+                          int kh, int kw, int sh, int sw, int ph, int pw, int dh, int dw,
+                          int oh_lo, int oh_hi, float *y)
+{
+    const int Ho = (H + 2 * ph - dh * (kh - 1) - 1) / sh + 1;
+    const int Wo = (W + 2 * pw - dw * (kw - 1) - 1) / sw + 1;
+    if (oh_lo < 0) oh_lo = 0;
+    if (oh_hi > Ho) oh_hi = Ho;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (int n = 0; n < N; ++n)
+        for (int oh = oh_lo; oh < oh_hi; ++oh)
+            for (int ow = 0; ow < Wo; ++ow)
+                for (int c = 0; c < C; ++c) {
+                    float m = -INFINITY;
+                    for (int a = 0; a < kh; ++a) {
+                        const int ih = oh * sh - ph + a * dh;
+                        if (ih < 0 || ih >= H) continue;
+                        for (int b = 0; b < kw; ++b) {
+                            const int iw = ow * sw - pw + b * dw;
+                            if (iw < 0 || iw >= W) continue;
+                            const float v = x[(((size_t)n * H + ih) * W + iw) * C + c];
+                            if (v > m) m = v;
+                        }
+                    }
+                    y[(((size_t)n * Ho + oh) * Wo + ow) * C + c] = m;
+                }
+}
+
+int lop_oracle_num_threads(void)
+{
+#ifdef _OPENMP
+    extern int omp_get_max_threads(void);
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}

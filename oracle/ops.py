@@ -1,0 +1,77 @@
+"""numpy front-end to the C oracle routines (see lop_oracle.c for the definitions)."""
+import ctypes
+
+import numpy as np
+
+from . import build as _build
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(_build.build())
+        _lib.lop_oracle_bf16_rne.restype = ctypes.c_float
+        _lib.lop_oracle_bf16_rne.argtypes = [ctypes.c_float]
+        _lib.lop_oracle_num_threads.restype = ctypes.c_int
+        _lib.lop_oracle_conv2d.restype = None
+        _lib.lop_oracle_maxpool2d.restype = None
+    return _lib
+
+
+def _fp(a):
+    return a.ctypes.data_as(ctypes.POINTER(ctypes.c_float)) if a is not None else None
+
+
+def _f32(a):
+    return None if a is None else np.ascontiguousarray(a, dtype=np.float32)
+
+
+def out_size(n, k, s, p, d):
+    """Floor-mode output extent of a strided, padded, dilated window (Sec. IV-A block-wise operators)."""
+    return (n + 2 * p - d * (k - 1) - 1) // s + 1
+
+
+def bf16_rne(v):
+    return float(lib().lop_oracle_bf16_rne(ctypes.c_float(v)))
+
+
+def num_threads():
+    return int(lib().lop_oracle_num_threads())
+
+
+def conv2d(x, w, stride=(1, 1), pad=(0, 0), dil=(1, 1), scale=None, shift=None, res=None, res_pos=0,
+           act=0, round_bf16=False, rows=None, out=None):
+    """Rows ``rows=(lo,hi)`` (default all) of the NHWC convolution with fused epilogue, into ``out``."""
+    x, w = _f32(x), _f32(w)
+    N, H, W, Cin = x.shape
+    Cout, kh, kw, cin2 = w.shape
+    assert cin2 == Cin
+    Ho, Wo = out_size(H, kh, stride[0], pad[0], dil[0]), out_size(W, kw, stride[1], pad[1], dil[1])
+    assert Ho > 0 and Wo > 0
+    if out is None:
+        out = np.zeros((N, Ho, Wo, Cout), dtype=np.float32)
+    assert out.shape == (N, Ho, Wo, Cout) and out.dtype == np.float32 and out.flags.c_contiguous
+    scale, shift, res = _f32(scale), _f32(shift), _f32(res)
+    if res is not None:
+        assert res.shape == out.shape
+    lo, hi = (0, Ho) if rows is None else rows
+    lib().lop_oracle_conv2d(_fp(x), N, H, W, Cin, _fp(w), Cout, kh, kw, stride[0], stride[1], pad[0], pad[1],
+                            dil[0], dil[1], _fp(scale), _fp(shift), _fp(res), int(res_pos), int(act),
+                            int(bool(round_bf16)), int(lo), int(hi), _fp(out))
+    return out
+
+
+def maxpool2d(x, k, stride, pad=(0, 0), dil=(1, 1), rows=None, out=None):
+    x = _f32(x)
+    N, H, W, C = x.shape
+    Ho, Wo = out_size(H, k[0], stride[0], pad[0], dil[0]), out_size(W, k[1], stride[1], pad[1], dil[1])
+    assert Ho > 0 and Wo > 0
+    if out is None:
+        out = np.zeros((N, Ho, Wo, C), dtype=np.float32)
+    assert out.shape == (N, Ho, Wo, C) and out.dtype == np.float32 and out.flags.c_contiguous
+    lo, hi = (0, Ho) if rows is None else rows
+    lib().lop_oracle_maxpool2d(_fp(x), N, H, W, C, k[0], k[1], stride[0], stride[1], pad[0], pad[1],
+                               dil[0], dil[1], int(lo), int(hi), _fp(out))
+    return out
