@@ -1,0 +1,178 @@
+/*
+ * lop.h -- C ABI of the band-wise local-operator library for NVIDIA B200 (sm_100a).
+ *
+ * The library executes a chain of LOCAL operators in the sense of Sec. IV-A of the
+ * Intra-DP paper (arxiv 2507.05829): block-wise operators (2-D convolution, max pooling),
+ * element-wise operators (ReLU, SiLU, folded batch-norm scale/shift) and the residual
+ * addition.  Following the paper's local-operation parallelism (Sec. IV-B), the rows of the
+ * chain's output are cut into contiguous bands; every band carries the halo rows its
+ * receptive field needs, so the input of band i+1 can still be in flight while band i is
+ * being computed, and the stitched result equals whole-tensor execution.
+ *
+ * Conventions
+ *   - Every function returns LOP_OK (0) or a negative lop_status; nothing throws or aborts.
+ *     A human-readable message for the calling thread's last failure: lop_last_error().
+ *   - "host" / "device" / "pinned host" say where a pointer must live.  The caller owns every
+ *     buffer and the stream; the library owns the opaque plan and what hangs off it (one side
+ *     stream, events, tensor maps), all released by lop_plan_destroy().
+ *   - Activations are NHWC, contiguous; weights are [cout][kh][kw][cin] (KRSC), contiguous,
+ *     in the plan's storage dtype; scale/shift are float32 [cout].  Accumulation is float32.
+ *   - Row ranges are half-open [lo, hi); the empty range is {0, 0}.
+ *   - A plan may be used by one thread at a time.  Work is enqueued on the caller's stream and
+ *     ordered after earlier and before later work on that stream; no function synchronises the
+ *     device unless its comment says so.
+ */
+#ifndef LOP_H
+#define LOP_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    LOP_OK = 0,
+    LOP_EINVAL = -1,        /* NULL pointer, index out of range, bad enum value                 */
+    LOP_ESHAPE = -2,        /* layer list does not type-check (channels, empty output, ...)     */
+    LOP_EUNSUPPORTED = -3,  /* valid request this build has no kernel for                        */
+    LOP_ENOMEM = -4,        /* host allocation failed                                           */
+    LOP_ECUDA = -5,         /* a CUDA call failed; lop_last_error() carries the CUDA string      */
+    LOP_EWORKSPACE = -6,    /* caller-provided scratch is NULL or misaligned                    */
+    LOP_EDEVICE = -7        /* a kernel reported a bounded wait that ran out (status word)      */
+} lop_status;
+
+enum { LOP_F32 = 0, LOP_BF16 = 1 };                         /* storage dtype                     */
+enum { LOP_CONV2D = 0, LOP_MAXPOOL2D = 1 };
+enum { LOP_ACT_NONE = 0, LOP_ACT_RELU = 1, LOP_ACT_SILU = 2 };
+enum { LOP_RES_NONE = 0, LOP_RES_PRE_ACT = 1, LOP_RES_POST_ACT = 2 };
+enum { LOP_INPUT = -1, LOP_NO_RESIDUAL = -2 };              /* special layer indices             */
+enum {
+    LOP_FLAG_REUSE_HALO = 1u,     /* bands run in ascending order and compute only rows no earlier
+                                     band produced ("only what is missing", Sec. IV-C data
+                                     dependency); otherwise every band recomputes its halo and is
+                                     independent of the others (operation replication, Sec. IV-C) */
+    LOP_FLAG_TIME_LAYERS = 2u,    /* record a CUDA event pair around every (band, layer) launch    */
+    LOP_FLAG_FORCE_SIMT = 4u      /* never use the tensor-core convolution (second on-GPU opinion) */
+};
+
+/*
+ * One local operator (Sec. IV-A).  Convolution:
+ *   acc[n,oh,ow,co] = sum_{a,b,ci} x[n, oh*sh-ph+a*dh, ow*sw-pw+b*dw, ci] * weight[co,a,b,ci]
+ *   t = scale[co]*acc + shift[co];  RES_PRE_ACT: t += r;  t = act(t);  RES_POST_ACT: t += r
+ * with taps outside the input contributing zero.  Max pooling takes the maximum over the
+ * in-bounds taps (padding never wins); cout must equal cin; act/residual are ignored.
+ * input_from / residual_from name an earlier layer of the same list, or LOP_INPUT for the
+ * chain input; residual_from == LOP_NO_RESIDUAL means none.  The list order is topological.
+ * The three pointers are DEVICE pointers; they are stored, never dereferenced on the host,
+ * and may be NULL at planning time (set them later with lop_plan_set_params).
+ */
+typedef struct {
+    int32_t op, cin, cout;
+    int32_t kh, kw, sh, sw, ph, pw, dh, dw;
+    int32_t act;
+    int32_t input_from;
+    int32_t residual_from, residual_pos;
+    int32_t reserved;
+    const void  *weight;   /* device, KRSC, storage dtype; NULL for pooling                       */
+    const float *scale;    /* device, [cout]; NULL => 1                                           */
+    const float *shift;    /* device, [cout]; NULL => 0                                           */
+} lop_layer;
+
+/*
+ * What one band does at one layer.  [out_lo,out_hi): output rows of this layer the band
+ * depends on; [in_lo,in_hi): rows of the layer's main input those outputs read (rows that
+ * exist and are touched by a tap; the inverse of the paper's child(.) relation);
+ * pad_top/pad_bot: how many rows above/below the input the taps reach; new_lo: first row of
+ * [out_lo,out_hi) that no earlier band has produced (reuse-halo mode computes [new_lo,out_hi)).
+ */
+typedef struct {
+    int32_t out_lo, out_hi, in_lo, in_hi, pad_top, pad_bot, new_lo, reserved;
+} lop_range;
+
+/* Times of the last lop_run_pipelined call, in milliseconds (see lop_plan_last_timing). */
+typedef struct {
+    float total_ms;        /* first enqueued operation to last, on the caller's stream            */
+    float copy_ms;         /* sum of the band copies' own durations (copy-stream events)          */
+    float first_copy_ms;   /* duration of band 0's copy: it can never be hidden                   */
+    int32_t n_copies;
+    int32_t reserved;
+} lop_timing;
+
+typedef struct lop_plan lop_plan_t;
+
+/* ---- planning: HOST ONLY, needs no GPU, dereferences no device pointer -------------------
+ * Validates the layer list, derives every layer's output shape (floor rounding), cuts the last
+ * layer's output rows into n_bands bands  [floor(i*H/B), floor((i+1)*H/B))  (bands may be empty
+ * when n_bands exceeds the row count) and back-propagates each band through every layer's
+ * kernel, stride, padding and dilation (Sec. IV-A block-wise operators; dependency rule of
+ * Sec. IV-B).  N,H,W,C: shape of the chain input.  On success *out owns the plan. */
+int lop_plan(const lop_layer *layers, int n_layers, int N, int H, int W, int C, int dtype,
+             int n_bands, unsigned flags, lop_plan_t **out);
+void lop_plan_destroy(lop_plan_t *plan);                       /* NULL is accepted              */
+int lop_plan_num_bands(const lop_plan_t *plan);                /* <0 on NULL                    */
+int lop_plan_num_layers(const lop_plan_t *plan);
+/* layer in [0, n_layers) or LOP_INPUT: for the chain input, out_* is the row range the band
+ * needs, new_lo the first row not already transferred for an earlier band, in_* and pad_* 0. */
+int lop_plan_get_range(const lop_plan_t *plan, int band, int layer, lop_range *out);
+int lop_plan_out_shape(const lop_plan_t *plan, int layer, int *H, int *W, int *C);
+/* Re-point a layer's device parameters (any may be NULL as in lop_layer). */
+int lop_plan_set_params(lop_plan_t *plan, int layer, const void *weight, const float *scale,
+                        const float *shift);
+/* Device scratch, in bytes, that every lop_run_* call must be given (256-byte aligned):
+ * full-size intermediate tensors, and a channel-padded copy of the input and first-layer
+ * weights where the tensor-core kernel needs one. */
+size_t lop_plan_workspace_bytes(const lop_plan_t *plan);
+/* Size of the device-side input tensor N*H*W*C in storage dtype (staging for pipelined runs). */
+size_t lop_plan_staging_bytes(const lop_plan_t *plan);
+/* 2 * multiply-accumulates of the unpartitioned convolutions of the chain. */
+double lop_plan_flops(const lop_plan_t *plan);
+
+/* ---- execution: every pointer below is a DEVICE pointer unless it says otherwise ----------
+ * in_dev and out_dev are FULL-SIZE tensors (chain input N*H*W*C, last layer's output); bands
+ * address row ranges inside them.  stream is a cudaStream_t passed as void* (NULL = legacy
+ * default stream).  The first execution call on a plan creates its side stream and events:
+ * make it outside any stream capture. */
+
+/* Whole-tensor execution: every layer over all its rows (the unpartitioned reference order). */
+int lop_run_whole(lop_plan_t *plan, const void *in_dev, void *out_dev, void *workspace, void *stream);
+/* One band (Sec. IV-B: the band's operations at every layer, in dependency order).  Rows
+ * [out_lo,out_hi) of the chain-input range must be present in in_dev; exactly the band's rows
+ * of the last layer are written to out_dev.  Without LOP_FLAG_REUSE_HALO bands may run in any
+ * order; with it, bands 0..band-1 must have run on the same workspace before. */
+int lop_run_band(lop_plan_t *plan, int band, const void *in_dev, void *out_dev, void *workspace,
+                 void *stream);
+/* All bands in ascending order from a device-resident input (no transfers). */
+int lop_run_banded(lop_plan_t *plan, const void *in_dev, void *out_dev, void *workspace, void *stream);
+/* The transfer step of one band (the paper's transmission, Sec. IV-B): asynchronously copies
+ * the chain-input rows the band needs and no earlier band has brought, for all N images, from
+ * in_host_pinned (PINNED HOST, full-size tensor) to the same rows of staging_dev. */
+int lop_copy_band(lop_plan_t *plan, int band, const void *in_host_pinned, void *staging_dev, void *stream);
+/* Band pipeline (Sec. IV-B computation/transmission overlap): band i+1's rows are copied on the
+ * plan's side stream while band i is computed on the caller's stream; CUDA events carry the
+ * dependencies.  Returns after enqueueing.  staging_dev: lop_plan_staging_bytes() bytes. */
+int lop_run_pipelined(lop_plan_t *plan, const void *in_host_pinned, void *staging_dev, void *out_dev,
+                      void *workspace, void *stream);
+/* Event times of the last lop_run_pipelined call.  SYNCHRONISES with that call's completion. */
+int lop_plan_last_timing(lop_plan_t *plan, lop_timing *out);
+/* With LOP_FLAG_TIME_LAYERS: device time in ms of the (band, layer) launch of the last
+ * lop_run_band / banded / pipelined call (band = -1: last lop_run_whole).  SYNCHRONISES.
+ * *ms = 0 when that band had nothing to do at that layer. */
+int lop_plan_layer_time(lop_plan_t *plan, int band, int layer, float *ms);
+/* Which kernel family serves a layer: 0 = pooling, 1 = CUDA-core convolution,
+ * 2 = tcgen05 tensor-core convolution.  <0 on error. */
+int lop_plan_layer_kernel(const lop_plan_t *plan, int layer);
+/* Number of kernel launches and async copies the last execution call enqueued. */
+int lop_plan_last_launches(const lop_plan_t *plan);
+/* Reads the plan's device status word (0 = no kernel gave up on a bounded wait).  SYNCHRONISES
+ * the stream of the last execution call. */
+int lop_plan_check_device(lop_plan_t *plan, void *workspace);
+
+const char *lop_strerror(int status);
+const char *lop_last_error(void);       /* thread-local; valid until the next failing call */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LOP_H */

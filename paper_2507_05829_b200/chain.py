@@ -1,0 +1,128 @@
+"""Device-side convenience around :class:`binding.Plan`: one plan per segment of a workload.
+
+torch is used for device / pinned memory and streams only; every operator runs in the C-ABI
+library.  A workload is any object with ``dtype, N, H, W, C, segments`` whose layers carry the
+lop_layer fields plus numpy ``weight / scale / shift`` (see the ``lop_inputs`` package).
+"""
+from types import SimpleNamespace
+
+import numpy as np
+import torch
+
+from . import binding as B
+
+_FIELDS = ("op", "cin", "cout", "kh", "kw", "sh", "sw", "ph", "pw", "dh", "dw", "act", "input_from",
+           "residual_from", "residual_pos")
+
+
+def to_device(a, dtype, device):
+    """float32 numpy array -> device tensor in the storage dtype (bf16 values must be representable)."""
+    t = torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32))
+    if dtype == "bf16":
+        t = t.to(torch.bfloat16)            # exact: the generators hand out bf16-representable values
+    return t.to(device).contiguous()
+
+
+def to_host_f32(t):
+    return t.detach().to("cpu", torch.float32).numpy()
+
+
+class DeviceChain:
+    def __init__(self, wl, flags=0, device="cuda:0", n_bands=None):
+        if not torch.cuda.is_available():
+            raise RuntimeError("DeviceChain needs a CUDA device; there is no CPU path")
+        self.wl, self.device = wl, torch.device(device)
+        self.dtype = B.LOP_BF16 if wl.dtype == "bf16" else B.LOP_F32
+        self.tdtype = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
+        self.keep = []                       # device tensors the plans point into
+        self.plans, self.ws, self.outs = [], [], []
+        H, W, C = wl.H, wl.W, wl.C
+        with torch.cuda.device(self.device):
+            for seg in wl.segments:
+                layers = []
+                for l in seg.layers:
+                    d = SimpleNamespace(**{f: getattr(l, f) for f in _FIELDS})
+                    d.weight_ptr = d.scale_ptr = d.shift_ptr = None
+                    if l.weight is not None:
+                        w = to_device(l.weight, wl.dtype, self.device)
+                        self.keep.append(w)
+                        d.weight_ptr = w.data_ptr()
+                    for name in ("scale", "shift"):
+                        v = getattr(l, name)
+                        if v is not None:
+                            t = torch.from_numpy(np.ascontiguousarray(v, dtype=np.float32)).to(self.device)
+                            self.keep.append(t)
+                            setattr(d, name + "_ptr", t.data_ptr())
+                    layers.append(d)
+                nb = seg.n_bands if n_bands is None else n_bands
+                plan = B.Plan(layers, wl.N, H, W, C, self.dtype, nb, flags)
+                self.plans.append(plan)
+                self.ws.append(torch.zeros(max(plan.workspace_bytes(), 256), dtype=torch.uint8, device=self.device))
+                H, W, C = plan.out_shape(plan.num_layers() - 1)
+                self.outs.append(torch.zeros((wl.N, H, W, C), dtype=self.tdtype, device=self.device))
+        self.staging = torch.zeros((wl.N, wl.H, wl.W, wl.C), dtype=self.tdtype, device=self.device)
+
+    # -- helpers -------------------------------------------------------------------------------
+    def input_tensor(self, x=None):
+        return to_device(self.wl.x if x is None else x, self.wl.dtype, self.device)
+
+    def pinned_input(self, x=None):
+        t = torch.from_numpy(np.ascontiguousarray(self.wl.x if x is None else x, dtype=np.float32))
+        if self.wl.dtype == "bf16":
+            t = t.to(torch.bfloat16)
+        return t.contiguous().pin_memory()
+
+    def _stream(self, stream):
+        s = torch.cuda.current_stream(self.device) if stream is None else stream
+        return s.cuda_stream
+
+    def layer_output(self, seg, layer):
+        """View of an intermediate full-size tensor inside a segment's workspace (tests only)."""
+        plan = self.plans[seg]
+        if layer == plan.num_layers() - 1:
+            return self.outs[seg]
+        raise NotImplementedError
+
+    # -- execution -----------------------------------------------------------------------------
+    def run_whole(self, x_dev, stream=None):
+        s = self._stream(stream)
+        for plan, ws, out in zip(self.plans, self.ws, self.outs):
+            plan.run_whole(x_dev.data_ptr(), out.data_ptr(), ws.data_ptr(), s)
+            x_dev = out
+        return self.outs[-1]
+
+    def run_banded(self, x_dev, stream=None):
+        s = self._stream(stream)
+        for plan, ws, out in zip(self.plans, self.ws, self.outs):
+            plan.run_banded(x_dev.data_ptr(), out.data_ptr(), ws.data_ptr(), s)
+            x_dev = out
+        return self.outs[-1]
+
+    def run_bands_one_by_one(self, x_dev, order=None, stream=None):
+        s = self._stream(stream)
+        for plan, ws, out in zip(self.plans, self.ws, self.outs):
+            for b in (range(plan.num_bands()) if order is None else order(plan.num_bands())):
+                plan.run_band(b, x_dev.data_ptr(), out.data_ptr(), ws.data_ptr(), s)
+            x_dev = out
+        return self.outs[-1]
+
+    def run_pipelined(self, x_pinned, stream=None):
+        """Segment 0 streams its input bands from pinned host memory; later segments run band-wise on the device."""
+        s = self._stream(stream)
+        self.plans[0].run_pipelined(x_pinned.data_ptr(), self.staging.data_ptr(), self.outs[0].data_ptr(),
+                                    self.ws[0].data_ptr(), s)
+        x_dev = self.outs[0]
+        for plan, ws, out in list(zip(self.plans, self.ws, self.outs))[1:]:
+            plan.run_banded(x_dev.data_ptr(), out.data_ptr(), ws.data_ptr(), s)
+            x_dev = out
+        return self.outs[-1]
+
+    def check_device(self):
+        for plan, ws in zip(self.plans, self.ws):
+            plan.check_device(ws.data_ptr())
+
+    def launches(self):
+        return sum(p.last_launches() for p in self.plans)
+
+    def flops(self):
+        return sum(p.flops() for p in self.plans)

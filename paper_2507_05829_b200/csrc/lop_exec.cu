@@ -1,0 +1,390 @@
+// Chain executor and band scheduler: lop_run_whole / lop_run_band / lop_run_banded /
+// lop_copy_band / lop_run_pipelined.
+//
+// Sec. IV-B of the paper: a band's operations at every layer run in dependency order as soon
+// as their inputs exist; the transfer of the next band's input overlaps the current band's
+// computation.  Here the "transmission" is an asynchronous pinned-host -> device copy on a side
+// stream, the dependency "input has arrived" is a CUDA event, and tensor "combining" is
+// addressing: every band writes its rows straight into full-size tensors.
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <map>
+#include <tuple>
+#include <vector>
+
+#include "lop_internal.h"
+#include "lop_kernels.cuh"
+
+namespace lop {
+
+struct MapKey {
+    int layer, TW, TR, TN, BN, BK;
+    const void *x, *w;
+    bool operator<(const MapKey &o) const
+    {
+        return std::tie(layer, TW, TR, TN, BN, BK, x, w) < std::tie(o.layer, o.TW, o.TR, o.TN, o.BN, o.BK, o.x, o.w);
+    }
+};
+
+struct ExecState {
+    cudaStream_t copy_stream = nullptr;
+    cudaEvent_t ev_fork = nullptr, ev_begin = nullptr, ev_end = nullptr;
+    std::vector<cudaEvent_t> ev_copy_start, ev_copy_end;       // [band]
+    std::vector<cudaEvent_t> ev_layer;                         // [(band+1) * L + layer] * 2, slot 0 = whole
+    std::vector<char> layer_timed;
+    std::map<MapKey, ConvTcMaps> maps;
+    const void *prepared_ws = nullptr;
+    std::vector<const void *> prepared_w;                      // weight pointers the padded copies were made from
+    cudaStream_t last_stream = nullptr;
+    int launches = 0;
+    bool timing_valid = false;
+    std::vector<char> copy_issued;
+};
+
+void exec_destroy(ExecState *e)
+{
+    if (!e) return;
+    if (e->copy_stream) cudaStreamDestroy(e->copy_stream);
+    for (cudaEvent_t ev : {e->ev_fork, e->ev_begin, e->ev_end})
+        if (ev) cudaEventDestroy(ev);
+    for (auto &v : {&e->ev_copy_start, &e->ev_copy_end, &e->ev_layer})
+        for (cudaEvent_t ev : *v)
+            if (ev) cudaEventDestroy(ev);
+    delete e;
+}
+
+namespace {
+
+#define LOP_CUDA(call)                                                                  \
+    do {                                                                                \
+        cudaError_t e__ = (call);                                                       \
+        if (e__ != cudaSuccess) {                                                       \
+            set_error("%s failed: %s", #call, cudaGetErrorString(e__));                 \
+            return LOP_ECUDA;                                                           \
+        }                                                                               \
+    } while (0)
+
+int ensure_exec(lop_plan_t *pl)
+{
+    if (pl->exec) return LOP_OK;
+    ExecState *e = new (std::nothrow) ExecState();
+    if (!e) { set_error("out of host memory"); return LOP_ENOMEM; }
+    pl->exec = e;
+    const int B = pl->n_bands, L = (int)pl->layers.size();
+    LOP_CUDA(cudaStreamCreateWithFlags(&e->copy_stream, cudaStreamNonBlocking));
+    LOP_CUDA(cudaEventCreateWithFlags(&e->ev_fork, cudaEventDisableTiming));
+    LOP_CUDA(cudaEventCreate(&e->ev_begin));
+    LOP_CUDA(cudaEventCreate(&e->ev_end));
+    e->ev_copy_start.assign(B, nullptr);
+    e->ev_copy_end.assign(B, nullptr);
+    e->copy_issued.assign(B, 0);
+    for (int b = 0; b < B; ++b) {
+        LOP_CUDA(cudaEventCreate(&e->ev_copy_start[b]));
+        LOP_CUDA(cudaEventCreate(&e->ev_copy_end[b]));
+    }
+    if (pl->flags & LOP_FLAG_TIME_LAYERS) {
+        e->ev_layer.assign((size_t)(B + 1) * L * 2, nullptr);
+        e->layer_timed.assign((size_t)(B + 1) * L, 0);
+        for (auto &ev : e->ev_layer) LOP_CUDA(cudaEventCreate(&ev));
+    }
+    e->prepared_w.assign(L, nullptr);
+    return LOP_OK;
+}
+
+int check_common(lop_plan_t *pl, const void *in, const void *out, const void *ws)
+{
+    if (!pl) { set_error("plan is NULL"); return LOP_EINVAL; }
+    if (!in || !out) { set_error("input/output pointer is NULL"); return LOP_EINVAL; }
+    if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255u)) { set_error("workspace is NULL or not 256-byte aligned"); return LOP_EWORKSPACE; }
+    if ((reinterpret_cast<uintptr_t>(in) & 15u) || (reinterpret_cast<uintptr_t>(out) & 15u)) {
+        set_error("input/output tensors must be 16-byte aligned");
+        return LOP_EINVAL;
+    }
+    for (size_t i = 0; i < pl->layers.size(); ++i)
+        if (pl->layers[i].l.op == LOP_CONV2D && !pl->layers[i].l.weight) {
+            set_error("layer %zu has no weight pointer (lop_plan_set_params)", i);
+            return LOP_EINVAL;
+        }
+    return ensure_exec(pl);
+}
+
+// One-time work per workspace: clear the status word, build channel-padded first-layer weights.
+int prepare_workspace(lop_plan_t *pl, void *ws, cudaStream_t s)
+{
+    ExecState *e = pl->exec;
+    char *base = static_cast<char *>(ws);
+    bool fresh = e->prepared_ws != ws;
+    if (fresh) {
+        LOP_CUDA(cudaMemsetAsync(base + pl->status_off, 0, 1024, s));
+        e->launches++;
+    }
+    for (size_t i = 0; i < pl->layers.size(); ++i) {
+        LayerInfo &li = pl->layers[i];
+        if (!li.reads_padded_input) continue;
+        if (!fresh && e->prepared_w[i] == li.l.weight) continue;
+        LOP_CUDA(launch_pad_weights(li.l.weight, base + li.wpad_off, (long long)li.l.cout * li.l.kh * li.l.kw, li.l.cin,
+                                    li.cin_eff, s));
+        e->prepared_w[i] = li.l.weight;
+        e->launches++;
+    }
+    e->prepared_ws = ws;
+    return LOP_OK;
+}
+
+const void *tensor_of(const lop_plan_t *pl, int idx, const void *in, void *out, void *ws)
+{
+    if (idx == LOP_INPUT) return in;
+    if (idx == (int)pl->layers.size() - 1) return out;
+    return static_cast<char *>(ws) + pl->layers[idx].out_off;
+}
+
+// Rows [lo, hi) of layer i.  slot: index into the per-layer timing events, or -1.
+int run_layer(lop_plan_t *pl, int i, int lo, int hi, const void *in, void *out, void *ws, cudaStream_t s, int slot)
+{
+    if (hi <= lo) return LOP_OK;
+    ExecState *e = pl->exec;
+    LayerInfo &li = pl->layers[i];
+    const lop_layer &l = li.l;
+    const bool timed = slot >= 0 && !e->ev_layer.empty();
+    if (timed) {
+        LOP_CUDA(cudaEventRecord(e->ev_layer[(size_t)slot * 2], s));
+        e->layer_timed[slot] = 1;
+    }
+    void *y = const_cast<void *>(tensor_of(pl, i, in, out, ws));
+    if (l.op == LOP_MAXPOOL2D) {
+        PoolArgs a;
+        a.x = tensor_of(pl, l.input_from, in, out, ws);
+        a.y = y;
+        a.N = pl->N; a.Hin = li.Hin; a.Win = li.Win; a.C = l.cin; a.Ho = li.Ho; a.Wo = li.Wo;
+        a.kh = l.kh; a.kw = l.kw; a.sh = l.sh; a.sw = l.sw; a.ph = l.ph; a.pw = l.pw; a.dh = l.dh; a.dw = l.dw;
+        a.oh_lo = lo; a.oh_hi = hi;
+        LOP_CUDA(launch_maxpool(a, pl->dtype, s));
+    } else {
+        ConvArgs a;
+        a.x = tensor_of(pl, l.input_from, in, out, ws);
+        a.w = l.weight;
+        a.scale = l.scale; a.shift = l.shift;
+        a.res = l.residual_from == LOP_NO_RESIDUAL ? nullptr : tensor_of(pl, l.residual_from, in, out, ws);
+        a.y = y;
+        a.N = pl->N; a.Hin = li.Hin; a.Win = li.Win; a.Cin = l.cin; a.Ho = li.Ho; a.Wo = li.Wo; a.Cout = l.cout;
+        a.kh = l.kh; a.kw = l.kw; a.sh = l.sh; a.sw = l.sw; a.ph = l.ph; a.pw = l.pw; a.dh = l.dh; a.dw = l.dw;
+        a.act = l.act; a.res_pos = a.res ? l.residual_pos : LOP_RES_NONE;
+        a.oh_lo = lo; a.oh_hi = hi;
+        if (li.kernel == K_CONV_TC) {
+            if (li.reads_padded_input) {
+                a.x = static_cast<char *>(ws) + pl->padin_off;
+                a.w = static_cast<char *>(ws) + li.wpad_off;
+            }
+            a.Cin = li.cin_eff;
+            const ConvTcGeom g = conv_tc_geometry(a, hi - lo);
+            const MapKey key{i, g.TW, g.TR, g.TN, g.BN, g.BK, a.x, a.w};
+            auto it = e->maps.find(key);
+            if (it == e->maps.end()) {
+                ConvTcMaps m;
+                int rc = conv_tc_encode(a, g, &m);
+                if (rc != LOP_OK) { set_error("layer %d: tensor-map encoding failed", i); return rc; }
+                it = e->maps.emplace(key, m).first;
+            }
+            LOP_CUDA(launch_conv_tc(a, g, it->second, reinterpret_cast<unsigned *>(static_cast<char *>(ws) + pl->status_off), s));
+        } else {
+            LOP_CUDA(launch_conv_simt(a, pl->dtype, s));
+        }
+    }
+    e->launches++;
+    if (timed) LOP_CUDA(cudaEventRecord(e->ev_layer[(size_t)slot * 2 + 1], s));
+    return LOP_OK;
+}
+
+int pad_input_rows(lop_plan_t *pl, int lo, int hi, const void *in, void *ws, cudaStream_t s)
+{
+    if (!pl->Cpad || hi <= lo) return LOP_OK;
+    LOP_CUDA(launch_pad_channels(in, static_cast<char *>(ws) + pl->padin_off, pl->N, pl->H, pl->W, pl->C, pl->Cpad, lo, hi, s));
+    pl->exec->launches++;
+    return LOP_OK;
+}
+
+int run_band_impl(lop_plan_t *pl, int band, const void *in, void *out, void *ws, cudaStream_t s)
+{
+    const int L = (int)pl->layers.size();
+    const bool reuse = (pl->flags & LOP_FLAG_REUSE_HALO) != 0;
+    const lop_range &need = pl->in_need[band];
+    int rc = pad_input_rows(pl, reuse ? need.new_lo : need.out_lo, need.out_hi, in, ws, s);
+    if (rc != LOP_OK) return rc;
+    for (int i = 0; i < L; ++i) {
+        const lop_range &r = pl->ranges[(size_t)band * L + i];
+        rc = run_layer(pl, i, reuse ? r.new_lo : r.out_lo, r.out_hi, in, out, ws, s, (band + 1) * L + i);
+        if (rc != LOP_OK) return rc;
+    }
+    return LOP_OK;
+}
+
+void reset_layer_timing(lop_plan_t *pl)
+{
+    for (auto &c : pl->exec->layer_timed) c = 0;
+}
+
+int copy_band_impl(lop_plan_t *pl, int band, const void *host, void *staging, cudaStream_t s)
+{
+    const lop_range &need = pl->in_need[band];
+    const int lo = need.new_lo, hi = need.out_hi;
+    if (hi <= lo) return LOP_OK;
+    const size_t row = (size_t)pl->W * pl->C * elem_size(pl->dtype);
+    const size_t img = row * pl->H;
+    LOP_CUDA(cudaMemcpy2DAsync(static_cast<char *>(staging) + lo * row, img, static_cast<const char *>(host) + lo * row, img,
+                               (size_t)(hi - lo) * row, pl->N, cudaMemcpyHostToDevice, s));
+    pl->exec->launches++;
+    return LOP_OK;
+}
+
+}  // namespace
+}  // namespace lop
+
+using namespace lop;
+
+extern "C" {
+
+int lop_run_whole(lop_plan_t *pl, const void *in, void *out, void *ws, void *stream)
+{
+    int rc = check_common(pl, in, out, ws);
+    if (rc != LOP_OK) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    pl->exec->launches = 0;
+    pl->exec->last_stream = s;
+    reset_layer_timing(pl);
+    if ((rc = prepare_workspace(pl, ws, s)) != LOP_OK) return rc;
+    if ((rc = pad_input_rows(pl, 0, pl->H, in, ws, s)) != LOP_OK) return rc;
+    for (int i = 0; i < (int)pl->layers.size(); ++i)
+        if ((rc = run_layer(pl, i, 0, pl->layers[i].Ho, in, out, ws, s, i)) != LOP_OK) return rc;
+    return LOP_OK;
+}
+
+int lop_run_band(lop_plan_t *pl, int band, const void *in, void *out, void *ws, void *stream)
+{
+    int rc = check_common(pl, in, out, ws);
+    if (rc != LOP_OK) return rc;
+    if (band < 0 || band >= pl->n_bands) { set_error("band %d out of range", band); return LOP_EINVAL; }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    pl->exec->launches = 0;
+    pl->exec->last_stream = s;
+    if ((rc = prepare_workspace(pl, ws, s)) != LOP_OK) return rc;
+    return run_band_impl(pl, band, in, out, ws, s);
+}
+
+int lop_run_banded(lop_plan_t *pl, const void *in, void *out, void *ws, void *stream)
+{
+    int rc = check_common(pl, in, out, ws);
+    if (rc != LOP_OK) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    pl->exec->launches = 0;
+    pl->exec->last_stream = s;
+    reset_layer_timing(pl);
+    if ((rc = prepare_workspace(pl, ws, s)) != LOP_OK) return rc;
+    for (int b = 0; b < pl->n_bands; ++b)
+        if ((rc = run_band_impl(pl, b, in, out, ws, s)) != LOP_OK) return rc;
+    return LOP_OK;
+}
+
+int lop_copy_band(lop_plan_t *pl, int band, const void *host, void *staging, void *stream)
+{
+    if (!pl || !host || !staging) { set_error("lop_copy_band: NULL argument"); return LOP_EINVAL; }
+    if (band < 0 || band >= pl->n_bands) { set_error("band %d out of range", band); return LOP_EINVAL; }
+    int rc = ensure_exec(pl);
+    if (rc != LOP_OK) return rc;
+    pl->exec->launches = 0;
+    return copy_band_impl(pl, band, host, staging, static_cast<cudaStream_t>(stream));
+}
+
+int lop_run_pipelined(lop_plan_t *pl, const void *host, void *staging, void *out, void *ws, void *stream)
+{
+    int rc = check_common(pl, staging, out, ws);
+    if (rc != LOP_OK) return rc;
+    if (!host) { set_error("lop_run_pipelined: host input is NULL"); return LOP_EINVAL; }
+    ExecState *e = pl->exec;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    e->launches = 0;
+    e->last_stream = s;
+    e->timing_valid = false;
+    reset_layer_timing(pl);
+    LOP_CUDA(cudaEventRecord(e->ev_begin, s));
+    // the side stream starts after everything already queued on the caller's stream
+    LOP_CUDA(cudaEventRecord(e->ev_fork, s));
+    LOP_CUDA(cudaStreamWaitEvent(e->copy_stream, e->ev_fork, 0));
+    if ((rc = prepare_workspace(pl, ws, s)) != LOP_OK) return rc;
+    // all transfers are queued up front on the side stream: band i+1 (and later) stream in while band i computes
+    for (int b = 0; b < pl->n_bands; ++b) {
+        const lop_range &need = pl->in_need[b];
+        e->copy_issued[b] = need.out_hi > need.new_lo;
+        if (!e->copy_issued[b]) continue;
+        LOP_CUDA(cudaEventRecord(e->ev_copy_start[b], e->copy_stream));
+        if ((rc = copy_band_impl(pl, b, host, staging, e->copy_stream)) != LOP_OK) return rc;
+        LOP_CUDA(cudaEventRecord(e->ev_copy_end[b], e->copy_stream));
+    }
+    bool joined = false;
+    for (int b = 0; b < pl->n_bands; ++b) {
+        if (e->copy_issued[b]) {
+            LOP_CUDA(cudaStreamWaitEvent(s, e->ev_copy_end[b], 0));
+            joined = true;
+        }
+        if ((rc = run_band_impl(pl, b, staging, out, ws, s)) != LOP_OK) return rc;
+    }
+    if (!joined) LOP_CUDA(cudaStreamWaitEvent(s, e->ev_fork, 0));
+    LOP_CUDA(cudaEventRecord(e->ev_end, s));
+    e->timing_valid = true;
+    return LOP_OK;
+}
+
+int lop_plan_last_timing(lop_plan_t *pl, lop_timing *out)
+{
+    if (!pl || !out) { set_error("lop_plan_last_timing: NULL argument"); return LOP_EINVAL; }
+    if (!pl->exec || !pl->exec->timing_valid) { set_error("no pipelined run to report"); return LOP_EINVAL; }
+    ExecState *e = pl->exec;
+    LOP_CUDA(cudaEventSynchronize(e->ev_end));
+    lop_timing t = {0, 0, 0, 0, 0};
+    LOP_CUDA(cudaEventElapsedTime(&t.total_ms, e->ev_begin, e->ev_end));
+    bool first = true;
+    for (int b = 0; b < pl->n_bands; ++b) {
+        if (!e->copy_issued[b]) continue;
+        float ms = 0;
+        LOP_CUDA(cudaEventElapsedTime(&ms, e->ev_copy_start[b], e->ev_copy_end[b]));
+        t.copy_ms += ms;
+        if (first) { t.first_copy_ms = ms; first = false; }
+        t.n_copies++;
+    }
+    *out = t;
+    return LOP_OK;
+}
+
+int lop_plan_layer_time(lop_plan_t *pl, int band, int layer, float *ms)
+{
+    if (!pl || !ms) { set_error("lop_plan_layer_time: NULL argument"); return LOP_EINVAL; }
+    const int L = (int)pl->layers.size();
+    if (band < -1 || band >= pl->n_bands || layer < 0 || layer >= L) { set_error("band/layer out of range"); return LOP_EINVAL; }
+    if (!pl->exec || pl->exec->ev_layer.empty()) { set_error("plan was not made with LOP_FLAG_TIME_LAYERS, or has not run"); return LOP_EINVAL; }
+    ExecState *e = pl->exec;
+    const size_t slot = (size_t)(band + 1) * L + layer;
+    *ms = 0.0f;
+    if (!e->layer_timed[slot]) return LOP_OK;
+    LOP_CUDA(cudaEventSynchronize(e->ev_layer[slot * 2 + 1]));
+    LOP_CUDA(cudaEventElapsedTime(ms, e->ev_layer[slot * 2], e->ev_layer[slot * 2 + 1]));
+    return LOP_OK;
+}
+
+int lop_plan_last_launches(const lop_plan_t *pl)
+{
+    if (!pl) { set_error("plan is NULL"); return LOP_EINVAL; }
+    return pl->exec ? pl->exec->launches : 0;
+}
+
+int lop_plan_check_device(lop_plan_t *pl, void *ws)
+{
+    if (!pl || !ws) { set_error("lop_plan_check_device: NULL argument"); return LOP_EINVAL; }
+    if (!pl->exec) return LOP_OK;
+    LOP_CUDA(cudaStreamSynchronize(pl->exec->last_stream));
+    unsigned status = 0;
+    LOP_CUDA(cudaMemcpy(&status, static_cast<char *>(ws) + pl->status_off, sizeof(status), cudaMemcpyDeviceToHost));
+    if (status) { set_error("device status word 0x%x: a bounded wait ran out", status); return LOP_EDEVICE; }
+    return LOP_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,50 @@
+// Internal declarations shared by the library's translation units (not part of the ABI).
+#pragma once
+#include <cstdint>
+#include <cstddef>
+#include <string>
+#include <vector>
+
+#include "lop.h"
+
+namespace lop {
+
+enum KernelFamily { K_POOL = 0, K_CONV_SIMT = 1, K_CONV_TC = 2 };
+
+struct LayerInfo {
+    lop_layer l;
+    int Hin = 0, Win = 0;          // spatial extent of the main input
+    int Ho = 0, Wo = 0, Co = 0;    // output shape
+    int kernel = K_CONV_SIMT;
+    int cin_eff = 0;               // channels the tensor-core kernel sees (chain input may be channel-padded)
+    bool reads_padded_input = false;
+    size_t out_off = 0;            // workspace offset of the full-size output (unused for the last layer)
+    size_t wpad_off = 0;           // workspace offset of the channel-padded weights (if reads_padded_input)
+};
+
+struct ExecState;                  // CUDA-side resources, defined in lop_exec.cu
+
+}  // namespace lop
+
+struct lop_plan {
+    std::vector<lop::LayerInfo> layers;
+    int N = 0, H = 0, W = 0, C = 0, dtype = 0, n_bands = 0;
+    unsigned flags = 0;
+    int Cpad = 0;                  // >0: a [N,H,W,Cpad] copy of the chain input lives in the workspace
+    std::vector<lop_range> ranges;     // [band][layer]
+    std::vector<lop_range> in_need;    // [band]: chain-input rows (out_lo,out_hi,new_lo)
+    size_t ws_bytes = 0, status_off = 0, padin_off = 0;
+    double flops = 0.0;
+    lop::ExecState *exec = nullptr;
+};
+
+namespace lop {
+
+void set_error(const char *fmt, ...);
+inline size_t elem_size(int dtype) { return dtype == LOP_BF16 ? 2 : 4; }
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// lop_exec.cu
+void exec_destroy(ExecState *e);
+
+}  // namespace lop

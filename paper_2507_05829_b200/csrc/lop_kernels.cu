@@ -1,0 +1,320 @@
+// CUDA-core kernels: general convolution (any kernel/stride/padding/dilation/channel count),
+// max pooling, channel padding of the chain input (the band "split" step) and of weights.
+//
+// The convolution here is the fp32 path and the fall-back for shapes the tensor-core kernel
+// does not take; it is also the library's second on-GPU opinion (LOP_FLAG_FORCE_SIMT).
+// Operators: Sec. IV-A of the paper (block-wise and element-wise local operators).
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "lop.h"
+#include "lop_kernels.cuh"
+
+namespace lop {
+
+namespace {
+
+__device__ __forceinline__ float to_f32(float v) { return v; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 v) { return __bfloat162float(v); }
+__device__ __forceinline__ void from_f32(float &d, float v) { d = v; }
+__device__ __forceinline__ void from_f32(__nv_bfloat16 &d, float v) { d = __float2bfloat16_rn(v); }
+
+__device__ __forceinline__ float activate(float t, int act)
+{
+    if (act == LOP_ACT_RELU) return fmaxf(t, 0.0f);
+    if (act == LOP_ACT_SILU) return t / (1.0f + expf(-t));
+    return t;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Implicit-GEMM convolution on CUDA cores.  M = N*rows*Wo output pixels, N = Cout, K = kh*kw*Cin.
+// 64x64 tile per 256-thread block, 16-wide K slabs staged through shared memory, 4x4 outputs per
+// thread.  K is walked in one fixed order, so a pixel's value does not depend on the band it is in.
+// ---------------------------------------------------------------------------------------------
+constexpr int SM_BM = 64, SM_BN = 64, SM_BK = 16;
+
+template <typename T>
+__global__ void __launch_bounds__(256) conv_simt_kernel(ConvArgs p)
+{
+    __shared__ float As[SM_BK][SM_BM + 4];
+    __shared__ float Bs[SM_BK][SM_BN + 4];
+
+    const T *__restrict__ x = static_cast<const T *>(p.x);
+    const T *__restrict__ w = static_cast<const T *>(p.w);
+    const int rows = p.oh_hi - p.oh_lo;
+    const long long M = (long long)p.N * rows * p.Wo;
+    const int K = p.kh * p.kw * p.Cin;
+    const long long m0 = (long long)blockIdx.x * SM_BM;
+    const int n0 = blockIdx.y * SM_BN;
+    const int t = threadIdx.x;
+    const int kk = t & 15;              // K index inside the slab this thread stages
+    const int lr = t >> 4;              // 0..15: first of the 4 tile rows (stride 16) this thread stages
+
+    // the four pixels / four output channels whose operands this thread stages
+    long long xbase[4];
+    int ih0[4], iw0[4];
+    bool mvalid[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const long long m = m0 + lr + e * 16;
+        mvalid[e] = m < M;
+        const long long mm = mvalid[e] ? m : 0;
+        const int ow = (int)(mm % p.Wo);
+        const long long q = mm / p.Wo;
+        const int oh = p.oh_lo + (int)(q % rows);
+        const int n = (int)(q / rows);
+        ih0[e] = oh * p.sh - p.ph;
+        iw0[e] = ow * p.sw - p.pw;
+        xbase[e] = (long long)n * p.Hin * p.Win * p.Cin;
+    }
+
+    const int tx = t & 15, ty = t >> 4;
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.0f;
+
+    for (int k0 = 0; k0 < K; k0 += SM_BK) {
+        const int k = k0 + kk;
+        const bool kvalid = k < K;
+        int ci = 0, a = 0, b = 0;
+        if (kvalid) {
+            ci = k % p.Cin;
+            const int tap = k / p.Cin;
+            b = tap % p.kw;
+            a = tap / p.kw;
+        }
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            float v = 0.0f;
+            if (kvalid && mvalid[e]) {
+                const int ih = ih0[e] + a * p.dh, iw = iw0[e] + b * p.dw;
+                if (ih >= 0 && ih < p.Hin && iw >= 0 && iw < p.Win)
+                    v = to_f32(x[xbase[e] + ((long long)ih * p.Win + iw) * p.Cin + ci]);
+            }
+            As[kk][lr + e * 16] = v;
+            float wv = 0.0f;
+            const int co = n0 + lr + e * 16;
+            if (kvalid && co < p.Cout) wv = to_f32(w[(long long)co * K + k]);
+            Bs[kk][lr + e * 16] = wv;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int q = 0; q < SM_BK; ++q) {
+            float av[4], bv[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) av[i] = As[q][ty * 4 + i];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) bv[j] = Bs[q][tx * 4 + j];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+
+    T *__restrict__ y = static_cast<T *>(p.y);
+    const T *__restrict__ res = static_cast<const T *>(p.res);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const long long m = m0 + ty * 4 + i;
+        if (m >= M) continue;
+        const int ow = (int)(m % p.Wo);
+        const long long q = m / p.Wo;
+        const int oh = p.oh_lo + (int)(q % rows);
+        const int n = (int)(q / rows);
+        const long long o = (((long long)n * p.Ho + oh) * p.Wo + ow) * p.Cout;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int co = n0 + tx * 4 + j;
+            if (co >= p.Cout) continue;
+            float v = acc[i][j];
+            v = fmaf(p.scale ? p.scale[co] : 1.0f, v, p.shift ? p.shift[co] : 0.0f);
+            if (res && p.res_pos == LOP_RES_PRE_ACT) v += to_f32(res[o + co]);
+            v = activate(v, p.act);
+            if (res && p.res_pos == LOP_RES_POST_ACT) v += to_f32(res[o + co]);
+            from_f32(y[o + co], v);
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Max pooling, NHWC.  One thread per (output pixel, group of VEC channels); a warp covers
+// consecutive channel groups of consecutive pixels, so loads and stores are 16-byte and coalesced.
+// HBM-bound: bytes = rows read once + rows written once.
+// ---------------------------------------------------------------------------------------------
+template <typename T, int VEC>
+struct alignas(sizeof(T) * VEC) Pack {
+    T v[VEC];
+};
+
+template <typename T, int VEC>
+__global__ void __launch_bounds__(256) maxpool_kernel(PoolArgs p)
+{
+    const int rows = p.oh_hi - p.oh_lo;
+    const int cg = p.C / VEC;
+    const long long total = (long long)p.N * rows * p.Wo * cg;
+    const T *__restrict__ x = static_cast<const T *>(p.x);
+    T *__restrict__ y = static_cast<T *>(p.y);
+    for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+         idx += (long long)gridDim.x * blockDim.x) {
+        const int g = (int)(idx % cg);
+        long long q = idx / cg;
+        const int ow = (int)(q % p.Wo);
+        q /= p.Wo;
+        const int oh = p.oh_lo + (int)(q % rows);
+        const int n = (int)(q / rows);
+        float m[VEC];
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) m[i] = -INFINITY;
+        for (int a = 0; a < p.kh; ++a) {
+            const int ih = oh * p.sh - p.ph + a * p.dh;
+            if (ih < 0 || ih >= p.Hin) continue;
+            for (int b = 0; b < p.kw; ++b) {
+                const int iw = ow * p.sw - p.pw + b * p.dw;
+                if (iw < 0 || iw >= p.Win) continue;
+                const Pack<T, VEC> v = *reinterpret_cast<const Pack<T, VEC> *>(
+                    x + (((long long)n * p.Hin + ih) * p.Win + iw) * p.C + (long long)g * VEC);
+#pragma unroll
+                for (int i = 0; i < VEC; ++i) m[i] = fmaxf(m[i], to_f32(v.v[i]));
+            }
+        }
+        Pack<T, VEC> o;
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) from_f32(o.v[i], m[i]);
+        *reinterpret_cast<Pack<T, VEC> *>(y + (((long long)n * p.Ho + oh) * p.Wo + ow) * p.C + (long long)g * VEC) = o;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Channel padding of a row band of the chain input (the tensor "split" an operator interceptor
+// performs, Sec. III-B): x[N,H,W,C] rows [lo,hi) -> y[N,H,W,Cpad], zero in channels C..Cpad-1.
+// A warp takes 32 consecutive pixels of one image's band: their C*32 input elements are one
+// contiguous run that the lanes load coalesced, then each lane collects its own pixel's channels
+// with warp shuffles and writes Cpad*2 bytes as 16-byte stores.  C <= 16 = Cpad.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) pad_channels_kernel(const uint16_t *__restrict__ x, uint16_t *__restrict__ y,
+                                                           int N, int H, int W, int C, int lo, int hi)
+{
+    constexpr int CP = 16;
+    const int lane = threadIdx.x & 31;
+    const long long per_img = (long long)(hi - lo) * W;          // pixels of one image's band
+    const long long warps_per_img = (per_img + 31) / 32;
+    const long long nwarps = warps_per_img * N;
+    const long long wstride = (long long)gridDim.x * (blockDim.x >> 5);
+    for (long long wid = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); wid < nwarps; wid += wstride) {
+        const int n = (int)(wid / warps_per_img);
+        const long long p0 = (wid % warps_per_img) * 32;
+        const int npix = (int)((per_img - p0) < 32 ? (per_img - p0) : 32);
+        const long long pix0 = ((long long)n * H + lo) * W + p0;  // first pixel, in whole-tensor pixel units
+        const uint16_t *src = x + pix0 * C;
+        const int nelem = npix * C;
+        uint16_t v[CP];
+#pragma unroll
+        for (int j = 0; j < CP; ++j) {
+            v[j] = 0;
+            if (j < C) {
+                const int e = lane + 32 * j;
+                if (e < nelem) v[j] = src[e];
+            }
+        }
+        uint16_t out[CP];
+#pragma unroll
+        for (int c = 0; c < CP; ++c) {
+            out[c] = 0;
+            if (c < C) {                                          // uniform across the warp
+                const int e = lane * C + c;
+                const int srcl = e & 31, srcj = e >> 5;
+                uint16_t got = 0;
+#pragma unroll
+                for (int j = 0; j < CP; ++j) {
+                    if (j < C) {                                  // uniform across the warp
+                        const unsigned tmp = __shfl_sync(0xffffffffu, (unsigned)v[j], srcl);
+                        if (srcj == j) got = (uint16_t)tmp;
+                    }
+                }
+                out[c] = got;
+            }
+        }
+        if (lane < npix) {
+            uint4 *dst = reinterpret_cast<uint4 *>(y + (pix0 + lane) * CP);
+            uint4 q0, q1;
+            q0.x = out[0] | ((unsigned)out[1] << 16);  q0.y = out[2] | ((unsigned)out[3] << 16);
+            q0.z = out[4] | ((unsigned)out[5] << 16);  q0.w = out[6] | ((unsigned)out[7] << 16);
+            q1.x = out[8] | ((unsigned)out[9] << 16);  q1.y = out[10] | ((unsigned)out[11] << 16);
+            q1.z = out[12] | ((unsigned)out[13] << 16); q1.w = out[14] | ((unsigned)out[15] << 16);
+            dst[0] = q0;
+            dst[1] = q1;
+        }
+    }
+}
+
+__global__ void pad_weights_kernel(const uint16_t *__restrict__ w, uint16_t *__restrict__ wp, long long rows, int C,
+                                   int Cpad)
+{
+    const long long total = rows * Cpad;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
+         i += (long long)gridDim.x * blockDim.x) {
+        const int c = (int)(i % Cpad);
+        const long long r = i / Cpad;
+        wp[i] = c < C ? w[r * C + c] : (uint16_t)0;
+    }
+}
+
+inline int grid_for(long long work_items, int block, int max_blocks = 148 * 8)
+{
+    long long b = (work_items + block - 1) / block;
+    if (b < 1) b = 1;
+    if (b > max_blocks) b = max_blocks;
+    return (int)b;
+}
+
+}  // namespace
+
+cudaError_t launch_conv_simt(const ConvArgs &a, int dtype, cudaStream_t s)
+{
+    const int rows = a.oh_hi - a.oh_lo;
+    if (rows <= 0) return cudaSuccess;
+    const long long M = (long long)a.N * rows * a.Wo;
+    dim3 grid((unsigned)((M + SM_BM - 1) / SM_BM), (unsigned)((a.Cout + SM_BN - 1) / SM_BN));
+    if (dtype == LOP_BF16) conv_simt_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>(a);
+    else conv_simt_kernel<float><<<grid, 256, 0, s>>>(a);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_maxpool(const PoolArgs &a, int dtype, cudaStream_t s)
+{
+    const int rows = a.oh_hi - a.oh_lo;
+    if (rows <= 0) return cudaSuccess;
+    const long long pix = (long long)a.N * rows * a.Wo;
+    if (dtype == LOP_BF16) {
+        if (a.C % 8 == 0) maxpool_kernel<__nv_bfloat16, 8><<<grid_for(pix * (a.C / 8), 256), 256, 0, s>>>(a);
+        else maxpool_kernel<__nv_bfloat16, 1><<<grid_for(pix * a.C, 256), 256, 0, s>>>(a);
+    } else {
+        if (a.C % 4 == 0) maxpool_kernel<float, 4><<<grid_for(pix * (a.C / 4), 256), 256, 0, s>>>(a);
+        else maxpool_kernel<float, 1><<<grid_for(pix * a.C, 256), 256, 0, s>>>(a);
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_pad_channels(const void *x, void *y, int N, int H, int W, int C, int Cpad, int lo, int hi,
+                                cudaStream_t s)
+{
+    if (hi <= lo) return cudaSuccess;
+    if (Cpad != 16 || C > 16) return cudaErrorInvalidValue;
+    const long long warps = (((long long)(hi - lo) * W + 31) / 32) * N;
+    pad_channels_kernel<<<grid_for(warps * 32, 256), 256, 0, s>>>(static_cast<const uint16_t *>(x),
+                                                                   static_cast<uint16_t *>(y), N, H, W, C, lo, hi);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_pad_weights(const void *w, void *wp, long long rows, int C, int Cpad, cudaStream_t s)
+{
+    pad_weights_kernel<<<grid_for(rows * Cpad, 256), 256, 0, s>>>(static_cast<const uint16_t *>(w),
+                                                                  static_cast<uint16_t *>(wp), rows, C, Cpad);
+    return cudaGetLastError();
+}
+
+}  // namespace lop

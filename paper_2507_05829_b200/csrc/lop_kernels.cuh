@@ -1,0 +1,57 @@
+// Launch interfaces of the device kernels (host-callable wrappers; each returns a cudaError_t).
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <cstdint>
+
+namespace lop {
+
+struct ConvArgs {
+    const void *x;          // [N, Hin, Win, Cin]
+    const void *w;          // [Cout, kh, kw, Cin]
+    const float *scale, *shift;
+    const void *res;        // [N, Ho, Wo, Cout] or nullptr
+    void *y;                // [N, Ho, Wo, Cout]
+    int N, Hin, Win, Cin, Ho, Wo, Cout;
+    int kh, kw, sh, sw, ph, pw, dh, dw;
+    int act, res_pos;
+    int oh_lo, oh_hi;       // rows to compute
+};
+
+struct PoolArgs {
+    const void *x;
+    void *y;
+    int N, Hin, Win, C, Ho, Wo;
+    int kh, kw, sh, sw, ph, pw, dh, dw;
+    int oh_lo, oh_hi;
+};
+
+// CUDA-core convolution (fp32 accumulate); dtype: LOP_F32 / LOP_BF16 storage.
+cudaError_t launch_conv_simt(const ConvArgs &a, int dtype, cudaStream_t s);
+cudaError_t launch_maxpool(const PoolArgs &a, int dtype, cudaStream_t s);
+// rows [lo,hi) of x[N,H,W,C] -> same rows of y[N,H,W,Cpad], channels C..Cpad-1 zero (bf16 only).
+cudaError_t launch_pad_channels(const void *x, void *y, int N, int H, int W, int C, int Cpad, int lo, int hi,
+                                cudaStream_t s);
+// w[rows][C] -> wp[rows][Cpad] zero-padded (bf16 only); rows = cout*kh*kw.
+cudaError_t launch_pad_weights(const void *w, void *wp, long long rows, int C, int Cpad, cudaStream_t s);
+
+// ---- tcgen05 tensor-core convolution ---------------------------------------------------------
+struct ConvTcGeom {
+    int TW, TR, TN;         // output tile = TN images x TR rows x TW columns, TW*TR*TN == 128 (powers of two)
+    int BN;                 // output channels per CTA (multiple of 16, <= 256)
+    int BK;                 // input channels per pipeline stage: 64, 32 or 16
+    int stages;
+};
+struct ConvTcMaps {
+    CUtensorMap a[4];       // activation maps, one per (row parity, column parity) of a strided window
+    CUtensorMap w;          // weights as a [Cout][kh*kw*Cin] matrix
+    int a_valid[4];
+};
+// Chooses the tile geometry for a layer and a number of rows.
+ConvTcGeom conv_tc_geometry(const ConvArgs &a, int rows);
+// Encodes the tensor maps for a layer (x, w pointers and geometry are baked in).  Host only.
+int conv_tc_encode(const ConvArgs &a, const ConvTcGeom &g, ConvTcMaps *maps);
+cudaError_t launch_conv_tc(const ConvArgs &a, const ConvTcGeom &g, const ConvTcMaps &maps, unsigned *status,
+                           cudaStream_t s);
+
+}  // namespace lop

@@ -1,0 +1,202 @@
+"""Parity of the CUDA library (through the C ABI) against the CPU oracle.  Needs a B200."""
+import numpy as np
+import pytest
+import torch
+
+import lop_inputs as li
+import paper_2507_05829_b200 as lop
+from lop_inputs.workloads import Layer, Segment, Workload, conv, pool
+from oracle import chain as ochain
+from paper_2507_05829_b200.chain import DeviceChain, to_host_f32
+
+pytestmark = pytest.mark.gpu
+
+TOL = {"f32": 1e-4, "bf16": 2e-2}       # max |gpu - oracle| / max |oracle|
+
+
+def rel_err(got, want):
+    scale = float(np.max(np.abs(want)))
+    return float(np.max(np.abs(got.astype(np.float64) - want.astype(np.float64)))) / (scale if scale > 0 else 1.0)
+
+
+def check_workload(wl, flags=0, modes=("whole", "banded", "pipelined"), n_bands=None, tol=None):
+    """Run every segment on the GPU in each mode and compare the segment outputs with the oracle."""
+    want = ochain.run_workload(wl, keep_segments=True)
+    tol = TOL[wl.dtype] if tol is None else tol
+    results = {}
+    for mode in modes:
+        dc = DeviceChain(wl, flags=flags, n_bands=n_bands)
+        if mode == "pipelined":
+            dc.run_pipelined(dc.pinned_input())
+        elif mode == "banded":
+            dc.run_banded(dc.input_tensor())
+        else:
+            dc.run_whole(dc.input_tensor())
+        torch.cuda.synchronize()
+        dc.check_device()
+        outs = [to_host_f32(o) for o in dc.outs]
+        for s, (g, w) in enumerate(zip(outs, want)):
+            assert g.shape == w.shape
+            assert np.all(np.isfinite(g)), (wl.name, mode, s)
+            e = rel_err(g, w)
+            assert e <= tol, (wl.name, mode, "segment", s, "rel err", e)
+        results[mode] = outs
+    base = results[modes[0]]
+    for mode in modes[1:]:                   # band-wise execution reproduces whole-tensor execution bit for bit
+        for a, b in zip(base, results[mode]):
+            assert np.array_equal(a, b), (wl.name, mode, "differs from", modes[0])
+    return results
+
+
+def one_layer(l, N, H, W, dtype="bf16", n_bands=3, seed=9, affine=True):
+    wl = Workload("one_layer", dtype, N, H, W, l.cin, [Segment([l], n_bands)], seed=seed, affine=affine)
+    l.input_from = -1
+    li.fill_parameters(wl)
+    li.make_input(wl)
+    return wl
+
+
+# ------------------------------------------------------------------------------------ fp32 path
+def test_single_conv_fp32_four_bands():
+    wl = li.build("single_conv")
+    check_workload(wl)
+
+
+@pytest.mark.parametrize("k,s,p,d,cin,cout,H,W", [
+    (3, 1, 1, 1, 5, 7, 11, 13), (5, 2, 2, 1, 3, 8, 17, 9), (3, 1, 2, 2, 4, 4, 12, 12), (1, 2, 0, 1, 9, 3, 10, 7),
+    (7, 3, 3, 1, 2, 5, 23, 23), (2, 2, 0, 1, 6, 70, 8, 8),
+])
+def test_fp32_conv_general_shapes(k, s, p, d, cin, cout, H, W):
+    wl = one_layer(conv(cin, cout, k, s=s, p=p, d=d, act=li.ACT_SILU), 2, H, W, dtype="f32")
+    check_workload(wl, modes=("whole", "banded"))
+
+
+def test_fp32_vgg_block_small():
+    check_workload(li.build("vgg_block", H=30, W=22, dtype="f32", width=16, n_bands=4))
+
+
+# ------------------------------------------------------------------------------------ bf16 tensor-core conv, per shape
+TC_CASES = [  # k, s, p, d, cin, cout, N, H, W
+    (3, 1, 1, 1, 64, 64, 1, 20, 32),
+    (3, 1, 1, 1, 64, 64, 2, 9, 56),        # ragged W against the tile width
+    (3, 1, 1, 1, 128, 256, 1, 14, 14),
+    (3, 2, 1, 1, 64, 128, 2, 28, 28),      # stride 2, even extent
+    (3, 2, 1, 1, 32, 64, 1, 31, 45),       # stride 2, odd extents, 32-channel slabs
+    (1, 1, 0, 1, 256, 64, 3, 7, 7),        # pointwise, tiny image, batch folded into the tile
+    (1, 2, 0, 1, 64, 256, 2, 15, 15),      # strided pointwise projection
+    (7, 2, 3, 1, 3, 64, 2, 38, 38),        # stem: 3 input channels, padded to 16
+    (3, 1, 1, 1, 3, 32, 1, 24, 40),
+    (3, 1, 2, 2, 64, 32, 1, 16, 16),       # dilation 2
+    (3, 1, 1, 1, 16, 16, 1, 10, 10),       # 16-channel slabs
+    (5, 1, 2, 1, 64, 48, 1, 12, 12),       # 48 output channels
+    (3, 1, 1, 1, 512, 512, 1, 7, 7),
+    (3, 1, 1, 1, 64, 64, 1, 5, 300),       # wider than two 128-pixel tiles
+]
+
+
+@pytest.mark.parametrize("case", TC_CASES)
+def test_bf16_tensor_core_conv_shapes(case):
+    k, s, p, d, cin, cout, N, H, W = case
+    wl = one_layer(conv(cin, cout, k, s=s, p=p, d=d, act=li.ACT_RELU), N, H, W)
+    dc = DeviceChain(wl)
+    assert dc.plans[0].layer_kernel(0) == 2
+    check_workload(wl, modes=("whole", "banded"))
+    check_workload(wl, modes=("whole",), flags=lop.LOP_FLAG_FORCE_SIMT)
+
+
+@pytest.mark.parametrize("pos,act", [(li.RES_PRE_ACT, li.ACT_RELU), (li.RES_POST_ACT, li.ACT_SILU)])
+def test_bf16_residual_and_activation_epilogues(pos, act):
+    layers = [conv(64, 64, 3, act=act), conv(64, 64, 3, act=act, residual_from=0, residual_pos=pos),
+              conv(64, 64, 1, p=0, act=li.ACT_NONE, residual_from=-1, residual_pos=pos)]
+    for i, l in enumerate(layers):
+        l.input_from = i - 1
+    wl = Workload("res", "bf16", 2, 18, 24, 64, [Segment(layers, 4)], seed=5)
+    li.fill_parameters(wl)
+    li.make_input(wl)
+    check_workload(wl)
+
+
+# ------------------------------------------------------------------------------------ pooling
+@pytest.mark.parametrize("dtype,C", [("bf16", 64), ("bf16", 6), ("f32", 8), ("f32", 3)])
+@pytest.mark.parametrize("k,s,p", [(2, 2, 0), (3, 2, 1)])
+def test_maxpool(dtype, C, k, s, p):
+    l = pool(C, k, s, p)
+    wl = one_layer(l, 2, 21, 18, dtype=dtype)
+    res = check_workload(wl, modes=("whole", "banded"), tol=0.0)   # pooling only selects: exact
+
+
+# ------------------------------------------------------------------------------------ chains, reduced sizes
+SMALL = [("vgg_block", dict(H=44, W=36)), ("resnet18", dict(H=64, W=64)),
+         ("resnet50", dict(N=2, H=64, W=64, depths=(2, 2, 2, 2))), ("csp_stack", dict(H=256, W=128))]
+
+
+@pytest.mark.parametrize("name,kw", SMALL)
+@pytest.mark.parametrize("flags", [0, lop.LOP_FLAG_REUSE_HALO])
+def test_chains_small(name, kw, flags):
+    check_workload(li.build(name, **kw), flags=flags)
+
+
+def test_tensor_core_and_cuda_core_paths_agree():
+    wl = li.build("resnet18", H=64, W=64)
+    a = check_workload(wl, modes=("whole",))["whole"]
+    b = check_workload(wl, modes=("whole",), flags=lop.LOP_FLAG_FORCE_SIMT)["whole"]
+    for x, y in zip(a, b):
+        assert rel_err(x, y) <= 2e-2
+
+
+# ------------------------------------------------------------------------------------ edge cases
+def test_more_bands_than_rows_and_single_band():
+    wl = li.build("vgg_block", H=12, W=20)
+    for nb in (1, 6, 7, 13):                                     # 6 output rows: empty bands from 7 on
+        check_workload(wl, n_bands=nb, modes=("whole", "banded", "pipelined"))
+
+
+def test_bands_in_any_order_without_reuse():
+    wl = li.build("vgg_block", H=44, W=36)
+    want = ochain.run_workload(wl)
+    dc = DeviceChain(wl)
+    dc.run_bands_one_by_one(dc.input_tensor(), order=lambda n: list(reversed(range(n))))
+    torch.cuda.synchronize()
+    assert rel_err(to_host_f32(dc.outs[-1]), want) <= TOL["bf16"]
+    ref = DeviceChain(wl)
+    ref.run_whole(ref.input_tensor())
+    torch.cuda.synchronize()
+    assert torch.equal(ref.outs[-1], dc.outs[-1])
+
+
+def test_run_band_writes_only_its_rows():
+    wl = li.build("vgg_block", H=44, W=36)
+    dc = DeviceChain(wl)
+    dc.outs[0].fill_(123.0)
+    plan = dc.plans[0]
+    plan.run_band(2, dc.input_tensor().data_ptr(), dc.outs[0].data_ptr(), dc.ws[0].data_ptr(),
+                  torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    r = plan.get_range(2, plan.num_layers() - 1)
+    out = to_host_f32(dc.outs[0])
+    want = ochain.run_workload(wl)
+    assert np.all(out[:, :r.out_lo] == 123.0) and np.all(out[:, r.out_hi:] == 123.0)
+    assert rel_err(out[:, r.out_lo:r.out_hi], want[:, r.out_lo:r.out_hi]) <= TOL["bf16"]
+
+
+def test_pipelined_timing_and_launch_count():
+    wl = li.build("vgg_block")
+    dc = DeviceChain(wl, flags=lop.LOP_FLAG_REUSE_HALO | lop.LOP_FLAG_TIME_LAYERS)
+    x = dc.pinned_input()
+    for _ in range(3):
+        dc.run_pipelined(x)
+    torch.cuda.synchronize()
+    t = dc.plans[0].last_timing()
+    assert t.n_copies == 8 and t.total_ms > 0 and 0 < t.first_copy_ms <= t.copy_ms
+    assert dc.plans[0].last_launches() == 8 * (1 + 1 + 3)        # copy + channel pad + three layers per band
+    assert dc.plans[0].layer_time(0, 1) > 0 and dc.plans[0].layer_time(3, 2) > 0
+
+
+# ------------------------------------------------------------------------------------ the named configurations, full size
+@pytest.mark.parametrize("name", ["vgg_block", "resnet18", "csp_stack"])
+def test_named_configurations_full_size(name):
+    check_workload(li.build(name), flags=lop.LOP_FLAG_REUSE_HALO, modes=("whole", "pipelined"))
+
+
+def test_resnet50_batch8_full_size():
+    check_workload(li.build("resnet50"), flags=lop.LOP_FLAG_REUSE_HALO, modes=("pipelined",))
