@@ -163,8 +163,9 @@ int lop_plan_layer_time(lop_plan_t *plan, int band, int layer, float *ms);
 /* Which kernel family serves a layer: 0 = pooling, 1 = CUDA-core convolution,
  * 2 = tcgen05 tensor-core convolution.  <0 on error. */
 int lop_plan_layer_kernel(const lop_plan_t *plan, int layer);
-/* Number of kernel launches and async copies the last execution call enqueued. */
+/* Number of kernels (this library's own) and of async copies the last execution call enqueued. */
 int lop_plan_last_launches(const lop_plan_t *plan);
+int lop_plan_last_copies(const lop_plan_t *plan);
 /* Reads the plan's device status word (0 = no kernel gave up on a bounded wait).  SYNCHRONISES
  * the stream of the last execution call. */
 int lop_plan_check_device(lop_plan_t *plan, void *workspace);

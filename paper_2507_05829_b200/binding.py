@@ -19,7 +19,7 @@ EXPORTS = [
     "lop_plan", "lop_plan_destroy", "lop_plan_num_bands", "lop_plan_num_layers", "lop_plan_get_range",
     "lop_plan_out_shape", "lop_plan_set_params", "lop_plan_workspace_bytes", "lop_plan_staging_bytes",
     "lop_plan_flops", "lop_run_whole", "lop_run_band", "lop_run_banded", "lop_copy_band", "lop_run_pipelined",
-    "lop_plan_last_timing", "lop_plan_layer_time", "lop_plan_layer_kernel", "lop_plan_last_launches",
+    "lop_plan_last_timing", "lop_plan_layer_time", "lop_plan_layer_kernel", "lop_plan_last_launches", "lop_plan_last_copies",
     "lop_plan_check_device", "lop_strerror", "lop_last_error",
 ]
 
@@ -87,6 +87,7 @@ def lib():
     L.lop_plan_layer_time.argtypes = [c_void_p, c_int, c_int, POINTER(c_float)]
     L.lop_plan_layer_kernel.argtypes = [c_void_p, c_int]
     L.lop_plan_last_launches.argtypes = [c_void_p]
+    L.lop_plan_last_copies.argtypes = [c_void_p]
     L.lop_plan_check_device.argtypes = [c_void_p, c_void_p]
     L.lop_strerror.argtypes = [c_int]
     L.lop_strerror.restype = c_char_p
@@ -192,6 +193,9 @@ class Plan:
 
     def last_launches(self):
         return _check(lib().lop_plan_last_launches(self._h))
+
+    def last_copies(self):
+        return _check(lib().lop_plan_last_copies(self._h))
 
     def check_device(self, ws):
         _check(lib().lop_plan_check_device(self._h, ws))

@@ -37,7 +37,8 @@ struct ExecState {
     const void *prepared_ws = nullptr;
     std::vector<const void *> prepared_w;                      // weight pointers the padded copies were made from
     cudaStream_t last_stream = nullptr;
-    int launches = 0;
+    int launches = 0;                                          // kernels enqueued by the last execution call
+    int copies = 0;                                            // async copies enqueued by it
     bool timing_valid = false;
     std::vector<char> copy_issued;
 };
@@ -117,7 +118,6 @@ int prepare_workspace(lop_plan_t *pl, void *ws, cudaStream_t s)
     bool fresh = e->prepared_ws != ws;
     if (fresh) {
         LOP_CUDA(cudaMemsetAsync(base + pl->status_off, 0, 1024, s));
-        e->launches++;
     }
     for (size_t i = 0; i < pl->layers.size(); ++i) {
         LayerInfo &li = pl->layers[i];
@@ -233,7 +233,7 @@ int copy_band_impl(lop_plan_t *pl, int band, const void *host, void *staging, cu
     const size_t img = row * pl->H;
     LOP_CUDA(cudaMemcpy2DAsync(static_cast<char *>(staging) + lo * row, img, static_cast<const char *>(host) + lo * row, img,
                                (size_t)(hi - lo) * row, pl->N, cudaMemcpyHostToDevice, s));
-    pl->exec->launches++;
+    pl->exec->copies++;
     return LOP_OK;
 }
 
@@ -249,7 +249,7 @@ int lop_run_whole(lop_plan_t *pl, const void *in, void *out, void *ws, void *str
     int rc = check_common(pl, in, out, ws);
     if (rc != LOP_OK) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    pl->exec->launches = 0;
+    pl->exec->launches = pl->exec->copies = 0;
     pl->exec->last_stream = s;
     reset_layer_timing(pl);
     if ((rc = prepare_workspace(pl, ws, s)) != LOP_OK) return rc;
@@ -265,7 +265,7 @@ int lop_run_band(lop_plan_t *pl, int band, const void *in, void *out, void *ws, 
     if (rc != LOP_OK) return rc;
     if (band < 0 || band >= pl->n_bands) { set_error("band %d out of range", band); return LOP_EINVAL; }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    pl->exec->launches = 0;
+    pl->exec->launches = pl->exec->copies = 0;
     pl->exec->last_stream = s;
     if ((rc = prepare_workspace(pl, ws, s)) != LOP_OK) return rc;
     return run_band_impl(pl, band, in, out, ws, s);
@@ -276,7 +276,7 @@ int lop_run_banded(lop_plan_t *pl, const void *in, void *out, void *ws, void *st
     int rc = check_common(pl, in, out, ws);
     if (rc != LOP_OK) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    pl->exec->launches = 0;
+    pl->exec->launches = pl->exec->copies = 0;
     pl->exec->last_stream = s;
     reset_layer_timing(pl);
     if ((rc = prepare_workspace(pl, ws, s)) != LOP_OK) return rc;
@@ -291,7 +291,7 @@ int lop_copy_band(lop_plan_t *pl, int band, const void *host, void *staging, voi
     if (band < 0 || band >= pl->n_bands) { set_error("band %d out of range", band); return LOP_EINVAL; }
     int rc = ensure_exec(pl);
     if (rc != LOP_OK) return rc;
-    pl->exec->launches = 0;
+    pl->exec->launches = pl->exec->copies = 0;
     return copy_band_impl(pl, band, host, staging, static_cast<cudaStream_t>(stream));
 }
 
@@ -302,7 +302,7 @@ int lop_run_pipelined(lop_plan_t *pl, const void *host, void *staging, void *out
     if (!host) { set_error("lop_run_pipelined: host input is NULL"); return LOP_EINVAL; }
     ExecState *e = pl->exec;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    e->launches = 0;
+    e->launches = e->copies = 0;
     e->last_stream = s;
     e->timing_valid = false;
     reset_layer_timing(pl);
@@ -374,6 +374,12 @@ int lop_plan_last_launches(const lop_plan_t *pl)
 {
     if (!pl) { set_error("plan is NULL"); return LOP_EINVAL; }
     return pl->exec ? pl->exec->launches : 0;
+}
+
+int lop_plan_last_copies(const lop_plan_t *pl)
+{
+    if (!pl) { set_error("plan is NULL"); return LOP_EINVAL; }
+    return pl->exec ? pl->exec->copies : 0;
 }
 
 int lop_plan_check_device(lop_plan_t *pl, void *ws)

@@ -188,7 +188,8 @@ def test_pipelined_timing_and_launch_count():
     torch.cuda.synchronize()
     t = dc.plans[0].last_timing()
     assert t.n_copies == 8 and t.total_ms > 0 and 0 < t.first_copy_ms <= t.copy_ms
-    assert dc.plans[0].last_launches() == 8 * (1 + 1 + 3)        # copy + channel pad + three layers per band
+    assert dc.plans[0].last_launches() == 8 * (1 + 3)            # channel pad + three layers per band
+    assert dc.plans[0].last_copies() == 8                        # one 2-D copy per band
     assert dc.plans[0].layer_time(0, 1) > 0 and dc.plans[0].layer_time(3, 2) > 0
 
 
