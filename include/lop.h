@@ -14,7 +14,8 @@
  *     A human-readable message for the calling thread's last failure: lop_last_error().
  *   - "host" / "device" / "pinned host" say where a pointer must live.  The caller owns every
  *     buffer and the stream; the library owns the opaque plan and what hangs off it (one side
- *     stream, events, tensor maps), all released by lop_plan_destroy().
+ *     stream, events, tensor maps and small device-side program tables it allocates on the first
+ *     execution call for a given set of buffers), all released by lop_plan_destroy().
  *   - Activations are NHWC, contiguous; weights are [cout][kh][kw][cin] (KRSC), contiguous,
  *     in the plan's storage dtype; scale/shift are float32 [cout].  Accumulation is float32.
  *   - Row ranges are half-open [lo, hi); the empty range is {0, 0}.
@@ -54,7 +55,9 @@ enum {
                                      dependency); otherwise every band recomputes its halo and is
                                      independent of the others (operation replication, Sec. IV-C) */
     LOP_FLAG_TIME_LAYERS = 2u,    /* record a CUDA event pair around every (band, layer) launch    */
-    LOP_FLAG_FORCE_SIMT = 4u      /* never use the tensor-core convolution (second on-GPU opinion) */
+    LOP_FLAG_FORCE_SIMT = 4u,     /* never use the tensor-core convolution (second on-GPU opinion) */
+    LOP_FLAG_PER_LAYER = 8u       /* one kernel launch per (band, layer) instead of one persistent
+                                     wavefront launch per call / per band                          */
 };
 
 /*
@@ -132,8 +135,9 @@ double lop_plan_flops(const lop_plan_t *plan);
 /* ---- execution: every pointer below is a DEVICE pointer unless it says otherwise ----------
  * in_dev and out_dev are FULL-SIZE tensors (chain input N*H*W*C, last layer's output); bands
  * address row ranges inside them.  stream is a cudaStream_t passed as void* (NULL = legacy
- * default stream).  The first execution call on a plan creates its side stream and events:
- * make it outside any stream capture. */
+ * default stream).  The first execution call on a plan for a given (input, output, workspace)
+ * triple creates the side stream, events and program tables (cudaMalloc + synchronous uploads):
+ * make it outside any stream capture; later calls with the same buffers allocate nothing. */
 
 /* Whole-tensor execution: every layer over all its rows (the unpartitioned reference order). */
 int lop_run_whole(lop_plan_t *plan, const void *in_dev, void *out_dev, void *workspace, void *stream);
@@ -156,7 +160,7 @@ int lop_run_pipelined(lop_plan_t *plan, const void *in_host_pinned, void *stagin
                       void *workspace, void *stream);
 /* Event times of the last lop_run_pipelined call.  SYNCHRONISES with that call's completion. */
 int lop_plan_last_timing(lop_plan_t *plan, lop_timing *out);
-/* With LOP_FLAG_TIME_LAYERS: device time in ms of the (band, layer) launch of the last
+/* With LOP_FLAG_TIME_LAYERS (implies per-layer launches): device time in ms of the (band, layer) launch of the last
  * lop_run_band / banded / pipelined call (band = -1: last lop_run_whole).  SYNCHRONISES.
  * *ms = 0 when that band had nothing to do at that layer. */
 int lop_plan_layer_time(lop_plan_t *plan, int band, int layer, float *ms);

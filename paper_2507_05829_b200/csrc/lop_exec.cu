@@ -15,6 +15,7 @@
 
 #include "lop_internal.h"
 #include "lop_kernels.cuh"
+#include "lop_program.h"
 
 namespace lop {
 
@@ -27,7 +28,15 @@ struct MapKey {
     }
 };
 
+struct ProgKey {
+    int kind;                        // -1 whole, -2 all bands, >= 0 one band
+    const void *in, *out, *ws;
+    bool operator<(const ProgKey &o) const { return std::tie(kind, in, out, ws) < std::tie(o.kind, o.in, o.out, o.ws); }
+};
+
 struct ExecState {
+    std::map<ProgKey, Program *> programs;
+    bool wavefront = false;
     cudaStream_t copy_stream = nullptr;
     cudaEvent_t ev_fork = nullptr, ev_begin = nullptr, ev_end = nullptr;
     std::vector<cudaEvent_t> ev_copy_start, ev_copy_end;       // [band]
@@ -52,6 +61,7 @@ void exec_destroy(ExecState *e)
     for (auto &v : {&e->ev_copy_start, &e->ev_copy_end, &e->ev_layer})
         for (cudaEvent_t ev : *v)
             if (ev) cudaEventDestroy(ev);
+    for (auto &kv : e->programs) program_destroy(kv.second);
     delete e;
 }
 
@@ -90,6 +100,7 @@ int ensure_exec(lop_plan_t *pl)
         for (auto &ev : e->ev_layer) LOP_CUDA(cudaEventCreate(&ev));
     }
     e->prepared_w.assign(L, nullptr);
+    e->wavefront = program_supported(pl) && !(pl->flags & (LOP_FLAG_PER_LAYER | LOP_FLAG_TIME_LAYERS));
     return LOP_OK;
 }
 
@@ -219,6 +230,46 @@ int run_band_impl(lop_plan_t *pl, int band, const void *in, void *out, void *ws,
     return LOP_OK;
 }
 
+// Requests of one band in dependency order: channel padding first, then every layer.
+void band_requests(const lop_plan_t *pl, int band, std::vector<StageReq> &reqs)
+{
+    const int L = (int)pl->layers.size();
+    const bool reuse = (pl->flags & LOP_FLAG_REUSE_HALO) != 0;
+    const lop_range &need = pl->in_need[band];
+    if (pl->Cpad) reqs.push_back(StageReq{band, -1, reuse ? need.new_lo : need.out_lo, need.out_hi});
+    for (int i = 0; i < L; ++i) {
+        const lop_range &r = pl->ranges[(size_t)band * L + i];
+        reqs.push_back(StageReq{band, i, reuse ? r.new_lo : r.out_lo, r.out_hi});
+    }
+}
+
+// kind: -1 whole tensor, -2 every band in ascending order, b >= 0 band b.  One persistent launch.
+int run_program(lop_plan_t *pl, int kind, const void *in, void *out, void *ws, cudaStream_t s)
+{
+    ExecState *e = pl->exec;
+    const ProgKey key{kind, in, out, ws};
+    auto it = e->programs.find(key);
+    if (it == e->programs.end()) {
+        std::vector<StageReq> reqs;
+        if (kind == -1) {
+            if (pl->Cpad) reqs.push_back(StageReq{0, -1, 0, pl->H});
+            for (int i = 0; i < (int)pl->layers.size(); ++i) reqs.push_back(StageReq{0, i, 0, pl->layers[i].Ho});
+        } else if (kind == -2) {
+            for (int b = 0; b < pl->n_bands; ++b) band_requests(pl, b, reqs);
+        } else {
+            band_requests(pl, kind, reqs);
+        }
+        Program *p = nullptr;
+        int rc = program_build(pl, reqs, in, out, ws, &p);
+        if (rc != LOP_OK) return rc;
+        it = e->programs.emplace(key, p).first;
+    }
+    if (program_empty(it->second)) return LOP_OK;
+    int rc = program_launch(it->second, s);
+    if (rc == LOP_OK) e->launches++;
+    return rc;
+}
+
 void reset_layer_timing(lop_plan_t *pl)
 {
     for (auto &c : pl->exec->layer_timed) c = 0;
@@ -253,6 +304,7 @@ int lop_run_whole(lop_plan_t *pl, const void *in, void *out, void *ws, void *str
     pl->exec->last_stream = s;
     reset_layer_timing(pl);
     if ((rc = prepare_workspace(pl, ws, s)) != LOP_OK) return rc;
+    if (pl->exec->wavefront) return run_program(pl, -1, in, out, ws, s);
     if ((rc = pad_input_rows(pl, 0, pl->H, in, ws, s)) != LOP_OK) return rc;
     for (int i = 0; i < (int)pl->layers.size(); ++i)
         if ((rc = run_layer(pl, i, 0, pl->layers[i].Ho, in, out, ws, s, i)) != LOP_OK) return rc;
@@ -268,6 +320,7 @@ int lop_run_band(lop_plan_t *pl, int band, const void *in, void *out, void *ws, 
     pl->exec->launches = pl->exec->copies = 0;
     pl->exec->last_stream = s;
     if ((rc = prepare_workspace(pl, ws, s)) != LOP_OK) return rc;
+    if (pl->exec->wavefront) return run_program(pl, band, in, out, ws, s);
     return run_band_impl(pl, band, in, out, ws, s);
 }
 
@@ -280,6 +333,7 @@ int lop_run_banded(lop_plan_t *pl, const void *in, void *out, void *ws, void *st
     pl->exec->last_stream = s;
     reset_layer_timing(pl);
     if ((rc = prepare_workspace(pl, ws, s)) != LOP_OK) return rc;
+    if (pl->exec->wavefront) return run_program(pl, -2, in, out, ws, s);
     for (int b = 0; b < pl->n_bands; ++b)
         if ((rc = run_band_impl(pl, b, in, out, ws, s)) != LOP_OK) return rc;
     return LOP_OK;
@@ -326,7 +380,8 @@ int lop_run_pipelined(lop_plan_t *pl, const void *host, void *staging, void *out
             LOP_CUDA(cudaStreamWaitEvent(s, e->ev_copy_end[b], 0));
             joined = true;
         }
-        if ((rc = run_band_impl(pl, b, staging, out, ws, s)) != LOP_OK) return rc;
+        rc = e->wavefront ? run_program(pl, b, staging, out, ws, s) : run_band_impl(pl, b, staging, out, ws, s);
+        if (rc != LOP_OK) return rc;
     }
     if (!joined) LOP_CUDA(cudaStreamWaitEvent(s, e->ev_fork, 0));
     LOP_CUDA(cudaEventRecord(e->ev_end, s));

@@ -47,8 +47,9 @@ struct ConvTcMaps {
     CUtensorMap w;          // weights as a [Cout][kh*kw*Cin] matrix
     int a_valid[4];
 };
-// Chooses the tile geometry for a layer and a number of rows.
-ConvTcGeom conv_tc_geometry(const ConvArgs &a, int rows);
+// Chooses the tile geometry for a layer and a number of rows.  fill_sms: a stand-alone launch prefers
+// narrower channel tiles when there are too few pixel tiles to occupy every SM.
+ConvTcGeom conv_tc_geometry(const ConvArgs &a, int rows, bool fill_sms = true);
 // Encodes the tensor maps for a layer (x, w pointers and geometry are baked in).  Host only.
 int conv_tc_encode(const ConvArgs &a, const ConvTcGeom &g, ConvTcMaps *maps);
 cudaError_t launch_conv_tc(const ConvArgs &a, const ConvTcGeom &g, const ConvTcMaps &maps, unsigned *status,

@@ -100,7 +100,8 @@ def test_bf16_tensor_core_conv_shapes(case):
     wl = one_layer(conv(cin, cout, k, s=s, p=p, d=d, act=li.ACT_RELU), N, H, W)
     dc = DeviceChain(wl)
     assert dc.plans[0].layer_kernel(0) == 2
-    check_workload(wl, modes=("whole", "banded"))
+    check_workload(wl, modes=("whole", "banded"))                                   # persistent wavefront launch
+    check_workload(wl, modes=("whole", "banded"), flags=lop.LOP_FLAG_PER_LAYER)     # one launch per (band, layer)
     check_workload(wl, modes=("whole",), flags=lop.LOP_FLAG_FORCE_SIMT)
 
 
@@ -114,6 +115,7 @@ def test_bf16_residual_and_activation_epilogues(pos, act):
     li.fill_parameters(wl)
     li.make_input(wl)
     check_workload(wl)
+    check_workload(wl, flags=lop.LOP_FLAG_PER_LAYER | lop.LOP_FLAG_REUSE_HALO)
 
 
 # ------------------------------------------------------------------------------------ pooling
@@ -131,7 +133,8 @@ SMALL = [("vgg_block", dict(H=44, W=36)), ("resnet18", dict(H=64, W=64)),
 
 
 @pytest.mark.parametrize("name,kw", SMALL)
-@pytest.mark.parametrize("flags", [0, lop.LOP_FLAG_REUSE_HALO])
+@pytest.mark.parametrize("flags", [0, lop.LOP_FLAG_REUSE_HALO, lop.LOP_FLAG_PER_LAYER,
+                                   lop.LOP_FLAG_PER_LAYER | lop.LOP_FLAG_REUSE_HALO])
 def test_chains_small(name, kw, flags):
     check_workload(li.build(name, **kw), flags=flags)
 
@@ -191,6 +194,40 @@ def test_pipelined_timing_and_launch_count():
     assert dc.plans[0].last_launches() == 8 * (1 + 3)            # channel pad + three layers per band
     assert dc.plans[0].last_copies() == 8                        # one 2-D copy per band
     assert dc.plans[0].layer_time(0, 1) > 0 and dc.plans[0].layer_time(3, 2) > 0
+
+
+def test_wavefront_launch_counts_and_repeatability():
+    wl = li.build("vgg_block")
+    dc = DeviceChain(wl, flags=lop.LOP_FLAG_REUSE_HALO)
+    x, xd = dc.pinned_input(), dc.input_tensor()
+    first = None
+    for i in range(5):                                           # run counters advance from launch to launch
+        dc.run_pipelined(x)
+        torch.cuda.synchronize()
+        if i == 0:
+            assert dc.plans[0].last_launches() == 8 + 1          # one launch per band (+ weight padding once)
+        else:
+            assert dc.plans[0].last_launches() == 8 and dc.plans[0].last_copies() == 8
+        out = dc.outs[-1].clone()
+        first = out if first is None else first
+        assert torch.equal(out, first)
+        dc.outs[-1].zero_()
+    dc.run_banded(xd)
+    torch.cuda.synchronize()
+    assert dc.plans[0].last_launches() == 1 and torch.equal(dc.outs[-1], first)
+    dc.check_device()
+
+
+def test_wavefront_and_per_layer_executors_agree_bit_for_bit():
+    for name, kw in (("resnet18", dict(H=96, W=96)), ("csp_stack", dict(H=256, W=256))):
+        wl = li.build(name, **kw)
+        a = DeviceChain(wl, flags=lop.LOP_FLAG_REUSE_HALO)
+        b = DeviceChain(wl, flags=lop.LOP_FLAG_REUSE_HALO | lop.LOP_FLAG_PER_LAYER)
+        a.run_banded(a.input_tensor())
+        b.run_banded(b.input_tensor())
+        torch.cuda.synchronize()
+        for x, y in zip(a.outs, b.outs):
+            assert torch.equal(x, y)
 
 
 # ------------------------------------------------------------------------------------ the named configurations, full size
