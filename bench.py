@@ -28,6 +28,10 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one wavefront_kernel launch (ncu, see profiles/); None until captured
+# for the kernel as it stands
+TRAFFIC = {}
+
 METRIC = "band-pipelined conv-chain images/s"
 UNIT = "images/s"
 DEFAULT_WORKLOAD = "vgg_block"
@@ -266,48 +270,51 @@ def main():
     hidden = 100.0 * (1.0 - exposed / t_copy) if t_copy > 0 else None
     bound = 100.0 * min(1.0 - tm.first_copy_ms / tm.copy_ms if tm.copy_ms > 0 else 0.0, t_comp / t_copy if t_copy > 0 else 1.0)
 
-    # ---- dominant kernel: per-launch CUDA events inside an eager pass of the same workload
-    dct = DeviceChain(wl, flags=flags | lop.LOP_FLAG_TIME_LAYERS, device=dev)
-    conv_layers = []
-    for s, (seg, plan) in enumerate(zip(wl.segments, dct.plans)):
-        H, W, C = (wl.H, wl.W, wl.C) if s == 0 else dct.plans[s - 1].out_shape(dct.plans[s - 1].num_layers() - 1)
-        for i, l in enumerate(seg.layers):
-            if l.op == 0:
-                ho, wo, co = plan.out_shape(i)
-                conv_layers.append((s, i, 2.0 * wl.N * ho * wo * co * l.kh * l.kw * l.cin))
-    per_layer = {}
-    reps = 30
+    # ---- dominant kernel: the persistent wavefront kernel; in the `value` arm one step is exactly one launch of
+    # it, so the per-step CUDA events of the timed region are its launch durations
+    conv_fl = dc.flops()
+    achieved = conv_fl / (ms_res * 1e-3) / 1e12
+    roofline = {"bound": "tensor", "kernel": "wavefront_kernel (all-bands program: every conv / pool / pad stage of the step in one persistent launch)",
+                "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                "frac": achieved / peaks["bf16_tflops"],
+                "peak_source": "%s TFLOP/s burst bf16 (of %s)" % (peaks["bf16_tflops"], peaks["source"]),
+                "flops_per_launch": conv_fl, "avg_launch_us": ms_res * 1e3, "launches_per_step": launches_res,
+                "traffic": TRAFFIC.get(args.workload)}
+
+    # ---- per-layer view: whole-tensor launches, one kernel per layer, CUDA events around each (eager)
+    dct = DeviceChain(wl, flags=lop.LOP_FLAG_PER_LAYER | lop.LOP_FLAG_TIME_LAYERS, device=dev)
+    acc = {}
+    reps = 20
     for r in range(reps + 3):
         with torch.cuda.stream(stream):
             flush.zero_()
-            dct.run_banded(x_dev, stream)
+            dct.run_whole(x_dev, stream)
         stream.synchronize()
         if r < 3:
             continue
-        for (s, i, fl) in conv_layers:
-            plan = dct.plans[s]
-            tot, n = 0.0, 0
-            for b in range(plan.num_bands()):
-                ms = plan.layer_time(b, i)
-                if ms > 0:
-                    tot += ms
-                    n += 1
-            d = per_layer.setdefault((s, i), [0.0, 0, fl])
-            d[0] += tot
-            d[1] += n
-    dom = max(per_layer.items(), key=lambda kv: kv[1][2])           # the layer with the most FLOPs
-    (ds, di), (tot_ms, n_launch, fl) = dom
-    launches_per_pass = n_launch / reps
-    avg_ms = tot_ms / n_launch
-    flops_per_launch = fl / launches_per_pass
-    achieved = flops_per_launch / (avg_ms * 1e-3) / 1e12
-    conv_ms = sum(v[0] for v in per_layer.values()) / reps
-    conv_fl = sum(v[2] for v in per_layer.values())
-    roofline = {"bound": "tensor", "kernel": "conv_tc_kernel (segment %d layer %d)" % (ds, di),
-                "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                "frac": achieved / peaks["bf16_tflops"], "peak_source": "%s burst bf16 (of %s)" % (peaks["bf16_tflops"], peaks["source"]),
-                "flops_per_launch": flops_per_launch, "avg_launch_us": avg_ms * 1e3,
-                "launches_per_step": launches_per_pass, "traffic": None}
+        for s_, (seg, plan) in enumerate(zip(wl.segments, dct.plans)):
+            for i in range(len(seg.layers)):
+                acc[(s_, i)] = acc.get((s_, i), 0.0) + plan.layer_time(-1, i)
+    per_layer = []
+    es = 2 if wl.dtype == "bf16" else 4
+    for s_, (seg, plan) in enumerate(zip(wl.segments, dct.plans)):
+        for i, l in enumerate(seg.layers):
+            ms = acc[(s_, i)] / reps
+            ho, wo, co = plan.out_shape(i)
+            hi, wi, ci = plan.out_shape(l.input_from)
+            if l.op == 0:
+                fl = 2.0 * wl.N * ho * wo * co * l.kh * l.kw * l.cin
+                per_layer.append({"segment": s_, "layer": i, "op": "conv%dx%d s%d %d->%d" % (l.kh, l.kw, l.sh, l.cin, l.cout),
+                                  "kernel": ["pool", "cuda-core", "tcgen05"][plan.layer_kernel(i)], "us": ms * 1e3,
+                                  "tflops": fl / (ms * 1e-3) / 1e12,
+                                  "pct_of_burst_peak": 100.0 * fl / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"]})
+            else:
+                by = wl.N * (hi * wi * ci + ho * wo * co) * es
+                per_layer.append({"segment": s_, "layer": i, "op": "maxpool%dx%d s%d" % (l.kh, l.kw, l.sh), "kernel": "pool",
+                                  "us": ms * 1e3, "gbs": by / (ms * 1e-3) / 1e9,
+                                  "pct_of_hbm_peak": 100.0 * by / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]})
+    if len(per_layer) > 16:                                   # keep the line readable: the slowest layers only
+        per_layer = sorted(per_layer, key=lambda d: -d["us"])[:16]
 
     if rank != 0:
         if world > 1:
@@ -328,10 +335,9 @@ def main():
         "gpu_launches": int(launches_res * args.steps),
         "clocks": clocks,
         "roofline": roofline,
-        "conv_tflops": {"useful": conv_fl / (conv_ms * 1e-3) / 1e12, "sum_conv_kernel_ms": conv_ms,
-                        "pct_of_burst_peak": 100.0 * conv_fl / (conv_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
-                        "pct_of_sustained_peak": 100.0 * conv_fl / (conv_ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
-                        "whole_step_useful": dc.flops() / (ms_res * 1e-3) / 1e12},
+        "conv_tflops": {"whole_step_useful": achieved, "pct_of_burst_peak": 100.0 * achieved / peaks["bf16_tflops"],
+                        "pct_of_sustained_peak": 100.0 * achieved / peaks["bf16_tflops_sustained"],
+                        "per_layer_launches": per_layer},
         "pipeline": {"t_copy_ms": t_copy, "t_compute_ms": t_comp, "t_pipelined_ms": t_pipe, "exposed_ms": exposed,
                      "hidden_pct": hidden, "hidden_pct_bound": bound, "copy_events_ms": tm.copy_ms,
                      "first_copy_ms": tm.first_copy_ms, "launch": "eager"},

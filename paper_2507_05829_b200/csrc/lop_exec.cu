@@ -38,7 +38,8 @@ struct ExecState {
     std::map<ProgKey, Program *> programs;
     bool wavefront = false;
     cudaStream_t copy_stream = nullptr;
-    cudaEvent_t ev_fork = nullptr, ev_begin = nullptr, ev_end = nullptr;
+    cudaEvent_t ev_fork = nullptr, ev_begin = nullptr, ev_end = nullptr, ev_join = nullptr;
+    unsigned *pinned_one = nullptr;                            // pinned host word holding 1: source of arrival flags
     std::vector<cudaEvent_t> ev_copy_start, ev_copy_end;       // [band]
     std::vector<cudaEvent_t> ev_layer;                         // [(band+1) * L + layer] * 2, slot 0 = whole
     std::vector<char> layer_timed;
@@ -56,7 +57,8 @@ void exec_destroy(ExecState *e)
 {
     if (!e) return;
     if (e->copy_stream) cudaStreamDestroy(e->copy_stream);
-    for (cudaEvent_t ev : {e->ev_fork, e->ev_begin, e->ev_end})
+    if (e->pinned_one) cudaFreeHost(e->pinned_one);
+    for (cudaEvent_t ev : {e->ev_fork, e->ev_begin, e->ev_end, e->ev_join})
         if (ev) cudaEventDestroy(ev);
     for (auto &v : {&e->ev_copy_start, &e->ev_copy_end, &e->ev_layer})
         for (cudaEvent_t ev : *v)
@@ -85,6 +87,9 @@ int ensure_exec(lop_plan_t *pl)
     const int B = pl->n_bands, L = (int)pl->layers.size();
     LOP_CUDA(cudaStreamCreateWithFlags(&e->copy_stream, cudaStreamNonBlocking));
     LOP_CUDA(cudaEventCreateWithFlags(&e->ev_fork, cudaEventDisableTiming));
+    LOP_CUDA(cudaEventCreateWithFlags(&e->ev_join, cudaEventDisableTiming));
+    LOP_CUDA(cudaHostAlloc(reinterpret_cast<void **>(&e->pinned_one), 64, cudaHostAllocDefault));
+    *e->pinned_one = 1u;
     LOP_CUDA(cudaEventCreate(&e->ev_begin));
     LOP_CUDA(cudaEventCreate(&e->ev_end));
     e->ev_copy_start.assign(B, nullptr);
@@ -231,42 +236,63 @@ int run_band_impl(lop_plan_t *pl, int band, const void *in, void *out, void *ws,
 }
 
 // Requests of one band in dependency order: channel padding first, then every layer.
-void band_requests(const lop_plan_t *pl, int band, std::vector<StageReq> &reqs)
+void band_requests(const lop_plan_t *pl, int band, bool wait_arrival, std::vector<StageReq> &reqs)
 {
     const int L = (int)pl->layers.size();
     const bool reuse = (pl->flags & LOP_FLAG_REUSE_HALO) != 0;
     const lop_range &need = pl->in_need[band];
-    if (pl->Cpad) reqs.push_back(StageReq{band, -1, reuse ? need.new_lo : need.out_lo, need.out_hi});
+    if (pl->Cpad) reqs.push_back(StageReq{band, -1, reuse ? need.new_lo : need.out_lo, need.out_hi, wait_arrival});
     for (int i = 0; i < L; ++i) {
         const lop_range &r = pl->ranges[(size_t)band * L + i];
-        reqs.push_back(StageReq{band, i, reuse ? r.new_lo : r.out_lo, r.out_hi});
+        reqs.push_back(StageReq{band, i, reuse ? r.new_lo : r.out_lo, r.out_hi, wait_arrival});
     }
 }
 
-// kind: -1 whole tensor, -2 every band in ascending order, b >= 0 band b.  One persistent launch.
-int run_program(lop_plan_t *pl, int kind, const void *in, void *out, void *ws, cudaStream_t s)
+enum { PROG_WHOLE = -1, PROG_ALL_BANDS = -2, PROG_PIPELINED = -3 };
+
+// kind: PROG_WHOLE, PROG_ALL_BANDS, PROG_PIPELINED, or b >= 0 for band b alone.
+int get_program(lop_plan_t *pl, int kind, const void *in, void *out, void *ws, Program **prog)
 {
     ExecState *e = pl->exec;
     const ProgKey key{kind, in, out, ws};
     auto it = e->programs.find(key);
     if (it == e->programs.end()) {
+        const int L = (int)pl->layers.size(), B = pl->n_bands;
         std::vector<StageReq> reqs;
-        if (kind == -1) {
-            if (pl->Cpad) reqs.push_back(StageReq{0, -1, 0, pl->H});
-            for (int i = 0; i < (int)pl->layers.size(); ++i) reqs.push_back(StageReq{0, i, 0, pl->layers[i].Ho});
-        } else if (kind == -2) {
-            for (int b = 0; b < pl->n_bands; ++b) band_requests(pl, b, reqs);
+        if (kind == PROG_WHOLE) {
+            if (pl->Cpad) reqs.push_back(StageReq{0, -1, 0, pl->H, false});
+            for (int i = 0; i < L; ++i) reqs.push_back(StageReq{0, i, 0, pl->layers[i].Ho, false});
+        } else if (kind == PROG_ALL_BANDS) {
+            // Input resident: the bands' operations of one layer do not depend on each other, so they are
+            // batched layer by layer (operation batching, Sec. IV-C); dependencies stay per band row group.
+            std::vector<std::vector<StageReq>> per_band(B);
+            for (int b = 0; b < B; ++b) band_requests(pl, b, false, per_band[b]);
+            const size_t per = per_band.empty() ? 0 : per_band[0].size();
+            for (size_t j = 0; j < per; ++j)
+                for (int b = 0; b < B; ++b) reqs.push_back(per_band[b][j]);
+        } else if (kind == PROG_PIPELINED) {
+            // Bands arrive one after the other: band-major order, each band gated by its arrival flag.
+            for (int b = 0; b < B; ++b) band_requests(pl, b, true, reqs);
         } else {
-            band_requests(pl, kind, reqs);
+            band_requests(pl, kind, false, reqs);
         }
         Program *p = nullptr;
         int rc = program_build(pl, reqs, in, out, ws, &p);
         if (rc != LOP_OK) return rc;
         it = e->programs.emplace(key, p).first;
     }
-    if (program_empty(it->second)) return LOP_OK;
-    int rc = program_launch(it->second, s);
-    if (rc == LOP_OK) e->launches++;
+    *prog = it->second;
+    return LOP_OK;
+}
+
+int run_program(lop_plan_t *pl, int kind, const void *in, void *out, void *ws, cudaStream_t s)
+{
+    Program *p = nullptr;
+    int rc = get_program(pl, kind, in, out, ws, &p);
+    if (rc != LOP_OK) return rc;
+    if (program_empty(p)) return LOP_OK;
+    rc = program_launch(p, s);
+    if (rc == LOP_OK) pl->exec->launches++;
     return rc;
 }
 
@@ -304,7 +330,7 @@ int lop_run_whole(lop_plan_t *pl, const void *in, void *out, void *ws, void *str
     pl->exec->last_stream = s;
     reset_layer_timing(pl);
     if ((rc = prepare_workspace(pl, ws, s)) != LOP_OK) return rc;
-    if (pl->exec->wavefront) return run_program(pl, -1, in, out, ws, s);
+    if (pl->exec->wavefront) return run_program(pl, PROG_WHOLE, in, out, ws, s);
     if ((rc = pad_input_rows(pl, 0, pl->H, in, ws, s)) != LOP_OK) return rc;
     for (int i = 0; i < (int)pl->layers.size(); ++i)
         if ((rc = run_layer(pl, i, 0, pl->layers[i].Ho, in, out, ws, s, i)) != LOP_OK) return rc;
@@ -333,7 +359,7 @@ int lop_run_banded(lop_plan_t *pl, const void *in, void *out, void *ws, void *st
     pl->exec->last_stream = s;
     reset_layer_timing(pl);
     if ((rc = prepare_workspace(pl, ws, s)) != LOP_OK) return rc;
-    if (pl->exec->wavefront) return run_program(pl, -2, in, out, ws, s);
+    if (pl->exec->wavefront) return run_program(pl, PROG_ALL_BANDS, in, out, ws, s);
     for (int b = 0; b < pl->n_bands; ++b)
         if ((rc = run_band_impl(pl, b, in, out, ws, s)) != LOP_OK) return rc;
     return LOP_OK;
@@ -365,6 +391,32 @@ int lop_run_pipelined(lop_plan_t *pl, const void *host, void *staging, void *out
     LOP_CUDA(cudaEventRecord(e->ev_fork, s));
     LOP_CUDA(cudaStreamWaitEvent(e->copy_stream, e->ev_fork, 0));
     if ((rc = prepare_workspace(pl, ws, s)) != LOP_OK) return rc;
+    if (e->wavefront) {
+        // One persistent launch for the whole request: it starts at once and every band's first stage waits
+        // for that band's arrival flag, which the side stream sets right after the band's copy.
+        Program *p = nullptr;
+        if ((rc = get_program(pl, PROG_PIPELINED, staging, out, ws, &p)) != LOP_OK) return rc;
+        if (!program_empty(p)) {
+            if ((rc = program_launch(p, s)) != LOP_OK) return rc;
+            e->launches++;
+        }
+        for (int b = 0; b < pl->n_bands; ++b) {
+            const lop_range &need = pl->in_need[b];
+            e->copy_issued[b] = need.out_hi > need.new_lo;
+            if (e->copy_issued[b]) {
+                LOP_CUDA(cudaEventRecord(e->ev_copy_start[b], e->copy_stream));
+                if ((rc = copy_band_impl(pl, b, host, staging, e->copy_stream)) != LOP_OK) return rc;
+                LOP_CUDA(cudaEventRecord(e->ev_copy_end[b], e->copy_stream));
+            }
+            unsigned *flag = program_arrival_flag(p, b);
+            if (flag) LOP_CUDA(cudaMemcpyAsync(flag, e->pinned_one, sizeof(unsigned), cudaMemcpyHostToDevice, e->copy_stream));
+        }
+        LOP_CUDA(cudaEventRecord(e->ev_join, e->copy_stream));
+        LOP_CUDA(cudaStreamWaitEvent(s, e->ev_join, 0));
+        LOP_CUDA(cudaEventRecord(e->ev_end, s));
+        e->timing_valid = true;
+        return LOP_OK;
+    }
     // all transfers are queued up front on the side stream: band i+1 (and later) stream in while band i computes
     for (int b = 0; b < pl->n_bands; ++b) {
         const lop_range &need = pl->in_need[b];
@@ -380,8 +432,7 @@ int lop_run_pipelined(lop_plan_t *pl, const void *host, void *staging, void *out
             LOP_CUDA(cudaStreamWaitEvent(s, e->ev_copy_end[b], 0));
             joined = true;
         }
-        rc = e->wavefront ? run_program(pl, b, staging, out, ws, s) : run_band_impl(pl, b, staging, out, ws, s);
-        if (rc != LOP_OK) return rc;
+        if ((rc = run_band_impl(pl, b, staging, out, ws, s)) != LOP_OK) return rc;
     }
     if (!joined) LOP_CUDA(cudaStreamWaitEvent(s, e->ev_fork, 0));
     LOP_CUDA(cudaEventRecord(e->ev_end, s));

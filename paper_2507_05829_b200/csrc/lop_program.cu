@@ -20,6 +20,7 @@ struct Program {
     unsigned *counters = nullptr;
     WfParams params{};
     int grid = 0;
+    int flag_base = 0, n_flags = 0;
 };
 
 void program_destroy(Program *p)
@@ -102,6 +103,7 @@ int program_build(lop_plan_t *pl, const std::vector<StageReq> &reqs, const void 
     std::vector<std::vector<int>> by_layer(L + 1);      // stage indices per producing layer
     std::vector<int> expected;                         // completions per row group, per stage
     int n_items = 0, n_ctr = WF_CTR_FIRST;
+    bool uses_flags = false;
     uint32_t slot_bytes = 1024;
 
     for (const StageReq &rq : reqs) {
@@ -151,9 +153,13 @@ int program_build(lop_plan_t *pl, const std::vector<StageReq> &reqs, const void 
             st.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(g.BN >> 3) << 17) | ((128u >> 4) << 24);
             slot_bytes = std::max(slot_bytes, st.a_bytes + (st.b_bytes + 1023u) / 1024u * 1024u);
         } else {
+            // one output row of one image, cut into chunks of 128 pixels (padding) / 256 channel vectors (pooling)
             st.kind = rq.layer < 0 ? WF_PAD : WF_POOL;
             st.tw_log = 0; st.tr_log = 0;
-            st.tiles_w = 1; st.tiles_r = rows; st.tiles_n = pl->N; st.cout_tiles = 1;
+            const int per_row = rq.layer < 0 ? pl->W : pl->layers[rq.layer].Wo * (pl->layers[rq.layer].l.cin / 8);
+            const int per_item = rq.layer < 0 ? 128 : 256;
+            st.tiles_w = (per_row + per_item - 1) / per_item;
+            st.tiles_r = rows; st.tiles_n = pl->N; st.cout_tiles = 1;
         }
         st.n_items = st.tiles_w * st.tiles_r * st.tiles_n * st.cout_tiles;
         st.ctr_base = n_ctr;
@@ -181,6 +187,15 @@ int program_build(lop_plan_t *pl, const std::vector<StageReq> &reqs, const void 
                 if (l.op == LOP_CONV2D && l.residual_from >= 0) needs[nn++] = Need{l.residual_from, o0, o1};
             }
             const int first = (int)deps.size();
+            if (rq.wait_arrival) {
+                bool raw = rq.layer < 0;
+                if (rq.layer >= 0) {
+                    const LayerInfo &li = pl->layers[rq.layer];
+                    raw = (li.l.input_from == LOP_INPUT && !(li.kernel == K_CONV_TC && li.reads_padded_input)) ||
+                          (li.l.op == LOP_CONV2D && li.l.residual_from == LOP_INPUT);
+                }
+                if (raw) { deps.push_back(make_int2(-1 - rq.band, -1)); uses_flags = true; }   // patched below
+            }
             for (int q = 0; q < nn; ++q)
                 for (int ps : by_layer[needs[q].layer]) {
                     if (!reuse && stage_band[ps] != rq.band) continue;
@@ -201,6 +216,13 @@ int program_build(lop_plan_t *pl, const std::vector<StageReq> &reqs, const void 
 
     Program *p = new (std::nothrow) Program();
     if (!p) { set_error("out of host memory"); return LOP_ENOMEM; }
+    if (uses_flags) {                                        // arrival flags live after the row-group counters
+        p->flag_base = n_ctr;
+        p->n_flags = pl->n_bands;
+        for (int2 &d : deps)
+            if (d.x < 0) d.x = p->flag_base + (-1 - d.x);
+        n_ctr += p->n_flags;
+    }
     if (n_items == 0) { *result = p; return LOP_OK; }          // nothing to do: an empty program
 
     // ---- one device allocation for all tables
@@ -236,6 +258,7 @@ int program_build(lop_plan_t *pl, const std::vector<StageReq> &reqs, const void 
     P.deps = reinterpret_cast<const int2 *>(d + o_deps);
     P.counters = p->counters;
     P.status = reinterpret_cast<unsigned *>(wsb + pl->status_off);
+    P.flag_base = p->flag_base; P.n_flags = p->n_flags;
     P.n_stages = (int)stages.size();
     P.n_items = n_items;
     P.slot_bytes = slot_bytes;
@@ -258,5 +281,11 @@ int program_launch(Program *p, cudaStream_t s)
 }
 
 bool program_empty(const Program *p) { return !p || p->grid == 0; }
+
+unsigned *program_arrival_flag(Program *p, int band)
+{
+    if (!p || !p->counters || band < 0 || band >= p->n_flags) return nullptr;
+    return p->counters + p->flag_base + band;
+}
 
 }  // namespace lop

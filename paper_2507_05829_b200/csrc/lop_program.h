@@ -8,12 +8,16 @@
 
 namespace lop {
 
-struct StageReq { int band, layer, lo, hi; };     // layer -1: channel padding of the chain input
+// layer -1: channel padding of the chain input.  wait_arrival: stages that read the raw chain input wait for
+// their band's arrival flag (single-launch pipelined programs).
+struct StageReq { int band, layer, lo, hi; bool wait_arrival; };
 struct Program;
 
 bool program_supported(const lop_plan_t *pl);
 int program_build(lop_plan_t *pl, const std::vector<StageReq> &reqs, const void *in, void *out, void *ws, Program **result);
 int program_launch(Program *p, cudaStream_t s);
+// Device address of band b's arrival flag (a 4-byte word the copy stream sets non-zero), or nullptr.
+unsigned *program_arrival_flag(Program *p, int band);
 bool program_empty(const Program *p);
 void program_destroy(Program *p);
 

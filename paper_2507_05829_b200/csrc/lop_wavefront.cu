@@ -25,11 +25,6 @@ using namespace ptx;
 constexpr uint32_t SPIN_LIMIT = 1u << 22;
 constexpr int EPI_THREADS = 128;
 
-struct RoleCtx {
-    WfStage st;
-    WfLayer ly;
-};
-
 __device__ __forceinline__ unsigned ld_acquire(const unsigned *p)
 {
     unsigned v;
@@ -54,39 +49,35 @@ __device__ __forceinline__ bool wait_counter(const unsigned *ctr, unsigned targe
     return false;
 }
 
-__device__ __forceinline__ bool wait_deps(const WfParams &P, const WfStage &st, int tile_r, unsigned run)
+__device__ __forceinline__ bool wait_deps(const WfParams &P, int dep_slot, unsigned run)
 {
-    const int2 di = __ldg(&P.dep_index[st.dep_base + tile_r]);
+    const int2 di = __ldg(&P.dep_index[dep_slot]);
     for (int j = di.x; j < di.x + di.y; ++j) {
         const int2 d = __ldg(&P.deps[j]);
-        if (!wait_counter(P.counters + d.x, run * (unsigned)d.y, P.counters + 2)) return false;
+        // d.y > 0: a row-group counter that grows by d.y per run; d.y < 0: an arrival flag set to >= -d.y
+        const unsigned target = d.y > 0 ? run * (unsigned)d.y : (unsigned)(-d.y);
+        if (!wait_counter(P.counters + d.x, target, P.counters + 2)) return false;
     }
     return true;
 }
 
-__device__ __forceinline__ void copy_words(void *dst, const void *src, int words, int tid, int nthreads)
-{
-    const uint32_t *s = static_cast<const uint32_t *>(src);
-    uint32_t *d = static_cast<uint32_t *>(dst);
-    for (int i = tid; i < words; i += nthreads) d[i] = __ldg(s + i);
-}
-
 __device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
-struct ConvTile {
-    int cout_tile, tile_w, tile_n, tile_r;
+// Walks the stage list as the CTA's item index grows; touches global memory only on a stage change.
+struct StageCursor {
+    int sidx = -1, first = 0, end = 0, kind = -1;
+    __device__ __forceinline__ bool advance(const WfParams &P, int item)      // true when the stage changed
+    {
+        if (item < end) return false;
+        do {
+            ++sidx;
+            first = __ldg(&P.stages[sidx].first_item);
+            end = first + __ldg(&P.stages[sidx].n_items);
+        } while (item >= end);
+        kind = __ldg(&P.stages[sidx].kind);
+        return true;
+    }
 };
-__device__ __forceinline__ ConvTile decode_conv(const WfStage &st, int local)
-{
-    ConvTile t;
-    t.cout_tile = local % st.cout_tiles;
-    int q = local / st.cout_tiles;
-    t.tile_w = q % st.tiles_w;
-    q /= st.tiles_w;
-    t.tile_n = q % st.tiles_n;
-    t.tile_r = q / st.tiles_n;
-    return t;
-}
 
 __global__ void __launch_bounds__(WF_THREADS, 1) wavefront_kernel(const WfParams P)
 {
@@ -95,12 +86,14 @@ __global__ void __launch_bounds__(WF_THREADS, 1) wavefront_kernel(const WfParams
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t *smem = smem_raw + (base - raw);
     const int S = P.ring;
-    const uint32_t ring_bytes = (uint32_t)S * P.slot_bytes;
+    const uint32_t slot_bytes = P.slot_bytes;
+    const uint32_t ring_bytes = (uint32_t)S * slot_bytes;
     const uint32_t full0 = base + ring_bytes, empty0 = full0 + 8u * S;
     const uint32_t accf0 = empty0 + 8u * S, acce0 = accf0 + 16u;
     volatile uint32_t *misc = reinterpret_cast<volatile uint32_t *>(smem + ring_bytes + 16u * S + 32u);
     // misc[0] TMEM base, misc[1] abort, misc[2] run number
-    RoleCtx *ctx = reinterpret_cast<RoleCtx *>(smem + ring_bytes + 16u * S + 64u);
+    float *s_scale = reinterpret_cast<float *>(smem + ring_bytes + 16u * S + 64u);   // [256]
+    float *s_shift = s_scale + 256;                                                   // [256]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
@@ -128,95 +121,110 @@ __global__ void __launch_bounds__(WF_THREADS, 1) wavefront_kernel(const WfParams
     const uint32_t tmem_base = misc[0];
     const unsigned run = misc[2];
     volatile uint32_t *abort_flag = &misc[1];
+    const int G = gridDim.x;
 
     if (warp == 0) {
         if (lane == 0) {
             // ---------------- TMA producer ----------------
-            RoleCtx &c = ctx[0];
-            int sidx = 0, cur = -1;
-            uint32_t it = 0;
-            for (int item = blockIdx.x; item < P.n_items && !*abort_flag; item += gridDim.x) {
-                while (item >= __ldg(&P.stages[sidx].first_item) + __ldg(&P.stages[sidx].n_items)) ++sidx;
-                if (__ldg(&P.stages[sidx].kind) != WF_CONV) continue;
-                if (sidx != cur) {
-                    copy_words(&c.st, &P.stages[sidx], 32, 0, 1);
-                    copy_words(&c.ly, &P.layers[c.st.layer], 32, 0, 1);
-                    cur = sidx;
+            // Everything the inner loop needs lives in registers: the PTX wrappers clobber memory, so a field
+            // left in shared or global memory would be re-read after every one of them.
+            StageCursor cur;
+            uint32_t slot = 0, phase = 0;
+            int first_item = 0, oh_lo = 0, tw_log = 0, tr_log = 0, tiles_w = 1, tiles_n = 1, cout_tiles = 1, BN = 0, BK = 0,
+                amask = 0, dep_base = 0, slabs = 1, kh = 1, kw = 1, sh = 1, sw = 1, ph = 0, pw = 0, dh = 1, dw = 1, cin = 0;
+            uint32_t a_bytes = 0, tx_bytes = 0;
+            const CUtensorMap *maps = nullptr;
+            bool fail = false;
+            for (int item = blockIdx.x; item < P.n_items && !fail; item += G) {
+                if (cur.advance(P, item) && cur.kind == WF_CONV) {
+                    const WfStage *sp = &P.stages[cur.sidx];
+                    const WfLayer *lp = &P.layers[__ldg(&sp->layer)];
+                    first_item = cur.first;
+                    oh_lo = __ldg(&sp->oh_lo); tw_log = __ldg(&sp->tw_log); tr_log = __ldg(&sp->tr_log);
+                    tiles_w = __ldg(&sp->tiles_w); tiles_n = __ldg(&sp->tiles_n); cout_tiles = __ldg(&sp->cout_tiles);
+                    BN = __ldg(&sp->BN); BK = __ldg(&sp->BK); amask = __ldg(&sp->a_valid_mask); dep_base = __ldg(&sp->dep_base);
+                    a_bytes = __ldg(&sp->a_bytes); tx_bytes = a_bytes + __ldg(&sp->b_bytes);
+                    maps = P.maps + __ldg(&sp->map_base);
+                    kh = __ldg(&lp->kh); kw = __ldg(&lp->kw); sh = __ldg(&lp->sh); sw = __ldg(&lp->sw);
+                    ph = __ldg(&lp->ph); pw = __ldg(&lp->pw); dh = __ldg(&lp->dh); dw = __ldg(&lp->dw);
+                    cin = __ldg(&lp->Cin);
+                    slabs = cin / BK;
                 }
-                const WfStage &st = c.st;
-                const WfLayer &ly = c.ly;
-                const ConvTile t = decode_conv(st, item - st.first_item);
-                if (!wait_deps(P, st, t.tile_r, run)) {
+                if (cur.kind != WF_CONV) continue;
+                if (*abort_flag) break;
+                int q = item - first_item;
+                const int cout_tile = q % cout_tiles; q /= cout_tiles;
+                const int tile_w = q % tiles_w; q /= tiles_w;
+                const int tile_n = q % tiles_n;
+                const int tile_r = q / tiles_n;
+                if (!wait_deps(P, dep_base + tile_r, run)) {
                     atomicOr(P.status, 0x10u);
-                    atomicExch(P.counters + 2, 1u);
-                    *abort_flag = 1;
+                    fail = true;
                     break;
                 }
                 asm volatile("fence.proxy.async;" ::: "memory");       // producers' generic-proxy writes -> our TMA reads
-                const int ow0 = t.tile_w << st.tw_log;
-                const int oh0 = st.oh_lo + (t.tile_r << st.tr_log);
-                const int n0 = t.tile_n * (128 >> (st.tw_log + st.tr_log));
-                const int co0 = t.cout_tile * st.BN;
-                const int slabs = ly.Cin / st.BK;
-                const CUtensorMap *maps = P.maps + st.map_base;
-                bool fail = false;
-                for (int a = 0; a < ly.kh && !fail; ++a) {
-                    const int qh = a * ly.dh - ly.ph;
-                    const int offh = floor_div_i(qh, ly.sh), parh = qh - offh * ly.sh;
-                    for (int b = 0; b < ly.kw && !fail; ++b) {
-                        const int qw = b * ly.dw - ly.pw;
-                        const int offw = floor_div_i(qw, ly.sw), parw = qw - offw * ly.sw;
-                        const int mi = parh * ly.sw + parw;
-                        const bool have = (st.a_valid_mask >> mi) & 1;
-                        for (int cs = 0; cs < slabs; ++cs, ++it) {
-                            const uint32_t s = it % (uint32_t)S, round = it / (uint32_t)S;
-                            if (round > 0 && !mbar_wait(empty0 + 8u * s, (round - 1) & 1)) { fail = true; break; }
-                            const uint32_t sa = base + s * P.slot_bytes, sb = sa + st.a_bytes;
-                            const uint32_t fb = full0 + 8u * s;
-                            mbar_expect_tx(fb, st.a_bytes + st.b_bytes);
-                            tma_load_4d(sa, maps + mi, fb, cs * st.BK, have ? ow0 + offw : -65536, have ? oh0 + offh : -65536, n0);
-                            tma_load_2d(sb, maps + 4, fb, (a * ly.kw + b) * ly.Cin + cs * st.BK, co0);
+                const int ow0 = tile_w << tw_log;
+                const int oh0 = oh_lo + (tile_r << tr_log);
+                const int n0 = tile_n * (128 >> (tw_log + tr_log));
+                const int co0 = cout_tile * BN;
+                for (int a = 0; a < kh && !fail; ++a) {
+                    const int qh = a * dh - ph;
+                    const int offh = floor_div_i(qh, sh), parh = qh - offh * sh;
+                    for (int b = 0; b < kw && !fail; ++b) {
+                        const int qw = b * dw - pw;
+                        const int offw = floor_div_i(qw, sw), parw = qw - offw * sw;
+                        const int mi = parh * sw + parw;
+                        const bool have = (amask >> mi) & 1;
+                        const int cw = have ? ow0 + offw : -65536, chh = have ? oh0 + offh : -65536;
+                        const int kbase = (a * kw + b) * cin;
+                        for (int cs = 0; cs < slabs; ++cs) {
+                            if (!mbar_wait(empty0 + 8u * slot, phase ^ 1u)) { atomicOr(P.status, 0x1u); fail = true; break; }
+                            const uint32_t sa = base + slot * slot_bytes;
+                            const uint32_t fb = full0 + 8u * slot;
+                            mbar_expect_tx(fb, tx_bytes);
+                            tma_load_4d(sa, maps + mi, fb, cs * BK, cw, chh, n0);
+                            tma_load_2d(sa + a_bytes, maps + 4, fb, kbase + cs * BK, co0);
+                            if (++slot == (uint32_t)S) { slot = 0; phase ^= 1u; }
                         }
                     }
                 }
-                if (fail) {
-                    atomicOr(P.status, 0x1u);
-                    atomicExch(P.counters + 2, 1u);
-                    *abort_flag = 1;
-                    break;
-                }
+            }
+            if (fail) {
+                atomicExch(P.counters + 2, 1u);
+                *abort_flag = 1;
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
             // ---------------- MMA issuer ----------------
-            RoleCtx &c = ctx[1];
-            int sidx = 0, cur = -1;
-            uint32_t it = 0, cnt = 0;
+            StageCursor cur;
+            uint32_t slot = 0, phase = 0, cnt = 0;
+            int k_iters = 0, ksteps = 0;
+            uint32_t a_bytes = 0, idesc = 0, layout_code = 0, sbo = 0;
             bool fail = false;
-            for (int item = blockIdx.x; item < P.n_items && !fail; item += gridDim.x) {
-                while (item >= __ldg(&P.stages[sidx].first_item) + __ldg(&P.stages[sidx].n_items)) ++sidx;
-                if (__ldg(&P.stages[sidx].kind) != WF_CONV) continue;
-                if (sidx != cur) {
-                    copy_words(&c.st, &P.stages[sidx], 32, 0, 1);
-                    cur = sidx;
+            for (int item = blockIdx.x; item < P.n_items && !fail; item += G) {
+                if (cur.advance(P, item) && cur.kind == WF_CONV) {
+                    const WfStage *sp = &P.stages[cur.sidx];
+                    k_iters = __ldg(&sp->k_iters); ksteps = __ldg(&sp->BK) / 16;
+                    a_bytes = __ldg(&sp->a_bytes); idesc = __ldg(&sp->idesc);
+                    layout_code = __ldg(&sp->layout_code); sbo = __ldg(&sp->sbo_bytes);
                 }
-                const WfStage &st = c.st;
+                if (cur.kind != WF_CONV) continue;
                 const uint32_t buf = cnt & 1u;
-                if (cnt >= 2 && !mbar_wait(acce0 + 8u * buf, ((cnt >> 1) - 1) & 1)) { fail = true; break; }
+                if (!mbar_wait(acce0 + 8u * buf, ((cnt >> 1) & 1u) ^ 1u)) { fail = true; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t acc = tmem_base + buf * 256u;
-                for (int k = 0; k < st.k_iters; ++k, ++it) {
-                    const uint32_t s = it % (uint32_t)S, round = it / (uint32_t)S;
-                    if (*abort_flag || !mbar_wait(full0 + 8u * s, round & 1)) { fail = true; break; }
+                for (int k = 0; k < k_iters; ++k) {
+                    if (*abort_flag || !mbar_wait(full0 + 8u * slot, phase)) { fail = true; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    const uint32_t sa = base + s * P.slot_bytes, sb = sa + st.a_bytes;
-                    for (int kk = 0; kk < st.BK / 16; ++kk) {
-                        const uint64_t ad = smem_desc(sa + 32u * kk, st.sbo_bytes, st.layout_code);
-                        const uint64_t bd = smem_desc(sb + 32u * kk, st.sbo_bytes, st.layout_code);
-                        umma_bf16(acc, ad, bd, st.idesc, (k > 0 || kk > 0) ? 1u : 0u);
+                    const uint32_t sa = base + slot * slot_bytes, sb = sa + a_bytes;
+                    for (int kk = 0; kk < ksteps; ++kk) {
+                        const uint64_t ad = smem_desc(sa + 32u * kk, sbo, layout_code);
+                        const uint64_t bd = smem_desc(sb + 32u * kk, sbo, layout_code);
+                        umma_bf16(acc, ad, bd, idesc, (k > 0 || kk > 0) ? 1u : 0u);
                     }
-                    umma_commit(empty0 + 8u * s);
+                    umma_commit(empty0 + 8u * slot);
+                    if (++slot == (uint32_t)S) { slot = 0; phase ^= 1u; }
                 }
                 if (fail) break;
                 umma_commit(accf0 + 8u * buf);
@@ -230,57 +238,74 @@ __global__ void __launch_bounds__(WF_THREADS, 1) wavefront_kernel(const WfParams
         }
     } else {
         // ---------------- epilogue / SIMT warps ----------------
-        RoleCtx &c = ctx[2];
         const int tid = threadIdx.x - 64;
         const int g = warp & 3;
-        int sidx = 0, cur = -1;
+        StageCursor cur;
         uint32_t cnt = 0;
         bool fail = false;
-        for (int item = blockIdx.x; item < P.n_items; item += gridDim.x) {
-            while (item >= __ldg(&P.stages[sidx].first_item) + __ldg(&P.stages[sidx].n_items)) ++sidx;
-            if (sidx != cur) {
-                epi_bar();                                           // everyone is done with the old context
-                copy_words(&c.st, &P.stages[sidx], 32, tid, EPI_THREADS);
-                epi_bar();
-                copy_words(&c.ly, &P.layers[c.st.layer], 32, tid, EPI_THREADS);
-                epi_bar();
-                cur = sidx;
+        int first_item = 0, oh_lo = 0, oh_hi = 0, tw_log = 0, tr_log = 0, tiles_w = 1, tiles_n = 1, cout_tiles = 1, BN = 0,
+            dep_base = 0, ctr_base = 0;
+        int N = 0, Hin = 0, Win = 0, Cin = 0, Ho = 0, Wo = 0, Cout = 0, kh = 1, kw = 1, sh = 1, sw = 1, ph = 0, pw = 0, dh = 1,
+            dw = 1, act = 0, res_pos = 0;
+        const void *xin = nullptr, *resp = nullptr;
+        const float *scale = nullptr, *shift = nullptr;
+        void *yout = nullptr;
+        for (int item = blockIdx.x; item < P.n_items; item += G) {
+            if (cur.advance(P, item)) {
+                const WfStage *sp = &P.stages[cur.sidx];
+                const WfLayer *lp = &P.layers[__ldg(&sp->layer)];
+                first_item = cur.first;
+                oh_lo = __ldg(&sp->oh_lo); oh_hi = __ldg(&sp->oh_hi); tw_log = __ldg(&sp->tw_log); tr_log = __ldg(&sp->tr_log);
+                tiles_w = __ldg(&sp->tiles_w); tiles_n = __ldg(&sp->tiles_n); cout_tiles = __ldg(&sp->cout_tiles);
+                BN = __ldg(&sp->BN); dep_base = __ldg(&sp->dep_base); ctr_base = __ldg(&sp->ctr_base);
+                N = __ldg(&lp->N); Hin = __ldg(&lp->Hin); Win = __ldg(&lp->Win); Cin = __ldg(&lp->Cin);
+                Ho = __ldg(&lp->Ho); Wo = __ldg(&lp->Wo); Cout = __ldg(&lp->Cout);
+                kh = __ldg(&lp->kh); kw = __ldg(&lp->kw); sh = __ldg(&lp->sh); sw = __ldg(&lp->sw);
+                ph = __ldg(&lp->ph); pw = __ldg(&lp->pw); dh = __ldg(&lp->dh); dw = __ldg(&lp->dw);
+                act = __ldg(&lp->act); res_pos = __ldg(&lp->res_pos);
+                xin = reinterpret_cast<const void *>(__ldg(reinterpret_cast<const unsigned long long *>(&lp->x)));
+                resp = reinterpret_cast<const void *>(__ldg(reinterpret_cast<const unsigned long long *>(&lp->res)));
+                scale = reinterpret_cast<const float *>(__ldg(reinterpret_cast<const unsigned long long *>(&lp->scale)));
+                shift = reinterpret_cast<const float *>(__ldg(reinterpret_cast<const unsigned long long *>(&lp->shift)));
+                yout = reinterpret_cast<void *>(__ldg(reinterpret_cast<const unsigned long long *>(&lp->y)));
             }
-            const WfStage &st = c.st;
-            const WfLayer &ly = c.ly;
-            const int local = item - st.first_item;
+            int q = item - first_item;
             int tile_r;
-            if (st.kind == WF_CONV) {
-                const ConvTile t = decode_conv(st, local);
-                tile_r = t.tile_r;
+            if (cur.kind == WF_CONV) {
+                const int cout_tile = q % cout_tiles; q /= cout_tiles;
+                const int tile_w = q % tiles_w; q /= tiles_w;
+                const int tile_n = q % tiles_n;
+                tile_r = q / tiles_n;
                 const uint32_t buf = cnt & 1u;
-                const int TW = 1 << st.tw_log, TR = 1 << st.tr_log;
+                const int TW = 1 << tw_log, TR = 1 << tr_log;
                 const int m = g * 32 + lane;
-                const int ow = (t.tile_w << st.tw_log) + (m & (TW - 1));
-                const int oh = st.oh_lo + (t.tile_r << st.tr_log) + ((m >> st.tw_log) & (TR - 1));
-                const int n = t.tile_n * (128 >> (st.tw_log + st.tr_log)) + (m >> (st.tw_log + st.tr_log));
-                const bool valid = ow < ly.Wo && oh < st.oh_hi && n < ly.N;
-                const int co0 = t.cout_tile * st.BN;
-                const long long pix = (((long long)n * ly.Ho + oh) * ly.Wo + ow) * ly.Cout + co0;
-                if (!mbar_wait(accf0 + 8u * buf, (cnt >> 1) & 1)) { fail = true; }
+                const int ow = (tile_w << tw_log) + (m & (TW - 1));
+                const int oh = oh_lo + (tile_r << tr_log) + ((m >> tw_log) & (TR - 1));
+                const int n = tile_n * (128 >> (tw_log + tr_log)) + (m >> (tw_log + tr_log));
+                const bool valid = ow < Wo && oh < oh_hi && n < N;
+                const int co0 = cout_tile * BN;
+                const long long pix = (((long long)n * Ho + oh) * Wo + ow) * Cout + co0;
+                // this tile's scale/shift into shared memory while the main loop is still running
+                epi_bar();                                           // previous item's readers are done
+                for (int i = tid; i < BN; i += EPI_THREADS) {
+                    s_scale[i] = scale ? __ldg(scale + co0 + i) : 1.0f;
+                    s_shift[i] = shift ? __ldg(shift + co0 + i) : 0.0f;
+                }
+                epi_bar();
+                if (!mbar_wait(accf0 + 8u * buf, (cnt >> 1) & 1u)) fail = true;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 if (!fail) {
-                    __nv_bfloat16 *y = static_cast<__nv_bfloat16 *>(ly.y);
-                    const __nv_bfloat16 *res = static_cast<const __nv_bfloat16 *>(ly.res);
+                    __nv_bfloat16 *y = static_cast<__nv_bfloat16 *>(yout);
+                    const __nv_bfloat16 *res = static_cast<const __nv_bfloat16 *>(resp);
                     const uint32_t acc = tmem_base + buf * 256u + ((uint32_t)(g * 32) << 16);
-                    for (int j = 0; j < st.BN; j += 16) {
+                    for (int j = 0; j < BN; j += 16) {
                         uint32_t r[16];
                         tmem_ld16(acc + (uint32_t)j, r);
                         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
                         if (!valid) continue;
                         float v[16];
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) {
-                            const int co = co0 + j + i;
-                            const float sc = ly.scale ? __ldg(ly.scale + co) : 1.0f;
-                            const float sf = ly.shift ? __ldg(ly.shift + co) : 0.0f;
-                            v[i] = fmaf(sc, __uint_as_float(r[i]), sf);
-                        }
+                        for (int i = 0; i < 16; ++i) v[i] = fmaf(s_scale[j + i], __uint_as_float(r[i]), s_shift[j + i]);
                         if (res) {
                             // produced inside this launch by other SMs: read through L2, never a stale L1 line
                             const uint4 q0 = __ldcg(reinterpret_cast<const uint4 *>(res + pix + j));
@@ -292,16 +317,16 @@ __global__ void __launch_bounds__(WF_THREADS, 1) wavefront_kernel(const WfParams
                                 rv[2 * i] = __uint_as_float(rw[i] << 16);
                                 rv[2 * i + 1] = __uint_as_float(rw[i] & 0xFFFF0000u);
                             }
-                            if (ly.res_pos == LOP_RES_PRE_ACT) {
+                            if (res_pos == LOP_RES_PRE_ACT) {
 #pragma unroll
-                                for (int i = 0; i < 16; ++i) v[i] = activate(v[i] + rv[i], ly.act);
+                                for (int i = 0; i < 16; ++i) v[i] = activate(v[i] + rv[i], act);
                             } else {
 #pragma unroll
-                                for (int i = 0; i < 16; ++i) v[i] = activate(v[i], ly.act) + rv[i];
+                                for (int i = 0; i < 16; ++i) v[i] = activate(v[i], act) + rv[i];
                             }
                         } else {
 #pragma unroll
-                            for (int i = 0; i < 16; ++i) v[i] = activate(v[i], ly.act);
+                            for (int i = 0; i < 16; ++i) v[i] = activate(v[i], act);
                         }
                         uint32_t o[8];
 #pragma unroll
@@ -320,55 +345,82 @@ __global__ void __launch_bounds__(WF_THREADS, 1) wavefront_kernel(const WfParams
                     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(acce0 + 8u * buf) : "memory");
                 ++cnt;
             } else {
-                // pooling or channel padding: one (row, image) per item, all 128 threads
-                const int n = local % st.tiles_n;
-                tile_r = local / st.tiles_n;
-                const int oh = st.oh_lo + tile_r;
-                if (!wait_deps(P, st, tile_r, run)) fail = true;
-                if (!fail && st.kind == WF_POOL) {
-                    const int cg = ly.Cin >> 3;
-                    const __nv_bfloat16 *x = static_cast<const __nv_bfloat16 *>(ly.x);
-                    __nv_bfloat16 *y = static_cast<__nv_bfloat16 *>(ly.y);
-                    for (int idx = tid; idx < ly.Wo * cg; idx += EPI_THREADS) {
-                        const int gch = idx % cg, ow = idx / cg;
-                        float mx[8];
+                // pooling or channel padding: a chunk of one output row of one image per item, all 128 threads
+                const int chunk = q % tiles_w; q /= tiles_w;
+                const int n = q % tiles_n;
+                tile_r = q / tiles_n;
+                const int oh = oh_lo + tile_r;
+                if (!wait_deps(P, dep_base + tile_r, run)) fail = true;
+                if (!fail && cur.kind == WF_POOL) {
+                    // 2 channel-group vectors per thread, up to 3 taps of each in flight at once
+                    const int cg = Cin >> 3;
+                    const int total = Wo * cg;
+                    const __nv_bfloat16 *x = static_cast<const __nv_bfloat16 *>(xin);
+                    __nv_bfloat16 *y = static_cast<__nv_bfloat16 *>(yout);
+                    int idx[2], gch[2], ow[2];
+                    float mx[2][8];
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) mx[i] = -INFINITY;
-                        for (int a = 0; a < ly.kh; ++a) {
-                            const int ih = oh * ly.sh - ly.ph + a * ly.dh;
-                            if (ih < 0 || ih >= ly.Hin) continue;
-                            for (int b = 0; b < ly.kw; ++b) {
-                                const int iw = ow * ly.sw - ly.pw + b * ly.dw;
-                                if (iw < 0 || iw >= ly.Win) continue;
-                                const uint4 q = __ldcg(reinterpret_cast<const uint4 *>(
-                                    x + (((long long)n * ly.Hin + ih) * ly.Win + iw) * ly.Cin + gch * 8));
-                                const uint32_t w4[4] = {q.x, q.y, q.z, q.w};
+                    for (int u = 0; u < 2; ++u) {
+                        idx[u] = chunk * (2 * EPI_THREADS) + u * EPI_THREADS + tid;
+                        gch[u] = idx[u] % cg;
+                        ow[u] = idx[u] / cg;
 #pragma unroll
-                                for (int i = 0; i < 4; ++i) {
-                                    mx[2 * i] = fmaxf(mx[2 * i], __uint_as_float(w4[i] << 16));
-                                    mx[2 * i + 1] = fmaxf(mx[2 * i + 1], __uint_as_float(w4[i] & 0xFFFF0000u));
-                                }
-                            }
-                        }
-                        uint32_t o[4];
-#pragma unroll
-                        for (int i = 0; i < 4; ++i)          // values are bf16 already: truncation is exact
-                            o[i] = (__float_as_uint(mx[2 * i]) >> 16) | (__float_as_uint(mx[2 * i + 1]) & 0xFFFF0000u);
-                        *reinterpret_cast<uint4 *>(y + (((long long)n * ly.Ho + oh) * ly.Wo + ow) * ly.Cin + gch * 8) =
-                            make_uint4(o[0], o[1], o[2], o[3]);
+                        for (int i = 0; i < 8; ++i) mx[u][i] = -INFINITY;
                     }
+                    for (int a = 0; a < kh; ++a) {
+                        const int ih = oh * sh - ph + a * dh;
+                        if (ih < 0 || ih >= Hin) continue;
+                        const long long rowbase = ((long long)n * Hin + ih) * Win;
+                        for (int b0 = 0; b0 < kw; b0 += 3) {
+                            uint4 q4[2][3];
+                            bool ok[2][3];
+#pragma unroll
+                            for (int u = 0; u < 2; ++u)
+#pragma unroll
+                                for (int bb = 0; bb < 3; ++bb) {
+                                    const int iw = ow[u] * sw - pw + (b0 + bb) * dw;
+                                    ok[u][bb] = idx[u] < total && b0 + bb < kw && iw >= 0 && iw < Win;
+                                    if (ok[u][bb])
+                                        q4[u][bb] = __ldcg(reinterpret_cast<const uint4 *>(x + (rowbase + iw) * Cin + gch[u] * 8));
+                                }
+#pragma unroll
+                            for (int u = 0; u < 2; ++u)
+#pragma unroll
+                                for (int bb = 0; bb < 3; ++bb)
+                                    if (ok[u][bb]) {
+                                        const uint32_t w4[4] = {q4[u][bb].x, q4[u][bb].y, q4[u][bb].z, q4[u][bb].w};
+#pragma unroll
+                                        for (int i = 0; i < 4; ++i) {
+                                            mx[u][2 * i] = fmaxf(mx[u][2 * i], __uint_as_float(w4[i] << 16));
+                                            mx[u][2 * i + 1] = fmaxf(mx[u][2 * i + 1], __uint_as_float(w4[i] & 0xFFFF0000u));
+                                        }
+                                    }
+                        }
+                    }
+#pragma unroll
+                    for (int u = 0; u < 2; ++u)
+                        if (idx[u] < total) {
+                            uint32_t o[4];
+#pragma unroll
+                            for (int i = 0; i < 4; ++i)      // values are bf16 already: truncation is exact
+                                o[i] = (__float_as_uint(mx[u][2 * i]) >> 16) | (__float_as_uint(mx[u][2 * i + 1]) & 0xFFFF0000u);
+                            *reinterpret_cast<uint4 *>(y + (((long long)n * Ho + oh) * Wo + ow[u]) * Cin + gch[u] * 8) =
+                                make_uint4(o[0], o[1], o[2], o[3]);
+                        }
                 } else if (!fail) {
-                    // channel padding: ly.Cin real channels -> 16, one pixel per thread and step
-                    const uint16_t *x = static_cast<const uint16_t *>(ly.x);
-                    uint16_t *y = static_cast<uint16_t *>(ly.y);
-                    const long long row = ((long long)n * ly.Hin + oh) * ly.Win;
-                    for (int px = tid; px < ly.Win; px += EPI_THREADS) {
-                        uint32_t o[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-                        const uint16_t *src = x + (row + px) * ly.Cin;
-                        for (int ch = 0; ch < ly.Cin; ++ch) o[ch >> 1] |= (uint32_t)src[ch] << ((ch & 1) * 16);
+                    // channel padding: Cin real channels -> 16, one pixel per thread
+                    const uint16_t *x = static_cast<const uint16_t *>(xin);
+                    uint16_t *y = static_cast<uint16_t *>(yout);
+                    const long long row = ((long long)n * Hin + oh) * Win;
+                    const int px = chunk * EPI_THREADS + tid;
+                    if (px < Win) {
+                        const uint16_t *src = x + (row + px) * Cin;
+                        uint32_t h[16];
+#pragma unroll
+                        for (int ch = 0; ch < 16; ++ch) h[ch] = ch < Cin ? (uint32_t)src[ch] : 0u;
                         uint4 *dst = reinterpret_cast<uint4 *>(y + (row + px) * 16);
-                        dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
-                        dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+                        dst[0] = make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), h[4] | (h[5] << 16), h[6] | (h[7] << 16));
+                        dst[1] = make_uint4(h[8] | (h[9] << 16), h[10] | (h[11] << 16), h[12] | (h[13] << 16), h[14] | (h[15] << 16));
                     }
                 }
                 __threadfence();
@@ -382,7 +434,7 @@ __global__ void __launch_bounds__(WF_THREADS, 1) wavefront_kernel(const WfParams
                 }
                 break;
             }
-            if (tid == 0) atomicAdd(P.counters + st.ctr_base + tile_r, 1u);   // release: stores fenced above
+            if (tid == 0) atomicAdd(P.counters + ctr_base + tile_r, 1u);      // release: stores fenced above
         }
     }
 
@@ -395,6 +447,7 @@ __global__ void __launch_bounds__(WF_THREADS, 1) wavefront_kernel(const WfParams
         __threadfence();
         const unsigned done = atomicAdd(P.counters + 1, 1u);
         if (done == gridDim.x - 1) {                                  // last CTA out: this run is complete
+            for (int f = 0; f < P.n_flags; ++f) P.counters[P.flag_base + f] = 0u;   // arrival flags of the next run
             atomicExch(P.counters + 1, 0u);
             __threadfence();
             atomicAdd(P.counters, 1u);
@@ -406,7 +459,7 @@ __global__ void __launch_bounds__(WF_THREADS, 1) wavefront_kernel(const WfParams
 
 size_t wavefront_smem_bytes(int ring, uint32_t slot_bytes)
 {
-    return 1024 + (size_t)ring * slot_bytes + 16 * (size_t)ring + 64 + 3 * sizeof(RoleCtx) + 64;
+    return 1024 + (size_t)ring * slot_bytes + 16 * (size_t)ring + 64 + 2 * 256 * sizeof(float) + 64;
 }
 
 cudaError_t launch_wavefront(const WfParams &p, int grid, cudaStream_t s)

@@ -51,7 +51,9 @@ struct WfParams {
     const CUtensorMap *maps;
     const int2 *dep_index;    // per (stage, tile_r): first, count
     const int2 *deps;         // (counter index, completions expected per run)
-    unsigned *counters;       // [0] runs completed, [1] CTAs finished, [2] abort, [4..] row-group counters
+    unsigned *counters;       // [0] runs completed, [1] CTAs finished, [2] abort, [4..] row-group counters,
+                              // then n_flags band-arrival flags (set by the copy stream, cleared at run end)
+    int flag_base, n_flags;
     unsigned *status;
     int n_stages, n_items;
     int ring;                 // pipeline depth

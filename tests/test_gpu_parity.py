@@ -205,9 +205,9 @@ def test_wavefront_launch_counts_and_repeatability():
         dc.run_pipelined(x)
         torch.cuda.synchronize()
         if i == 0:
-            assert dc.plans[0].last_launches() == 8 + 1          # one launch per band (+ weight padding once)
+            assert dc.plans[0].last_launches() == 1 + 1          # one persistent launch (+ weight padding once)
         else:
-            assert dc.plans[0].last_launches() == 8 and dc.plans[0].last_copies() == 8
+            assert dc.plans[0].last_launches() == 1 and dc.plans[0].last_copies() == 8
         out = dc.outs[-1].clone()
         first = out if first is None else first
         assert torch.equal(out, first)
