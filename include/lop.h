@@ -174,6 +174,36 @@ int lop_plan_last_copies(const lop_plan_t *plan);
  * the stream of the last execution call. */
 int lop_plan_check_device(lop_plan_t *plan, void *workspace);
 
+/* ---- execution without any allocation --------------------------------------------------------
+ * (The paper has no counterpart: this entry point exists for how the library is deployed.)
+ * Some callers are not allowed to allocate: a plug-in running inside an application that forbids
+ * cudaMalloc once it has started, a control loop that must never wait on the allocator, a process
+ * whose device memory was handed out in full beforehand.  They cannot provide a workspace, and the
+ * other lop_run_* functions would also create a stream, events and device tables on first use.
+ *
+ * lop_run_whole_static computes what lop_run_whole computes (every layer over all its rows, one
+ * kernel launch per layer, the same kernels and therefore the same bits), but takes its scratch
+ * -- status word, channel-padded input and first-layer weights, the tensors between layers --
+ * from one array of LOP_STATIC_SCRATCH_BYTES bytes built into the library's device image.  It
+ * calls no cudaMalloc / cudaFree / cudaHostAlloc, creates no stream or event and caches nothing;
+ * the plan is only read.  in_dev, out_dev: DEVICE, full-size tensors as for lop_run_whole, owned
+ * by the caller.  status_dev: DEVICE, 4 bytes, may be NULL; when given it is cleared at the start
+ * of the call and afterwards holds 0, or a non-zero mask if a tensor-core kernel gave up on a
+ * bounded wait (read it after synchronising the stream).  stream: cudaStream_t as void*.
+ *
+ * Limits and rules:
+ *   - A plan with lop_plan_workspace_bytes() > LOP_STATIC_SCRATCH_BYTES is refused with
+ *     LOP_EUNSUPPORTED before anything is enqueued (16 MiB holds e.g. a 224x224 image through two
+ *     64-channel layers).  Every GPU on which the library is loaded holds the array until exit.
+ *   - The first call on each device looks the array's device address up (with that device
+ *     current); make that first call outside any stream capture.
+ *   - All calls on a device share the array.  Each call rewrites what it needs, so calls one
+ *     after the other on one stream are fine; calls whose kernels can overlap on the GPU (two
+ *     streams, two threads) race on the array and give wrong results. */
+#define LOP_STATIC_SCRATCH_BYTES (16u << 20)
+int lop_run_whole_static(lop_plan_t *plan, const void *in_dev, void *out_dev, unsigned *status_dev,
+                         void *stream);
+
 const char *lop_strerror(int status);
 const char *lop_last_error(void);       /* thread-local; valid until the next failing call */
 

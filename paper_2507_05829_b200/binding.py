@@ -20,8 +20,9 @@ EXPORTS = [
     "lop_plan_out_shape", "lop_plan_set_params", "lop_plan_workspace_bytes", "lop_plan_staging_bytes",
     "lop_plan_flops", "lop_run_whole", "lop_run_band", "lop_run_banded", "lop_copy_band", "lop_run_pipelined",
     "lop_plan_last_timing", "lop_plan_layer_time", "lop_plan_layer_kernel", "lop_plan_last_launches", "lop_plan_last_copies",
-    "lop_plan_check_device", "lop_strerror", "lop_last_error",
+    "lop_plan_check_device", "lop_run_whole_static", "lop_strerror", "lop_last_error",
 ]
+LOP_STATIC_SCRATCH_BYTES = 16 << 20
 
 
 class LopError(RuntimeError):
@@ -89,6 +90,7 @@ def lib():
     L.lop_plan_last_launches.argtypes = [c_void_p]
     L.lop_plan_last_copies.argtypes = [c_void_p]
     L.lop_plan_check_device.argtypes = [c_void_p, c_void_p]
+    L.lop_run_whole_static.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
     L.lop_strerror.argtypes = [c_int]
     L.lop_strerror.restype = c_char_p
     L.lop_last_error.restype = c_char_p
@@ -196,6 +198,10 @@ class Plan:
 
     def last_copies(self):
         return _check(lib().lop_plan_last_copies(self._h))
+
+    def run_whole_static(self, in_dev, out_dev, status_dev, stream):
+        """lop_run_whole_static: no workspace argument, nothing is allocated (see include/lop.h)."""
+        _check(lib().lop_run_whole_static(self._h, in_dev, out_dev, status_dev, stream))
 
     def check_device(self, ws):
         _check(lib().lop_plan_check_device(self._h, ws))
