@@ -124,8 +124,8 @@ int lop_plan_out_shape(const lop_plan_t *plan, int layer, int *H, int *W, int *C
 int lop_plan_set_params(lop_plan_t *plan, int layer, const void *weight, const float *scale,
                         const float *shift);
 /* Device scratch, in bytes, that every lop_run_* call must be given (256-byte aligned):
- * full-size intermediate tensors, and a channel-padded copy of the input and first-layer
- * weights where the tensor-core kernel needs one. */
+ * full-size intermediate tensors, and for a thin (image) input the first layer's gathered
+ * receptive patches and zero-padded weights, which the tensor-core kernel consumes. */
 size_t lop_plan_workspace_bytes(const lop_plan_t *plan);
 /* Size of the device-side input tensor N*H*W*C in storage dtype (staging for pipelined runs). */
 size_t lop_plan_staging_bytes(const lop_plan_t *plan);
@@ -183,7 +183,7 @@ int lop_plan_check_device(lop_plan_t *plan, void *workspace);
  *
  * lop_run_whole_static computes what lop_run_whole computes (every layer over all its rows, one
  * kernel launch per layer, the same kernels and therefore the same bits), but takes its scratch
- * -- status word, channel-padded input and first-layer weights, the tensors between layers --
+ * -- status word, the first layer's gathered patches and padded weights, the tensors between layers --
  * from one array of LOP_STATIC_SCRATCH_BYTES bytes built into the library's device image.  It
  * calls no cudaMalloc / cudaFree / cudaHostAlloc, creates no stream or event and caches nothing;
  * the plan is only read.  in_dev, out_dev: DEVICE, full-size tensors as for lop_run_whole, owned

@@ -16,7 +16,7 @@
 // A strided window (stride 2) reads every other row/column: the activation is exposed through
 // one tensor map per (row parity, column parity) whose base is offset by the parity and whose
 // strides are doubled, so each tap is again a dense box.  K is always walked in the order
-// (kh, kw, channel slab), whatever the tile position, so a pixel's value does not depend on the
+// (channel slab, kh, kw), whatever the tile position, so a pixel's value does not depend on the
 // band that computes it.  Every wait is bounded; a wait that runs out sets the status word.
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -102,17 +102,19 @@ __global__ void __launch_bounds__(TC_THREADS) conv_tc_kernel(const __grid_consta
 
     if (warp == 0 && lane == 0) {
         // ---------------- TMA producer ----------------
+        // K is walked as (channel slab, kh, kw): the order every executor of this library uses, so that a
+        // pixel's value does not depend on which of them computed it
         int it = 0;
-        for (int a = 0; a < p.kh && !*abort_flag; ++a) {
-            const int qh = a * p.dh - p.ph;
-            const int offh = floor_div_i(qh, p.sh), parh = qh - offh * p.sh;
-            for (int b = 0; b < p.kw; ++b) {
-                const int qw = b * p.dw - p.pw;
-                const int offw = floor_div_i(qw, p.sw), parw = qw - offw * p.sw;
-                const int mi = parh * p.sw + parw;
-                const CUtensorMap *amap = &maps.a[mi];
-                const bool have = maps.a_valid[mi] != 0;
-                for (int c = 0; c < slabs; ++c, ++it) {
+        for (int c = 0; c < slabs && !*abort_flag; ++c) {
+            for (int a = 0; a < p.kh && !*abort_flag; ++a) {
+                const int qh = a * p.dh - p.ph;
+                const int offh = floor_div_i(qh, p.sh), parh = qh - offh * p.sh;
+                for (int b = 0; b < p.kw; ++b, ++it) {
+                    const int qw = b * p.dw - p.pw;
+                    const int offw = floor_div_i(qw, p.sw), parw = qw - offw * p.sw;
+                    const int mi = parh * p.sw + parw;
+                    const CUtensorMap *amap = &maps.a[mi];
+                    const bool have = maps.a_valid[mi] != 0;
                     const int s = it % p.stages;
                     const uint32_t round = (uint32_t)(it / p.stages);
                     if (round > 0 && !mbar_wait(empty0 + 8u * s, (round - 1) & 1)) {
@@ -128,7 +130,6 @@ __global__ void __launch_bounds__(TC_THREADS) conv_tc_kernel(const __grid_consta
                     tma_load_4d(sa, amap, fb, c * p.BK, have ? ow0 + offw : -65536, have ? oh0 + offh : -65536, n0);
                     tma_load_2d(sb, &maps.w, fb, (a * p.kw + b) * p.cin + c * p.BK, co0);
                 }
-                if (*abort_flag) break;
             }
         }
     } else if (warp == 1 && lane == 0) {
@@ -183,27 +184,18 @@ __global__ void __launch_bounds__(TC_THREADS) conv_tc_kernel(const __grid_consta
                     const float sf = p.shift ? __ldg(p.shift + co) : 0.0f;
                     v[i] = fmaf(sc, __uint_as_float(r[i]), sf);
                 }
+                float rv[16];
                 if (res) {
                     const uint4 q0 = *reinterpret_cast<const uint4 *>(res + pix + j);
                     const uint4 q1 = *reinterpret_cast<const uint4 *>(res + pix + j + 8);
                     const uint32_t rw[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
-                    float rv[16];
 #pragma unroll
                     for (int i = 0; i < 8; ++i) {
                         rv[2 * i] = __uint_as_float(rw[i] << 16);
                         rv[2 * i + 1] = __uint_as_float(rw[i] & 0xFFFF0000u);
                     }
-                    if (p.res_pos == LOP_RES_PRE_ACT) {
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) v[i] = activate(v[i] + rv[i], p.act);
-                    } else {
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) v[i] = activate(v[i], p.act) + rv[i];
-                    }
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) v[i] = activate(v[i], p.act);
                 }
+                finish16(v, rv, res ? p.res_pos : LOP_RES_NONE, p.act);
                 uint32_t o[8];
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
@@ -223,26 +215,26 @@ __global__ void __launch_bounds__(TC_THREADS) conv_tc_kernel(const __grid_consta
     }
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+typedef TensorMapEncodeFn EncodeTiledFn;
 
-EncodeTiledFn encode_fn()
+EncodeTiledFn encode_fn() { return tensor_map_encoder(); }
+
+int ilog2(int v) { int l = 0; while ((1 << l) < v) ++l; return l; }
+
+}  // namespace
+
+TensorMapEncodeFn tensor_map_encoder()
 {
-    static EncodeTiledFn fn = nullptr;
+    static TensorMapEncodeFn fn = nullptr;
     if (!fn) {
         void *ptr = nullptr;
         cudaDriverEntryPointQueryResult q;
         if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
             q == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+            fn = reinterpret_cast<TensorMapEncodeFn>(ptr);
     }
     return fn;
 }
-
-int ilog2(int v) { int l = 0; while ((1 << l) < v) ++l; return l; }
-
-}  // namespace
 
 ConvTcGeom conv_tc_geometry(const ConvArgs &a, int rows, bool fill_sms)
 {

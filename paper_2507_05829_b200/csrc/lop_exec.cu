@@ -8,6 +8,7 @@
 // addressing: every band writes its rows straight into full-size tensors.
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cstdio>
 #include <map>
 #include <tuple>
@@ -15,6 +16,7 @@
 
 #include "lop_internal.h"
 #include "lop_kernels.cuh"
+#include "lop_layerargs.h"
 #include "lop_program.h"
 
 namespace lop {
@@ -126,7 +128,7 @@ int check_common(lop_plan_t *pl, const void *in, const void *out, const void *ws
     return ensure_exec(pl);
 }
 
-// One-time work per workspace: clear the status word, build channel-padded first-layer weights.
+// One-time work per workspace: clear the status word, build the zero-padded weights of a gathered stem.
 int prepare_workspace(lop_plan_t *pl, void *ws, cudaStream_t s)
 {
     ExecState *e = pl->exec;
@@ -137,22 +139,14 @@ int prepare_workspace(lop_plan_t *pl, void *ws, cudaStream_t s)
     }
     for (size_t i = 0; i < pl->layers.size(); ++i) {
         LayerInfo &li = pl->layers[i];
-        if (!li.reads_padded_input) continue;
+        if (!li.stem_gather) continue;
         if (!fresh && e->prepared_w[i] == li.l.weight) continue;
-        LOP_CUDA(launch_pad_weights(li.l.weight, base + li.wpad_off, (long long)li.l.cout * li.l.kh * li.l.kw, li.l.cin,
-                                    li.cin_eff, s));
+        LOP_CUDA(launch_pad_weights(li.l.weight, base + li.wpad_off, li.l.cout, li.l.kh * li.l.kw * li.l.cin, li.cin_eff, s));
         e->prepared_w[i] = li.l.weight;
         e->launches++;
     }
     e->prepared_ws = ws;
     return LOP_OK;
-}
-
-const void *tensor_of(const lop_plan_t *pl, int idx, const void *in, void *out, void *ws)
-{
-    if (idx == LOP_INPUT) return in;
-    if (idx == (int)pl->layers.size() - 1) return out;
-    return static_cast<char *>(ws) + pl->layers[idx].out_off;
 }
 
 // Rows [lo, hi) of layer i.  slot: index into the per-layer timing events, or -1.
@@ -167,32 +161,15 @@ int run_layer(lop_plan_t *pl, int i, int lo, int hi, const void *in, void *out, 
         LOP_CUDA(cudaEventRecord(e->ev_layer[(size_t)slot * 2], s));
         e->layer_timed[slot] = 1;
     }
-    void *y = const_cast<void *>(tensor_of(pl, i, in, out, ws));
     if (l.op == LOP_MAXPOOL2D) {
-        PoolArgs a;
-        a.x = tensor_of(pl, l.input_from, in, out, ws);
-        a.y = y;
-        a.N = pl->N; a.Hin = li.Hin; a.Win = li.Win; a.C = l.cin; a.Ho = li.Ho; a.Wo = li.Wo;
-        a.kh = l.kh; a.kw = l.kw; a.sh = l.sh; a.sw = l.sw; a.ph = l.ph; a.pw = l.pw; a.dh = l.dh; a.dw = l.dw;
-        a.oh_lo = lo; a.oh_hi = hi;
-        LOP_CUDA(launch_maxpool(a, pl->dtype, s));
+        LOP_CUDA(launch_maxpool(pool_args(pl, i, in, out, ws, lo, hi), pl->dtype, s));
     } else {
-        ConvArgs a;
-        a.x = tensor_of(pl, l.input_from, in, out, ws);
-        a.w = l.weight;
-        a.scale = l.scale; a.shift = l.shift;
-        a.res = l.residual_from == LOP_NO_RESIDUAL ? nullptr : tensor_of(pl, l.residual_from, in, out, ws);
-        a.y = y;
-        a.N = pl->N; a.Hin = li.Hin; a.Win = li.Win; a.Cin = l.cin; a.Ho = li.Ho; a.Wo = li.Wo; a.Cout = l.cout;
-        a.kh = l.kh; a.kw = l.kw; a.sh = l.sh; a.sw = l.sw; a.ph = l.ph; a.pw = l.pw; a.dh = l.dh; a.dw = l.dw;
-        a.act = l.act; a.res_pos = a.res ? l.residual_pos : LOP_RES_NONE;
-        a.oh_lo = lo; a.oh_hi = hi;
+        const ConvArgs a = conv_args(pl, i, in, out, ws, lo, hi);
         if (li.kernel == K_CONV_TC) {
-            if (li.reads_padded_input) {
-                a.x = static_cast<char *>(ws) + pl->padin_off;
-                a.w = static_cast<char *>(ws) + li.wpad_off;
+            if (li.stem_gather) {                      // the band's patches first (the split step), same stream
+                LOP_CUDA(launch_stem_gather(in, static_cast<char *>(ws) + pl->col_off, gather_geom(pl, i), lo, hi, s));
+                e->launches++;
             }
-            a.Cin = li.cin_eff;
             const ConvTcGeom g = conv_tc_geometry(a, hi - lo);
             const MapKey key{i, g.TW, g.TR, g.TN, g.BN, g.BK, a.x, a.w};
             auto it = e->maps.find(key);
@@ -212,21 +189,11 @@ int run_layer(lop_plan_t *pl, int i, int lo, int hi, const void *in, void *out, 
     return LOP_OK;
 }
 
-int pad_input_rows(lop_plan_t *pl, int lo, int hi, const void *in, void *ws, cudaStream_t s)
-{
-    if (!pl->Cpad || hi <= lo) return LOP_OK;
-    LOP_CUDA(launch_pad_channels(in, static_cast<char *>(ws) + pl->padin_off, pl->N, pl->H, pl->W, pl->C, pl->Cpad, lo, hi, s));
-    pl->exec->launches++;
-    return LOP_OK;
-}
-
 int run_band_impl(lop_plan_t *pl, int band, const void *in, void *out, void *ws, cudaStream_t s)
 {
     const int L = (int)pl->layers.size();
     const bool reuse = (pl->flags & LOP_FLAG_REUSE_HALO) != 0;
-    const lop_range &need = pl->in_need[band];
-    int rc = pad_input_rows(pl, reuse ? need.new_lo : need.out_lo, need.out_hi, in, ws, s);
-    if (rc != LOP_OK) return rc;
+    int rc = LOP_OK;
     for (int i = 0; i < L; ++i) {
         const lop_range &r = pl->ranges[(size_t)band * L + i];
         rc = run_layer(pl, i, reuse ? r.new_lo : r.out_lo, r.out_hi, in, out, ws, s, (band + 1) * L + i);
@@ -235,16 +202,16 @@ int run_band_impl(lop_plan_t *pl, int band, const void *in, void *out, void *ws,
     return LOP_OK;
 }
 
-// Requests of one band in dependency order: channel padding first, then every layer.
+// Requests of one band in dependency order; a gathered stem is preceded by its patch-gather stage over the same rows.
 void band_requests(const lop_plan_t *pl, int band, bool wait_arrival, std::vector<StageReq> &reqs)
 {
     const int L = (int)pl->layers.size();
     const bool reuse = (pl->flags & LOP_FLAG_REUSE_HALO) != 0;
-    const lop_range &need = pl->in_need[band];
-    if (pl->Cpad) reqs.push_back(StageReq{band, -1, reuse ? need.new_lo : need.out_lo, need.out_hi, wait_arrival});
     for (int i = 0; i < L; ++i) {
         const lop_range &r = pl->ranges[(size_t)band * L + i];
-        reqs.push_back(StageReq{band, i, reuse ? r.new_lo : r.out_lo, r.out_hi, wait_arrival});
+        const int lo = reuse ? r.new_lo : r.out_lo;
+        if (pl->layers[i].stem_gather) reqs.push_back(StageReq{band, i, lo, r.out_hi, wait_arrival, true});
+        reqs.push_back(StageReq{band, i, lo, r.out_hi, wait_arrival, false});
     }
 }
 
@@ -260,8 +227,10 @@ int get_program(lop_plan_t *pl, int kind, const void *in, void *out, void *ws, P
         const int L = (int)pl->layers.size(), B = pl->n_bands;
         std::vector<StageReq> reqs;
         if (kind == PROG_WHOLE) {
-            if (pl->Cpad) reqs.push_back(StageReq{0, -1, 0, pl->H, false});
-            for (int i = 0; i < L; ++i) reqs.push_back(StageReq{0, i, 0, pl->layers[i].Ho, false});
+            for (int i = 0; i < L; ++i) {
+                if (pl->layers[i].stem_gather) reqs.push_back(StageReq{0, i, 0, pl->layers[i].Ho, false, true});
+                reqs.push_back(StageReq{0, i, 0, pl->layers[i].Ho, false, false});
+            }
         } else if (kind == PROG_ALL_BANDS) {
             // Input resident: the bands' operations of one layer do not depend on each other, so they are
             // batched layer by layer (operation batching, Sec. IV-C); dependencies stay per band row group.
@@ -271,8 +240,15 @@ int get_program(lop_plan_t *pl, int kind, const void *in, void *out, void *ws, P
             for (size_t j = 0; j < per; ++j)
                 for (int b = 0; b < B; ++b) reqs.push_back(per_band[b][j]);
         } else if (kind == PROG_PIPELINED) {
-            // Bands arrive one after the other: band-major order, each band gated by its arrival flag.
-            for (int b = 0; b < B; ++b) band_requests(pl, b, true, reqs);
+            // Bands arrive one after the other and each band's stages form a dependency chain, so the stages
+            // are ordered along the diagonals of the (band, stage) grid: while band b is at its first stage,
+            // band b-1 is at its second, and so on -- the pipeline of Sec. IV-B.  Inside a diagonal the deeper
+            // stages come first, so a CTA does not sit on a band that has not arrived while older bands have work.
+            std::vector<std::vector<StageReq>> per_band(B);
+            for (int b = 0; b < B; ++b) band_requests(pl, b, true, per_band[b]);
+            const int per = per_band.empty() ? 0 : (int)per_band[0].size();
+            for (int t = 0; t < B + per - 1; ++t)
+                for (int b = std::max(0, t - per + 1); b <= std::min(t, B - 1); ++b) reqs.push_back(per_band[b][t - b]);
         } else {
             band_requests(pl, kind, false, reqs);
         }
@@ -331,7 +307,6 @@ int lop_run_whole(lop_plan_t *pl, const void *in, void *out, void *ws, void *str
     reset_layer_timing(pl);
     if ((rc = prepare_workspace(pl, ws, s)) != LOP_OK) return rc;
     if (pl->exec->wavefront) return run_program(pl, PROG_WHOLE, in, out, ws, s);
-    if ((rc = pad_input_rows(pl, 0, pl->H, in, ws, s)) != LOP_OK) return rc;
     for (int i = 0; i < (int)pl->layers.size(); ++i)
         if ((rc = run_layer(pl, i, 0, pl->layers[i].Ho, in, out, ws, s, i)) != LOP_OK) return rc;
     return LOP_OK;

@@ -16,10 +16,11 @@ struct LayerInfo {
     int Hin = 0, Win = 0;          // spatial extent of the main input
     int Ho = 0, Wo = 0, Co = 0;    // output shape
     int kernel = K_CONV_SIMT;
-    int cin_eff = 0;               // channels the tensor-core kernel sees (chain input may be channel-padded)
-    bool reads_padded_input = false;
+    int cin_eff = 0;               // channels the tensor-core kernel sees (= the patch length Kcol for a gathered stem)
+    bool stem_gather = false;      // thin chain input: the layer's receptive patches are gathered into a
+                                   // [N, Ho, Wo, Kcol] tensor first and the convolution runs as 1x1 over it
     size_t out_off = 0;            // workspace offset of the full-size output (unused for the last layer)
-    size_t wpad_off = 0;           // workspace offset of the channel-padded weights (if reads_padded_input)
+    size_t wpad_off = 0;           // workspace offset of the [cout][Kcol] zero-padded weights (if stem_gather)
 };
 
 struct ExecState;                  // CUDA-side resources, defined in lop_exec.cu
@@ -30,10 +31,10 @@ struct lop_plan {
     std::vector<lop::LayerInfo> layers;
     int N = 0, H = 0, W = 0, C = 0, dtype = 0, n_bands = 0;
     unsigned flags = 0;
-    int Cpad = 0;                  // >0: a [N,H,W,Cpad] copy of the chain input lives in the workspace
+    int stem = -1;                 // index of the stem_gather layer, or -1
     std::vector<lop_range> ranges;     // [band][layer]
     std::vector<lop_range> in_need;    // [band]: chain-input rows (out_lo,out_hi,new_lo)
-    size_t ws_bytes = 0, status_off = 0, padin_off = 0;
+    size_t ws_bytes = 0, status_off = 0, col_off = 0;   // col_off: the gathered patch tensor
     double flops = 0.0;
     lop::ExecState *exec = nullptr;
 };

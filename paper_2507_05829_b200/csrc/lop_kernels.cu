@@ -1,5 +1,5 @@
 // CUDA-core kernels: general convolution (any kernel/stride/padding/dilation/channel count),
-// max pooling, channel padding of the chain input (the band "split" step) and of weights.
+// max pooling, patch gather of a thin chain input (the band "split" step), zero-padding of weight rows.
 //
 // The convolution here is the fp32 path and the fall-back for shapes the tensor-core kernel
 // does not take; it is also the library's second on-GPU opinion (LOP_FLAG_FORCE_SIMT).
@@ -9,6 +9,7 @@
 
 #include "lop.h"
 #include "lop_kernels.cuh"
+#include "lop_gather.cuh"
 
 namespace lop {
 
@@ -189,65 +190,25 @@ __global__ void __launch_bounds__(256) maxpool_kernel(PoolArgs p)
 }
 
 // ---------------------------------------------------------------------------------------------
-// Channel padding of a row band of the chain input (the tensor "split" an operator interceptor
-// performs, Sec. III-B): x[N,H,W,C] rows [lo,hi) -> y[N,H,W,Cpad], zero in channels C..Cpad-1.
-// A warp takes 32 consecutive pixels of one image's band: their C*32 input elements are one
-// contiguous run that the lanes load coalesced, then each lane collects its own pixel's channels
-// with warp shuffles and writes Cpad*2 bytes as 16-byte stores.  C <= 16 = Cpad.
+// Patch gather for a thin chain input, rows [lo, hi) of the patch tensor (see lop_gather.cuh).
+// One thread per 16-byte group of eight patch elements: consecutive threads write consecutive
+// 16 bytes, reads hit the few image rows of the band in L1/L2.  HBM-bound on the write.
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) pad_channels_kernel(const uint16_t *__restrict__ x, uint16_t *__restrict__ y,
-                                                           int N, int H, int W, int C, int lo, int hi)
+__global__ void __launch_bounds__(256) stem_gather_kernel(const uint16_t *__restrict__ x, uint16_t *__restrict__ y,
+                                                          GatherGeom g, int lo, int hi)
 {
-    constexpr int CP = 16;
-    const int lane = threadIdx.x & 31;
-    const long long per_img = (long long)(hi - lo) * W;          // pixels of one image's band
-    const long long warps_per_img = (per_img + 31) / 32;
-    const long long nwarps = warps_per_img * N;
-    const long long wstride = (long long)gridDim.x * (blockDim.x >> 5);
-    for (long long wid = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); wid < nwarps; wid += wstride) {
-        const int n = (int)(wid / warps_per_img);
-        const long long p0 = (wid % warps_per_img) * 32;
-        const int npix = (int)((per_img - p0) < 32 ? (per_img - p0) : 32);
-        const long long pix0 = ((long long)n * H + lo) * W + p0;  // first pixel, in whole-tensor pixel units
-        const uint16_t *src = x + pix0 * C;
-        const int nelem = npix * C;
-        uint16_t v[CP];
-#pragma unroll
-        for (int j = 0; j < CP; ++j) {
-            v[j] = 0;
-            if (j < C) {
-                const int e = lane + 32 * j;
-                if (e < nelem) v[j] = src[e];
-            }
-        }
-        uint16_t out[CP];
-#pragma unroll
-        for (int c = 0; c < CP; ++c) {
-            out[c] = 0;
-            if (c < C) {                                          // uniform across the warp
-                const int e = lane * C + c;
-                const int srcl = e & 31, srcj = e >> 5;
-                uint16_t got = 0;
-#pragma unroll
-                for (int j = 0; j < CP; ++j) {
-                    if (j < C) {                                  // uniform across the warp
-                        const unsigned tmp = __shfl_sync(0xffffffffu, (unsigned)v[j], srcl);
-                        if (srcj == j) got = (uint16_t)tmp;
-                    }
-                }
-                out[c] = got;
-            }
-        }
-        if (lane < npix) {
-            uint4 *dst = reinterpret_cast<uint4 *>(y + (pix0 + lane) * CP);
-            uint4 q0, q1;
-            q0.x = out[0] | ((unsigned)out[1] << 16);  q0.y = out[2] | ((unsigned)out[3] << 16);
-            q0.z = out[4] | ((unsigned)out[5] << 16);  q0.w = out[6] | ((unsigned)out[7] << 16);
-            q1.x = out[8] | ((unsigned)out[9] << 16);  q1.y = out[10] | ((unsigned)out[11] << 16);
-            q1.z = out[12] | ((unsigned)out[13] << 16); q1.w = out[14] | ((unsigned)out[15] << 16);
-            dst[0] = q0;
-            dst[1] = q1;
-        }
+    const int k8n = g.Kcol >> 3;
+    const long long total = (long long)g.N * (hi - lo) * g.Wo * k8n;
+    for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+         idx += (long long)gridDim.x * blockDim.x) {
+        const int k8 = (int)(idx % k8n);
+        long long q = idx / k8n;
+        const int ow = (int)(q % g.Wo);
+        q /= g.Wo;
+        const int oh = lo + (int)(q % (hi - lo));
+        const int n = (int)(q / (hi - lo));
+        const uint4 v = gather8<false>(x, g, n, oh, ow, k8);
+        *reinterpret_cast<uint4 *>(y + (((long long)n * g.Ho + oh) * g.Wo + ow) * g.Kcol + k8 * 8) = v;
     }
 }
 
@@ -299,14 +260,12 @@ cudaError_t launch_maxpool(const PoolArgs &a, int dtype, cudaStream_t s)
     return cudaGetLastError();
 }
 
-cudaError_t launch_pad_channels(const void *x, void *y, int N, int H, int W, int C, int Cpad, int lo, int hi,
-                                cudaStream_t s)
+cudaError_t launch_stem_gather(const void *x, void *y, const GatherGeom &g, int lo, int hi, cudaStream_t s)
 {
     if (hi <= lo) return cudaSuccess;
-    if (Cpad != 16 || C > 16) return cudaErrorInvalidValue;
-    const long long warps = (((long long)(hi - lo) * W + 31) / 32) * N;
-    pad_channels_kernel<<<grid_for(warps * 32, 256), 256, 0, s>>>(static_cast<const uint16_t *>(x),
-                                                                   static_cast<uint16_t *>(y), N, H, W, C, lo, hi);
+    if (g.Kcol % 8 != 0) return cudaErrorInvalidValue;
+    const long long work = (long long)g.N * (hi - lo) * g.Wo * (g.Kcol / 8);
+    stem_gather_kernel<<<grid_for(work, 256), 256, 0, s>>>(static_cast<const uint16_t *>(x), static_cast<uint16_t *>(y), g, lo, hi);
     return cudaGetLastError();
 }
 

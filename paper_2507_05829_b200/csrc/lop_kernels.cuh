@@ -29,11 +29,17 @@ struct PoolArgs {
 // CUDA-core convolution (fp32 accumulate); dtype: LOP_F32 / LOP_BF16 storage.
 cudaError_t launch_conv_simt(const ConvArgs &a, int dtype, cudaStream_t s);
 cudaError_t launch_maxpool(const PoolArgs &a, int dtype, cudaStream_t s);
-// rows [lo,hi) of x[N,H,W,C] -> same rows of y[N,H,W,Cpad], channels C..Cpad-1 zero (bf16 only).
-cudaError_t launch_pad_channels(const void *x, void *y, int N, int H, int W, int C, int Cpad, int lo, int hi,
-                                cudaStream_t s);
-// w[rows][C] -> wp[rows][Cpad] zero-padded (bf16 only); rows = cout*kh*kw.
+// rows [lo,hi) of the patch tensor y[N,Ho,Wo,Kcol] of a thin chain input x[N,H,W,C] (bf16 only).
+struct GatherGeom;
+cudaError_t launch_stem_gather(const void *x, void *y, const GatherGeom &g, int lo, int hi, cudaStream_t s);
+// w[rows][C] -> wp[rows][Cpad] zero-padded (bf16 only).
 cudaError_t launch_pad_weights(const void *w, void *wp, long long rows, int C, int Cpad, cudaStream_t s);
+
+// cuTensorMapEncodeTiled, looked up through the runtime (no link-time dependency on the driver library); nullptr if absent.
+typedef CUresult (*TensorMapEncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                      const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                      CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+TensorMapEncodeFn tensor_map_encoder();
 
 // ---- tcgen05 tensor-core convolution ---------------------------------------------------------
 struct ConvTcGeom {

@@ -169,38 +169,41 @@ static void choose_kernels(lop_plan_t &pl)
 {
     const int L = (int)pl.layers.size();
     const size_t es = elem_size(pl.dtype);
-    pl.Cpad = 0;
+    pl.stem = -1;
     const bool tc_ok = pl.dtype == LOP_BF16 && !(pl.flags & LOP_FLAG_FORCE_SIMT);
     for (int i = 0; i < L; ++i) {
         LayerInfo &li = pl.layers[i];
         const lop_layer &l = li.l;
         li.cin_eff = l.cin;
-        li.reads_padded_input = false;
+        li.stem_gather = false;
         if (l.op == LOP_MAXPOOL2D) { li.kernel = K_POOL; continue; }
         li.kernel = K_CONV_SIMT;
         if (!tc_ok) continue;
         if (l.cout % 16 != 0 || l.sh * l.sw > 4) continue;
         int cin = l.cin;
         if (cin % 16 != 0) {
-            if (l.input_from != LOP_INPUT || cin > 16) continue;   // only a thin chain input is channel-padded
-            cin = 16;
-            li.reads_padded_input = true;
+            // a thin chain input (an image): gather each output pixel's kh*kw*cin patch, zero-padded to a multiple
+            // of 16, and run the layer as a pointwise convolution over the patches
+            const long long patch = (long long)l.kh * l.kw * cin;
+            if (l.input_from != LOP_INPUT || cin > 16 || patch > 1024 || pl.stem >= 0) continue;
+            cin = (int)align_up((size_t)patch, 16);
+            li.stem_gather = true;
+            pl.stem = i;
         }
         if ((long long)l.kh * l.kw * cin > (1LL << 20)) continue;
         li.cin_eff = cin;
         li.kernel = K_CONV_TC;
     }
-    for (auto &li : pl.layers)
-        if (li.reads_padded_input) pl.Cpad = li.cin_eff;
 
     size_t off = 0;
     pl.status_off = off; off += 1024;
-    if (pl.Cpad) { pl.padin_off = off; off += align_up((size_t)pl.N * pl.H * pl.W * pl.Cpad * es, 1024); }
     for (int i = 0; i < L; ++i) {
         LayerInfo &li = pl.layers[i];
-        if (li.reads_padded_input) {
+        if (li.stem_gather) {
+            pl.col_off = off;
+            off += align_up((size_t)pl.N * li.Ho * li.Wo * li.cin_eff * es, 1024);
             li.wpad_off = off;
-            off += align_up((size_t)li.l.cout * li.l.kh * li.l.kw * li.cin_eff * es, 1024);
+            off += align_up((size_t)li.l.cout * li.cin_eff * es, 1024);
         }
         if (i != L - 1) {
             li.out_off = off;

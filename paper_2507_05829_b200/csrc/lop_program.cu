@@ -1,5 +1,5 @@
 // Host side of the wavefront kernel: turns a list of (band, layer, row range) requests into a
-// device-resident program (stages, bound layers, tensor maps, dependency lists, counters).
+// device-resident program (stages, item records, tensor maps, dependency lists, counters).
 //
 // Dependencies follow Sec. IV-B of the paper: a tile depends on a producer row group as soon as
 // any row of that group lies inside the tile's receptive rows (for the residual: its own rows).
@@ -10,6 +10,7 @@
 
 #include "lop_internal.h"
 #include "lop_kernels.cuh"
+#include "lop_layerargs.h"
 #include "lop_program.h"
 #include "lop_wavefront.cuh"
 
@@ -32,25 +33,116 @@ void program_destroy(Program *p)
 
 namespace {
 
-#define PROG_CUDA(call)                                                                 \
-    do {                                                                                \
-        cudaError_t e__ = (call);                                                       \
-        if (e__ != cudaSuccess) {                                                       \
-            set_error("%s failed: %s", #call, cudaGetErrorString(e__));                 \
-            return LOP_ECUDA;                                                           \
-        }                                                                               \
-    } while (0)
-
-struct MapSet { int layer, TW, TR, TN, BN, BK, base; };
-
-const void *tensor_ptr(const lop_plan_t *pl, int idx, const void *in, void *out, void *ws)
-{
-    if (idx == LOP_INPUT) return in;
-    if (idx == (int)pl->layers.size() - 1) return out;
-    return static_cast<char *>(ws) + pl->layers[idx].out_off;
-}
+constexpr uint32_t A_BOX_MAX = 48u * 1024u;     // largest activation box a ring slot is sized for
+constexpr uint32_t B_BOX_MAX = 32u * 1024u;     // largest weight box
 
 int ilog2i(int v) { int l = 0; while ((1 << l) < v) ++l; return l; }
+uint32_t round_up_u32(uint32_t v, uint32_t a) { return (v + a - 1) / a * a; }
+
+// Tile geometry of one convolution stage.
+struct Geom {
+    int mode;
+    int P, TR, TN;            // anchors: TN images x TR rows x P columns = 128
+    int tw_valid;             // output columns per tile
+    int RI;                   // rows of the activation box
+    int BN, BK, tb, n_taps, n_chunks;
+    uint32_t a_bytes, b_bytes, a_slot, b_slot;
+};
+
+// a: the convolution as its kernel sees it (a gathered stem already reduced to 1x1).
+Geom choose_geom(const ConvArgs &a, int rows)
+{
+    Geom g{};
+    g.BK = a.Cin % 64 == 0 ? 64 : (a.Cin % 32 == 0 ? 32 : 16);
+    g.BN = 16;
+    for (int bn = 128; bn >= 16; bn -= 16)
+        if (a.Cout % bn == 0) { g.BN = bn; break; }
+    g.n_taps = a.kh * a.kw;
+    g.n_chunks = a.Cin / g.BK;
+    const uint32_t row_bytes = (uint32_t)g.BK * 2u;
+    const bool pointwise = a.kh == 1 && a.kw == 1;
+    const int halo_w = (a.kw - 1) * a.dw, halo_h = (a.kh - 1) * a.dh;
+    bool slab = false;
+    if (!pointwise && a.sh == 1 && a.sw == 1 && g.BK == 64) {
+        // pitch P: the split of 128 anchors into rows of P pixels that needs the fewest tiles, then the smallest box
+        long long best_tiles = -1, best_box = 0;
+        for (int P = 16; P <= 128; P <<= 1) {
+            const int twv = P - halo_w, TR = 128 / P, RI = TR + halo_h;
+            if (twv < 8 || RI > 256) continue;
+            const uint32_t box = (uint32_t)RI * P * row_bytes;
+            if (box > A_BOX_MAX) continue;
+            const long long tiles = (long long)((a.Wo + twv - 1) / twv) * ((rows + TR - 1) / TR);
+            if (best_tiles < 0 || tiles < best_tiles || (tiles == best_tiles && box < best_box)) {
+                best_tiles = tiles; best_box = box;
+                g.P = P; g.TR = TR; g.TN = 1; g.tw_valid = twv; g.RI = RI;
+                slab = true;
+            }
+        }
+    }
+    if (slab || pointwise) g.mode = WF_SLAB;
+    else g.mode = WF_TAP;
+    if (!slab) {
+        // dense tile: the (TW, TR, TN) split of 128 pixels that needs the fewest tiles
+        const ConvTcGeom d = conv_tc_geometry(a, rows, /*fill_sms=*/false);
+        g.P = d.TW; g.TR = d.TR; g.TN = d.TN; g.tw_valid = d.TW; g.RI = d.TR;
+    }
+    g.a_bytes = (uint32_t)g.RI * g.P * g.TN * row_bytes;
+    // a shifted tap reads up to halo_w pixels past the box: the slot's padding takes that
+    g.a_slot = round_up_u32(g.a_bytes + (slab ? (uint32_t)halo_w * row_bytes : 0u), 1024u);
+    g.tb = 1;
+    if (g.mode == WF_SLAB && g.n_taps > 1) {
+        const int cap = std::max(1, (int)(B_BOX_MAX / ((uint32_t)g.BN * row_bytes)));
+        const int nblk = (g.n_taps + cap - 1) / cap;
+        g.tb = (g.n_taps + nblk - 1) / nblk;
+    }
+    g.b_bytes = (uint32_t)g.tb * g.BN * row_bytes;
+    g.b_slot = round_up_u32(g.b_bytes, 1024u);
+    return g;
+}
+
+struct MapSet { int layer, P, RI, TN, BN, BK, tb, base; };
+
+// Five tensor maps of a convolution stage: the activation seen through the (row parity, column parity)
+// classes of its stride, and the weights as [tap][cout][cin].
+int encode_maps(const ConvArgs &a, const Geom &g, CUtensorMap *out, int *valid_mask)
+{
+    TensorMapEncodeFn enc = tensor_map_encoder();
+    if (!enc) return LOP_ECUDA;
+    const CUtensorMapSwizzle swz = g.BK == 64 ? CU_TENSOR_MAP_SWIZZLE_128B
+                                   : (g.BK == 32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
+    const cuuint32_t ones[4] = {1, 1, 1, 1};
+    int mask = 0;
+    for (int ph = 0; ph < a.sh; ++ph)
+        for (int pw = 0; pw < a.sw; ++pw) {
+            const int idx = ph * a.sw + pw;
+            if (idx >= 4) continue;
+            const long long Hp = (a.Hin - ph + a.sh - 1) / a.sh, Wp = (a.Win - pw + a.sw - 1) / a.sw;
+            if (a.Hin - ph <= 0 || a.Win - pw <= 0 || Hp <= 0 || Wp <= 0) continue;
+            const cuuint64_t dims[4] = {(cuuint64_t)a.Cin, (cuuint64_t)Wp, (cuuint64_t)Hp, (cuuint64_t)a.N};
+            const cuuint64_t strides[3] = {(cuuint64_t)a.sw * a.Cin * 2, (cuuint64_t)a.sh * a.Win * a.Cin * 2,
+                                           (cuuint64_t)a.Hin * a.Win * a.Cin * 2};
+            const cuuint32_t box[4] = {(cuuint32_t)g.BK, (cuuint32_t)g.P, (cuuint32_t)g.RI, (cuuint32_t)g.TN};
+            void *basep = (void *)(static_cast<const char *>(a.x) + ((size_t)ph * a.Win + pw) * a.Cin * 2);
+            if (enc(&out[idx], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, basep, dims, strides, box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+                return LOP_ECUDA;
+            mask |= 1 << idx;
+        }
+    if (!mask) return LOP_ECUDA;
+    for (int i = 0; i < 4; ++i)
+        if (!((mask >> i) & 1))
+            for (int j = 0; j < 4; ++j)
+                if ((mask >> j) & 1) { out[i] = out[j]; break; }
+    const cuuint64_t taps = (cuuint64_t)a.kh * a.kw;
+    const cuuint64_t wd[3] = {(cuuint64_t)a.Cin, (cuuint64_t)a.Cout, taps};
+    const cuuint64_t ws[2] = {taps * a.Cin * 2, (cuuint64_t)a.Cin * 2};
+    const cuuint32_t wb[3] = {(cuuint32_t)g.BK, (cuuint32_t)g.BN, (cuuint32_t)g.tb};
+    if (enc(&out[4], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(a.w), wd, ws, wb, ones, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return LOP_ECUDA;
+    *valid_mask = mask;
+    return LOP_OK;
+}
 
 }  // namespace
 
@@ -71,147 +163,138 @@ int program_build(lop_plan_t *pl, const std::vector<StageReq> &reqs, const void 
     const bool reuse = (pl->flags & LOP_FLAG_REUSE_HALO) != 0;
     char *wsb = static_cast<char *>(ws);
 
-    // ---- bound layers; index L is the channel-padding pseudo-layer
-    std::vector<WfLayer> layers(L + 1);
-    for (int i = 0; i < L; ++i) {
-        const LayerInfo &li = pl->layers[i];
-        const lop_layer &l = li.l;
-        WfLayer w{};
-        w.x = (li.kernel == K_CONV_TC && li.reads_padded_input) ? wsb + pl->padin_off : tensor_ptr(pl, l.input_from, in, out, ws);
-        w.res = (l.op == LOP_CONV2D && l.residual_from != LOP_NO_RESIDUAL) ? tensor_ptr(pl, l.residual_from, in, out, ws) : nullptr;
-        w.scale = l.scale; w.shift = l.shift;
-        w.y = const_cast<void *>(tensor_ptr(pl, i, in, out, ws));
-        w.N = pl->N; w.Hin = li.Hin; w.Win = li.Win; w.Cin = l.op == LOP_CONV2D ? li.cin_eff : l.cin;
-        w.Ho = li.Ho; w.Wo = li.Wo; w.Cout = l.cout;
-        w.kh = l.kh; w.kw = l.kw; w.sh = l.sh; w.sw = l.sw; w.ph = l.ph; w.pw = l.pw; w.dh = l.dh; w.dw = l.dw;
-        w.act = l.act; w.res_pos = w.res ? l.residual_pos : LOP_RES_NONE;
-        layers[i] = w;
-    }
-    {
-        WfLayer w{};
-        w.x = in; w.y = wsb + pl->padin_off;
-        w.N = pl->N; w.Hin = pl->H; w.Win = pl->W; w.Cin = pl->C; w.Ho = pl->H; w.Wo = pl->W; w.Cout = pl->Cpad;
-        w.kh = w.kw = w.sh = w.sw = w.dh = w.dw = 1;
-        layers[L] = w;
-    }
-
     std::vector<WfStage> stages;
-    std::vector<int> stage_band;
+    std::vector<int> stage_band, stage_rows_per_group;
+    std::vector<int4> items;
     std::vector<CUtensorMap> maps;
     std::vector<MapSet> mapsets;
-    std::vector<int2> dep_index, deps;
-    std::vector<std::vector<int>> by_layer(L + 1);      // stage indices per producing layer
+    std::vector<int2> deps;
+    std::vector<std::vector<int>> by_tensor(L + 1);     // stage indices per produced tensor; index L: the stem's patches
     std::vector<int> expected;                         // completions per row group, per stage
-    int n_items = 0, n_ctr = WF_CTR_FIRST;
+    int n_ctr = WF_CTR_FIRST;
     bool uses_flags = false;
-    uint32_t slot_bytes = 1024;
+    uint32_t a_slot = 1024, b_slot = 1024, stg_bytes = 1024;
 
     for (const StageReq &rq : reqs) {
         if (rq.hi <= rq.lo) continue;
+        if (stages.size() >= 65535) { set_error("program has too many stages"); return LOP_EUNSUPPORTED; }
+        const LayerInfo &li = pl->layers[rq.layer];
+        const lop_layer &l = li.l;
         WfStage st{};
-        const int lidx = rq.layer < 0 ? L : rq.layer;
-        st.layer = lidx;
         st.oh_lo = rq.lo; st.oh_hi = rq.hi;
-        st.first_item = n_items;
         const int rows = rq.hi - rq.lo;
-        if (rq.layer >= 0 && pl->layers[rq.layer].l.op == LOP_CONV2D) {
-            const LayerInfo &li = pl->layers[rq.layer];
-            const lop_layer &l = li.l;
+        int group_rows = 1, tiles_r = rows, tiles_w = 1, tiles_n = pl->N, cout_tiles = 1;
+        const int produces = rq.gather ? L : rq.layer;
+        if (rq.gather) {
+            st.kind = WF_GATHER;
+            st.x = in; st.y = wsb + pl->col_off;
+            st.N = pl->N; st.Hin = pl->H; st.Win = pl->W; st.Cin = pl->C; st.Ho = li.Ho; st.Wo = li.Wo; st.Cout = li.cin_eff;
+            st.kh = l.kh; st.kw = l.kw; st.sh = l.sh; st.sw = l.sw; st.ph = l.ph; st.pw = l.pw; st.dh = l.dh; st.dw = l.dw;
+            // the kh image rows an output row reads are staged in shared memory when they fit (mode 0), else read in place
+            const uint32_t pitch = ((uint32_t)pl->W * pl->C * 2u + 31u + 15u) & ~15u;
+            const uint32_t need = round_up_u32((uint32_t)l.kh * pitch + 4u * (uint32_t)li.cin_eff, 1024u);
+            if (need <= 48u * 1024u && l.kh <= 64) stg_bytes = std::max(stg_bytes, need);
+            else st.mode = 1;
+        } else if (l.op == LOP_MAXPOOL2D) {
+            const PoolArgs a = pool_args(pl, rq.layer, in, out, ws, rq.lo, rq.hi);
+            st.kind = WF_POOL;
+            st.x = a.x; st.y = a.y;
+            st.N = a.N; st.Hin = a.Hin; st.Win = a.Win; st.Cin = a.C; st.Ho = a.Ho; st.Wo = a.Wo; st.Cout = a.C;
+            st.kh = a.kh; st.kw = a.kw; st.sh = a.sh; st.sw = a.sw; st.ph = a.ph; st.pw = a.pw; st.dh = a.dh; st.dw = a.dw;
+        } else {
+            const ConvArgs a = conv_args(pl, rq.layer, in, out, ws, rq.lo, rq.hi);
+            const Geom g = choose_geom(a, rows);
             st.kind = WF_CONV;
-            ConvArgs a{};
-            a.x = layers[lidx].x;
-            a.w = li.reads_padded_input ? (const void *)(wsb + li.wpad_off) : l.weight;
-            a.N = pl->N; a.Hin = li.Hin; a.Win = li.Win; a.Cin = li.cin_eff; a.Ho = li.Ho; a.Wo = li.Wo; a.Cout = l.cout;
-            a.kh = l.kh; a.kw = l.kw; a.sh = l.sh; a.sw = l.sw; a.ph = l.ph; a.pw = l.pw; a.dh = l.dh; a.dw = l.dw;
-            a.oh_lo = rq.lo; a.oh_hi = rq.hi;
-            const ConvTcGeom g = conv_tc_geometry(a, rows, /*fill_sms=*/false);
+            st.mode = g.mode;
+            st.x = a.x; st.res = a.res; st.scale = a.scale; st.shift = a.shift; st.y = a.y;
+            st.N = a.N; st.Hin = a.Hin; st.Win = a.Win; st.Cin = a.Cin; st.Ho = a.Ho; st.Wo = a.Wo; st.Cout = a.Cout;
+            st.kh = a.kh; st.kw = a.kw; st.sh = a.sh; st.sw = a.sw; st.ph = a.ph; st.pw = a.pw; st.dh = a.dh; st.dw = a.dw;
+            st.act = a.act; st.res_pos = a.res_pos;
             int base = -1;
             for (const MapSet &m : mapsets)
-                if (m.layer == rq.layer && m.TW == g.TW && m.TR == g.TR && m.TN == g.TN && m.BN == g.BN && m.BK == g.BK) base = m.base;
-            ConvTcMaps cm;
-            const int rc = conv_tc_encode(a, g, &cm);               // also tells which parity classes exist
+                if (m.layer == rq.layer && m.P == g.P && m.RI == g.RI && m.TN == g.TN && m.BN == g.BN && m.BK == g.BK && m.tb == g.tb)
+                    base = m.base;
+            CUtensorMap cm[5];
+            int mask = 0;
+            const int rc = encode_maps(a, g, cm, &mask);            // also tells which parity classes exist
             if (rc != LOP_OK) { set_error("layer %d: tensor-map encoding failed", rq.layer); return rc; }
             if (base < 0) {
                 base = (int)maps.size();
-                for (int i = 0; i < 4; ++i) maps.push_back(cm.a[i]);
-                maps.push_back(cm.w);
-                mapsets.push_back(MapSet{rq.layer, g.TW, g.TR, g.TN, g.BN, g.BK, base});
+                for (int i = 0; i < 5; ++i) maps.push_back(cm[i]);
+                mapsets.push_back(MapSet{rq.layer, g.P, g.RI, g.TN, g.BN, g.BK, g.tb, base});
             }
             st.map_base = base;
-            st.a_valid_mask = cm.a_valid[0] | (cm.a_valid[1] << 1) | (cm.a_valid[2] << 2) | (cm.a_valid[3] << 3);
-            st.tw_log = ilog2i(g.TW); st.tr_log = ilog2i(g.TR);
-            st.tiles_w = (li.Wo + g.TW - 1) / g.TW;
-            st.tiles_r = (rows + g.TR - 1) / g.TR;
-            st.tiles_n = (pl->N + g.TN - 1) / g.TN;
-            st.cout_tiles = l.cout / g.BN;
-            st.BN = g.BN; st.BK = g.BK;
-            st.k_iters = l.kh * l.kw * (li.cin_eff / g.BK);
-            st.a_bytes = 128u * g.BK * 2u;
-            st.b_bytes = (uint32_t)(g.BN * g.BK * 2);
+            st.a_valid_mask = mask;
+            st.p_log = ilog2i(g.P); st.tr_log = ilog2i(g.TR); st.tw_valid = g.tw_valid;
+            st.BN = g.BN; st.BK = g.BK; st.n_chunks = g.n_chunks; st.n_taps = g.n_taps; st.tb = g.tb;
+            st.a_bytes = g.a_bytes; st.b_bytes = g.b_bytes;
+            st.row_bytes = (uint32_t)g.BK * 2u;
             st.layout_code = g.BK == 64 ? 2u : (g.BK == 32 ? 4u : 6u);
-            st.sbo_bytes = 8u * g.BK * 2u;
+            st.sbo_bytes = 8u * st.row_bytes;
+            // instruction descriptor: fp32 accumulate, bf16 x bf16, both operands K-major, N = BN, M = 128
             st.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(g.BN >> 3) << 17) | ((128u >> 4) << 24);
-            slot_bytes = std::max(slot_bytes, st.a_bytes + (st.b_bytes + 1023u) / 1024u * 1024u);
-        } else {
-            // one output row of one image, cut into chunks of 128 pixels (padding) / 256 channel vectors (pooling)
-            st.kind = rq.layer < 0 ? WF_PAD : WF_POOL;
-            st.tw_log = 0; st.tr_log = 0;
-            const int per_row = rq.layer < 0 ? pl->W : pl->layers[rq.layer].Wo * (pl->layers[rq.layer].l.cin / 8);
-            const int per_item = rq.layer < 0 ? 128 : 256;
-            st.tiles_w = (per_row + per_item - 1) / per_item;
-            st.tiles_r = rows; st.tiles_n = pl->N; st.cout_tiles = 1;
+            a_slot = std::max(a_slot, g.a_slot);
+            b_slot = std::max(b_slot, g.b_slot);
+            stg_bytes = std::max(stg_bytes, round_up_u32(128u * (uint32_t)g.BN * 2u, 1024u));
+            group_rows = g.TR;
+            tiles_r = (rows + g.TR - 1) / g.TR;
+            tiles_w = (a.Wo + g.tw_valid - 1) / g.tw_valid;
+            tiles_n = (a.N + g.TN - 1) / g.TN;
+            cout_tiles = a.Cout / g.BN;
         }
-        st.n_items = st.tiles_w * st.tiles_r * st.tiles_n * st.cout_tiles;
+        if (tiles_w > 65535 || tiles_n > 65535 || cout_tiles > 65535 || tiles_r >= (1 << 20)) {
+            set_error("layer %d: too many tiles for one stage", rq.layer);
+            return LOP_EUNSUPPORTED;
+        }
         st.ctr_base = n_ctr;
-        n_ctr += st.tiles_r;
-        st.dep_base = (int)dep_index.size();
-        const int exp_here = st.tiles_w * st.tiles_n * st.cout_tiles;
+        n_ctr += tiles_r;
+        const int exp_here = tiles_w * tiles_n * cout_tiles;
+        const int sidx = (int)stages.size();
 
         // ---- dependencies of every row group of this stage on earlier stages of this program
-        struct Need { int layer, lo, hi; };
-        for (int tr = 0; tr < st.tiles_r; ++tr) {
-            const int TR = 1 << st.tr_log;
-            const int o0 = rq.lo + tr * TR, o1 = std::min(o0 + TR, rq.hi);
+        struct Need { int tensor, lo, hi; };
+        for (int tr = 0; tr < tiles_r; ++tr) {
+            const int o0 = rq.lo + tr * group_rows, o1 = std::min(o0 + group_rows, rq.hi);
             Need needs[2];
             int nn = 0;
-            if (rq.layer >= 0) {
-                const LayerInfo &li = pl->layers[rq.layer];
-                const lop_layer &l = li.l;
-                int prod = l.input_from;
-                if (prod == LOP_INPUT) prod = (li.kernel == K_CONV_TC && li.reads_padded_input) ? L : -1;
-                if (prod >= 0) {
+            bool raw = rq.gather;                                   // reads the chain input itself
+            if (!rq.gather) {
+                if (li.stem_gather) {
+                    needs[nn++] = Need{L, o0, o1};                  // the patches of exactly these rows
+                } else if (l.input_from == LOP_INPUT) {
+                    raw = true;
+                } else {
                     long long a = (long long)o0 * l.sh - l.ph, b = (long long)(o1 - 1) * l.sh - l.ph + (long long)(l.kh - 1) * l.dh;
                     a = std::max(a, 0LL); b = std::min(b, (long long)li.Hin - 1);
-                    if (a <= b) needs[nn++] = Need{prod, (int)a, (int)b + 1};
+                    if (a <= b) needs[nn++] = Need{l.input_from, (int)a, (int)b + 1};
                 }
                 if (l.op == LOP_CONV2D && l.residual_from >= 0) needs[nn++] = Need{l.residual_from, o0, o1};
+                if (l.op == LOP_CONV2D && l.residual_from == LOP_INPUT) raw = true;
             }
             const int first = (int)deps.size();
-            if (rq.wait_arrival) {
-                bool raw = rq.layer < 0;
-                if (rq.layer >= 0) {
-                    const LayerInfo &li = pl->layers[rq.layer];
-                    raw = (li.l.input_from == LOP_INPUT && !(li.kernel == K_CONV_TC && li.reads_padded_input)) ||
-                          (li.l.op == LOP_CONV2D && li.l.residual_from == LOP_INPUT);
-                }
-                if (raw) { deps.push_back(make_int2(-1 - rq.band, -1)); uses_flags = true; }   // patched below
-            }
+            if (rq.wait_arrival && raw) { deps.push_back(make_int2(-1 - rq.band, -1)); uses_flags = true; }   // patched below
             for (int q = 0; q < nn; ++q)
-                for (int ps : by_layer[needs[q].layer]) {
+                for (int ps : by_tensor[needs[q].tensor]) {
                     if (!reuse && stage_band[ps] != rq.band) continue;
                     const WfStage &p = stages[ps];
                     const int lo = std::max(needs[q].lo, p.oh_lo), hi = std::min(needs[q].hi, p.oh_hi);
                     if (lo >= hi) continue;
-                    for (int g = (lo - p.oh_lo) >> p.tr_log; g <= (hi - 1 - p.oh_lo) >> p.tr_log; ++g)
+                    const int gr = stage_rows_per_group[ps];
+                    for (int g = (lo - p.oh_lo) / gr; g <= (hi - 1 - p.oh_lo) / gr; ++g)
                         deps.push_back(make_int2(p.ctr_base + g, expected[ps]));
                 }
-            dep_index.push_back(make_int2(first, (int)deps.size() - first));
+            const int count = (int)deps.size() - first;
+            if (count > WF_MAX_DEPS) { set_error("layer %d: a tile depends on too many row groups", rq.layer); return LOP_EUNSUPPORTED; }
+            for (int tn = 0; tn < tiles_n; ++tn)
+                for (int tw = 0; tw < tiles_w; ++tw)
+                    for (int ct = 0; ct < cout_tiles; ++ct)
+                        items.push_back(make_int4(sidx | (ct << 16), tw | (tn << 16), tr | (count << 20), first));
         }
-        by_layer[lidx].push_back((int)stages.size());
+        by_tensor[produces].push_back(sidx);
         stages.push_back(st);
         stage_band.push_back(rq.band);
+        stage_rows_per_group.push_back(group_rows);
         expected.push_back(exp_here);
-        n_items += st.n_items;
     }
 
     Program *p = new (std::nothrow) Program();
@@ -223,15 +306,26 @@ int program_build(lop_plan_t *pl, const std::vector<StageReq> &reqs, const void 
             if (d.x < 0) d.x = p->flag_base + (-1 - d.x);
         n_ctr += p->n_flags;
     }
+    const int n_items = (int)items.size();
     if (n_items == 0) { *result = p; return LOP_OK; }          // nothing to do: an empty program
+
+    // ---- shared-memory rings: as many slots as fit beside the staging tile, weights first
+    const size_t fixed = 1024 + stg_bytes + 8 * (2 * 8 + 2 * 8 + 4) + 64 + 2048 + 1024 + 64;
+    const size_t budget = 227 * 1024 - fixed;
+    int sa = 2, sb = 2;
+    if ((size_t)sa * a_slot + (size_t)sb * b_slot > budget) { delete p; set_error("tile buffers do not fit shared memory"); return LOP_EUNSUPPORTED; }
+    for (bool grew = true; grew;) {
+        grew = false;
+        if (sb < 8 && (size_t)sa * a_slot + (size_t)(sb + 1) * b_slot <= budget) { ++sb; grew = true; }
+        if (sa < 4 && (size_t)(sa + 1) * a_slot + (size_t)sb * b_slot <= budget) { ++sa; grew = true; }
+    }
 
     // ---- one device allocation for all tables
     auto al = [](size_t v) { return (v + 255) / 256 * 256; };
     const size_t o_stages = 0;
-    const size_t o_layers = o_stages + al(stages.size() * sizeof(WfStage));
-    const size_t o_maps = o_layers + al(layers.size() * sizeof(WfLayer));
-    const size_t o_depi = o_maps + al(std::max<size_t>(maps.size(), 1) * sizeof(CUtensorMap));
-    const size_t o_deps = o_depi + al(std::max<size_t>(dep_index.size(), 1) * sizeof(int2));
+    const size_t o_items = o_stages + al(stages.size() * sizeof(WfStage));
+    const size_t o_maps = o_items + al(items.size() * sizeof(int4));
+    const size_t o_deps = o_maps + al(std::max<size_t>(maps.size(), 1) * sizeof(CUtensorMap));
     const size_t o_ctr = o_deps + al(std::max<size_t>(deps.size(), 1) * sizeof(int2));
     const size_t total = o_ctr + al((size_t)n_ctr * sizeof(unsigned));
     cudaError_t e = cudaMalloc(&p->dev, total);
@@ -241,9 +335,8 @@ int program_build(lop_plan_t *pl, const std::vector<StageReq> &reqs, const void 
         return bytes ? cudaMemcpy(d + off, src, bytes, cudaMemcpyHostToDevice) : cudaSuccess;
     };
     if ((e = cudaMemset(d, 0, total)) != cudaSuccess || (e = up(o_stages, stages.data(), stages.size() * sizeof(WfStage))) != cudaSuccess ||
-        (e = up(o_layers, layers.data(), layers.size() * sizeof(WfLayer))) != cudaSuccess ||
+        (e = up(o_items, items.data(), items.size() * sizeof(int4))) != cudaSuccess ||
         (e = up(o_maps, maps.data(), maps.size() * sizeof(CUtensorMap))) != cudaSuccess ||
-        (e = up(o_depi, dep_index.data(), dep_index.size() * sizeof(int2))) != cudaSuccess ||
         (e = up(o_deps, deps.data(), deps.size() * sizeof(int2))) != cudaSuccess) {
         program_destroy(p);
         set_error("program upload failed: %s", cudaGetErrorString(e));
@@ -252,18 +345,16 @@ int program_build(lop_plan_t *pl, const std::vector<StageReq> &reqs, const void 
     p->counters = reinterpret_cast<unsigned *>(d + o_ctr);
     WfParams &P = p->params;
     P.stages = reinterpret_cast<const WfStage *>(d + o_stages);
-    P.layers = reinterpret_cast<const WfLayer *>(d + o_layers);
+    P.items = reinterpret_cast<const int4 *>(d + o_items);
     P.maps = reinterpret_cast<const CUtensorMap *>(d + o_maps);
-    P.dep_index = reinterpret_cast<const int2 *>(d + o_depi);
     P.deps = reinterpret_cast<const int2 *>(d + o_deps);
     P.counters = p->counters;
     P.status = reinterpret_cast<unsigned *>(wsb + pl->status_off);
     P.flag_base = p->flag_base; P.n_flags = p->n_flags;
     P.n_stages = (int)stages.size();
     P.n_items = n_items;
-    P.slot_bytes = slot_bytes;
-    int ring = (int)((200u * 1024u) / slot_bytes);
-    P.ring = std::max(2, std::min(8, ring));
+    P.sa = sa; P.sb = sb;
+    P.a_slot_bytes = a_slot; P.b_slot_bytes = b_slot; P.stg_bytes = stg_bytes;
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);

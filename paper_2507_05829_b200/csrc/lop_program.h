@@ -8,9 +8,10 @@
 
 namespace lop {
 
-// layer -1: channel padding of the chain input.  wait_arrival: stages that read the raw chain input wait for
-// their band's arrival flag (single-launch pipelined programs).
-struct StageReq { int band, layer, lo, hi; bool wait_arrival; };
+// Rows [lo, hi) of a layer for one band.  gather: the patch-gather stage that precedes a gathered stem layer
+// (same rows).  wait_arrival: stages that read the raw chain input wait for their band's arrival flag
+// (single-launch pipelined programs).
+struct StageReq { int band, layer, lo, hi; bool wait_arrival; bool gather; };
 struct Program;
 
 bool program_supported(const lop_plan_t *pl);

@@ -58,6 +58,14 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
         : "memory");
 }
 
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+}
+
 // Shared-memory matrix descriptor of a K-major operand tile (rows of `row bytes` = swizzle span).
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t sbo_bytes, uint32_t layout_code)
 {
@@ -66,6 +74,8 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t sbo_bytes,
     d |= (uint64_t)1 << 16;                                // leading-dimension offset: unused for swizzled K-major
     d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;      // stride between 8-row groups
     d |= (uint64_t)1 << 46;                                // descriptor version of this architecture
+    // base-offset field (bits 49-51) stays 0: the swizzle is a function of the shared-memory address itself, so
+    // an operand may start at any row of a 1024-byte-aligned box (the slab convolution's shifted taps rely on it)
     d |= (uint64_t)layout_code << 61;                      // swizzle mode
     return d;
 }
@@ -94,11 +104,50 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16])
         : "memory");
 }
 
-__device__ __forceinline__ float activate(float t, int act)
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
 {
-    if (act == LOP_ACT_RELU) return fmaxf(t, 0.0f);
-    if (act == LOP_ACT_SILU) return t / (1.0f + __expf(-t));
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+
+// Activation with the kind fixed at compile time: selected once per tile, outside the per-element loops (a
+// run-time `act` inside them makes the compiler evaluate the SiLU division for every element of every kind).
+template <int ACT>
+__device__ __forceinline__ float activate_t(float t)
+{
+    if (ACT == LOP_ACT_RELU) return fmaxf(t, 0.0f);
+    if (ACT == LOP_ACT_SILU) return __fdividef(t, 1.0f + __expf(-t));
     return t;
+}
+
+// Last step of the fused epilogue on 16 channels: v = scale*acc + shift already; rv = residual values.
+template <int ACT>
+__device__ __forceinline__ void finish16_t(float (&v)[16], const float (&rv)[16], int res_pos)
+{
+    if (res_pos == LOP_RES_PRE_ACT) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) v[i] = activate_t<ACT>(v[i] + rv[i]);
+    } else if (res_pos == LOP_RES_POST_ACT) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) v[i] = activate_t<ACT>(v[i]) + rv[i];
+    } else {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) v[i] = activate_t<ACT>(v[i]);
+    }
+}
+// res_pos must be LOP_RES_NONE when there is no residual (rv is then not read).
+__device__ __forceinline__ void finish16(float (&v)[16], const float (&rv)[16], int res_pos, int act)
+{
+    if (act == LOP_ACT_RELU) finish16_t<LOP_ACT_RELU>(v, rv, res_pos);
+    else if (act == LOP_ACT_SILU) finish16_t<LOP_ACT_SILU>(v, rv, res_pos);
+    else finish16_t<LOP_ACT_NONE>(v, rv, res_pos);
 }
 
 __device__ __forceinline__ int floor_div_i(int a, int b) { int q = a / b; return (a % b != 0 && a < 0) ? q - 1 : q; }

@@ -4,14 +4,14 @@
 // creates a side stream, events and device tables.  A caller that lives inside someone else's
 // memory budget -- a plug-in of a host application that forbids cudaMalloc after start-up, a
 // real-time loop that must not take the allocator's lock, a process whose device memory is
-// fully pre-assigned -- cannot do either.  For them the scratch (status word, channel-padded
-// input and first-layer weights, the intermediate tensors between layers) lives in one
+// fully pre-assigned -- cannot do either.  For them the scratch (status word, the stem's patch
+// tensor and zero-padded weights, the intermediate tensors between layers) lives in one
 // fixed-size array in the library's own device image, and the layers are launched one kernel
 // after the other with nothing created, cached or freed.
 //
 // The array exists once per device that loads the library and is shared by every call: a call
 // overwrites whatever the previous one left, so everything that has to start from a known value
-// (the status word, the padded weights, the padded input) is rewritten by each call, and two calls
+// (the status word, the padded weights, the stem patches) is rewritten by each call, and two calls
 // whose kernels may overlap on the GPU (different streams, different threads) corrupt each other.
 #include <cuda_runtime.h>
 
@@ -19,6 +19,7 @@
 
 #include "lop_internal.h"
 #include "lop_kernels.cuh"
+#include "lop_layerargs.h"
 
 namespace lop {
 namespace {
@@ -56,13 +57,6 @@ int scratch_for_current_device(unsigned char **out)
     return LOP_OK;
 }
 
-const void *tensor_at(const lop_plan_t *pl, int idx, const void *in, void *out, unsigned char *ws)
-{
-    if (idx == LOP_INPUT) return in;
-    if (idx == (int)pl->layers.size() - 1) return out;
-    return ws + pl->layers[idx].out_off;
-}
-
 }  // namespace
 }  // namespace lop
 
@@ -96,43 +90,23 @@ extern "C" int lop_run_whole_static(lop_plan_t *pl, const void *in, void *out, u
     // the previous call's leftovers: the status word must read 0 before any kernel can raise it
     unsigned *status = status_dev ? status_dev : reinterpret_cast<unsigned *>(ws + pl->status_off);
     ST_CUDA(cudaMemsetAsync(status, 0, sizeof(unsigned), s));
-    if (pl->Cpad)
-        ST_CUDA(launch_pad_channels(in, ws + pl->padin_off, pl->N, pl->H, pl->W, pl->C, pl->Cpad, 0, pl->H, s));
     for (int i = 0; i < L; ++i) {
         const LayerInfo &li = pl->layers[i];
         const lop_layer &l = li.l;
-        void *y = const_cast<void *>(tensor_at(pl, i, in, out, ws));
         if (l.op == LOP_MAXPOOL2D) {
-            PoolArgs a;
-            a.x = tensor_at(pl, l.input_from, in, out, ws);
-            a.y = y;
-            a.N = pl->N; a.Hin = li.Hin; a.Win = li.Win; a.C = l.cin; a.Ho = li.Ho; a.Wo = li.Wo;
-            a.kh = l.kh; a.kw = l.kw; a.sh = l.sh; a.sw = l.sw; a.ph = l.ph; a.pw = l.pw; a.dh = l.dh; a.dw = l.dw;
-            a.oh_lo = 0; a.oh_hi = li.Ho;
-            ST_CUDA(launch_maxpool(a, pl->dtype, s));
+            ST_CUDA(launch_maxpool(pool_args(pl, i, in, out, ws, 0, li.Ho), pl->dtype, s));
             continue;
         }
-        ConvArgs a;
-        a.x = tensor_at(pl, l.input_from, in, out, ws);
-        a.w = l.weight;
-        a.scale = l.scale; a.shift = l.shift;
-        a.res = l.residual_from == LOP_NO_RESIDUAL ? nullptr : tensor_at(pl, l.residual_from, in, out, ws);
-        a.y = y;
-        a.N = pl->N; a.Hin = li.Hin; a.Win = li.Win; a.Cin = l.cin; a.Ho = li.Ho; a.Wo = li.Wo; a.Cout = l.cout;
-        a.kh = l.kh; a.kw = l.kw; a.sh = l.sh; a.sw = l.sw; a.ph = l.ph; a.pw = l.pw; a.dh = l.dh; a.dw = l.dw;
-        a.act = l.act; a.res_pos = a.res ? l.residual_pos : LOP_RES_NONE;
-        a.oh_lo = 0; a.oh_hi = li.Ho;
+        const ConvArgs a = conv_args(pl, i, in, out, ws, 0, li.Ho);
         if (li.kernel != K_CONV_TC) {
             ST_CUDA(launch_conv_simt(a, pl->dtype, s));
             continue;
         }
-        if (li.reads_padded_input) {
-            // another plan may have used the array since: the padded weights are rebuilt by every call
-            ST_CUDA(launch_pad_weights(l.weight, ws + li.wpad_off, (long long)l.cout * l.kh * l.kw, l.cin, li.cin_eff, s));
-            a.x = ws + pl->padin_off;
-            a.w = ws + li.wpad_off;
+        if (li.stem_gather) {
+            // another plan may have used the array since: padded weights and patches are rebuilt by every call
+            ST_CUDA(launch_pad_weights(l.weight, ws + li.wpad_off, l.cout, l.kh * l.kw * l.cin, li.cin_eff, s));
+            ST_CUDA(launch_stem_gather(in, ws + pl->col_off, gather_geom(pl, i), 0, li.Ho, s));
         }
-        a.Cin = li.cin_eff;
         const ConvTcGeom g = conv_tc_geometry(a, li.Ho);
         ConvTcMaps maps;                                   // encoded on the stack: nothing is cached between calls
         rc = conv_tc_encode(a, g, &maps);

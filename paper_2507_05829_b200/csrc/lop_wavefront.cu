@@ -1,18 +1,31 @@
 // Persistent wavefront kernel (see lop_wavefront.cuh for the execution model).
 //
-// CTA layout (192 threads, one CTA per SM):
-//   warp 0, one lane   waits for the item's producer row groups, then streams the item's activation and
-//                      weight boxes by TMA into a shared-memory ring that lives across items
-//   warp 1, one lane   tcgen05.mma into one of two fp32 accumulators in tensor memory, so the next
-//                      item's main loop overlaps this item's epilogue
-//   warps 2..5         epilogue of convolution items (TMEM -> scale/shift/residual/activation -> bf16),
-//                      and the whole of pooling / channel-padding items; they publish each finished
-//                      tile by a release increment of its row group's counter
+// CTA layout (two special warps + WF_WORKER_WARPS worker warps, one CTA per SM):
+//   warp 0      all lanes poll the item's producer row groups in parallel (the dependency list of the
+//               next item is prefetched while this one runs); lane 0 then streams the item's activation
+//               and weight boxes by TMA into two shared-memory rings that live across items
+//   warp 1      one lane issues tcgen05.mma into one of two fp32 accumulators in tensor memory, so the
+//               next item's main loop overlaps this item's epilogue
+//   workers     epilogue of convolution items: TMEM -> scale/shift/residual/activation -> bf16 rows in a
+//               shared staging tile -> coalesced 16-byte stores; and the whole of pooling / patch-gather
+//               items.  They publish each finished item by a release increment of its row group's counter.
+//               Many of them because straight-line per-element code needs several warps per scheduler to
+//               hide its own latency; the four warps that share a TMEM lane group split a tile's columns.
+//
+// Convolution as implicit GEMM: accumulator row m is an *anchor*, a position in a flat list of pixels
+// with a row pitch of P pixels.  In slab mode the activation box holds the tile's rows plus the halo of
+// the filter, P pixels wide; filter tap (a, b) reads the same box starting (a*dh*P + b*dw) pixels later,
+// so one TMA box per 64-channel chunk serves all taps (the shared-memory matrix descriptor simply starts
+// later: the swizzle is a function of the address).  Anchors in the last (kw-1)*dw columns of a
+// pitch would wrap into the next row; they are computed and dropped.  K is walked as (channel chunk, kh,
+// kw, 16-channel step) whatever the tile, so a pixel's bits do not depend on who computes it.
+//
 // Deadlock freedom: items are numbered in a topological order, every CTA is resident and takes its
 // items in increasing order, so the lowest unfinished item never waits on an unstarted one.  All
 // waits are bounded all the same; one that runs out raises the status word and the abort flag.
 #include <cuda_bf16.h>
 
+#include "lop_gather.cuh"
 #include "lop_ptx.cuh"
 #include "lop_wavefront.cuh"
 
@@ -23,7 +36,8 @@ namespace {
 using namespace ptx;
 
 constexpr uint32_t SPIN_LIMIT = 1u << 22;
-constexpr int EPI_THREADS = 128;
+constexpr int EPI_THREADS = 32 * WF_WORKER_WARPS;
+constexpr int COL_GROUPS = WF_WORKER_WARPS / 4;            // worker warps sharing a TMEM lane group split the columns
 
 __device__ __forceinline__ unsigned ld_acquire(const unsigned *p)
 {
@@ -38,46 +52,105 @@ __device__ __forceinline__ unsigned ld_relaxed(const unsigned *p)
     return v;
 }
 
-// Bounded wait until *ctr has reached target (counters only grow; compare modulo 2^32).
-__device__ __forceinline__ bool wait_counter(const unsigned *ctr, unsigned target, const unsigned *abort_word)
+#ifdef LOP_WF_TRACE
+// Developer build only: per-item time stamps (global timer, ns) of the three roles.
+constexpr int TRACE_ITEMS = 1 << 15;
+__device__ unsigned long long g_wf_trace[TRACE_ITEMS * 16];
+__device__ __forceinline__ void tr(int item, int slot)
 {
-    for (uint32_t i = 0; i < SPIN_LIMIT; ++i) {
-        if ((int)(ld_acquire(ctr) - target) >= 0) return true;
-        if ((i & 127u) == 127u && ld_relaxed(abort_word)) return false;
-        __nanosleep(40);
+    if (item < TRACE_ITEMS) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+        g_wf_trace[item * 16 + slot] = t;
+    }
+}
+#else
+#define tr(item, slot) ((void)0)
+#endif
+
+// ---- item records -------------------------------------------------------------------------------
+__device__ __forceinline__ int rec_stage(const int4 &r) { return r.x & 0xFFFF; }
+__device__ __forceinline__ int rec_cout(const int4 &r) { return (int)((unsigned)r.x >> 16); }
+__device__ __forceinline__ int rec_tw(const int4 &r) { return r.y & 0xFFFF; }
+__device__ __forceinline__ int rec_tn(const int4 &r) { return (int)((unsigned)r.y >> 16); }
+__device__ __forceinline__ int rec_tr(const int4 &r) { return r.z & 0xFFFFF; }
+__device__ __forceinline__ int rec_ndep(const int4 &r) { return (int)((unsigned)r.z >> 20); }
+__device__ __forceinline__ int rec_dep0(const int4 &r) { return r.w; }
+
+// Bounded wait of a whole warp for an item's dependencies: lane j polls entry j of the list (its first
+// 32 entries were prefetched into `mine`).  Counters only grow (compare modulo 2^32).  The result is
+// uniform across the warp.
+__device__ __forceinline__ bool wait_deps_warp(const WfParams &P, int first, int count, int2 mine, unsigned run, int lane)
+{
+    for (int j0 = 0; j0 < count; j0 += 32) {
+        const bool have = j0 + lane < count;
+        int2 d = mine;
+        if (j0 > 0 && have) d = __ldg(&P.deps[first + j0 + lane]);
+        // d.y > 0: a row-group counter that grows by d.y per run; d.y < 0: an arrival flag set to >= -d.y
+        const unsigned target = !have ? 0u : (d.y > 0 ? run * (unsigned)d.y : (unsigned)(-d.y));
+        const unsigned *ctr = P.counters + (have ? d.x : 0);
+        bool done = !have;
+        for (uint32_t i = 0;; ++i) {
+            if (!done) done = (int)(ld_acquire(ctr) - target) >= 0;
+            if (__all_sync(0xffffffffu, done)) break;
+            if (i >= SPIN_LIMIT) return false;
+            if ((i & 63u) == 63u && __any_sync(0xffffffffu, ld_relaxed(P.counters + 2) != 0u)) return false;
+            __nanosleep(32);
+        }
+    }
+    __syncwarp();            // every lane's acquire now orders the whole warp's later reads
+    return true;
+}
+
+// Bounded mbarrier wait that also gives up when the CTA's abort flag is raised.
+__device__ __forceinline__ bool mbar_wait_abortable(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag)
+{
+    for (uint32_t i = 0; i < WAIT_LIMIT; ++i) {
+        uint32_t done;
+        asm volatile(
+            "{\n"
+            ".reg .pred p;\n"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+            "selp.u32 %0, 1, 0, p;\n"
+            "}\n"
+            : "=r"(done)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (done) return true;
+        if ((i & 255u) == 255u && *abort_flag) return false;
     }
     return false;
 }
 
-__device__ __forceinline__ bool wait_deps(const WfParams &P, int dep_slot, unsigned run)
+// The 16-channel MMA steps of one (tap, channel chunk): descriptors differ only in their start-address field.
+// desc_hi: upper word of the operand descriptors (stride between 8-row groups, version, swizzle mode).
+template <int KSTEPS>
+__device__ __forceinline__ void mma_ksteps(uint32_t acc, uint32_t pa, uint32_t pb, uint32_t desc_hi, uint32_t idesc, uint32_t &accumulate)
 {
-    const int2 di = __ldg(&P.dep_index[dep_slot]);
-    for (int j = di.x; j < di.x + di.y; ++j) {
-        const int2 d = __ldg(&P.deps[j]);
-        // d.y > 0: a row-group counter that grows by d.y per run; d.y < 0: an arrival flag set to >= -d.y
-        const unsigned target = d.y > 0 ? run * (unsigned)d.y : (unsigned)(-d.y);
-        if (!wait_counter(P.counters + d.x, target, P.counters + 2)) return false;
+    const uint32_t la = ((pa & 0x3FFFFu) >> 4) | (1u << 16), lb = ((pb & 0x3FFFFu) >> 4) | (1u << 16);
+#pragma unroll
+    for (int kk = 0; kk < KSTEPS; ++kk) {
+        const uint64_t ad = ((uint64_t)desc_hi << 32) | (uint64_t)(la + 2u * kk);
+        const uint64_t bd = ((uint64_t)desc_hi << 32) | (uint64_t)(lb + 2u * kk);
+        umma_bf16(acc, ad, bd, idesc, accumulate);
+        accumulate = 1u;
     }
-    return true;
+}
+__device__ __forceinline__ void mma_tap(uint32_t acc, uint32_t pa, uint32_t pb, uint32_t desc_hi, uint32_t idesc, int ksteps,
+                                        uint32_t &accumulate)
+{
+    if (ksteps == 4) mma_ksteps<4>(acc, pa, pb, desc_hi, idesc, accumulate);
+    else if (ksteps == 2) mma_ksteps<2>(acc, pa, pb, desc_hi, idesc, accumulate);
+    else mma_ksteps<1>(acc, pa, pb, desc_hi, idesc, accumulate);
 }
 
-__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, %0;" ::"n"(EPI_THREADS) : "memory"); }
 
-// Walks the stage list as the CTA's item index grows; touches global memory only on a stage change.
-struct StageCursor {
-    int sidx = -1, first = 0, end = 0, kind = -1;
-    __device__ __forceinline__ bool advance(const WfParams &P, int item)      // true when the stage changed
-    {
-        if (item < end) return false;
-        do {
-            ++sidx;
-            first = __ldg(&P.stages[sidx].first_item);
-            end = first + __ldg(&P.stages[sidx].n_items);
-        } while (item >= end);
-        kind = __ldg(&P.stages[sidx].kind);
-        return true;
-    }
-};
+template <typename T>
+__device__ __forceinline__ T ldg_ptr(const void *const *p)
+{
+    return reinterpret_cast<T>(__ldg(reinterpret_cast<const unsigned long long *>(p)));
+}
 
 __global__ void __launch_bounds__(WF_THREADS, 1) wavefront_kernel(const WfParams P)
 {
@@ -85,21 +158,28 @@ __global__ void __launch_bounds__(WF_THREADS, 1) wavefront_kernel(const WfParams
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t *smem = smem_raw + (base - raw);
-    const int S = P.ring;
-    const uint32_t slot_bytes = P.slot_bytes;
-    const uint32_t ring_bytes = (uint32_t)S * slot_bytes;
-    const uint32_t full0 = base + ring_bytes, empty0 = full0 + 8u * S;
-    const uint32_t accf0 = empty0 + 8u * S, acce0 = accf0 + 16u;
-    volatile uint32_t *misc = reinterpret_cast<volatile uint32_t *>(smem + ring_bytes + 16u * S + 32u);
-    // misc[0] TMEM base, misc[1] abort, misc[2] run number
-    float *s_scale = reinterpret_cast<float *>(smem + ring_bytes + 16u * S + 64u);   // [256]
-    float *s_shift = s_scale + 256;                                                   // [256]
+    const int SA = P.sa, SB = P.sb;
+    const uint32_t a_slot_bytes = P.a_slot_bytes, b_slot_bytes = P.b_slot_bytes;
+    const uint32_t a0 = base, b0 = a0 + (uint32_t)SA * a_slot_bytes, stg0 = b0 + (uint32_t)SB * b_slot_bytes;
+    const uint32_t bars = stg0 + P.stg_bytes;
+    const uint32_t full_a = bars, empty_a = full_a + 8u * SA, full_b = empty_a + 8u * SA, empty_b = full_b + 8u * SB;
+    const uint32_t accf0 = empty_b + 8u * SB, acce0 = accf0 + 16u;
+    uint8_t *tail = smem + (acce0 + 16u - base);
+    volatile uint32_t *misc = reinterpret_cast<volatile uint32_t *>(tail);      // [0] TMEM base, [1] abort, [2] run, [3] epilogue failure
+    float *s_scale = reinterpret_cast<float *>(tail + 64);                       // [256]
+    float *s_shift = s_scale + 256;                                              // [256]
+    long long *row_pix = reinterpret_cast<long long *>(tail + 64 + 2048);        // [128]: element offset of anchor m's output, or -1
+    uint8_t *stg = smem + (stg0 - base);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
-        for (int s = 0; s < S; ++s) {
-            mbar_init(full0 + 8u * s, 1);
-            mbar_init(empty0 + 8u * s, 1);
+        for (int s = 0; s < SA; ++s) {
+            mbar_init(full_a + 8u * s, 1);
+            mbar_init(empty_a + 8u * s, 1);
+        }
+        for (int s = 0; s < SB; ++s) {
+            mbar_init(full_b + 8u * s, 1);
+            mbar_init(empty_b + 8u * s, 1);
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(accf0 + 8u * b, 1);
@@ -107,6 +187,7 @@ __global__ void __launch_bounds__(WF_THREADS, 1) wavefront_kernel(const WfParams
         }
         misc[1] = 0;
         misc[2] = ld_acquire(P.counters) + 1u;                 // this launch is run number (completed runs + 1)
+        misc[3] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
@@ -121,114 +202,183 @@ __global__ void __launch_bounds__(WF_THREADS, 1) wavefront_kernel(const WfParams
     const uint32_t tmem_base = misc[0];
     const unsigned run = misc[2];
     volatile uint32_t *abort_flag = &misc[1];
+    volatile uint32_t *epi_fail = &misc[3];
     const int G = gridDim.x;
+    const int NI = P.n_items;
+    const int4 zero4 = make_int4(0, 0, 0, 0);
 
     if (warp == 0) {
-        if (lane == 0) {
-            // ---------------- TMA producer ----------------
-            // Everything the inner loop needs lives in registers: the PTX wrappers clobber memory, so a field
-            // left in shared or global memory would be re-read after every one of them.
-            StageCursor cur;
-            uint32_t slot = 0, phase = 0;
-            int first_item = 0, oh_lo = 0, tw_log = 0, tr_log = 0, tiles_w = 1, tiles_n = 1, cout_tiles = 1, BN = 0, BK = 0,
-                amask = 0, dep_base = 0, slabs = 1, kh = 1, kw = 1, sh = 1, sw = 1, ph = 0, pw = 0, dh = 1, dw = 1, cin = 0;
-            uint32_t a_bytes = 0, tx_bytes = 0;
-            const CUtensorMap *maps = nullptr;
-            bool fail = false;
-            for (int item = blockIdx.x; item < P.n_items && !fail; item += G) {
-                if (cur.advance(P, item) && cur.kind == WF_CONV) {
-                    const WfStage *sp = &P.stages[cur.sidx];
-                    const WfLayer *lp = &P.layers[__ldg(&sp->layer)];
-                    first_item = cur.first;
-                    oh_lo = __ldg(&sp->oh_lo); tw_log = __ldg(&sp->tw_log); tr_log = __ldg(&sp->tr_log);
-                    tiles_w = __ldg(&sp->tiles_w); tiles_n = __ldg(&sp->tiles_n); cout_tiles = __ldg(&sp->cout_tiles);
-                    BN = __ldg(&sp->BN); BK = __ldg(&sp->BK); amask = __ldg(&sp->a_valid_mask); dep_base = __ldg(&sp->dep_base);
-                    a_bytes = __ldg(&sp->a_bytes); tx_bytes = a_bytes + __ldg(&sp->b_bytes);
-                    maps = P.maps + __ldg(&sp->map_base);
-                    kh = __ldg(&lp->kh); kw = __ldg(&lp->kw); sh = __ldg(&lp->sh); sw = __ldg(&lp->sw);
-                    ph = __ldg(&lp->ph); pw = __ldg(&lp->pw); dh = __ldg(&lp->dh); dw = __ldg(&lp->dw);
-                    cin = __ldg(&lp->Cin);
-                    slabs = cin / BK;
-                }
-                if (cur.kind != WF_CONV) continue;
-                if (*abort_flag) break;
-                int q = item - first_item;
-                const int cout_tile = q % cout_tiles; q /= cout_tiles;
-                const int tile_w = q % tiles_w; q /= tiles_w;
-                const int tile_n = q % tiles_n;
-                const int tile_r = q / tiles_n;
-                if (!wait_deps(P, dep_base + tile_r, run)) {
-                    atomicOr(P.status, 0x10u);
-                    fail = true;
-                    break;
-                }
-                asm volatile("fence.proxy.async;" ::: "memory");       // producers' generic-proxy writes -> our TMA reads
-                const int ow0 = tile_w << tw_log;
-                const int oh0 = oh_lo + (tile_r << tr_log);
-                const int n0 = tile_n * (128 >> (tw_log + tr_log));
-                const int co0 = cout_tile * BN;
-                for (int a = 0; a < kh && !fail; ++a) {
-                    const int qh = a * dh - ph;
-                    const int offh = floor_div_i(qh, sh), parh = qh - offh * sh;
-                    for (int b = 0; b < kw && !fail; ++b) {
-                        const int qw = b * dw - pw;
-                        const int offw = floor_div_i(qw, sw), parw = qw - offw * sw;
-                        const int mi = parh * sw + parw;
-                        const bool have = (amask >> mi) & 1;
-                        const int cw = have ? ow0 + offw : -65536, chh = have ? oh0 + offh : -65536;
-                        const int kbase = (a * kw + b) * cin;
-                        for (int cs = 0; cs < slabs; ++cs) {
-                            if (!mbar_wait(empty0 + 8u * slot, phase ^ 1u)) { atomicOr(P.status, 0x1u); fail = true; break; }
-                            const uint32_t sa = base + slot * slot_bytes;
-                            const uint32_t fb = full0 + 8u * slot;
-                            mbar_expect_tx(fb, tx_bytes);
-                            tma_load_4d(sa, maps + mi, fb, cs * BK, cw, chh, n0);
-                            tma_load_2d(sa + a_bytes, maps + 4, fb, kbase + cs * BK, co0);
-                            if (++slot == (uint32_t)S) { slot = 0; phase ^= 1u; }
+        // ---------------- dependency wait (all lanes) + TMA producer (lane 0) ----------------
+        int item = blockIdx.x;
+        int4 cur = item < NI ? __ldg(&P.items[item]) : zero4;
+        int4 nxt = item + G < NI ? __ldg(&P.items[item + G]) : zero4;
+        int2 dep_cur = (item < NI && lane < rec_ndep(cur)) ? __ldg(&P.deps[rec_dep0(cur) + lane]) : make_int2(0, 0);
+        int sidx = -1;
+        int kind = -1, mode = 0, oh_lo = 0, tr_log = 0, p_log = 0, tw_valid = 0, BN = 0, BK = 0, n_chunks = 1, n_taps = 1, tbx = 1,
+            amask = 0, kh = 1, kw = 1, sh = 1, sw = 1, ph = 0, pw = 0, dh = 1, dw = 1;
+        uint32_t a_bytes = 0, b_bytes = 0;
+        const CUtensorMap *maps = nullptr;
+        uint32_t a_slot = 0, a_phase = 0, b_slot = 0, b_phase = 0;
+        for (; item < NI; item += G) {
+            // two items ahead: the record; one item ahead: this lane's dependency entry
+            const int4 nn = item + 2 * G < NI ? __ldg(&P.items[item + 2 * G]) : zero4;
+            const int2 dep_nxt = (item + G < NI && lane < rec_ndep(nxt)) ? __ldg(&P.deps[rec_dep0(nxt) + lane]) : make_int2(0, 0);
+            if (rec_stage(cur) != sidx) {
+                sidx = rec_stage(cur);
+                const WfStage *sp = &P.stages[sidx];
+                kind = __ldg(&sp->kind); mode = __ldg(&sp->mode); oh_lo = __ldg(&sp->oh_lo);
+                tr_log = __ldg(&sp->tr_log); p_log = __ldg(&sp->p_log); tw_valid = __ldg(&sp->tw_valid);
+                BN = __ldg(&sp->BN); BK = __ldg(&sp->BK); n_chunks = __ldg(&sp->n_chunks); n_taps = __ldg(&sp->n_taps);
+                tbx = __ldg(&sp->tb); amask = __ldg(&sp->a_valid_mask);
+                a_bytes = __ldg(&sp->a_bytes); b_bytes = __ldg(&sp->b_bytes);
+                maps = P.maps + __ldg(&sp->map_base);
+                kh = __ldg(&sp->kh); kw = __ldg(&sp->kw); sh = __ldg(&sp->sh); sw = __ldg(&sp->sw);
+                ph = __ldg(&sp->ph); pw = __ldg(&sp->pw); dh = __ldg(&sp->dh); dw = __ldg(&sp->dw);
+            }
+            if (kind == WF_CONV) {
+                if (lane == 0) tr(item, 0);
+                const bool ok = wait_deps_warp(P, rec_dep0(cur), rec_ndep(cur), dep_cur, run, lane);
+                int fail = 0;
+                if (!ok) {
+                    if (lane == 0) atomicOr(P.status, 0x10u);
+                    fail = 1;
+                } else if (lane == 0) {
+                    tr(item, 1);
+                    asm volatile("fence.proxy.async;" ::: "memory");       // producers' generic-proxy writes -> our TMA reads
+                    const int ow0 = rec_tw(cur) * tw_valid;
+                    const int oh0 = oh_lo + (rec_tr(cur) << tr_log);
+                    const int n0 = rec_tn(cur) * (128 >> (p_log + tr_log));
+                    const int co0 = rec_cout(cur) * BN;
+                    for (int ch = 0; ch < n_chunks && !fail; ++ch) {
+                        if (mode == WF_SLAB) {
+                            // the whole receptive window of the tile in one box: its first tap's offset places it
+                            const int qh = -ph, qw = -pw;
+                            const int offh = floor_div_i(qh, sh), parh = qh - offh * sh;
+                            const int offw = floor_div_i(qw, sw), parw = qw - offw * sw;
+                            const int mi = parh * sw + parw;
+                            const bool have = (amask >> mi) & 1;
+                            if (!mbar_wait_abortable(empty_a + 8u * a_slot, a_phase ^ 1u, abort_flag)) { fail = 1; break; }
+                            const uint32_t fa = full_a + 8u * a_slot;
+                            mbar_expect_tx(fa, a_bytes);
+                            tma_load_4d(a0 + a_slot * a_slot_bytes, maps + mi, fa, ch * BK, have ? ow0 + offw : -65536,
+                                        have ? oh0 + offh : -65536, n0);
+                            if (++a_slot == (uint32_t)SA) { a_slot = 0; a_phase ^= 1u; }
+                            for (int t0 = 0; t0 < n_taps; t0 += tbx) {
+                                if (!mbar_wait_abortable(empty_b + 8u * b_slot, b_phase ^ 1u, abort_flag)) { fail = 1; break; }
+                                const uint32_t fb = full_b + 8u * b_slot;
+                                mbar_expect_tx(fb, b_bytes);
+                                tma_load_3d(b0 + b_slot * b_slot_bytes, maps + 4, fb, ch * BK, co0, t0);
+                                if (++b_slot == (uint32_t)SB) { b_slot = 0; b_phase ^= 1u; }
+                            }
+                        } else {
+                            for (int a = 0; a < kh && !fail; ++a) {
+                                const int qh = a * dh - ph;
+                                const int offh = floor_div_i(qh, sh), parh = qh - offh * sh;
+                                for (int b = 0; b < kw; ++b) {
+                                    const int qw = b * dw - pw;
+                                    const int offw = floor_div_i(qw, sw), parw = qw - offw * sw;
+                                    const int mi = parh * sw + parw;
+                                    const bool have = (amask >> mi) & 1;
+                                    if (!mbar_wait_abortable(empty_a + 8u * a_slot, a_phase ^ 1u, abort_flag) ||
+                                        !mbar_wait_abortable(empty_b + 8u * b_slot, b_phase ^ 1u, abort_flag)) { fail = 1; break; }
+                                    const uint32_t fa = full_a + 8u * a_slot, fb = full_b + 8u * b_slot;
+                                    mbar_expect_tx(fa, a_bytes);
+                                    tma_load_4d(a0 + a_slot * a_slot_bytes, maps + mi, fa, ch * BK, have ? ow0 + offw : -65536,
+                                                have ? oh0 + offh : -65536, n0);
+                                    mbar_expect_tx(fb, b_bytes);
+                                    tma_load_3d(b0 + b_slot * b_slot_bytes, maps + 4, fb, ch * BK, co0, a * kw + b);
+                                    if (++a_slot == (uint32_t)SA) { a_slot = 0; a_phase ^= 1u; }
+                                    if (++b_slot == (uint32_t)SB) { b_slot = 0; b_phase ^= 1u; }
+                                }
+                            }
                         }
                     }
+                    if (fail) atomicOr(P.status, 0x1u);
+                    tr(item, 2);
+                }
+                if (__any_sync(0xffffffffu, fail | (int)*abort_flag)) {
+                    if (lane == 0) {
+                        atomicExch(P.counters + 2, 1u);
+                        *abort_flag = 1;
+                    }
+                    break;
                 }
             }
-            if (fail) {
-                atomicExch(P.counters + 2, 1u);
-                *abort_flag = 1;
-            }
+            cur = nxt; dep_cur = dep_nxt; nxt = nn;
         }
     } else if (warp == 1) {
         if (lane == 0) {
             // ---------------- MMA issuer ----------------
-            StageCursor cur;
-            uint32_t slot = 0, phase = 0, cnt = 0;
-            int k_iters = 0, ksteps = 0;
-            uint32_t a_bytes = 0, idesc = 0, layout_code = 0, sbo = 0;
+            int item = blockIdx.x;
+            int4 cur = item < NI ? __ldg(&P.items[item]) : zero4;
+            int sidx = -1;
+            int kind = -1, mode = 0, n_chunks = 1, n_taps = 1, tbx = 1, kw = 1, dh = 1, dw = 1, p_log = 0, ksteps = 1;
+            uint32_t idesc = 0, desc_hi = 0, row_bytes = 0, tap_bytes = 0;
+            uint32_t a_slot = 0, a_phase = 0, b_slot = 0, b_phase = 0, cnt = 0;
             bool fail = false;
-            for (int item = blockIdx.x; item < P.n_items && !fail; item += G) {
-                if (cur.advance(P, item) && cur.kind == WF_CONV) {
-                    const WfStage *sp = &P.stages[cur.sidx];
-                    k_iters = __ldg(&sp->k_iters); ksteps = __ldg(&sp->BK) / 16;
-                    a_bytes = __ldg(&sp->a_bytes); idesc = __ldg(&sp->idesc);
-                    layout_code = __ldg(&sp->layout_code); sbo = __ldg(&sp->sbo_bytes);
+            for (; item < NI && !fail; item += G) {
+                const int4 nxt = item + G < NI ? __ldg(&P.items[item + G]) : zero4;
+                if (rec_stage(cur) != sidx) {
+                    sidx = rec_stage(cur);
+                    const WfStage *sp = &P.stages[sidx];
+                    kind = __ldg(&sp->kind); mode = __ldg(&sp->mode);
+                    n_chunks = __ldg(&sp->n_chunks); n_taps = __ldg(&sp->n_taps); tbx = __ldg(&sp->tb);
+                    kw = __ldg(&sp->kw); dh = __ldg(&sp->dh); dw = __ldg(&sp->dw); p_log = __ldg(&sp->p_log);
+                    ksteps = __ldg(&sp->BK) / 16;
+                    idesc = __ldg(&sp->idesc);
+                    desc_hi = ((__ldg(&sp->sbo_bytes) >> 4) & 0x3FFFu) | (1u << 14) | (__ldg(&sp->layout_code) << 29);
+                    row_bytes = __ldg(&sp->row_bytes);
+                    tap_bytes = (uint32_t)__ldg(&sp->BN) * row_bytes;
                 }
-                if (cur.kind != WF_CONV) continue;
-                const uint32_t buf = cnt & 1u;
-                if (!mbar_wait(acce0 + 8u * buf, ((cnt >> 1) & 1u) ^ 1u)) { fail = true; break; }
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t acc = tmem_base + buf * 256u;
-                for (int k = 0; k < k_iters; ++k) {
-                    if (*abort_flag || !mbar_wait(full0 + 8u * slot, phase)) { fail = true; break; }
+                if (kind == WF_CONV) {
+                    const uint32_t buf = cnt & 1u;
+                    if (!mbar_wait_abortable(acce0 + 8u * buf, ((cnt >> 1) & 1u) ^ 1u, abort_flag)) { fail = true; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    const uint32_t sa = base + slot * slot_bytes, sb = sa + a_bytes;
-                    for (int kk = 0; kk < ksteps; ++kk) {
-                        const uint64_t ad = smem_desc(sa + 32u * kk, sbo, layout_code);
-                        const uint64_t bd = smem_desc(sb + 32u * kk, sbo, layout_code);
-                        umma_bf16(acc, ad, bd, idesc, (k > 0 || kk > 0) ? 1u : 0u);
+                    tr(item, 3);
+                    const uint32_t acc = tmem_base + buf * 256u;
+                    uint32_t accumulate = 0;
+                    for (int ch = 0; ch < n_chunks && !fail; ++ch) {
+                        if (mode == WF_SLAB) {
+                            if (!mbar_wait_abortable(full_a + 8u * a_slot, a_phase, abort_flag)) { fail = true; break; }
+                            const uint32_t sa = a0 + a_slot * a_slot_bytes;
+                            for (int t0 = 0; t0 < n_taps; t0 += tbx) {
+                                if (!mbar_wait_abortable(full_b + 8u * b_slot, b_phase, abort_flag)) { fail = true; break; }
+                                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                                const uint32_t sb = b0 + b_slot * b_slot_bytes;
+                                const int t1 = min(t0 + tbx, n_taps);
+                                int ta = t0 / kw, tb = t0 - ta * kw;
+                                for (int t = t0; t < t1; ++t) {
+                                    // tap (ta, tb): the same box, read (ta*dh*P + tb*dw) pixels further on
+                                    const uint32_t pa = sa + (uint32_t)(((ta * dh) << p_log) + tb * dw) * row_bytes;
+                                    const uint32_t pb = sb + (uint32_t)(t - t0) * tap_bytes;
+                                    mma_tap(acc, pa, pb, desc_hi, idesc, ksteps, accumulate);
+                                    if (++tb == kw) { tb = 0; ++ta; }
+                                }
+                                umma_commit(empty_b + 8u * b_slot);
+                                if (++b_slot == (uint32_t)SB) { b_slot = 0; b_phase ^= 1u; }
+                            }
+                            umma_commit(empty_a + 8u * a_slot);
+                            if (++a_slot == (uint32_t)SA) { a_slot = 0; a_phase ^= 1u; }
+                        } else {
+                            for (int t = 0; t < n_taps; ++t) {
+                                if (!mbar_wait_abortable(full_a + 8u * a_slot, a_phase, abort_flag) ||
+                                    !mbar_wait_abortable(full_b + 8u * b_slot, b_phase, abort_flag)) { fail = true; break; }
+                                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                                const uint32_t sa = a0 + a_slot * a_slot_bytes, sb = b0 + b_slot * b_slot_bytes;
+                                mma_tap(acc, sa, sb, desc_hi, idesc, ksteps, accumulate);
+                                umma_commit(empty_a + 8u * a_slot);
+                                umma_commit(empty_b + 8u * b_slot);
+                                if (++a_slot == (uint32_t)SA) { a_slot = 0; a_phase ^= 1u; }
+                                if (++b_slot == (uint32_t)SB) { b_slot = 0; b_phase ^= 1u; }
+                            }
+                        }
                     }
-                    umma_commit(empty0 + 8u * slot);
-                    if (++slot == (uint32_t)S) { slot = 0; phase ^= 1u; }
+                    if (fail) break;
+                    umma_commit(accf0 + 8u * buf);
+                    tr(item, 4);
+                    ++cnt;
                 }
-                if (fail) break;
-                umma_commit(accf0 + 8u * buf);
-                ++cnt;
+                cur = nxt;
             }
             if (fail) {
                 atomicOr(P.status, 0x2u);
@@ -239,156 +389,187 @@ __global__ void __launch_bounds__(WF_THREADS, 1) wavefront_kernel(const WfParams
     } else {
         // ---------------- epilogue / SIMT warps ----------------
         const int tid = threadIdx.x - 64;
-        const int g = warp & 3;
-        StageCursor cur;
+        const int g = warp & 3;                               // TMEM lane group this warp may read
+        const int m = g * 32 + lane;                          // accumulator row = anchor of this thread
+        const int cgrp = (warp - 2) >> 2;                     // which share of the tile's 16-column chunks is this warp's
+        int item = blockIdx.x;
+        int4 cur = item < NI ? __ldg(&P.items[item]) : zero4;
+        int4 nxt = item + G < NI ? __ldg(&P.items[item + G]) : zero4;
+        int2 dep_cur = (warp == 2 && item < NI && lane < rec_ndep(cur)) ? __ldg(&P.deps[rec_dep0(cur) + lane]) : make_int2(0, 0);
+        int sidx = -1;
         uint32_t cnt = 0;
-        bool fail = false;
-        int first_item = 0, oh_lo = 0, oh_hi = 0, tw_log = 0, tr_log = 0, tiles_w = 1, tiles_n = 1, cout_tiles = 1, BN = 0,
-            dep_base = 0, ctr_base = 0;
+        int kind = -1, oh_lo = 0, oh_hi = 0, p_log = 0, tr_log = 0, tw_valid = 0, BN = 0, ctr_base = 0, gather_direct = 0;
         int N = 0, Hin = 0, Win = 0, Cin = 0, Ho = 0, Wo = 0, Cout = 0, kh = 1, kw = 1, sh = 1, sw = 1, ph = 0, pw = 0, dh = 1,
             dw = 1, act = 0, res_pos = 0;
         const void *xin = nullptr, *resp = nullptr;
         const float *scale = nullptr, *shift = nullptr;
         void *yout = nullptr;
-        for (int item = blockIdx.x; item < P.n_items; item += G) {
-            if (cur.advance(P, item)) {
-                const WfStage *sp = &P.stages[cur.sidx];
-                const WfLayer *lp = &P.layers[__ldg(&sp->layer)];
-                first_item = cur.first;
-                oh_lo = __ldg(&sp->oh_lo); oh_hi = __ldg(&sp->oh_hi); tw_log = __ldg(&sp->tw_log); tr_log = __ldg(&sp->tr_log);
-                tiles_w = __ldg(&sp->tiles_w); tiles_n = __ldg(&sp->tiles_n); cout_tiles = __ldg(&sp->cout_tiles);
-                BN = __ldg(&sp->BN); dep_base = __ldg(&sp->dep_base); ctr_base = __ldg(&sp->ctr_base);
-                N = __ldg(&lp->N); Hin = __ldg(&lp->Hin); Win = __ldg(&lp->Win); Cin = __ldg(&lp->Cin);
-                Ho = __ldg(&lp->Ho); Wo = __ldg(&lp->Wo); Cout = __ldg(&lp->Cout);
-                kh = __ldg(&lp->kh); kw = __ldg(&lp->kw); sh = __ldg(&lp->sh); sw = __ldg(&lp->sw);
-                ph = __ldg(&lp->ph); pw = __ldg(&lp->pw); dh = __ldg(&lp->dh); dw = __ldg(&lp->dw);
-                act = __ldg(&lp->act); res_pos = __ldg(&lp->res_pos);
-                xin = reinterpret_cast<const void *>(__ldg(reinterpret_cast<const unsigned long long *>(&lp->x)));
-                resp = reinterpret_cast<const void *>(__ldg(reinterpret_cast<const unsigned long long *>(&lp->res)));
-                scale = reinterpret_cast<const float *>(__ldg(reinterpret_cast<const unsigned long long *>(&lp->scale)));
-                shift = reinterpret_cast<const float *>(__ldg(reinterpret_cast<const unsigned long long *>(&lp->shift)));
-                yout = reinterpret_cast<void *>(__ldg(reinterpret_cast<const unsigned long long *>(&lp->y)));
+        for (; item < NI; item += G) {
+            const int4 nn = item + 2 * G < NI ? __ldg(&P.items[item + 2 * G]) : zero4;
+            const int2 dep_nxt =
+                (warp == 2 && item + G < NI && lane < rec_ndep(nxt)) ? __ldg(&P.deps[rec_dep0(nxt) + lane]) : make_int2(0, 0);
+            if (rec_stage(cur) != sidx) {
+                sidx = rec_stage(cur);
+                const WfStage *sp = &P.stages[sidx];
+                kind = __ldg(&sp->kind); gather_direct = __ldg(&sp->mode); oh_lo = __ldg(&sp->oh_lo); oh_hi = __ldg(&sp->oh_hi);
+                p_log = __ldg(&sp->p_log); tr_log = __ldg(&sp->tr_log); tw_valid = __ldg(&sp->tw_valid);
+                BN = __ldg(&sp->BN); ctr_base = __ldg(&sp->ctr_base);
+                N = __ldg(&sp->N); Hin = __ldg(&sp->Hin); Win = __ldg(&sp->Win); Cin = __ldg(&sp->Cin);
+                Ho = __ldg(&sp->Ho); Wo = __ldg(&sp->Wo); Cout = __ldg(&sp->Cout);
+                kh = __ldg(&sp->kh); kw = __ldg(&sp->kw); sh = __ldg(&sp->sh); sw = __ldg(&sp->sw);
+                ph = __ldg(&sp->ph); pw = __ldg(&sp->pw); dh = __ldg(&sp->dh); dw = __ldg(&sp->dw);
+                act = __ldg(&sp->act); res_pos = __ldg(&sp->res_pos);
+                xin = ldg_ptr<const void *>(&sp->x);
+                resp = ldg_ptr<const void *>(&sp->res);
+                scale = ldg_ptr<const float *>(reinterpret_cast<const void *const *>(&sp->scale));
+                shift = ldg_ptr<const float *>(reinterpret_cast<const void *const *>(&sp->shift));
+                yout = ldg_ptr<void *>(reinterpret_cast<const void *const *>(&sp->y));
             }
-            int q = item - first_item;
-            int tile_r;
-            if (cur.kind == WF_CONV) {
-                const int cout_tile = q % cout_tiles; q /= cout_tiles;
-                const int tile_w = q % tiles_w; q /= tiles_w;
-                const int tile_n = q % tiles_n;
-                tile_r = q / tiles_n;
+            const int tile_r = rec_tr(cur);
+            if (tid == 0) tr(item, 7);
+            if (kind == WF_CONV) {
                 const uint32_t buf = cnt & 1u;
-                const int TW = 1 << tw_log, TR = 1 << tr_log;
-                const int m = g * 32 + lane;
-                const int ow = (tile_w << tw_log) + (m & (TW - 1));
-                const int oh = oh_lo + (tile_r << tr_log) + ((m >> tw_log) & (TR - 1));
-                const int n = tile_n * (128 >> (tw_log + tr_log)) + (m >> (tw_log + tr_log));
-                const bool valid = ow < Wo && oh < oh_hi && n < N;
-                const int co0 = cout_tile * BN;
-                const long long pix = (((long long)n * Ho + oh) * Wo + ow) * Cout + co0;
-                // this tile's scale/shift into shared memory while the main loop is still running
-                epi_bar();                                           // previous item's readers are done
-                for (int i = tid; i < BN; i += EPI_THREADS) {
+                const int c = m & ((1 << p_log) - 1);
+                const int r = (m >> p_log) & ((1 << tr_log) - 1);
+                const int ow = rec_tw(cur) * tw_valid + c;
+                const int oh = oh_lo + (tile_r << tr_log) + r;
+                const int n = rec_tn(cur) * (128 >> (p_log + tr_log)) + (m >> (p_log + tr_log));
+                const bool valid = c < tw_valid && ow < Wo && oh < oh_hi && n < N;
+                const int co0 = rec_cout(cur) * BN;
+                if (cgrp == 0) row_pix[m] = valid ? (((long long)n * Ho + oh) * Wo + ow) * Cout + co0 : -1LL;
+                for (int i = tid; i < BN; i += EPI_THREADS) {          // this tile's scale/shift while the main loop runs
                     s_scale[i] = scale ? __ldg(scale + co0 + i) : 1.0f;
                     s_shift[i] = shift ? __ldg(shift + co0 + i) : 0.0f;
                 }
                 epi_bar();
-                if (!mbar_wait(accf0 + 8u * buf, (cnt >> 1) & 1u)) fail = true;
+                const int cpr = BN >> 3;                               // 16-byte chunks per staged row
+                const int cpr_log = (cpr & (cpr - 1)) == 0 ? 31 - __clz(cpr) : -1;
+                const uint32_t row_stride = (uint32_t)BN * 2u;
+                const int swz = (cpr & 7) == 0 ? 7 : 0;                // chunk position = chunk ^ (row & 7): conflict-free columns
+                __nv_bfloat16 *y = static_cast<__nv_bfloat16 *>(yout);
+                if (!mbar_wait_abortable(accf0 + 8u * buf, (cnt >> 1) & 1u, abort_flag)) *epi_fail = 1;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                if (!fail) {
-                    __nv_bfloat16 *y = static_cast<__nv_bfloat16 *>(yout);
+                if (tid == 0) tr(item, 5);
+                // (only now: the finished accumulator implies that warp 0 saw this item's producers, the residual's included)
+                if (resp) {
+                    // residual tile -> staging, coalesced; produced inside this launch by other SMs: read through L2
                     const __nv_bfloat16 *res = static_cast<const __nv_bfloat16 *>(resp);
+#pragma unroll 4
+                    for (int idx = tid; idx < 128 * cpr; idx += EPI_THREADS) {
+                        const int row = cpr_log >= 0 ? idx >> cpr_log : idx / cpr, j = idx - row * cpr;
+                        const long long rp = row_pix[row];
+                        if (rp >= 0)
+                            *reinterpret_cast<uint4 *>(stg + row * row_stride + ((j ^ (row & swz)) << 4)) =
+                                __ldcg(reinterpret_cast<const uint4 *>(res + rp) + j);
+                    }
+                    epi_bar();
+                }
+                {
                     const uint32_t acc = tmem_base + buf * 256u + ((uint32_t)(g * 32) << 16);
-                    for (int j = 0; j < BN; j += 16) {
-                        uint32_t r[16];
-                        tmem_ld16(acc + (uint32_t)j, r);
+                    uint8_t *my_row = stg + m * row_stride;
+                    for (int j = 16 * cgrp; j < BN; j += 16 * COL_GROUPS) {
+                        uint32_t rr[16];
+                        tmem_ld16(acc + (uint32_t)j, rr);
                         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                        if (tid == 0 && j == 0) tr(item, 8);
+                        if (tid == 0 && j == 16 * COL_GROUPS) tr(item, 10);
                         if (!valid) continue;
                         float v[16];
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) v[i] = fmaf(s_scale[j + i], __uint_as_float(r[i]), s_shift[j + i]);
-                        if (res) {
-                            // produced inside this launch by other SMs: read through L2, never a stale L1 line
-                            const uint4 q0 = __ldcg(reinterpret_cast<const uint4 *>(res + pix + j));
-                            const uint4 q1 = __ldcg(reinterpret_cast<const uint4 *>(res + pix + j + 8));
+                        for (int i = 0; i < 16; ++i) v[i] = fmaf(s_scale[j + i], __uint_as_float(rr[i]), s_shift[j + i]);
+                        uint4 *c0p = reinterpret_cast<uint4 *>(my_row + ((((j >> 3)) ^ (m & swz)) << 4));
+                        uint4 *c1p = reinterpret_cast<uint4 *>(my_row + ((((j >> 3) + 1) ^ (m & swz)) << 4));
+                        float rv[16];
+                        if (resp) {
+                            const uint4 q0 = *c0p, q1 = *c1p;
                             const uint32_t rw[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
-                            float rv[16];
 #pragma unroll
                             for (int i = 0; i < 8; ++i) {
                                 rv[2 * i] = __uint_as_float(rw[i] << 16);
                                 rv[2 * i + 1] = __uint_as_float(rw[i] & 0xFFFF0000u);
                             }
-                            if (res_pos == LOP_RES_PRE_ACT) {
-#pragma unroll
-                                for (int i = 0; i < 16; ++i) v[i] = activate(v[i] + rv[i], act);
-                            } else {
-#pragma unroll
-                                for (int i = 0; i < 16; ++i) v[i] = activate(v[i], act) + rv[i];
-                            }
-                        } else {
-#pragma unroll
-                            for (int i = 0; i < 16; ++i) v[i] = activate(v[i], act);
                         }
+                        finish16(v, rv, resp ? res_pos : LOP_RES_NONE, act);
                         uint32_t o[8];
 #pragma unroll
                         for (int i = 0; i < 8; ++i) {
                             const __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
                             o[i] = *reinterpret_cast<const uint32_t *>(&h);
                         }
-                        *reinterpret_cast<uint4 *>(y + pix + j) = make_uint4(o[0], o[1], o[2], o[3]);
-                        *reinterpret_cast<uint4 *>(y + pix + j + 8) = make_uint4(o[4], o[5], o[6], o[7]);
+                        *c0p = make_uint4(o[0], o[1], o[2], o[3]);
+                        *c1p = make_uint4(o[4], o[5], o[6], o[7]);
+                        if (tid == 0 && j == 0) tr(item, 9);
                     }
                 }
                 asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-                __threadfence();
-                epi_bar();
-                if (tid == 0 && !fail)
-                    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(acce0 + 8u * buf) : "memory");
+                if (tid == 0) tr(item, 11);
+                epi_bar();                                             // accumulator drained, staging tile complete
+                if (tid == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(acce0 + 8u * buf) : "memory");
                 ++cnt;
+                if (!*epi_fail) {
+                    // staged rows -> global: consecutive threads write consecutive 16 bytes of a pixel's channels
+#pragma unroll 4
+                    for (int idx = tid; idx < 128 * cpr; idx += EPI_THREADS) {
+                        const int row = cpr_log >= 0 ? idx >> cpr_log : idx / cpr, j = idx - row * cpr;
+                        const long long rp = row_pix[row];
+                        if (rp >= 0)
+                            *(reinterpret_cast<uint4 *>(y + rp) + j) =
+                                *reinterpret_cast<const uint4 *>(stg + row * row_stride + ((j ^ (row & swz)) << 4));
+                    }
+                }
+                if (tid == 0) tr(item, 12);
             } else {
-                // pooling or channel padding: a chunk of one output row of one image per item, all 128 threads
-                const int chunk = q % tiles_w; q /= tiles_w;
-                const int n = q % tiles_n;
-                tile_r = q / tiles_n;
+                // pooling or patch gather: one output row of one image per item, all worker threads
+                if (warp == 2 && !wait_deps_warp(P, rec_dep0(cur), rec_ndep(cur), dep_cur, run, lane) && lane == 0) *epi_fail = 1;
+                epi_bar();
+                if (tid == 0) tr(item, 1);
+                const int n = rec_tn(cur);
                 const int oh = oh_lo + tile_r;
-                if (!wait_deps(P, dep_base + tile_r, run)) fail = true;
-                if (!fail && cur.kind == WF_POOL) {
-                    // 2 channel-group vectors per thread, up to 3 taps of each in flight at once
+                if (*epi_fail) {
+                    // fall through to the common exit below
+                } else if (kind == WF_POOL) {
                     const int cg = Cin >> 3;
                     const int total = Wo * cg;
                     const __nv_bfloat16 *x = static_cast<const __nv_bfloat16 *>(xin);
                     __nv_bfloat16 *y = static_cast<__nv_bfloat16 *>(yout);
-                    int idx[2], gch[2], ow[2];
-                    float mx[2][8];
+                    // two channel-group vectors per thread
+                    for (int idx0 = 0; idx0 < total; idx0 += 2 * EPI_THREADS) {
+                        int gch[2], ow[2];
+                        bool live[2];
+                        float mx[2][8];
 #pragma unroll
-                    for (int u = 0; u < 2; ++u) {
-                        idx[u] = chunk * (2 * EPI_THREADS) + u * EPI_THREADS + tid;
-                        gch[u] = idx[u] % cg;
-                        ow[u] = idx[u] / cg;
+                        for (int u = 0; u < 2; ++u) {
+                            const int idx = idx0 + u * EPI_THREADS + tid;
+                            live[u] = idx < total;
+                            ow[u] = idx / cg;
+                            gch[u] = idx - ow[u] * cg;
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) mx[u][i] = -INFINITY;
-                    }
-                    for (int a = 0; a < kh; ++a) {
-                        const int ih = oh * sh - ph + a * dh;
-                        if (ih < 0 || ih >= Hin) continue;
-                        const long long rowbase = ((long long)n * Hin + ih) * Win;
-                        for (int b0 = 0; b0 < kw; b0 += 3) {
-                            uint4 q4[2][3];
-                            bool ok[2][3];
+                            for (int i = 0; i < 8; ++i) mx[u][i] = -INFINITY;
+                        }
+                        const int nt = kh * kw;
+                        for (int t0 = 0; t0 < nt; t0 += 4) {                 // four filter taps of both vectors in flight
+                            uint4 q4[2][4];
+                            bool ok[2][4];
 #pragma unroll
-                            for (int u = 0; u < 2; ++u)
+                            for (int tt = 0; tt < 4; ++tt) {
+                                const int t = t0 + tt;
+                                const int a = t / kw, b = t - a * kw;
+                                const int ih = oh * sh - ph + a * dh;
+                                const bool rowok = t < nt && ih >= 0 && ih < Hin;
+                                const long long rowbase = ((long long)n * Hin + ih) * Win;
 #pragma unroll
-                                for (int bb = 0; bb < 3; ++bb) {
-                                    const int iw = ow[u] * sw - pw + (b0 + bb) * dw;
-                                    ok[u][bb] = idx[u] < total && b0 + bb < kw && iw >= 0 && iw < Win;
-                                    if (ok[u][bb])
-                                        q4[u][bb] = __ldcg(reinterpret_cast<const uint4 *>(x + (rowbase + iw) * Cin + gch[u] * 8));
+                                for (int u = 0; u < 2; ++u) {
+                                    const int iw = ow[u] * sw - pw + b * dw;
+                                    ok[u][tt] = live[u] && rowok && iw >= 0 && iw < Win;
+                                    if (ok[u][tt]) q4[u][tt] = __ldcg(reinterpret_cast<const uint4 *>(x + (rowbase + iw) * Cin + gch[u] * 8));
                                 }
+                            }
 #pragma unroll
                             for (int u = 0; u < 2; ++u)
 #pragma unroll
-                                for (int bb = 0; bb < 3; ++bb)
-                                    if (ok[u][bb]) {
-                                        const uint32_t w4[4] = {q4[u][bb].x, q4[u][bb].y, q4[u][bb].z, q4[u][bb].w};
+                                for (int tt = 0; tt < 4; ++tt)
+                                    if (ok[u][tt]) {
+                                        const uint32_t w4[4] = {q4[u][tt].x, q4[u][tt].y, q4[u][tt].z, q4[u][tt].w};
 #pragma unroll
                                         for (int i = 0; i < 4; ++i) {
                                             mx[u][2 * i] = fmaxf(mx[u][2 * i], __uint_as_float(w4[i] << 16));
@@ -396,37 +577,104 @@ __global__ void __launch_bounds__(WF_THREADS, 1) wavefront_kernel(const WfParams
                                         }
                                     }
                         }
+#pragma unroll
+                        for (int u = 0; u < 2; ++u)
+                            if (live[u]) {
+                                uint32_t o[4];
+#pragma unroll
+                                for (int i = 0; i < 4; ++i)      // values are bf16 already: truncation is exact
+                                    o[i] = (__float_as_uint(mx[u][2 * i]) >> 16) | (__float_as_uint(mx[u][2 * i + 1]) & 0xFFFF0000u);
+                                *reinterpret_cast<uint4 *>(y + (((long long)n * Ho + oh) * Wo + ow[u]) * Cin + gch[u] * 8) =
+                                    make_uint4(o[0], o[1], o[2], o[3]);
+                            }
                     }
-#pragma unroll
-                    for (int u = 0; u < 2; ++u)
-                        if (idx[u] < total) {
-                            uint32_t o[4];
-#pragma unroll
-                            for (int i = 0; i < 4; ++i)      // values are bf16 already: truncation is exact
-                                o[i] = (__float_as_uint(mx[u][2 * i]) >> 16) | (__float_as_uint(mx[u][2 * i + 1]) & 0xFFFF0000u);
-                            *reinterpret_cast<uint4 *>(y + (((long long)n * Ho + oh) * Wo + ow[u]) * Cin + gch[u] * 8) =
-                                make_uint4(o[0], o[1], o[2], o[3]);
-                        }
-                } else if (!fail) {
-                    // channel padding: Cin real channels -> 16, one pixel per thread
+                } else {
+                    // patch gather: Cout holds the patch length Kcol; x is the chain input, possibly still arriving
+                    GatherGeom gg;
+                    gg.N = N; gg.H = Hin; gg.W = Win; gg.C = Cin; gg.Ho = Ho; gg.Wo = Wo; gg.Kcol = Cout;
+                    gg.kh = kh; gg.kw = kw; gg.sh = sh; gg.sw = sw; gg.ph = ph; gg.pw = pw; gg.dh = dh; gg.dw = dw;
+                    const int k8n = Cout >> 3;
+                    const int total = Wo * k8n;
                     const uint16_t *x = static_cast<const uint16_t *>(xin);
                     uint16_t *y = static_cast<uint16_t *>(yout);
-                    const long long row = ((long long)n * Hin + oh) * Win;
-                    const int px = chunk * EPI_THREADS + tid;
-                    if (px < Win) {
-                        const uint16_t *src = x + (row + px) * Cin;
-                        uint32_t h[16];
+                    if (gather_direct) {
+                        for (int idx = tid; idx < total; idx += EPI_THREADS) {
+                            const int ow = idx / k8n, k8 = idx - ow * k8n;
+                            *reinterpret_cast<uint4 *>(y + (((long long)n * Ho + oh) * Wo + ow) * Cout + k8 * 8) =
+                                gather8<true>(x, gg, n, oh, ow, k8);
+                        }
+                    } else {
+                        // the kh image rows this output row reads, copied once into the staging tile with 16-byte
+                        // loads (around L1: the rows may have arrived while the kernel was running), then the
+                        // patches are put together from shared memory
+                        const int row_bytes_in = Win * Cin * 2;
+                        const int pitch = (row_bytes_in + 31 + 15) & ~15;
+                        const long long tensor_bytes = (long long)N * Hin * row_bytes_in;
+                        int *s_mis = reinterpret_cast<int *>(row_pix);       // per filter row: byte offset of the row's first element in staging, or -1
+                        const uint8_t *xb = reinterpret_cast<const uint8_t *>(x);
+                        const int nvec_max = (row_bytes_in + 30) >> 4;
+                        for (int idx = tid; idx < kh * nvec_max; idx += EPI_THREADS) {
+                            const int a = idx / nvec_max, v = idx - a * nvec_max;
+                            const int ih = oh * sh - ph + a * dh;
+                            const bool have = ih >= 0 && ih < Hin;
+                            const long long off = ((long long)n * Hin + ih) * row_bytes_in;
+                            const int mis = (int)(off & 15);
+                            if (v == 0) s_mis[a] = have ? a * pitch + mis : -1;
+                            if (!have || v >= ((mis + row_bytes_in + 15) >> 4)) continue;
+                            const long long off_al = off - mis;
+                            uint4 q;
+                            if (off_al + 16LL * (v + 1) <= tensor_bytes) {
+                                q = __ldcg(reinterpret_cast<const uint4 *>(xb + off_al) + v);
+                            } else {                                          // the tensor ends inside this vector
+                                uint32_t h[8];
 #pragma unroll
-                        for (int ch = 0; ch < 16; ++ch) h[ch] = ch < Cin ? (uint32_t)src[ch] : 0u;
-                        uint4 *dst = reinterpret_cast<uint4 *>(y + (row + px) * 16);
-                        dst[0] = make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), h[4] | (h[5] << 16), h[6] | (h[7] << 16));
-                        dst[1] = make_uint4(h[8] | (h[9] << 16), h[10] | (h[11] << 16), h[12] | (h[13] << 16), h[14] | (h[15] << 16));
+                                for (int e = 0; e < 8; ++e) {
+                                    const long long o = off_al + 16LL * v + 2 * e;
+                                    h[e] = o < tensor_bytes ? (uint32_t)__ldcg(reinterpret_cast<const uint16_t *>(xb + o)) : 0u;
+                                }
+                                q = make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), h[4] | (h[5] << 16), h[6] | (h[7] << 16));
+                            }
+                            *reinterpret_cast<uint4 *>(stg + a * pitch + 16 * v) = q;
+                        }
+                        // per patch element: filter row << 16 | element offset inside that row's run of kw*C values, or -1
+                        int *tab = reinterpret_cast<int *>(stg + kh * pitch);
+                        const int klen = kh * kw * Cin;
+                        for (int k = tid; k < Cout; k += EPI_THREADS) {
+                            int t = -1;
+                            if (k < klen) {
+                                const int tap = k / Cin, ci = k - tap * Cin;
+                                const int a = tap / kw, b = tap - a * kw;
+                                t = (a << 16) | (b * dw * Cin + ci);
+                            }
+                            tab[k] = t;
+                        }
+                        epi_bar();
+                        const int row_elems = Win * Cin;
+                        for (int idx = tid; idx < total; idx += EPI_THREADS) {
+                            const int ow = idx / k8n, k8 = idx - ow * k8n;
+                            const int base_e = (ow * sw - pw) * Cin;                  // first element of the pixel's runs
+                            const int4 t0 = *reinterpret_cast<const int4 *>(tab + k8 * 8);
+                            const int4 t1 = *reinterpret_cast<const int4 *>(tab + k8 * 8 + 4);
+                            const int tt[8] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
+                            uint32_t h[8];
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) {
+                                const int fa = tt[e] >> 16, src = base_e + (tt[e] & 0xFFFF);
+                                const int rowoff = s_mis[fa < 0 ? 0 : fa];          // byte offset of the row in staging, or -1
+                                const bool ok = tt[e] >= 0 && rowoff >= 0 && src >= 0 && src < row_elems;
+                                h[e] = ok ? (uint32_t)*reinterpret_cast<const uint16_t *>(stg + rowoff + src * 2) : 0u;
+                            }
+                            *reinterpret_cast<uint4 *>(y + (((long long)n * Ho + oh) * Wo + ow) * Cout + k8 * 8) =
+                                make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), h[4] | (h[5] << 16), h[6] | (h[7] << 16));
+                        }
                     }
                 }
-                __threadfence();
-                epi_bar();
             }
-            if (fail) {
+            if (kind != WF_CONV && lane == 0 && warp < 6) tr(item, 8 + (warp - 2) + (warp == 5 ? 2 : 0));   // 8, 9, 10, 13
+            __threadfence();
+            if (kind != WF_CONV && tid == 0) tr(item, 12);
+            epi_bar();
+            if (*epi_fail) {                                           // uniform: written only before the barrier above
                 if (tid == 0) {
                     atomicOr(P.status, 0x4u);
                     atomicExch(P.counters + 2, 1u);
@@ -434,7 +682,11 @@ __global__ void __launch_bounds__(WF_THREADS, 1) wavefront_kernel(const WfParams
                 }
                 break;
             }
-            if (tid == 0) atomicAdd(P.counters + ctr_base + tile_r, 1u);      // release: stores fenced above
+            if (tid == 0) {
+                atomicAdd(P.counters + ctr_base + tile_r, 1u);        // release: stores fenced above
+                tr(item, 6);
+            }
+            cur = nxt; dep_cur = dep_nxt; nxt = nn;
         }
     }
 
@@ -455,16 +707,46 @@ __global__ void __launch_bounds__(WF_THREADS, 1) wavefront_kernel(const WfParams
     }
 }
 
+#ifdef LOP_WF_TRACE
+static WfParams g_last_params;
+#endif
+
 }  // namespace
 
-size_t wavefront_smem_bytes(int ring, uint32_t slot_bytes)
+#ifdef LOP_WF_TRACE
+extern "C" int lop_debug_last_stages(void *host, int max_stages)
 {
-    return 1024 + (size_t)ring * slot_bytes + 16 * (size_t)ring + 64 + 2 * 256 * sizeof(float) + 64;
+    const int n = g_last_params.n_stages < max_stages ? g_last_params.n_stages : max_stages;
+    if (cudaMemcpy(host, g_last_params.stages, (size_t)n * sizeof(WfStage), cudaMemcpyDeviceToHost) != cudaSuccess) return -1;
+    return n;
+}
+extern "C" int lop_debug_last_items(void *host, int max_items)
+{
+    const int n = g_last_params.n_items < max_items ? g_last_params.n_items : max_items;
+    if (cudaMemcpy(host, g_last_params.items, (size_t)n * sizeof(int4), cudaMemcpyDeviceToHost) != cudaSuccess) return -1;
+    return n;
+}
+extern "C" int lop_debug_trace_copy(void *host, size_t bytes, int clear)
+{
+    if (bytes > sizeof(unsigned long long) * TRACE_ITEMS * 16) bytes = sizeof(unsigned long long) * TRACE_ITEMS * 16;
+    if (clear) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_wf_trace) != cudaSuccess) return -1;
+        return cudaMemset(p, 0, sizeof(unsigned long long) * TRACE_ITEMS * 16) == cudaSuccess ? 0 : -1;
+    }
+    return cudaMemcpyFromSymbol(host, g_wf_trace, bytes) == cudaSuccess ? 0 : -1;
+}
+#endif
+
+size_t wavefront_smem_bytes(const WfParams &p)
+{
+    return 1024 + (size_t)p.sa * p.a_slot_bytes + (size_t)p.sb * p.b_slot_bytes + p.stg_bytes + 8 * (size_t)(2 * p.sa + 2 * p.sb + 4) + 64 +
+           2 * 256 * sizeof(float) + 128 * sizeof(long long) + 64;
 }
 
 cudaError_t launch_wavefront(const WfParams &p, int grid, cudaStream_t s)
 {
-    const size_t smem = wavefront_smem_bytes(p.ring, p.slot_bytes);
+    const size_t smem = wavefront_smem_bytes(p);
     static bool configured = false;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(wavefront_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
@@ -472,6 +754,9 @@ cudaError_t launch_wavefront(const WfParams &p, int grid, cudaStream_t s)
         configured = true;
     }
     if (smem > 227 * 1024) return cudaErrorInvalidValue;
+#ifdef LOP_WF_TRACE
+    g_last_params = p;
+#endif
     wavefront_kernel<<<grid, WF_THREADS, smem, s>>>(p);
     return cudaGetLastError();
 }

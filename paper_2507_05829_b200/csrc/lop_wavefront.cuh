@@ -2,9 +2,10 @@
 //
 // Sec. III-A / IV-B of the paper: the operations of later layers start as soon as the rows they
 // depend on exist, without waiting for the whole earlier layer.  A *program* is the topologically
-// ordered list of stages of one launch; every stage is cut into items (output tiles); resident
-// CTAs take items round-robin in program order and an item waits -- with a bounded spin -- only
-// for the producer row groups its receptive field touches.
+// ordered list of stages of one launch; every stage is cut into items (output tiles of a
+// convolution, output rows of a pooling or patch-gather stage); resident CTAs take items
+// round-robin in program order and an item waits -- with a bounded spin -- only for the producer
+// row groups its receptive field touches.
 #pragma once
 #include <cuda.h>
 #include <cuda_runtime.h>
@@ -12,58 +13,65 @@
 
 namespace lop {
 
-enum WfKind { WF_PAD = 0, WF_CONV = 1, WF_POOL = 2 };
+enum WfKind { WF_GATHER = 0, WF_CONV = 1, WF_POOL = 2 };
+// How a convolution stage feeds the tensor cores.
+//   WF_SLAB  one activation box per channel chunk: the output tile's receptive window (tile plus halo),
+//            laid out in shared memory as rows of P pixels; every filter tap is the same box read at a
+//            shifted start address.  Weights arrive as boxes of several taps.
+//   WF_TAP   one activation box and one weight box per (channel chunk, tap): strided windows and
+//            channel chunks narrower than 64.
+enum WfMode { WF_SLAB = 0, WF_TAP = 1 };
 
-// One operator instance with its tensors bound (device pointers).
-struct WfLayer {
+// One (band, layer) stage: rows [oh_lo, oh_hi) of a bound operator.
+struct WfStage {
+    int kind, mode;
+    int oh_lo, oh_hi;
+    int ctr_base;             // counters[ctr_base + tile_r]: finished items of that row group
+    // convolution tile: accumulator row m is the anchor at column m & (P-1), row (m >> p_log) & (TR-1),
+    // image m >> (p_log + tr_log) of the tile; columns >= tw_valid are the slab's halo gap and are dropped
+    int p_log, tr_log, tw_valid;
+    int BN, BK, n_chunks, n_taps, tb;     // tb: taps per weight box
+    int map_base;             // first of 5 tensor maps (4 activation parity classes + weights)
+    int a_valid_mask;
+    uint32_t a_bytes, b_bytes;            // bytes of one activation / weight box
+    uint32_t idesc, layout_code, sbo_bytes, row_bytes;
+    // the operator, with its tensors bound (a gathered stem appears as the pointwise convolution it runs as)
+    int N, Hin, Win, Cin, Ho, Wo, Cout;
+    int kh, kw, sh, sw, ph, pw, dh, dw;
+    int act, res_pos;
     const void *x;            // main input, full-size NHWC tensor
     const void *res;          // residual tensor or nullptr
     const float *scale, *shift;
     void *y;                  // full-size output
-    int N, Hin, Win, Cin, Ho, Wo, Cout;
-    int kh, kw, sh, sw, ph, pw, dh, dw;
-    int act, res_pos;
-    int pad_[5];
+    int pad_[16];
 };
-static_assert(sizeof(WfLayer) == 128, "WfLayer is copied as 32 words");
+static_assert(sizeof(WfStage) == 256, "WfStage layout");
 
-// One (band, layer) stage: rows [oh_lo, oh_hi) of a layer, cut into n_items tiles.
-struct WfStage {
-    int kind, layer;
-    int oh_lo, oh_hi;
-    int first_item, n_items;
-    int tw_log, tr_log;       // conv tile = TN images x 2^tr_log rows x 2^tw_log columns (128 pixels)
-    int tiles_w, tiles_r, tiles_n, cout_tiles;
-    int BN, BK;
-    int map_base;             // first of 5 tensor maps (4 activation parity classes + weights)
-    int a_valid_mask;
-    int dep_base;             // dep_index[dep_base + tile_r] = (first, count) into the dependency list
-    int ctr_base;             // counters[ctr_base + tile_r]: completed tiles of that row group
-    int k_iters;
-    uint32_t a_bytes, b_bytes, idesc, layout_code, sbo_bytes;
-    int pad_[8];
-};
-static_assert(sizeof(WfStage) == 128, "WfStage is copied as 32 words");
-
+// One item, 16 bytes: x = stage | cout_tile << 16, y = tile_w | tile_n << 16, z = tile_r | dep_count << 20,
+// w = first entry of its dependency list.
 struct WfParams {
     const WfStage *stages;
-    const WfLayer *layers;
+    const int4 *items;
     const CUtensorMap *maps;
-    const int2 *dep_index;    // per (stage, tile_r): first, count
-    const int2 *deps;         // (counter index, completions expected per run)
+    const int2 *deps;         // (counter index, completions expected per run); y < 0: an arrival flag, target -y
     unsigned *counters;       // [0] runs completed, [1] CTAs finished, [2] abort, [4..] row-group counters,
                               // then n_flags band-arrival flags (set by the copy stream, cleared at run end)
     int flag_base, n_flags;
     unsigned *status;
     int n_stages, n_items;
-    int ring;                 // pipeline depth
-    uint32_t slot_bytes;      // bytes of one ring slot (activation tile + weight tile)
+    int sa, sb;               // slots of the activation / weight ring
+    uint32_t a_slot_bytes, b_slot_bytes, stg_bytes;
 };
 
-constexpr int WF_THREADS = 192;
+#ifndef LOP_WF_WORKER_WARPS
+#define LOP_WF_WORKER_WARPS 8
+#endif
+constexpr int WF_WORKER_WARPS = LOP_WF_WORKER_WARPS;      // epilogue / SIMT warps (a multiple of 4)
+constexpr int WF_THREADS = 64 + 32 * WF_WORKER_WARPS;
 constexpr int WF_CTR_FIRST = 4;
+constexpr int WF_MAX_DEPS = 4095;
 
-size_t wavefront_smem_bytes(int ring, uint32_t slot_bytes);
+size_t wavefront_smem_bytes(const WfParams &p);
 cudaError_t launch_wavefront(const WfParams &p, int grid, cudaStream_t s);
 
 }  // namespace lop
