@@ -97,8 +97,10 @@ typedef struct {
 /* Times of the last lop_run_pipelined call, in milliseconds (see lop_plan_last_timing). */
 typedef struct {
     float total_ms;        /* first enqueued operation to last, on the caller's stream            */
-    float copy_ms;         /* sum of the band copies' own durations (copy-stream events)          */
-    float first_copy_ms;   /* duration of band 0's copy: it can never be hidden                   */
+    float copy_ms;         /* sum of the band copies' own durations (copy-stream events); 0 unless
+                              the plan has LOP_FLAG_TIME_LAYERS: timing events on the side stream
+                              cost more than a small band's copy, so the fast path records none  */
+    float first_copy_ms;   /* duration of band 0's copy (it can never be hidden); 0 likewise       */
     int32_t n_copies;
     int32_t reserved;
 } lop_timing;
@@ -154,8 +156,10 @@ int lop_run_banded(lop_plan_t *plan, const void *in_dev, void *out_dev, void *wo
  * in_host_pinned (PINNED HOST, full-size tensor) to the same rows of staging_dev. */
 int lop_copy_band(lop_plan_t *plan, int band, const void *in_host_pinned, void *staging_dev, void *stream);
 /* Band pipeline (Sec. IV-B computation/transmission overlap): band i+1's rows are copied on the
- * plan's side stream while band i is computed on the caller's stream; CUDA events carry the
- * dependencies.  Returns after enqueueing.  staging_dev: lop_plan_staging_bytes() bytes. */
+ * plan's side stream while band i is computed on the caller's stream.  CUDA events fork and join
+ * the side stream; inside the run a band's arrival is a 4-byte stream-ordered write behind its
+ * copy that the persistent kernel polls (per-layer launches wait on one event per band instead).
+ * Returns after enqueueing.  staging_dev: lop_plan_staging_bytes() bytes. */
 int lop_run_pipelined(lop_plan_t *plan, const void *in_host_pinned, void *staging_dev, void *out_dev,
                       void *workspace, void *stream);
 /* Event times of the last lop_run_pipelined call.  SYNCHRONISES with that call's completion. */

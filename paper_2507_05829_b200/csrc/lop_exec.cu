@@ -6,6 +6,7 @@
 // computation.  Here the "transmission" is an asynchronous pinned-host -> device copy on a side
 // stream, the dependency "input has arrived" is a CUDA event, and tensor "combining" is
 // addressing: every band writes its rows straight into full-size tensors.
+#include <cuda.h>
 #include <cuda_runtime.h>
 
 #include <algorithm>
@@ -39,10 +40,13 @@ struct ProgKey {
 struct ExecState {
     std::map<ProgKey, Program *> programs;
     bool wavefront = false;
-    cudaStream_t copy_stream = nullptr;
+    cudaStream_t copy_stream = nullptr;                        // the side stream of the transfers
+    cudaStream_t signal_stream = nullptr;                      // performs the arrival writes of the single-launch pipeline
+    cudaEvent_t ev_signal_join = nullptr;
     cudaEvent_t ev_fork = nullptr, ev_begin = nullptr, ev_end = nullptr, ev_join = nullptr;
     unsigned *pinned_one = nullptr;                            // pinned host word holding 1: source of arrival flags
     std::vector<cudaEvent_t> ev_copy_start, ev_copy_end;       // [band]
+    std::vector<cudaEvent_t> ev_arrive;                        // [band], no timing
     std::vector<cudaEvent_t> ev_layer;                         // [(band+1) * L + layer] * 2, slot 0 = whole
     std::vector<char> layer_timed;
     std::map<MapKey, ConvTcMaps> maps;
@@ -52,6 +56,9 @@ struct ExecState {
     int launches = 0;                                          // kernels enqueued by the last execution call
     int copies = 0;                                            // async copies enqueued by it
     bool timing_valid = false;
+    std::map<std::tuple<const void *, const void *, const void *, const void *>, cudaGraphExec_t> pipe_graphs;   // (host, staging, out, ws)
+    cudaStream_t capture_stream = nullptr;
+    bool copies_timed = false;                                 // per-band copy events were recorded by the last pipelined run
     std::vector<char> copy_issued;
 };
 
@@ -59,12 +66,17 @@ void exec_destroy(ExecState *e)
 {
     if (!e) return;
     if (e->copy_stream) cudaStreamDestroy(e->copy_stream);
+    if (e->signal_stream) cudaStreamDestroy(e->signal_stream);
+    if (e->ev_signal_join) cudaEventDestroy(e->ev_signal_join);
     if (e->pinned_one) cudaFreeHost(e->pinned_one);
     for (cudaEvent_t ev : {e->ev_fork, e->ev_begin, e->ev_end, e->ev_join})
         if (ev) cudaEventDestroy(ev);
-    for (auto &v : {&e->ev_copy_start, &e->ev_copy_end, &e->ev_layer})
+    for (auto &v : {&e->ev_copy_start, &e->ev_copy_end, &e->ev_layer, &e->ev_arrive})
         for (cudaEvent_t ev : *v)
             if (ev) cudaEventDestroy(ev);
+    for (auto &kv : e->pipe_graphs)
+        if (kv.second) cudaGraphExecDestroy(kv.second);
+    if (e->capture_stream) cudaStreamDestroy(e->capture_stream);
     for (auto &kv : e->programs) program_destroy(kv.second);
     delete e;
 }
@@ -80,6 +92,23 @@ namespace {
         }                                                                               \
     } while (0)
 
+// cuStreamWriteValue32 through the runtime's entry-point lookup: a stream-ordered 4-byte write with a fence in front of
+// it, far cheaper than a 4-byte copy on the copy engine.  nullptr when the driver does not offer it.
+typedef CUresult (*StreamWriteValue32Fn)(CUstream, CUdeviceptr, cuuint32_t, unsigned int);
+StreamWriteValue32Fn stream_write_fn()
+{
+    static StreamWriteValue32Fn fn = nullptr;
+    static bool looked = false;
+    if (!looked) {
+        looked = true;
+        void *ptr = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuStreamWriteValue32", &ptr, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<StreamWriteValue32Fn>(ptr);
+    }
+    return fn;
+}
+
 int ensure_exec(lop_plan_t *pl)
 {
     if (pl->exec) return LOP_OK;
@@ -88,18 +117,23 @@ int ensure_exec(lop_plan_t *pl)
     pl->exec = e;
     const int B = pl->n_bands, L = (int)pl->layers.size();
     LOP_CUDA(cudaStreamCreateWithFlags(&e->copy_stream, cudaStreamNonBlocking));
+    LOP_CUDA(cudaStreamCreateWithFlags(&e->capture_stream, cudaStreamNonBlocking));
     LOP_CUDA(cudaEventCreateWithFlags(&e->ev_fork, cudaEventDisableTiming));
     LOP_CUDA(cudaEventCreateWithFlags(&e->ev_join, cudaEventDisableTiming));
+    LOP_CUDA(cudaStreamCreateWithFlags(&e->signal_stream, cudaStreamNonBlocking));
+    LOP_CUDA(cudaEventCreateWithFlags(&e->ev_signal_join, cudaEventDisableTiming));
     LOP_CUDA(cudaHostAlloc(reinterpret_cast<void **>(&e->pinned_one), 64, cudaHostAllocDefault));
     *e->pinned_one = 1u;
     LOP_CUDA(cudaEventCreate(&e->ev_begin));
     LOP_CUDA(cudaEventCreate(&e->ev_end));
     e->ev_copy_start.assign(B, nullptr);
     e->ev_copy_end.assign(B, nullptr);
+    e->ev_arrive.assign(B, nullptr);
     e->copy_issued.assign(B, 0);
     for (int b = 0; b < B; ++b) {
         LOP_CUDA(cudaEventCreate(&e->ev_copy_start[b]));
         LOP_CUDA(cudaEventCreate(&e->ev_copy_end[b]));
+        LOP_CUDA(cudaEventCreateWithFlags(&e->ev_arrive[b], cudaEventDisableTiming));
     }
     if (pl->flags & LOP_FLAG_TIME_LAYERS) {
         e->ev_layer.assign((size_t)(B + 1) * L * 2, nullptr);
@@ -284,9 +318,70 @@ int copy_band_impl(lop_plan_t *pl, int band, const void *host, void *staging, cu
     if (hi <= lo) return LOP_OK;
     const size_t row = (size_t)pl->W * pl->C * elem_size(pl->dtype);
     const size_t img = row * pl->H;
-    LOP_CUDA(cudaMemcpy2DAsync(static_cast<char *>(staging) + lo * row, img, static_cast<const char *>(host) + lo * row, img,
-                               (size_t)(hi - lo) * row, pl->N, cudaMemcpyHostToDevice, s));
+    if (pl->N == 1)
+        LOP_CUDA(cudaMemcpyAsync(static_cast<char *>(staging) + lo * row, static_cast<const char *>(host) + lo * row, (size_t)(hi - lo) * row,
+                                 cudaMemcpyHostToDevice, s));
+    else
+        LOP_CUDA(cudaMemcpy2DAsync(static_cast<char *>(staging) + lo * row, img, static_cast<const char *>(host) + lo * row, img,
+                                   (size_t)(hi - lo) * row, pl->N, cudaMemcpyHostToDevice, s));
     pl->exec->copies++;
+    return LOP_OK;
+}
+
+// Launch counts of one pipelined request (what enqueue_pipelined enqueues).
+void count_pipelined(lop_plan_t *pl, Program *p)
+{
+    ExecState *e = pl->exec;
+    if (!program_empty(p)) e->launches++;
+    for (int b = 0; b < pl->n_bands; ++b) {
+        const lop_range &need = pl->in_need[b];
+        e->copy_issued[b] = need.out_hi > need.new_lo;
+        if (e->copy_issued[b]) e->copies++;
+    }
+    e->copies_timed = false;
+}
+
+// The single-launch band pipeline on stream s (which may be capturing): fork the side streams, launch the
+// persistent kernel, enqueue every band's copy and arrival write, join.
+int enqueue_pipelined(lop_plan_t *pl, Program *p, const void *host, void *staging, cudaStream_t s)
+{
+    ExecState *e = pl->exec;
+    int rc = LOP_OK;
+    // the side streams start after everything already queued on the caller's stream
+    LOP_CUDA(cudaEventRecord(e->ev_fork, s));
+    LOP_CUDA(cudaStreamWaitEvent(e->copy_stream, e->ev_fork, 0));
+    if (!program_empty(p)) {
+        if ((rc = program_launch(p, s)) != LOP_OK) return rc;
+        e->launches++;
+    }
+    // Every command on a stream costs a few microseconds whatever its size -- as much as a small band's copy, more
+    // than its compute -- and commands of one stream run strictly one after the other.  So the copy stream carries,
+    // per band, the copy and an event record and nothing else (no timing events), and a second stream waits for that
+    // event and performs the 4-byte arrival write the kernel polls: the write of band b overlaps the copy of band b+1.
+    StreamWriteValue32Fn write32 = stream_write_fn();
+    LOP_CUDA(cudaStreamWaitEvent(e->signal_stream, e->ev_fork, 0));
+    for (int b = 0; b < pl->n_bands; ++b) {
+        const lop_range &need = pl->in_need[b];
+        e->copy_issued[b] = need.out_hi > need.new_lo;
+        if (e->copy_issued[b] && (rc = copy_band_impl(pl, b, host, staging, e->copy_stream)) != LOP_OK) return rc;
+        unsigned *flag = program_arrival_flag(p, b);
+        if (!flag) continue;
+        LOP_CUDA(cudaEventRecord(e->ev_arrive[b], e->copy_stream));
+        LOP_CUDA(cudaStreamWaitEvent(e->signal_stream, e->ev_arrive[b], 0));
+        if (write32) {
+            if (write32(reinterpret_cast<CUstream>(e->signal_stream), reinterpret_cast<CUdeviceptr>(flag), 1u, 0u) != CUDA_SUCCESS) {
+                set_error("cuStreamWriteValue32 failed");
+                return LOP_ECUDA;
+            }
+        } else {
+            LOP_CUDA(cudaMemcpyAsync(flag, e->pinned_one, sizeof(unsigned), cudaMemcpyHostToDevice, e->signal_stream));
+        }
+    }
+    e->copies_timed = false;
+    LOP_CUDA(cudaEventRecord(e->ev_signal_join, e->signal_stream));
+    LOP_CUDA(cudaStreamWaitEvent(s, e->ev_signal_join, 0));
+    LOP_CUDA(cudaEventRecord(e->ev_join, e->copy_stream));
+    LOP_CUDA(cudaStreamWaitEvent(s, e->ev_join, 0));
     return LOP_OK;
 }
 
@@ -362,37 +457,47 @@ int lop_run_pipelined(lop_plan_t *pl, const void *host, void *staging, void *out
     e->timing_valid = false;
     reset_layer_timing(pl);
     LOP_CUDA(cudaEventRecord(e->ev_begin, s));
-    // the side stream starts after everything already queued on the caller's stream
-    LOP_CUDA(cudaEventRecord(e->ev_fork, s));
-    LOP_CUDA(cudaStreamWaitEvent(e->copy_stream, e->ev_fork, 0));
     if ((rc = prepare_workspace(pl, ws, s)) != LOP_OK) return rc;
     if (e->wavefront) {
         // One persistent launch for the whole request: it starts at once and every band's first stage waits
-        // for that band's arrival flag, which the side stream sets right after the band's copy.
+        // for that band's arrival flag, which a side stream sets right after the band's copy.  The schedule is
+        // static, so it is captured once per buffer set into a CUDA graph and replayed: one host call per
+        // request instead of some twenty, each of which would cost the host more than a band costs the GPU.
         Program *p = nullptr;
         if ((rc = get_program(pl, PROG_PIPELINED, staging, out, ws, &p)) != LOP_OK) return rc;
-        if (!program_empty(p)) {
-            if ((rc = program_launch(p, s)) != LOP_OK) return rc;
-            e->launches++;
-        }
-        for (int b = 0; b < pl->n_bands; ++b) {
-            const lop_range &need = pl->in_need[b];
-            e->copy_issued[b] = need.out_hi > need.new_lo;
-            if (e->copy_issued[b]) {
-                LOP_CUDA(cudaEventRecord(e->ev_copy_start[b], e->copy_stream));
-                if ((rc = copy_band_impl(pl, b, host, staging, e->copy_stream)) != LOP_OK) return rc;
-                LOP_CUDA(cudaEventRecord(e->ev_copy_end[b], e->copy_stream));
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        LOP_CUDA(cudaStreamIsCapturing(s, &cap));
+        if (cap != cudaStreamCaptureStatusNone) {
+            if ((rc = enqueue_pipelined(pl, p, host, staging, s)) != LOP_OK) return rc;      // becomes part of the caller's graph
+        } else {
+            const auto key = std::make_tuple(host, (const void *)staging, (const void *)out, (const void *)ws);
+            auto it = e->pipe_graphs.find(key);
+            if (it == e->pipe_graphs.end()) {
+                cudaGraph_t graph = nullptr;
+                LOP_CUDA(cudaStreamBeginCapture(e->capture_stream, cudaStreamCaptureModeRelaxed));
+                rc = enqueue_pipelined(pl, p, host, staging, e->capture_stream);
+                const cudaError_t ce = cudaStreamEndCapture(e->capture_stream, &graph);
+                if (rc != LOP_OK) { if (graph) cudaGraphDestroy(graph); return rc; }
+                if (ce != cudaSuccess) { set_error("capturing the band pipeline failed: %s", cudaGetErrorString(ce)); return LOP_ECUDA; }
+                cudaGraphExec_t exec = nullptr;
+                const cudaError_t ie = cudaGraphInstantiate(&exec, graph, 0);
+                cudaGraphDestroy(graph);
+                if (ie != cudaSuccess) { set_error("cudaGraphInstantiate failed: %s", cudaGetErrorString(ie)); return LOP_ECUDA; }
+                it = e->pipe_graphs.emplace(key, exec).first;
+            } else {
+                count_pipelined(pl, p);
             }
-            unsigned *flag = program_arrival_flag(p, b);
-            if (flag) LOP_CUDA(cudaMemcpyAsync(flag, e->pinned_one, sizeof(unsigned), cudaMemcpyHostToDevice, e->copy_stream));
+            LOP_CUDA(cudaGraphLaunch(it->second, s));
         }
-        LOP_CUDA(cudaEventRecord(e->ev_join, e->copy_stream));
-        LOP_CUDA(cudaStreamWaitEvent(s, e->ev_join, 0));
         LOP_CUDA(cudaEventRecord(e->ev_end, s));
         e->timing_valid = true;
         return LOP_OK;
     }
-    // all transfers are queued up front on the side stream: band i+1 (and later) stream in while band i computes
+    // the side stream starts after everything already queued on the caller's stream; all transfers are queued
+    // up front on it: band i+1 (and later) stream in while band i computes
+    LOP_CUDA(cudaEventRecord(e->ev_fork, s));
+    LOP_CUDA(cudaStreamWaitEvent(e->copy_stream, e->ev_fork, 0));
+    e->copies_timed = true;
     for (int b = 0; b < pl->n_bands; ++b) {
         const lop_range &need = pl->in_need[b];
         e->copy_issued[b] = need.out_hi > need.new_lo;
@@ -427,7 +532,7 @@ int lop_plan_last_timing(lop_plan_t *pl, lop_timing *out)
     for (int b = 0; b < pl->n_bands; ++b) {
         if (!e->copy_issued[b]) continue;
         float ms = 0;
-        LOP_CUDA(cudaEventElapsedTime(&ms, e->ev_copy_start[b], e->ev_copy_end[b]));
+        if (e->copies_timed) LOP_CUDA(cudaEventElapsedTime(&ms, e->ev_copy_start[b], e->ev_copy_end[b]));
         t.copy_ms += ms;
         if (first) { t.first_copy_ms = ms; first = false; }
         t.n_copies++;

@@ -272,7 +272,17 @@ int program_build(lop_plan_t *pl, const std::vector<StageReq> &reqs, const void 
                 if (l.op == LOP_CONV2D && l.residual_from == LOP_INPUT) raw = true;
             }
             const int first = (int)deps.size();
-            if (rq.wait_arrival && raw) { deps.push_back(make_int2(-1 - rq.band, -1)); uses_flags = true; }   // patched below
+            if (rq.wait_arrival && raw) {
+                // every band whose transfer brought rows this band reads (its own, and earlier ones for the halo); no
+                // assumption is made about the order in which arrivals become visible
+                const lop_range &mine = pl->in_need[rq.band];
+                for (int b2 = 0; b2 <= rq.band; ++b2) {
+                    const lop_range &o = pl->in_need[b2];
+                    if (b2 != rq.band && (o.out_hi <= o.new_lo || o.out_hi <= mine.out_lo || o.new_lo >= mine.out_hi)) continue;
+                    deps.push_back(make_int2(-1 - b2, -1));             // patched below
+                }
+                uses_flags = true;
+            }
             for (int q = 0; q < nn; ++q)
                 for (int ps : by_tensor[needs[q].tensor]) {
                     if (!reuse && stage_band[ps] != rq.band) continue;
