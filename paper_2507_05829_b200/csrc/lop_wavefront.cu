@@ -1,14 +1,16 @@
 // Persistent wavefront kernel (see lop_wavefront.cuh for the execution model).
 //
-// CTA layout (two special warps + WF_WORKER_WARPS worker warps, one CTA per SM):
+// CTA layout (three special warps + WF_WORKER_WARPS worker warps, one CTA per SM):
 //   warp 0      all lanes poll the item's producer row groups in parallel (the dependency list of the
 //               next item is prefetched while this one runs); lane 0 then streams the item's activation
 //               and weight boxes by TMA into two shared-memory rings that live across items
 //   warp 1      one lane issues tcgen05.mma into one of two fp32 accumulators in tensor memory, so the
 //               next item's main loop overlaps this item's epilogue
+//   warp 2      one lane publishes finished items: after the workers' barrier it fences and does the release
+//               increment of the item's row-group counter, so that memory-fence latency is off the workers' path
 //   workers     epilogue of convolution items: TMEM -> scale/shift/residual/activation -> bf16 rows in a
 //               shared staging tile -> coalesced 16-byte stores; and the whole of pooling / patch-gather
-//               items.  They publish each finished item by a release increment of its row group's counter.
+//               items.
 //               Many of them because straight-line per-element code needs several warps per scheduler to
 //               hide its own latency; the four warps that share a TMEM lane group split a tile's columns.
 //
@@ -164,7 +166,8 @@ __global__ void __launch_bounds__(WF_THREADS, 1) wavefront_kernel(const WfParams
     const uint32_t bars = stg0 + P.stg_bytes;
     const uint32_t full_a = bars, empty_a = full_a + 8u * SA, full_b = empty_a + 8u * SA, empty_b = full_b + 8u * SB;
     const uint32_t accf0 = empty_b + 8u * SB, acce0 = accf0 + 16u;
-    uint8_t *tail = smem + (acce0 + 16u - base);
+    const uint32_t pubf0 = acce0 + 16u, pube0 = pubf0 + 8u * WF_PUBQ;
+    uint8_t *tail = smem + (pube0 + 8u * WF_PUBQ - base);
     volatile uint32_t *misc = reinterpret_cast<volatile uint32_t *>(tail);      // [0] TMEM base, [1] abort, [2] run, [3] epilogue failure
     float *s_scale = reinterpret_cast<float *>(tail + 64);                       // [256]
     float *s_shift = s_scale + 256;                                              // [256]
@@ -184,6 +187,10 @@ __global__ void __launch_bounds__(WF_THREADS, 1) wavefront_kernel(const WfParams
         for (int b = 0; b < 2; ++b) {
             mbar_init(accf0 + 8u * b, 1);
             mbar_init(acce0 + 8u * b, 1);
+        }
+        for (int q = 0; q < WF_PUBQ; ++q) {
+            mbar_init(pubf0 + 8u * q, 1);
+            mbar_init(pube0 + 8u * q, 1);
         }
         misc[1] = 0;
         misc[2] = ld_acquire(P.counters) + 1u;                 // this launch is run number (completed runs + 1)
@@ -244,7 +251,7 @@ __global__ void __launch_bounds__(WF_THREADS, 1) wavefront_kernel(const WfParams
                     fail = 1;
                 } else if (lane == 0) {
                     tr(item, 1);
-                    asm volatile("fence.proxy.async;" ::: "memory");       // producers' generic-proxy writes -> our TMA reads
+                    asm volatile("fence.proxy.async.global;" ::: "memory");       // producers' generic-proxy writes -> our TMA reads
                     const int ow0 = rec_tw(cur) * tw_valid;
                     const int oh0 = oh_lo + (rec_tr(cur) << tr_log);
                     const int n0 = rec_tn(cur) * (128 >> (p_log + tr_log));
@@ -386,19 +393,47 @@ __global__ void __launch_bounds__(WF_THREADS, 1) wavefront_kernel(const WfParams
                 *abort_flag = 1;
             }
         }
+    } else if (warp == 2) {
+        if (lane == 0) {
+            // ---------------- publisher ----------------
+            // Makes finished items visible: the workers' stores happen before their barrier and the arrive that
+            // this thread waits for, so its fence orders them before the release increment of the counter.
+            int item = blockIdx.x;
+            int4 cur = item < NI ? __ldg(&P.items[item]) : zero4;
+            int sidx = -1, ctr_base = 0;
+            bool fail = false;
+            for (uint32_t k = 0; item < NI; item += G, ++k) {
+                const int4 nxt = item + G < NI ? __ldg(&P.items[item + G]) : zero4;
+                if (rec_stage(cur) != sidx) {
+                    sidx = rec_stage(cur);
+                    ctr_base = __ldg(&P.stages[sidx].ctr_base);
+                }
+                const uint32_t q = k % WF_PUBQ, round = k / WF_PUBQ;
+                if (!mbar_wait_abortable(pubf0 + 8u * q, round & 1u, abort_flag)) { fail = !*abort_flag; break; }
+                __threadfence();
+                atomicAdd(P.counters + ctr_base + rec_tr(cur), 1u);
+                asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(pube0 + 8u * q) : "memory");
+                cur = nxt;
+            }
+            if (fail) {
+                atomicOr(P.status, 0x8u);
+                atomicExch(P.counters + 2, 1u);
+                *abort_flag = 1;
+            }
+        }
     } else {
         // ---------------- epilogue / SIMT warps ----------------
-        const int tid = threadIdx.x - 64;
+        const int tid = threadIdx.x - 32 * WF_FIRST_WORKER;
         const int g = warp & 3;                               // TMEM lane group this warp may read
         const int m = g * 32 + lane;                          // accumulator row = anchor of this thread
-        const int cgrp = (warp - 2) >> 2;                     // which share of the tile's 16-column chunks is this warp's
+        const int cgrp = (warp - WF_FIRST_WORKER) >> 2;                     // which share of the tile's 16-column chunks is this warp's
         int item = blockIdx.x;
         int4 cur = item < NI ? __ldg(&P.items[item]) : zero4;
         int4 nxt = item + G < NI ? __ldg(&P.items[item + G]) : zero4;
-        int2 dep_cur = (warp == 2 && item < NI && lane < rec_ndep(cur)) ? __ldg(&P.deps[rec_dep0(cur) + lane]) : make_int2(0, 0);
+        int2 dep_cur = (warp == WF_FIRST_WORKER && item < NI && lane < rec_ndep(cur)) ? __ldg(&P.deps[rec_dep0(cur) + lane]) : make_int2(0, 0);
         int sidx = -1;
-        uint32_t cnt = 0;
-        int kind = -1, oh_lo = 0, oh_hi = 0, p_log = 0, tr_log = 0, tw_valid = 0, BN = 0, ctr_base = 0, gather_direct = 0;
+        uint32_t cnt = 0, done_items = 0;
+        int kind = -1, oh_lo = 0, oh_hi = 0, p_log = 0, tr_log = 0, tw_valid = 0, BN = 0, gather_direct = 0;
         int N = 0, Hin = 0, Win = 0, Cin = 0, Ho = 0, Wo = 0, Cout = 0, kh = 1, kw = 1, sh = 1, sw = 1, ph = 0, pw = 0, dh = 1,
             dw = 1, act = 0, res_pos = 0;
         const void *xin = nullptr, *resp = nullptr;
@@ -407,13 +442,13 @@ __global__ void __launch_bounds__(WF_THREADS, 1) wavefront_kernel(const WfParams
         for (; item < NI; item += G) {
             const int4 nn = item + 2 * G < NI ? __ldg(&P.items[item + 2 * G]) : zero4;
             const int2 dep_nxt =
-                (warp == 2 && item + G < NI && lane < rec_ndep(nxt)) ? __ldg(&P.deps[rec_dep0(nxt) + lane]) : make_int2(0, 0);
+                (warp == WF_FIRST_WORKER && item + G < NI && lane < rec_ndep(nxt)) ? __ldg(&P.deps[rec_dep0(nxt) + lane]) : make_int2(0, 0);
             if (rec_stage(cur) != sidx) {
                 sidx = rec_stage(cur);
                 const WfStage *sp = &P.stages[sidx];
                 kind = __ldg(&sp->kind); gather_direct = __ldg(&sp->mode); oh_lo = __ldg(&sp->oh_lo); oh_hi = __ldg(&sp->oh_hi);
                 p_log = __ldg(&sp->p_log); tr_log = __ldg(&sp->tr_log); tw_valid = __ldg(&sp->tw_valid);
-                BN = __ldg(&sp->BN); ctr_base = __ldg(&sp->ctr_base);
+                BN = __ldg(&sp->BN);
                 N = __ldg(&sp->N); Hin = __ldg(&sp->Hin); Win = __ldg(&sp->Win); Cin = __ldg(&sp->Cin);
                 Ho = __ldg(&sp->Ho); Wo = __ldg(&sp->Wo); Cout = __ldg(&sp->Cout);
                 kh = __ldg(&sp->kh); kw = __ldg(&sp->kw); sh = __ldg(&sp->sh); sw = __ldg(&sp->sw);
@@ -520,7 +555,7 @@ __global__ void __launch_bounds__(WF_THREADS, 1) wavefront_kernel(const WfParams
                 if (tid == 0) tr(item, 12);
             } else {
                 // pooling or patch gather: one output row of one image per item, all worker threads
-                if (warp == 2 && !wait_deps_warp(P, rec_dep0(cur), rec_ndep(cur), dep_cur, run, lane) && lane == 0) *epi_fail = 1;
+                if (warp == WF_FIRST_WORKER && !wait_deps_warp(P, rec_dep0(cur), rec_ndep(cur), dep_cur, run, lane) && lane == 0) *epi_fail = 1;
                 epi_bar();
                 if (tid == 0) tr(item, 1);
                 const int n = rec_tn(cur);
@@ -670,11 +705,9 @@ __global__ void __launch_bounds__(WF_THREADS, 1) wavefront_kernel(const WfParams
                     }
                 }
             }
-            if (kind != WF_CONV && lane == 0 && warp < 6) tr(item, 8 + (warp - 2) + (warp == 5 ? 2 : 0));   // 8, 9, 10, 13
-            __threadfence();
             if (kind != WF_CONV && tid == 0) tr(item, 12);
-            epi_bar();
-            if (*epi_fail) {                                           // uniform: written only before the barrier above
+            epi_bar();                                                 // every worker's stores of this item are issued
+            if (*epi_fail) {                                           // uniform: written only before a barrier
                 if (tid == 0) {
                     atomicOr(P.status, 0x4u);
                     atomicExch(P.counters + 2, 1u);
@@ -683,9 +716,14 @@ __global__ void __launch_bounds__(WF_THREADS, 1) wavefront_kernel(const WfParams
                 break;
             }
             if (tid == 0) {
-                atomicAdd(P.counters + ctr_base + tile_r, 1u);        // release: stores fenced above
+                // hand the item to the publisher warp, which fences and increments the row group's counter while
+                // the workers go on; it may lag WF_PUBQ items behind
+                const uint32_t q = done_items % WF_PUBQ, round = done_items / WF_PUBQ;
+                if (!mbar_wait_abortable(pube0 + 8u * q, (round & 1u) ^ 1u, abort_flag)) *epi_fail = 1;
+                asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(pubf0 + 8u * q) : "memory");
                 tr(item, 6);
             }
+            ++done_items;
             cur = nxt; dep_cur = dep_nxt; nxt = nn;
         }
     }
@@ -740,7 +778,7 @@ extern "C" int lop_debug_trace_copy(void *host, size_t bytes, int clear)
 
 size_t wavefront_smem_bytes(const WfParams &p)
 {
-    return 1024 + (size_t)p.sa * p.a_slot_bytes + (size_t)p.sb * p.b_slot_bytes + p.stg_bytes + 8 * (size_t)(2 * p.sa + 2 * p.sb + 4) + 64 +
+    return 1024 + (size_t)p.sa * p.a_slot_bytes + (size_t)p.sb * p.b_slot_bytes + p.stg_bytes + 8 * (size_t)(2 * p.sa + 2 * p.sb + 4 + 2 * WF_PUBQ) + 64 +
            2 * 256 * sizeof(float) + 128 * sizeof(long long) + 64;
 }
 

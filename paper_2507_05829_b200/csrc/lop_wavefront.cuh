@@ -67,7 +67,9 @@ struct WfParams {
 #define LOP_WF_WORKER_WARPS 8
 #endif
 constexpr int WF_WORKER_WARPS = LOP_WF_WORKER_WARPS;      // epilogue / SIMT warps (a multiple of 4)
-constexpr int WF_THREADS = 64 + 32 * WF_WORKER_WARPS;
+constexpr int WF_FIRST_WORKER = 3;                         // warps 0..2: loader, MMA issuer, publisher
+constexpr int WF_THREADS = 32 * (WF_FIRST_WORKER + WF_WORKER_WARPS);
+constexpr int WF_PUBQ = 4;                                 // finished items the publisher may lag behind the workers
 constexpr int WF_CTR_FIRST = 4;
 constexpr int WF_MAX_DEPS = 4095;
 
