@@ -56,8 +56,6 @@ struct ExecState {
     int launches = 0;                                          // kernels enqueued by the last execution call
     int copies = 0;                                            // async copies enqueued by it
     bool timing_valid = false;
-    std::map<std::tuple<const void *, const void *, const void *, const void *>, cudaGraphExec_t> pipe_graphs;   // (host, staging, out, ws)
-    cudaStream_t capture_stream = nullptr;
     bool copies_timed = false;                                 // per-band copy events were recorded by the last pipelined run
     std::vector<char> copy_issued;
 };
@@ -74,9 +72,6 @@ void exec_destroy(ExecState *e)
     for (auto &v : {&e->ev_copy_start, &e->ev_copy_end, &e->ev_layer, &e->ev_arrive})
         for (cudaEvent_t ev : *v)
             if (ev) cudaEventDestroy(ev);
-    for (auto &kv : e->pipe_graphs)
-        if (kv.second) cudaGraphExecDestroy(kv.second);
-    if (e->capture_stream) cudaStreamDestroy(e->capture_stream);
     for (auto &kv : e->programs) program_destroy(kv.second);
     delete e;
 }
@@ -117,7 +112,6 @@ int ensure_exec(lop_plan_t *pl)
     pl->exec = e;
     const int B = pl->n_bands, L = (int)pl->layers.size();
     LOP_CUDA(cudaStreamCreateWithFlags(&e->copy_stream, cudaStreamNonBlocking));
-    LOP_CUDA(cudaStreamCreateWithFlags(&e->capture_stream, cudaStreamNonBlocking));
     LOP_CUDA(cudaEventCreateWithFlags(&e->ev_fork, cudaEventDisableTiming));
     LOP_CUDA(cudaEventCreateWithFlags(&e->ev_join, cudaEventDisableTiming));
     LOP_CUDA(cudaStreamCreateWithFlags(&e->signal_stream, cudaStreamNonBlocking));
@@ -328,19 +322,6 @@ int copy_band_impl(lop_plan_t *pl, int band, const void *host, void *staging, cu
     return LOP_OK;
 }
 
-// Launch counts of one pipelined request (what enqueue_pipelined enqueues).
-void count_pipelined(lop_plan_t *pl, Program *p)
-{
-    ExecState *e = pl->exec;
-    if (!program_empty(p)) e->launches++;
-    for (int b = 0; b < pl->n_bands; ++b) {
-        const lop_range &need = pl->in_need[b];
-        e->copy_issued[b] = need.out_hi > need.new_lo;
-        if (e->copy_issued[b]) e->copies++;
-    }
-    e->copies_timed = false;
-}
-
 // The single-launch band pipeline on stream s (which may be capturing): fork the side streams, launch the
 // persistent kernel, enqueue every band's copy and arrival write, join.
 int enqueue_pipelined(lop_plan_t *pl, Program *p, const void *host, void *staging, cudaStream_t s)
@@ -460,35 +441,13 @@ int lop_run_pipelined(lop_plan_t *pl, const void *host, void *staging, void *out
     if ((rc = prepare_workspace(pl, ws, s)) != LOP_OK) return rc;
     if (e->wavefront) {
         // One persistent launch for the whole request: it starts at once and every band's first stage waits
-        // for that band's arrival flag, which a side stream sets right after the band's copy.  The schedule is
-        // static, so it is captured once per buffer set into a CUDA graph and replayed: one host call per
-        // request instead of some twenty, each of which would cost the host more than a band costs the GPU.
+        // for that band's arrival flag, which a side stream sets right after the band's copy.  Plain stream
+        // calls: replaying the same schedule from a CUDA graph was measured slower (and stalled for hundreds of
+        // microseconds with 32 bands of 196 KB), so no graph is built here; a caller whose stream is capturing
+        // simply gets these operations into its own graph.
         Program *p = nullptr;
         if ((rc = get_program(pl, PROG_PIPELINED, staging, out, ws, &p)) != LOP_OK) return rc;
-        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
-        LOP_CUDA(cudaStreamIsCapturing(s, &cap));
-        if (cap != cudaStreamCaptureStatusNone) {
-            if ((rc = enqueue_pipelined(pl, p, host, staging, s)) != LOP_OK) return rc;      // becomes part of the caller's graph
-        } else {
-            const auto key = std::make_tuple(host, (const void *)staging, (const void *)out, (const void *)ws);
-            auto it = e->pipe_graphs.find(key);
-            if (it == e->pipe_graphs.end()) {
-                cudaGraph_t graph = nullptr;
-                LOP_CUDA(cudaStreamBeginCapture(e->capture_stream, cudaStreamCaptureModeRelaxed));
-                rc = enqueue_pipelined(pl, p, host, staging, e->capture_stream);
-                const cudaError_t ce = cudaStreamEndCapture(e->capture_stream, &graph);
-                if (rc != LOP_OK) { if (graph) cudaGraphDestroy(graph); return rc; }
-                if (ce != cudaSuccess) { set_error("capturing the band pipeline failed: %s", cudaGetErrorString(ce)); return LOP_ECUDA; }
-                cudaGraphExec_t exec = nullptr;
-                const cudaError_t ie = cudaGraphInstantiate(&exec, graph, 0);
-                cudaGraphDestroy(graph);
-                if (ie != cudaSuccess) { set_error("cudaGraphInstantiate failed: %s", cudaGetErrorString(ie)); return LOP_ECUDA; }
-                it = e->pipe_graphs.emplace(key, exec).first;
-            } else {
-                count_pipelined(pl, p);
-            }
-            LOP_CUDA(cudaGraphLaunch(it->second, s));
-        }
+        if ((rc = enqueue_pipelined(pl, p, host, staging, s)) != LOP_OK) return rc;
         LOP_CUDA(cudaEventRecord(e->ev_end, s));
         e->timing_valid = true;
         return LOP_OK;
