@@ -50,7 +50,8 @@ struct Geom {
 };
 
 // a: the convolution as its kernel sees it (a gathered stem already reduced to 1x1).
-Geom choose_geom(const ConvArgs &a, int rows)
+// even_tiles: tiles must hold whole 2x2 windows (rows and valid columns even, at least two rows).
+Geom choose_geom(const ConvArgs &a, int rows, bool even_tiles)
 {
     Geom g{};
     g.BK = a.Cin % 64 == 0 ? 64 : (a.Cin % 32 == 0 ? 32 : 16);
@@ -68,7 +69,7 @@ Geom choose_geom(const ConvArgs &a, int rows)
         long long best_tiles = -1, best_box = 0;
         for (int P = 16; P <= 128; P <<= 1) {
             const int twv = P - halo_w, TR = 128 / P, RI = TR + halo_h;
-            if (twv < 8 || RI > 256) continue;
+            if (twv < 8 || RI > 256 || (even_tiles && (TR < 2 || (twv & 1)))) continue;
             const uint32_t box = (uint32_t)RI * P * row_bytes;
             if (box > A_BOX_MAX) continue;
             const long long tiles = (long long)((a.Wo + twv - 1) / twv) * ((rows + TR - 1) / TR);
@@ -83,8 +84,18 @@ Geom choose_geom(const ConvArgs &a, int rows)
     else g.mode = WF_TAP;
     if (!slab) {
         // dense tile: the (TW, TR, TN) split of 128 pixels that needs the fewest tiles
-        const ConvTcGeom d = conv_tc_geometry(a, rows, /*fill_sms=*/false);
-        g.P = d.TW; g.TR = d.TR; g.TN = d.TN; g.tw_valid = d.TW; g.RI = d.TR;
+        int nmax = 1;
+        while (nmax * 2 <= a.N) nmax *= 2;
+        long long best = -1;
+        g.P = 128; g.TR = 1; g.TN = 1;
+        for (int tw = 128; tw >= 1; tw >>= 1)
+            for (int tr = 128 / tw; tr >= 1; tr >>= 1) {
+                const int tn = 128 / (tw * tr);
+                if (tn > nmax || (even_tiles && (tw < 2 || tr < 2))) continue;
+                const long long tiles = (long long)((a.Wo + tw - 1) / tw) * ((rows + tr - 1) / tr) * ((a.N + tn - 1) / tn);
+                if (best < 0 || tiles < best) { best = tiles; g.P = tw; g.TR = tr; g.TN = tn; }
+            }
+        g.tw_valid = g.P; g.RI = g.TR;
     }
     g.a_bytes = (uint32_t)g.RI * g.P * g.TN * row_bytes;
     // a shifted tap reads up to halo_w pixels past the box: the slot's padding takes that
@@ -144,6 +155,20 @@ int encode_maps(const ConvArgs &a, const Geom &g, CUtensorMap *out, int *valid_m
     return LOP_OK;
 }
 
+// Layer i is a tensor-core convolution whose output is read by nothing but a 2x2 stride-2 unpadded max pooling
+// right behind it: the persistent kernel can then pool inside the convolution's epilogue.
+bool pool_fusable(const lop_plan_t *pl, int i)
+{
+    const int L = (int)pl->layers.size();
+    if (i + 1 >= L) return false;
+    const LayerInfo &c = pl->layers[i], &q = pl->layers[i + 1];
+    if (c.l.op != LOP_CONV2D || c.kernel != K_CONV_TC || q.l.op != LOP_MAXPOOL2D || q.l.input_from != i) return false;
+    if (q.l.kh != 2 || q.l.kw != 2 || q.l.sh != 2 || q.l.sw != 2 || q.l.ph != 0 || q.l.pw != 0) return false;
+    for (int j = i + 2; j < L; ++j)
+        if (pl->layers[j].l.input_from == i || pl->layers[j].l.residual_from == i) return false;
+    return true;
+}
+
 }  // namespace
 
 bool program_supported(const lop_plan_t *pl)
@@ -175,8 +200,11 @@ int program_build(lop_plan_t *pl, const std::vector<StageReq> &reqs, const void 
     bool uses_flags = false;
     uint32_t a_slot = 1024, b_slot = 1024, stg_bytes = 1024;
 
-    for (const StageReq &rq : reqs) {
-        if (rq.hi <= rq.lo) continue;
+    std::vector<char> consumed(reqs.size(), 0);            // pooling requests folded into their convolution's stage
+    std::vector<int> prod_lo, prod_hi;                     // per stage: rows of the tensor it produces
+    for (size_t ri = 0; ri < reqs.size(); ++ri) {
+        const StageReq &rq = reqs[ri];
+        if (rq.hi <= rq.lo || consumed[ri]) continue;
         if (stages.size() >= 65535) { set_error("program has too many stages"); return LOP_EUNSUPPORTED; }
         const LayerInfo &li = pl->layers[rq.layer];
         const lop_layer &l = li.l;
@@ -184,7 +212,8 @@ int program_build(lop_plan_t *pl, const std::vector<StageReq> &reqs, const void 
         st.oh_lo = rq.lo; st.oh_hi = rq.hi;
         const int rows = rq.hi - rq.lo;
         int group_rows = 1, tiles_r = rows, tiles_w = 1, tiles_n = pl->N, cout_tiles = 1;
-        const int produces = rq.gather ? L : rq.layer;
+        int produces = rq.gather ? L : rq.layer;
+        int out_lo = rq.lo, out_hi = rq.hi;                    // rows of the produced tensor
         if (rq.gather) {
             st.kind = WF_GATHER;
             st.x = in; st.y = wsb + pl->col_off;
@@ -203,7 +232,14 @@ int program_build(lop_plan_t *pl, const std::vector<StageReq> &reqs, const void 
             st.kh = a.kh; st.kw = a.kw; st.sh = a.sh; st.sw = a.sw; st.ph = a.ph; st.pw = a.pw; st.dh = a.dh; st.dw = a.dw;
         } else {
             const ConvArgs a = conv_args(pl, rq.layer, in, out, ws, rq.lo, rq.hi);
-            const Geom g = choose_geom(a, rows);
+            // a 2x2 pooling that is this convolution's only reader, asked for exactly the rows this stage feeds it
+            size_t rj = reqs.size();
+            if (pool_fusable(pl, rq.layer))
+                for (size_t k = 0; k < reqs.size(); ++k)
+                    if (!consumed[k] && !reqs[k].gather && reqs[k].band == rq.band && reqs[k].layer == rq.layer + 1 &&
+                        reqs[k].hi > reqs[k].lo && rq.lo == 2 * reqs[k].lo && rq.hi == 2 * reqs[k].hi) { rj = k; break; }
+            const bool fuse = rj < reqs.size();
+            const Geom g = choose_geom(a, rows, fuse);
             st.kind = WF_CONV;
             st.mode = g.mode;
             st.x = a.x; st.res = a.res; st.scale = a.scale; st.shift = a.shift; st.y = a.y;
@@ -236,6 +272,14 @@ int program_build(lop_plan_t *pl, const std::vector<StageReq> &reqs, const void 
             a_slot = std::max(a_slot, g.a_slot);
             b_slot = std::max(b_slot, g.b_slot);
             stg_bytes = std::max(stg_bytes, round_up_u32(128u * (uint32_t)g.BN * 2u, 1024u));
+            if (fuse) {
+                const LayerInfo &pool = pl->layers[rq.layer + 1];
+                consumed[rj] = 1;
+                st.fuse_pool = 1; st.pool_Ho = pool.Ho; st.pool_Wo = pool.Wo;
+                st.y = const_cast<void *>(tensor_of(pl, rq.layer + 1, in, out, ws));
+                produces = rq.layer + 1;
+                out_lo = reqs[rj].lo; out_hi = reqs[rj].hi;
+            }
             group_rows = g.TR;
             tiles_r = (rows + g.TR - 1) / g.TR;
             tiles_w = (a.Wo + g.tw_valid - 1) / g.tw_valid;
@@ -287,10 +331,10 @@ int program_build(lop_plan_t *pl, const std::vector<StageReq> &reqs, const void 
                 for (int ps : by_tensor[needs[q].tensor]) {
                     if (!reuse && stage_band[ps] != rq.band) continue;
                     const WfStage &p = stages[ps];
-                    const int lo = std::max(needs[q].lo, p.oh_lo), hi = std::min(needs[q].hi, p.oh_hi);
+                    const int lo = std::max(needs[q].lo, prod_lo[ps]), hi = std::min(needs[q].hi, prod_hi[ps]);
                     if (lo >= hi) continue;
                     const int gr = stage_rows_per_group[ps];
-                    for (int g = (lo - p.oh_lo) / gr; g <= (hi - 1 - p.oh_lo) / gr; ++g)
+                    for (int g = (lo - prod_lo[ps]) / gr; g <= (hi - 1 - prod_lo[ps]) / gr; ++g)
                         deps.push_back(make_int2(p.ctr_base + g, expected[ps]));
                 }
             const int count = (int)deps.size() - first;
@@ -303,7 +347,9 @@ int program_build(lop_plan_t *pl, const std::vector<StageReq> &reqs, const void 
         by_tensor[produces].push_back(sidx);
         stages.push_back(st);
         stage_band.push_back(rq.band);
-        stage_rows_per_group.push_back(group_rows);
+        stage_rows_per_group.push_back(st.fuse_pool ? group_rows / 2 : group_rows);    // in rows of the produced tensor
+        prod_lo.push_back(out_lo);
+        prod_hi.push_back(out_hi);
         expected.push_back(exp_here);
     }
 
@@ -320,7 +366,7 @@ int program_build(lop_plan_t *pl, const std::vector<StageReq> &reqs, const void 
     if (n_items == 0) { *result = p; return LOP_OK; }          // nothing to do: an empty program
 
     // ---- shared-memory rings: as many slots as fit beside the staging tile, weights first
-    const size_t fixed = 1024 + stg_bytes + 8 * (2 * 8 + 2 * 8 + 4 + 2 * WF_PUBQ) + 64 + 2048 + 1024 + 64;
+    const size_t fixed = 1024 + stg_bytes + 8 * (2 * 8 + 2 * 8 + 4 + 2 * WF_PUBQ) + 64 + 2048 + 1280 + 64;
     const size_t budget = 227 * 1024 - fixed;
     int sa = 2, sb = 2;
     if ((size_t)sa * a_slot + (size_t)sb * b_slot > budget) { delete p; set_error("tile buffers do not fit shared memory"); return LOP_EUNSUPPORTED; }

@@ -172,6 +172,7 @@ __global__ void __launch_bounds__(WF_THREADS, 1) wavefront_kernel(const WfParams
     float *s_scale = reinterpret_cast<float *>(tail + 64);                       // [256]
     float *s_shift = s_scale + 256;                                              // [256]
     long long *row_pix = reinterpret_cast<long long *>(tail + 64 + 2048);        // [128]: element offset of anchor m's output, or -1
+    long long *pool_pix = row_pix + 128;                                         // [32]: element offset of a 2x2 window's pooled output, or -1
     uint8_t *stg = smem + (stg0 - base);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -433,7 +434,7 @@ __global__ void __launch_bounds__(WF_THREADS, 1) wavefront_kernel(const WfParams
         int2 dep_cur = (warp == WF_FIRST_WORKER && item < NI && lane < rec_ndep(cur)) ? __ldg(&P.deps[rec_dep0(cur) + lane]) : make_int2(0, 0);
         int sidx = -1;
         uint32_t cnt = 0, done_items = 0;
-        int kind = -1, oh_lo = 0, oh_hi = 0, p_log = 0, tr_log = 0, tw_valid = 0, BN = 0, gather_direct = 0;
+        int kind = -1, oh_lo = 0, oh_hi = 0, p_log = 0, tr_log = 0, tw_valid = 0, BN = 0, gather_direct = 0, fuse_pool = 0, pool_Ho = 0, pool_Wo = 0;
         int N = 0, Hin = 0, Win = 0, Cin = 0, Ho = 0, Wo = 0, Cout = 0, kh = 1, kw = 1, sh = 1, sw = 1, ph = 0, pw = 0, dh = 1,
             dw = 1, act = 0, res_pos = 0;
         const void *xin = nullptr, *resp = nullptr;
@@ -454,6 +455,7 @@ __global__ void __launch_bounds__(WF_THREADS, 1) wavefront_kernel(const WfParams
                 kh = __ldg(&sp->kh); kw = __ldg(&sp->kw); sh = __ldg(&sp->sh); sw = __ldg(&sp->sw);
                 ph = __ldg(&sp->ph); pw = __ldg(&sp->pw); dh = __ldg(&sp->dh); dw = __ldg(&sp->dw);
                 act = __ldg(&sp->act); res_pos = __ldg(&sp->res_pos);
+                fuse_pool = __ldg(&sp->fuse_pool); pool_Ho = __ldg(&sp->pool_Ho); pool_Wo = __ldg(&sp->pool_Wo);
                 xin = ldg_ptr<const void *>(&sp->x);
                 resp = ldg_ptr<const void *>(&sp->res);
                 scale = ldg_ptr<const float *>(reinterpret_cast<const void *const *>(&sp->scale));
@@ -472,6 +474,12 @@ __global__ void __launch_bounds__(WF_THREADS, 1) wavefront_kernel(const WfParams
                 const bool valid = c < tw_valid && ow < Wo && oh < oh_hi && n < N;
                 const int co0 = rec_cout(cur) * BN;
                 if (cgrp == 0) row_pix[m] = valid ? (((long long)n * Ho + oh) * Wo + ow) * Cout + co0 : -1LL;
+                if (fuse_pool && cgrp == 0 && !((r | c) & 1)) {
+                    // top-left anchor of a 2x2 window: where its maximum goes, if the whole window is inside the stage
+                    const int q = (((m >> (p_log + tr_log)) << (tr_log - 1)) + (r >> 1)) * ((1 << p_log) >> 1) + (c >> 1);
+                    const bool ok = valid && c + 1 < tw_valid && ow + 1 < Wo && oh + 1 < oh_hi;
+                    pool_pix[q] = ok ? (((long long)n * pool_Ho + (oh >> 1)) * pool_Wo + (ow >> 1)) * Cout + co0 : -1LL;
+                }
                 for (int i = tid; i < BN; i += EPI_THREADS) {          // this tile's scale/shift while the main loop runs
                     s_scale[i] = scale ? __ldg(scale + co0 + i) : 1.0f;
                     s_shift[i] = shift ? __ldg(shift + co0 + i) : 0.0f;
@@ -541,7 +549,28 @@ __global__ void __launch_bounds__(WF_THREADS, 1) wavefront_kernel(const WfParams
                 epi_bar();                                             // accumulator drained, staging tile complete
                 if (tid == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(acce0 + 8u * buf) : "memory");
                 ++cnt;
-                if (!*epi_fail) {
+                if (!*epi_fail && fuse_pool) {
+                    // 2x2 windows of staged rows -> their maxima (exact in bf16) -> the pooled tensor, 16 bytes per thread
+                    const int P_ = 1 << p_log, half_p = P_ >> 1, half_tr = (1 << tr_log) >> 1;
+                    for (int idx = tid; idx < 32 * cpr; idx += EPI_THREADS) {
+                        const int q = cpr_log >= 0 ? idx >> cpr_log : idx / cpr, j = idx - q * cpr;
+                        const long long pp = pool_pix[q];
+                        if (pp < 0) continue;
+                        const int pc = q % half_p, t = q / half_p;
+                        const int m0 = ((t / half_tr) << (p_log + tr_log)) + ((2 * (t % half_tr)) << p_log) + 2 * pc;
+                        const int rows4[4] = {m0, m0 + 1, m0 + P_, m0 + P_ + 1};
+                        uint4 acc4 = *reinterpret_cast<const uint4 *>(stg + rows4[0] * row_stride + ((j ^ (rows4[0] & swz)) << 4));
+#pragma unroll
+                        for (int k = 1; k < 4; ++k) {
+                            const uint4 v4 = *reinterpret_cast<const uint4 *>(stg + rows4[k] * row_stride + ((j ^ (rows4[k] & swz)) << 4));
+                            __nv_bfloat162 *pa = reinterpret_cast<__nv_bfloat162 *>(&acc4);
+                            const __nv_bfloat162 *pv = reinterpret_cast<const __nv_bfloat162 *>(&v4);
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) pa[e] = __hmax2(pa[e], pv[e]);
+                        }
+                        *(reinterpret_cast<uint4 *>(y + pp) + j) = acc4;
+                    }
+                } else if (!*epi_fail) {
                     // staged rows -> global: consecutive threads write consecutive 16 bytes of a pixel's channels
 #pragma unroll 4
                     for (int idx = tid; idx < 128 * cpr; idx += EPI_THREADS) {
@@ -779,7 +808,7 @@ extern "C" int lop_debug_trace_copy(void *host, size_t bytes, int clear)
 size_t wavefront_smem_bytes(const WfParams &p)
 {
     return 1024 + (size_t)p.sa * p.a_slot_bytes + (size_t)p.sb * p.b_slot_bytes + p.stg_bytes + 8 * (size_t)(2 * p.sa + 2 * p.sb + 4 + 2 * WF_PUBQ) + 64 +
-           2 * 256 * sizeof(float) + 128 * sizeof(long long) + 64;
+           2 * 256 * sizeof(float) + (128 + 32) * sizeof(long long) + 64;
 }
 
 cudaError_t launch_wavefront(const WfParams &p, int grid, cudaStream_t s)

@@ -42,8 +42,11 @@ struct WfStage {
     const void *x;            // main input, full-size NHWC tensor
     const void *res;          // residual tensor or nullptr
     const float *scale, *shift;
-    void *y;                  // full-size output
-    int pad_[16];
+    void *y;                  // full-size output (of the pooling layer when fuse_pool is set)
+    // fuse_pool: the convolution's only consumer is a 2x2 stride-2 max pooling; the tile's epilogue takes the
+    // maximum of each 2x2 window of staged rows and writes the pooled tensor [N, pool_Ho, pool_Wo, Cout] instead
+    int fuse_pool, pool_Ho, pool_Wo;
+    int pad_[13];
 };
 static_assert(sizeof(WfStage) == 256, "WfStage layout");
 

@@ -118,6 +118,41 @@ def test_bf16_residual_and_activation_epilogues(pos, act):
     check_workload(wl, flags=lop.LOP_FLAG_PER_LAYER | lop.LOP_FLAG_REUSE_HALO)
 
 
+# ------------------------------------------------------------------------------------ convolution + 2x2 pooling in one stage
+POOL_FUSE_CASES = [  # layers (cin, cout, k) of the convolution in front of the pooling, N, H, W, C
+    ((64, 64, 3), 2, 20, 27, 64),          # odd width: the last column has no partner
+    ((64, 32, 1), 3, 6, 6, 64),            # pointwise, tiny images folded into one tile
+    ((3, 64, 3), 1, 24, 40, 3),            # gathered stem straight into the pooling
+    ((64, 128, 5), 1, 16, 16, 64),         # wider halo, two channel tiles
+]
+
+
+@pytest.mark.parametrize("case", POOL_FUSE_CASES)
+def test_conv_then_pool2x2_is_pooled_in_the_epilogue(case):
+    (cin, cout, k), N, H, W, C = case
+    layers = [conv(cin, cout, k, act=li.ACT_RELU), pool(cout, 2, 2, 0)]
+    for i, l in enumerate(layers):
+        l.input_from = i - 1
+    wl = Workload("convpool", "bf16", N, H, W, C, [Segment(layers, 3)], seed=11)
+    li.fill_parameters(wl)
+    li.make_input(wl)
+    a = check_workload(wl, flags=lop.LOP_FLAG_REUSE_HALO)["whole"]
+    b = check_workload(wl, flags=lop.LOP_FLAG_REUSE_HALO | lop.LOP_FLAG_PER_LAYER, modes=("whole", "banded"))["whole"]
+    for x, y in zip(a, b):
+        assert np.array_equal(x, y)
+    check_workload(wl)                                           # independent bands
+
+
+def test_pooling_is_not_folded_when_the_convolution_has_another_reader():
+    layers = [conv(64, 64, 3, act=li.ACT_RELU), pool(64, 2, 2, 0),
+              conv(64, 64, 3, s=2, act=li.ACT_NONE, residual_from=1, residual_pos=li.RES_POST_ACT)]
+    layers[0].input_from, layers[1].input_from, layers[2].input_from = -1, 0, 0     # layer 2 also reads the convolution
+    wl = Workload("convpool2", "bf16", 1, 16, 24, 64, [Segment(layers, 2)], seed=12)
+    li.fill_parameters(wl)
+    li.make_input(wl)
+    check_workload(wl, flags=lop.LOP_FLAG_REUSE_HALO)
+
+
 # ------------------------------------------------------------------------------------ pooling
 @pytest.mark.parametrize("dtype,C", [("bf16", 64), ("bf16", 6), ("f32", 8), ("f32", 3)])
 @pytest.mark.parametrize("k,s,p", [(2, 2, 0), (3, 2, 1)])
