@@ -120,6 +120,22 @@ def time_oracle(wl, min_seconds):
             "sample": "%d whole pass(es) of the workload (N=%d), %.1f s" % (runs, wl.N, dt)}, dt / runs
 
 
+def max_over_ranks(ms, device=None):
+    """The slowest rank's time: every rank runs its own replica, the job is as slow as the slowest of them."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(ms)
+    t = torch.tensor([float(ms)], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_images_per_s(images_per_rank, world, ms_per_step):
+    """Whole-job throughput of `world` independent replicas (weak scaling, no data-path collective)."""
+    return images_per_rank * world / (ms_per_step * 1e-3)
+
+
 def run_reference(args):
     """The reference arm: the CPU oracle timed on the host cores, rank 0 only."""
     if int(os.environ.get("RANK", "0")) != 0:
@@ -236,11 +252,7 @@ def main():
             torch.cuda.synchronize()
             barrier()
         total = sum(a.elapsed_time(b) for a, b in evs)
-        if world > 1:
-            t = torch.tensor([total], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            total = float(t.item())
-        return total / steps
+        return max_over_ranks(total, dev) / steps
 
     sampler = ClockSampler(local)
     if rank == 0:
@@ -330,15 +342,14 @@ def main():
             dist.destroy_process_group()
         return
 
-    images = wl.N * world
     line = {
-        "metric": METRIC, "value": images / (ms_res * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "metric": METRIC, "value": job_images_per_s(wl.N, world, ms_res), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_res, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16" if wl.dtype == "bf16" else "f32", "data": "synthetic",
         "config": {"workload": WORKLOAD_NOTES[args.workload], "images_per_step_per_gpu": wl.N,
                    "mode": "reuse-halo bands", "launch": "eager" if args.no_graph else "value: cuda-graph replay of one step; e2e: eager calls",
                    "l2": "256 MiB buffer written between timed steps", "multi_gpu": "independent replicas"},
-        "e2e": {"value": images / (ms_e2e * 1e-3), "unit": UNIT, "ms_per_step": ms_e2e,
+        "e2e": {"value": job_images_per_s(wl.N, world, ms_e2e), "unit": UNIT, "ms_per_step": ms_e2e,
                 "h2d_bytes_per_step": int(x_pin.numel() * x_pin.element_size()),
                 "d2h_bytes_per_step": int(out_pin.numel() * out_pin.element_size())},
         "gpu_launches": int(launches_res * args.steps),

@@ -146,6 +146,24 @@ __device__ __forceinline__ void mma_tap(uint32_t acc, uint32_t pa, uint32_t pb, 
     else mma_ksteps<1>(acc, pa, pb, desc_hi, idesc, accumulate);
 }
 
+// One weight box of three taps of a 3x3 filter row over a 64-channel chunk: twelve MMAs whose descriptors differ
+// from the first one by compile-time constants.  One thread issues every MMA of the CTA and each instruction it
+// executes in between costs as much as a quarter of an N = 64 MMA, so the common case gets straight-line code.
+// la, lb: start-address fields (address >> 4) of the slab row this filter row starts at and of the weight box;
+// tap16: bytes of one tap's weights >> 4.
+__device__ __forceinline__ void mma_row3x64(uint32_t acc, uint32_t la, uint32_t lb, uint32_t tap16, uint32_t desc_hi, uint32_t idesc,
+                                            uint32_t &accumulate)
+{
+    const uint64_t hi = (uint64_t)desc_hi << 32;
+#pragma unroll
+    for (int tb = 0; tb < 3; ++tb)
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) {
+            umma_bf16(acc, hi | (uint64_t)(la + 8u * tb + 2u * kk), hi | (uint64_t)(lb + tap16 * tb + 2u * kk), idesc, accumulate);
+            accumulate = 1u;
+        }
+}
+
 __device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, %0;" ::"n"(EPI_THREADS) : "memory"); }
 
 template <typename T>
@@ -323,7 +341,7 @@ __global__ void __launch_bounds__(WF_THREADS, 1) wavefront_kernel(const WfParams
             int kind = -1, mode = 0, n_chunks = 1, n_taps = 1, tbx = 1, kw = 1, dh = 1, dw = 1, p_log = 0, ksteps = 1;
             uint32_t idesc = 0, desc_hi = 0, row_bytes = 0, tap_bytes = 0;
             uint32_t a_slot = 0, a_phase = 0, b_slot = 0, b_phase = 0, cnt = 0;
-            bool fail = false;
+            bool fail = false, row3x64 = false;
             for (; item < NI && !fail; item += G) {
                 const int4 nxt = item + G < NI ? __ldg(&P.items[item + G]) : zero4;
                 if (rec_stage(cur) != sidx) {
@@ -337,6 +355,7 @@ __global__ void __launch_bounds__(WF_THREADS, 1) wavefront_kernel(const WfParams
                     desc_hi = ((__ldg(&sp->sbo_bytes) >> 4) & 0x3FFFu) | (1u << 14) | (__ldg(&sp->layout_code) << 29);
                     row_bytes = __ldg(&sp->row_bytes);
                     tap_bytes = (uint32_t)__ldg(&sp->BN) * row_bytes;
+                    row3x64 = mode == WF_SLAB && n_taps == 9 && kw == 3 && tbx == 3 && ksteps == 4 && dw == 1;
                 }
                 if (kind == WF_CONV) {
                     const uint32_t buf = cnt & 1u;
@@ -355,6 +374,12 @@ __global__ void __launch_bounds__(WF_THREADS, 1) wavefront_kernel(const WfParams
                                 const uint32_t sb = b0 + b_slot * b_slot_bytes;
                                 const int t1 = min(t0 + tbx, n_taps);
                                 int ta = t0 / kw, tb = t0 - ta * kw;
+                                if (row3x64) {
+                                    // box = filter row t0 / 3 of a 3x3 filter: the slab row it starts at, then constants
+                                    const uint32_t pa = sa + (uint32_t)((ta * dh) << p_log) * 128u;
+                                    mma_row3x64(acc, ((pa & 0x3FFFFu) >> 4) | (1u << 16), ((sb & 0x3FFFFu) >> 4) | (1u << 16), tap_bytes >> 4,
+                                                desc_hi, idesc, accumulate);
+                                } else
                                 for (int t = t0; t < t1; ++t) {
                                     // tap (ta, tb): the same box, read (ta*dh*P + tb*dw) pixels further on
                                     const uint32_t pa = sa + (uint32_t)(((ta * dh) << p_log) + tb * dw) * row_bytes;
