@@ -175,7 +175,8 @@ int lop_plan_layer_kernel(const lop_plan_t *plan, int layer);
 int lop_plan_last_launches(const lop_plan_t *plan);
 int lop_plan_last_copies(const lop_plan_t *plan);
 /* Reads the plan's device status word (0 = no kernel gave up on a bounded wait).  SYNCHRONISES
- * the stream of the last execution call. */
+ * the stream of the last execution call.  On LOP_EDEVICE the outputs of that call are invalid; the
+ * library drops its cached device tables and clears the word, so the plan can be used again. */
 int lop_plan_check_device(lop_plan_t *plan, void *workspace);
 
 /* ---- execution without any allocation --------------------------------------------------------

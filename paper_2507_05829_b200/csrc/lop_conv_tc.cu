@@ -332,11 +332,15 @@ cudaError_t launch_conv_tc(const ConvArgs &a, const ConvTcGeom &g, const ConvTcM
     // instruction descriptor: fp32 accumulate, bf16 x bf16, both operands K-major, N = BN, M = 128
     p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(g.BN >> 3) << 17) | ((128u >> 4) << 24);
     const size_t smem = 1024 + (size_t)g.stages * (p.a_stage_bytes + p.b_stage_bytes) + 16 * g.stages + 32;
-    static size_t configured = 0;
-    if (smem > configured) {
-        cudaError_t e = cudaFuncSetAttribute(conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(200 * 1024));
+    // the attribute is per device: set it once on each device a launch is made from
+    static bool configured[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64 || !configured[dev]) {
+        e = cudaFuncSetAttribute(conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(200 * 1024));
         if (e != cudaSuccess) return e;
-        configured = 200 * 1024;
+        if (dev >= 0 && dev < 64) configured[dev] = true;
     }
     dim3 grid((unsigned)(p.tiles_w * p.tiles_r * tiles_n), (unsigned)(a.Cout / g.BN));
     conv_tc_kernel<<<grid, TC_THREADS, smem, s>>>(maps, p);

@@ -76,6 +76,15 @@ void exec_destroy(ExecState *e)
     delete e;
 }
 
+void exec_invalidate(ExecState *e)
+{
+    if (!e) return;
+    for (auto &kv : e->programs) program_destroy(kv.second);      // cudaFree waits for launches still in flight
+    e->programs.clear();
+    e->maps.clear();
+    e->prepared_ws = nullptr;                                      // padded stem weights are rebuilt on the next call
+}
+
 namespace {
 
 #define LOP_CUDA(call)                                                                  \
@@ -202,6 +211,7 @@ int run_layer(lop_plan_t *pl, int i, int lo, int hi, const void *in, void *out, 
             const MapKey key{i, g.TW, g.TR, g.TN, g.BN, g.BK, a.x, a.w};
             auto it = e->maps.find(key);
             if (it == e->maps.end()) {
+                if (e->maps.size() >= 4096) e->maps.clear();        // tensor maps are passed by value at launch: safe to drop
                 ConvTcMaps m;
                 int rc = conv_tc_encode(a, g, &m);
                 if (rc != LOP_OK) { set_error("layer %d: tensor-map encoding failed", i); return rc; }
@@ -252,6 +262,12 @@ int get_program(lop_plan_t *pl, int kind, const void *in, void *out, void *ws, P
     const ProgKey key{kind, in, out, ws};
     auto it = e->programs.find(key);
     if (it == e->programs.end()) {
+        if (e->programs.size() >= 64) {
+            // a caller that keeps changing buffers: start over rather than grow without bound (cudaFree waits for
+            // launches still in flight)
+            for (auto &kv : e->programs) program_destroy(kv.second);
+            e->programs.clear();
+        }
         const int L = (int)pl->layers.size(), B = pl->n_bands;
         std::vector<StageReq> reqs;
         if (kind == PROG_WHOLE) {
@@ -534,7 +550,15 @@ int lop_plan_check_device(lop_plan_t *pl, void *ws)
     LOP_CUDA(cudaStreamSynchronize(pl->exec->last_stream));
     unsigned status = 0;
     LOP_CUDA(cudaMemcpy(&status, static_cast<char *>(ws) + pl->status_off, sizeof(status), cudaMemcpyDeviceToHost));
-    if (status) { set_error("device status word 0x%x: a bounded wait ran out", status); return LOP_EDEVICE; }
+    if (status) {
+        // the run was abandoned half way: its row-group counters are meaningless now, so the programs (and their
+        // counters) are dropped and rebuilt on the next call; the status word is cleared for that call
+        for (auto &kv : pl->exec->programs) program_destroy(kv.second);
+        pl->exec->programs.clear();
+        cudaMemset(static_cast<char *>(ws) + pl->status_off, 0, sizeof(status));
+        set_error("device status word 0x%x: a bounded wait ran out", status);
+        return LOP_EDEVICE;
+    }
     return LOP_OK;
 }
 

@@ -47,5 +47,7 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 // lop_exec.cu
 void exec_destroy(ExecState *e);
+// Drops what was built from the layers' device pointers (programs, tensor maps, padded weights), after lop_plan_set_params.
+void exec_invalidate(ExecState *e);
 
 }  // namespace lop

@@ -311,6 +311,7 @@ int lop_plan_set_params(lop_plan_t *plan, int layer, const void *weight, const f
     if (layer < 0 || layer >= (int)plan->layers.size()) { set_error("lop_plan_set_params: layer %d out of range", layer); return LOP_EINVAL; }
     lop_layer &l = plan->layers[layer].l;
     l.weight = weight; l.scale = scale; l.shift = shift;
+    exec_invalidate(plan->exec);           // device tables and tensor maps were built from the old pointers
     return LOP_OK;
 }
 

@@ -839,11 +839,15 @@ size_t wavefront_smem_bytes(const WfParams &p)
 cudaError_t launch_wavefront(const WfParams &p, int grid, cudaStream_t s)
 {
     const size_t smem = wavefront_smem_bytes(p);
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(wavefront_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    // the attribute is per device: set it once on each device a launch is made from
+    static bool configured[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64 || !configured[dev]) {
+        e = cudaFuncSetAttribute(wavefront_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
         if (e != cudaSuccess) return e;
-        configured = true;
+        if (dev >= 0 && dev < 64) configured[dev] = true;
     }
     if (smem > 227 * 1024) return cudaErrorInvalidValue;
 #ifdef LOP_WF_TRACE

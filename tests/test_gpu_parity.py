@@ -183,6 +183,40 @@ def test_tensor_core_and_cuda_core_paths_agree():
 
 
 # ------------------------------------------------------------------------------------ edge cases
+def test_very_wide_image_gathers_patches_without_staging_rows():
+    """Three rows of a 4200-pixel image do not fit the shared staging tile: the gather reads the image in place."""
+    wl = one_layer(conv(3, 32, 3, act=li.ACT_RELU), 1, 6, 4200, n_bands=2)
+    check_workload(wl, flags=lop.LOP_FLAG_REUSE_HALO)
+
+
+def test_set_params_takes_effect_on_a_plan_that_has_already_run():
+    wl = li.build("vgg_block", H=44, W=36)
+    dc = DeviceChain(wl, flags=lop.LOP_FLAG_REUSE_HALO)
+    x = dc.input_tensor()
+    first = dc.run_banded(x).clone()
+    torch.cuda.synchronize()
+    seg = wl.segments[0]
+    for l in seg.layers:                                  # new weights: the old ones negated
+        if l.weight is not None:
+            l.weight = -l.weight
+    want = ochain.run_workload(wl)
+    keep = []
+    for i, l in enumerate(seg.layers):
+        if l.weight is None:
+            continue
+        w = torch.from_numpy(l.weight).to(torch.bfloat16).cuda().contiguous()
+        sc = torch.from_numpy(l.scale).cuda() if l.scale is not None else None
+        sh = torch.from_numpy(l.shift).cuda() if l.shift is not None else None
+        keep += [w, sc, sh]
+        dc.plans[0].set_params(i, w.data_ptr(), sc.data_ptr() if sc is not None else None, sh.data_ptr() if sh is not None else None)
+    for mode in ("banded", "whole"):
+        got = dc.run_banded(x) if mode == "banded" else dc.run_whole(x)
+        torch.cuda.synchronize()
+        dc.check_device()
+        assert rel_err(to_host_f32(got), want) <= TOL["bf16"], mode
+    assert not torch.equal(first, dc.outs[-1])
+
+
 def test_more_bands_than_rows_and_single_band():
     wl = li.build("vgg_block", H=12, W=20)
     for nb in (1, 6, 7, 13):                                     # 6 output rows: empty bands from 7 on
