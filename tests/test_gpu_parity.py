@@ -86,6 +86,9 @@ TC_CASES = [  # k, s, p, d, cin, cout, N, H, W
     (1, 2, 0, 1, 64, 256, 2, 15, 15),      # strided pointwise projection
     (7, 2, 3, 1, 3, 64, 2, 38, 38),        # stem: 3 input channels, padded to 16
     (3, 1, 1, 1, 3, 32, 1, 24, 40),
+    (3, 1, 1, 1, 5, 32, 2, 9, 21),         # 45 patch values -> 48: 16-channel chunks, tiny images
+    (3, 2, 1, 1, 7, 64, 3, 13, 13),        # 63 -> 64: one 64-channel chunk, strided stem
+    (5, 1, 2, 2, 3, 48, 1, 20, 20),        # dilated stem, 75 -> 80
     (3, 1, 2, 2, 64, 32, 1, 16, 16),       # dilation 2
     (3, 1, 1, 1, 16, 16, 1, 10, 10),       # 16-channel slabs
     (5, 1, 2, 1, 64, 48, 1, 12, 12),       # 48 output channels
