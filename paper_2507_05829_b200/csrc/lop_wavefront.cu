@@ -544,7 +544,14 @@ __global__ void __launch_bounds__(WF_THREADS, 1) wavefront_kernel(const WfParams
                         if (!valid) continue;
                         float v[16];
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) v[i] = fmaf(s_scale[j + i], __uint_as_float(rr[i]), s_shift[j + i]);
+                        for (int i = 0; i < 16; i += 4) {                  // 16-byte broadcast reads of the tile's scale / shift
+                            const float4 sc = *reinterpret_cast<const float4 *>(s_scale + j + i);
+                            const float4 sf = *reinterpret_cast<const float4 *>(s_shift + j + i);
+                            v[i] = fmaf(sc.x, __uint_as_float(rr[i]), sf.x);
+                            v[i + 1] = fmaf(sc.y, __uint_as_float(rr[i + 1]), sf.y);
+                            v[i + 2] = fmaf(sc.z, __uint_as_float(rr[i + 2]), sf.z);
+                            v[i + 3] = fmaf(sc.w, __uint_as_float(rr[i + 3]), sf.w);
+                        }
                         uint4 *c0p = reinterpret_cast<uint4 *>(my_row + ((((j >> 3)) ^ (m & swz)) << 4));
                         uint4 *c1p = reinterpret_cast<uint4 *>(my_row + ((((j >> 3) + 1) ^ (m & swz)) << 4));
                         float rv[16];
