@@ -295,12 +295,23 @@ def main():
     # it, so the per-step CUDA events of the timed region are its launch durations
     conv_fl = dc.flops()
     achieved = conv_fl / (ms_res * 1e-3) / 1e12
-    roofline = {"bound": "tensor", "kernel": "wavefront_kernel (all-bands program: every gather / conv / pool stage of the step in one persistent launch)",
-                "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                "frac": achieved / peaks["bf16_tflops"],
-                "peak_source": "%s TFLOP/s burst bf16 (of %s)" % (peaks["bf16_tflops"], peaks["source"]),
-                "flops_per_launch": conv_fl, "avg_launch_us": ms_res * 1e3, "launches_per_step": launches_res,
-                "traffic": TRAFFIC.get(args.workload)}
+    if wl.dtype == "bf16":
+        roofline = {"bound": "tensor", "kernel": "wavefront_kernel (all-bands program: every gather / conv / pool stage of the step in one persistent launch per segment)",
+                    "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                    "frac": achieved / peaks["bf16_tflops"],
+                    "peak_source": "%s TFLOP/s burst bf16 (of %s)" % (peaks["bf16_tflops"], peaks["source"]),
+                    "flops_per_launch": conv_fl, "avg_launch_us": ms_res * 1e3, "launches_per_step": launches_res,
+                    "traffic": TRAFFIC.get(args.workload)}
+    else:
+        # fp32 storage runs on the CUDA cores: plain-ALU peak = SMs x 128 FMA lanes x 2 flop x max SM clock
+        props = torch.cuda.get_device_properties(dev)
+        mhz = (clocks or {}).get("sm_max_mhz") or 1965.0
+        alu_peak = props.multi_processor_count * 128 * 2 * mhz * 1e6 / 1e12
+        roofline = {"bound": "alu", "kernel": "conv_simt_kernel (one launch per band)", "achieved": achieved, "peak": alu_peak,
+                    "unit": "TFLOP/s", "frac": achieved / alu_peak,
+                    "peak_source": "derived: %d SMs x 128 fp32 FMA lanes x 2 x %.0f MHz" % (props.multi_processor_count, mhz),
+                    "flops_per_launch": conv_fl / max(launches_res, 1), "avg_launch_us": ms_res * 1e3 / max(launches_res, 1),
+                    "launches_per_step": launches_res, "traffic": None}
 
     # ---- per-layer view: whole-tensor launches, one kernel per layer, CUDA events around each (eager)
     dct = DeviceChain(wl, flags=lop.LOP_FLAG_PER_LAYER | lop.LOP_FLAG_TIME_LAYERS, device=dev)
