@@ -162,6 +162,27 @@ int lop_copy_band(lop_plan_t *plan, int band, const void *in_host_pinned, void *
  * Returns after enqueueing.  staging_dev: lop_plan_staging_bytes() bytes. */
 int lop_run_pipelined(lop_plan_t *plan, const void *in_host_pinned, void *staging_dev, void *out_dev,
                       void *workspace, void *stream);
+/* ---- several plans as one chain (Sec. III-A: later operators start as soon as the rows they
+ * depend on exist) ---------------------------------------------------------------------------
+ * A long network is planned in pieces (one plan per stage of the network, each with its own bands);
+ * plan s+1 reads the full-size output tensor of plan s.  Run one after the other with the
+ * functions above, each plan waits for the whole previous one.  These two functions run all plans
+ * in ONE persistent launch with dependencies tracked per row group across plan boundaries, so a
+ * band of plan s+1 starts as soon as the rows of plan s it reads are written.
+ * plans[0..n_plans): HOST array; outs_dev[i], workspaces[i]: DEVICE, plan i's output tensor and
+ * workspace (HOST arrays of pointers).  Requirements: every plan runs on the tensor-core kernels
+ * (bf16, every convolution served by them), plan i+1's input shape equals plan i's output shape,
+ * all plans agree in N, dtype and LOP_FLAG_REUSE_HALO; otherwise LOP_EUNSUPPORTED / LOP_ESHAPE is
+ * returned before anything is enqueued and the caller runs the plans one by one.  The device status
+ * word of the launch is plan 0's (lop_plan_check_device(plans[0], workspaces[0])). */
+/* All bands of all plans from a device-resident input. */
+int lop_run_chain_banded(lop_plan_t *const *plans, int n_plans, const void *in_dev, void *const *outs_dev,
+                         void *const *workspaces, void *stream);
+/* Band pipeline over the whole chain: plan 0's input bands stream from PINNED HOST memory as in
+ * lop_run_pipelined while the rows already there flow through every plan. */
+int lop_run_chain_pipelined(lop_plan_t *const *plans, int n_plans, const void *in_host_pinned, void *staging_dev,
+                            void *const *outs_dev, void *const *workspaces, void *stream);
+
 /* Event times of the last lop_run_pipelined call.  SYNCHRONISES with that call's completion. */
 int lop_plan_last_timing(lop_plan_t *plan, lop_timing *out);
 /* With LOP_FLAG_TIME_LAYERS (implies per-layer launches): device time in ms of the (band, layer) launch of the last

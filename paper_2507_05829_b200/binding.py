@@ -20,7 +20,7 @@ EXPORTS = [
     "lop_plan_out_shape", "lop_plan_set_params", "lop_plan_workspace_bytes", "lop_plan_staging_bytes",
     "lop_plan_flops", "lop_run_whole", "lop_run_band", "lop_run_banded", "lop_copy_band", "lop_run_pipelined",
     "lop_plan_last_timing", "lop_plan_layer_time", "lop_plan_layer_kernel", "lop_plan_last_launches", "lop_plan_last_copies",
-    "lop_plan_check_device", "lop_run_whole_static", "lop_strerror", "lop_last_error",
+    "lop_plan_check_device", "lop_run_whole_static", "lop_run_chain_banded", "lop_run_chain_pipelined", "lop_strerror", "lop_last_error",
 ]
 LOP_STATIC_SCRATCH_BYTES = 16 << 20
 
@@ -91,6 +91,8 @@ def lib():
     L.lop_plan_last_copies.argtypes = [c_void_p]
     L.lop_plan_check_device.argtypes = [c_void_p, c_void_p]
     L.lop_run_whole_static.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
+    L.lop_run_chain_banded.argtypes = [POINTER(c_void_p), c_int, c_void_p, POINTER(c_void_p), POINTER(c_void_p), c_void_p]
+    L.lop_run_chain_pipelined.argtypes = [POINTER(c_void_p), c_int, c_void_p, c_void_p, POINTER(c_void_p), POINTER(c_void_p), c_void_p]
     L.lop_strerror.argtypes = [c_int]
     L.lop_strerror.restype = c_char_p
     L.lop_last_error.restype = c_char_p
@@ -115,6 +117,22 @@ def make_layer_array(layers):
         a.scale = getattr(l, "scale_ptr", None)
         a.shift = getattr(l, "shift_ptr", None)
     return arr
+
+
+def _ptr_array(values):
+    return (c_void_p * len(values))(*values)
+
+
+def run_chain_banded(plans, in_dev, outs_dev, workspaces, stream):
+    """lop_run_chain_banded: ``plans`` are :class:`Plan` objects, the rest device addresses."""
+    _check(lib().lop_run_chain_banded(_ptr_array([p._h.value for p in plans]), len(plans), in_dev, _ptr_array(outs_dev),
+                                      _ptr_array(workspaces), stream))
+
+
+def run_chain_pipelined(plans, in_host, staging_dev, outs_dev, workspaces, stream):
+    """lop_run_chain_pipelined."""
+    _check(lib().lop_run_chain_pipelined(_ptr_array([p._h.value for p in plans]), len(plans), in_host, staging_dev,
+                                         _ptr_array(outs_dev), _ptr_array(workspaces), stream))
 
 
 class Plan:

@@ -35,6 +35,7 @@ class DeviceChain:
         self.dtype = B.LOP_BF16 if wl.dtype == "bf16" else B.LOP_F32
         self.tdtype = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
         self.keep = []                       # device tensors the plans point into
+        self.per_plan = False                # set once the library declines to run the plans as one chain
         self.plans, self.ws, self.outs = [], [], []
         H, W, C = wl.H, wl.W, wl.C
         with torch.cuda.device(self.device):
@@ -91,8 +92,20 @@ class DeviceChain:
             x_dev = out
         return self.outs[-1]
 
+    def _chain(self):
+        """Several tensor-core plans run as one launch; False when the library wants them one by one."""
+        return len(self.plans) > 1 and not self.per_plan
+
     def run_banded(self, x_dev, stream=None):
         s = self._stream(stream)
+        if self._chain():
+            try:
+                B.run_chain_banded(self.plans, x_dev.data_ptr(), [o.data_ptr() for o in self.outs], [w.data_ptr() for w in self.ws], s)
+                return self.outs[-1]
+            except B.LopError as e:
+                if e.status != -3:
+                    raise
+                self.per_plan = True
         for plan, ws, out in zip(self.plans, self.ws, self.outs):
             plan.run_banded(x_dev.data_ptr(), out.data_ptr(), ws.data_ptr(), s)
             x_dev = out
@@ -109,6 +122,15 @@ class DeviceChain:
     def run_pipelined(self, x_pinned, stream=None):
         """Segment 0 streams its input bands from pinned host memory; later segments run band-wise on the device."""
         s = self._stream(stream)
+        if self._chain():
+            try:
+                B.run_chain_pipelined(self.plans, x_pinned.data_ptr(), self.staging.data_ptr(), [o.data_ptr() for o in self.outs],
+                                      [w.data_ptr() for w in self.ws], s)
+                return self.outs[-1]
+            except B.LopError as e:
+                if e.status != -3:
+                    raise
+                self.per_plan = True
         self.plans[0].run_pipelined(x_pinned.data_ptr(), self.staging.data_ptr(), self.outs[0].data_ptr(),
                                     self.ws[0].data_ptr(), s)
         x_dev = self.outs[0]

@@ -32,9 +32,10 @@ struct MapKey {
 };
 
 struct ProgKey {
-    int kind;                        // -1 whole, -2 all bands, >= 0 one band
-    const void *in, *out, *ws;
-    bool operator<(const ProgKey &o) const { return std::tie(kind, in, out, ws) < std::tie(o.kind, o.in, o.out, o.ws); }
+    int kind;                        // -1 whole, -2 all bands, -3 pipelined, >= 0 one band
+    int n_plans;                     // plans of the chain the program spans
+    const void *in, *out, *ws;       // first plan's input and workspace, last plan's output
+    bool operator<(const ProgKey &o) const { return std::tie(kind, n_plans, in, out, ws) < std::tie(o.kind, o.n_plans, o.in, o.out, o.ws); }
 };
 
 struct ExecState {
@@ -240,26 +241,29 @@ int run_band_impl(lop_plan_t *pl, int band, const void *in, void *out, void *ws,
     return LOP_OK;
 }
 
-// Requests of one band in dependency order; a gathered stem is preceded by its patch-gather stage over the same rows.
-void band_requests(const lop_plan_t *pl, int band, bool wait_arrival, std::vector<StageReq> &reqs)
+// Requests of one band of plan `seg` in dependency order; a gathered stem is preceded by its patch-gather stage over
+// the same rows.
+void band_requests(const lop_plan_t *pl, int seg, int band, bool wait_arrival, std::vector<StageReq> &reqs)
 {
     const int L = (int)pl->layers.size();
     const bool reuse = (pl->flags & LOP_FLAG_REUSE_HALO) != 0;
     for (int i = 0; i < L; ++i) {
         const lop_range &r = pl->ranges[(size_t)band * L + i];
         const int lo = reuse ? r.new_lo : r.out_lo;
-        if (pl->layers[i].stem_gather) reqs.push_back(StageReq{band, i, lo, r.out_hi, wait_arrival, true});
-        reqs.push_back(StageReq{band, i, lo, r.out_hi, wait_arrival, false});
+        if (pl->layers[i].stem_gather) reqs.push_back(StageReq{seg, band, i, lo, r.out_hi, wait_arrival && seg == 0, true, 0});
+        reqs.push_back(StageReq{seg, band, i, lo, r.out_hi, wait_arrival && seg == 0, false, 0});
     }
 }
 
 enum { PROG_WHOLE = -1, PROG_ALL_BANDS = -2, PROG_PIPELINED = -3 };
 
-// kind: PROG_WHOLE, PROG_ALL_BANDS, PROG_PIPELINED, or b >= 0 for band b alone.
-int get_program(lop_plan_t *pl, int kind, const void *in, void *out, void *ws, Program **prog)
+// kind: PROG_WHOLE, PROG_ALL_BANDS, PROG_PIPELINED, or b >= 0 for band b alone (single plan only).  segs: the plans of
+// a chain with their buffers; the program is cached in the first plan.
+int get_program(const std::vector<SegBind> &segs, int kind, Program **prog)
 {
-    ExecState *e = pl->exec;
-    const ProgKey key{kind, in, out, ws};
+    lop_plan_t *pl0 = segs[0].pl;
+    ExecState *e = pl0->exec;
+    const ProgKey key{kind, (int)segs.size(), segs.front().in, segs.back().out, segs.front().ws};
     auto it = e->programs.find(key);
     if (it == e->programs.end()) {
         if (e->programs.size() >= 64) {
@@ -268,41 +272,71 @@ int get_program(lop_plan_t *pl, int kind, const void *in, void *out, void *ws, P
             for (auto &kv : e->programs) program_destroy(kv.second);
             e->programs.clear();
         }
-        const int L = (int)pl->layers.size(), B = pl->n_bands;
         std::vector<StageReq> reqs;
+        long long next = 0;
         if (kind == PROG_WHOLE) {
-            for (int i = 0; i < L; ++i) {
-                if (pl->layers[i].stem_gather) reqs.push_back(StageReq{0, i, 0, pl->layers[i].Ho, false, true});
-                reqs.push_back(StageReq{0, i, 0, pl->layers[i].Ho, false, false});
+            for (int sg = 0; sg < (int)segs.size(); ++sg) {
+                const lop_plan_t *pl = segs[sg].pl;
+                for (int i = 0; i < (int)pl->layers.size(); ++i) {
+                    if (pl->layers[i].stem_gather) reqs.push_back(StageReq{sg, 0, i, 0, pl->layers[i].Ho, false, true, next++});
+                    reqs.push_back(StageReq{sg, 0, i, 0, pl->layers[i].Ho, false, false, next++});
+                }
             }
-        } else if (kind == PROG_ALL_BANDS) {
-            // Input resident: the bands' operations of one layer do not depend on each other, so they are
+        } else if (kind == PROG_ALL_BANDS || kind == PROG_PIPELINED) {
+            // ALL_BANDS (input resident): the bands' operations of one layer do not depend on each other, so they are
             // batched layer by layer (operation batching, Sec. IV-C); dependencies stay per band row group.
-            std::vector<std::vector<StageReq>> per_band(B);
-            for (int b = 0; b < B; ++b) band_requests(pl, b, false, per_band[b]);
-            const size_t per = per_band.empty() ? 0 : per_band[0].size();
-            for (size_t j = 0; j < per; ++j)
-                for (int b = 0; b < B; ++b) reqs.push_back(per_band[b][j]);
-        } else if (kind == PROG_PIPELINED) {
-            // Bands arrive one after the other and each band's stages form a dependency chain, so the stages
-            // are ordered along the diagonals of the (band, stage) grid: while band b is at its first stage,
-            // band b-1 is at its second, and so on -- the pipeline of Sec. IV-B.  Inside a diagonal the deeper
-            // stages come first, so a CTA does not sit on a band that has not arrived while older bands have work.
-            std::vector<std::vector<StageReq>> per_band(B);
-            for (int b = 0; b < B; ++b) band_requests(pl, b, true, per_band[b]);
-            const int per = per_band.empty() ? 0 : (int)per_band[0].size();
-            for (int t = 0; t < B + per - 1; ++t)
-                for (int b = std::max(0, t - per + 1); b <= std::min(t, B - 1); ++b) reqs.push_back(per_band[b][t - b]);
+            // PIPELINED: bands arrive one after the other and each band's stages form a dependency chain, so the
+            // stages are ordered along the diagonals of the (band, stage) grid: while band b is at its first stage,
+            // band b-1 is at its second, and so on -- the pipeline of Sec. IV-B -- and the plans of a chain follow
+            // one another on the same diagonals (a later plan's band needs the previous plan's rows around it, so it
+            // lags by a band; the builder moves a stage back wherever its producers come later still).  Inside a
+            // diagonal the deeper stages come first, so a CTA does not sit on a band that has not arrived while
+            // older bands have work.
+            long long joff = 0;
+            for (int sg = 0; sg < (int)segs.size(); ++sg) {
+                const lop_plan_t *pl = segs[sg].pl;
+                size_t per = 0;
+                for (int b = 0; b < pl->n_bands; ++b) {
+                    std::vector<StageReq> one;
+                    band_requests(pl, sg, b, kind == PROG_PIPELINED, one);
+                    per = one.size();
+                    for (size_t j = 0; j < one.size(); ++j) {
+                        const long long depth = joff + (long long)j;
+                        one[j].prio = kind == PROG_ALL_BANDS ? depth * 65536 + b : (b + depth + sg) * 65536 + (65535 - depth);
+                        reqs.push_back(one[j]);
+                    }
+                }
+                joff += (long long)per;
+            }
+            std::stable_sort(reqs.begin(), reqs.end(), [](const StageReq &x, const StageReq &y) { return x.prio < y.prio; });
         } else {
-            band_requests(pl, kind, false, reqs);
+            band_requests(pl0, 0, kind, false, reqs);
+            for (StageReq &r : reqs) r.prio = next++;
+        }
+        // pipelined: when each band should be on the device.  Measured on the copy stream: a command costs ~4.7 us and
+        // overlaps the previous copy's transfer, which runs at ~64 GB/s; the flag write follows ~5 us behind.
+        std::vector<double> arrival;
+        if (kind == PROG_PIPELINED) {
+            const double row_bytes = (double)pl0->W * pl0->C * elem_size(pl0->dtype) * pl0->N;
+            double t = 5.0;
+            for (int b = 0; b < pl0->n_bands; ++b) {
+                const lop_range &need = pl0->in_need[b];
+                if (need.out_hi > need.new_lo) t += std::max(4.7, (need.out_hi - need.new_lo) * row_bytes / 64e3);
+                arrival.push_back(t + 5.0);
+            }
         }
         Program *p = nullptr;
-        int rc = program_build(pl, reqs, in, out, ws, &p);
+        int rc = program_build(segs, reqs, &p, kind == PROG_PIPELINED ? &arrival : nullptr);
         if (rc != LOP_OK) return rc;
         it = e->programs.emplace(key, p).first;
     }
     *prog = it->second;
     return LOP_OK;
+}
+
+int get_program(lop_plan_t *pl, int kind, const void *in, void *out, void *ws, Program **prog)
+{
+    return get_program(std::vector<SegBind>{SegBind{pl, in, out, ws}}, kind, prog);
 }
 
 int run_program(lop_plan_t *pl, int kind, const void *in, void *out, void *ws, cudaStream_t s)
@@ -490,6 +524,73 @@ int lop_run_pipelined(lop_plan_t *pl, const void *host, void *staging, void *out
         if ((rc = run_band_impl(pl, b, staging, out, ws, s)) != LOP_OK) return rc;
     }
     if (!joined) LOP_CUDA(cudaStreamWaitEvent(s, e->ev_fork, 0));
+    LOP_CUDA(cudaEventRecord(e->ev_end, s));
+    e->timing_valid = true;
+    return LOP_OK;
+}
+
+namespace {
+
+// Validates a chain of plans (plan s+1 consumes plan s's output) and readies every plan for the persistent kernel.
+int chain_prepare(lop_plan_t *const *plans, int n, const void *in0, void *const *outs, void *const *wss, cudaStream_t s,
+                  std::vector<SegBind> &segs)
+{
+    if (!plans || !outs || !wss || n < 1) { set_error("chain: NULL argument or no plan"); return LOP_EINVAL; }
+    const void *in = in0;
+    for (int i = 0; i < n; ++i) {
+        lop_plan_t *pl = plans[i];
+        int rc = check_common(pl, in, outs[i], wss[i]);
+        if (rc != LOP_OK) return rc;
+        if (!pl->exec->wavefront) { set_error("chain: plan %d has a layer the persistent kernel does not take; run the plans one by one", i); return LOP_EUNSUPPORTED; }
+        if (i > 0) {
+            const lop_plan_t *pv = plans[i - 1];
+            const LayerInfo &last = pv->layers.back();
+            if (pl->N != pv->N || pl->H != last.Ho || pl->W != last.Wo || pl->C != last.Co || pl->dtype != pv->dtype ||
+                (pl->flags & LOP_FLAG_REUSE_HALO) != (pv->flags & LOP_FLAG_REUSE_HALO)) {
+                set_error("chain: plan %d does not take plan %d's output (shape, dtype or halo mode differ)", i, i - 1);
+                return LOP_ESHAPE;
+            }
+        }
+        pl->exec->launches = pl->exec->copies = 0;
+        pl->exec->last_stream = s;
+        if ((rc = prepare_workspace(pl, wss[i], s)) != LOP_OK) return rc;
+        segs.push_back(SegBind{pl, in, outs[i], wss[i]});
+        in = outs[i];
+    }
+    return LOP_OK;
+}
+
+}  // namespace
+
+int lop_run_chain_banded(lop_plan_t *const *plans, int n_plans, const void *in_dev, void *const *outs_dev, void *const *workspaces,
+                         void *stream)
+{
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    std::vector<SegBind> segs;
+    int rc = chain_prepare(plans, n_plans, in_dev, outs_dev, workspaces, s, segs);
+    if (rc != LOP_OK) return rc;
+    Program *p = nullptr;
+    if ((rc = get_program(segs, PROG_ALL_BANDS, &p)) != LOP_OK) return rc;
+    if (program_empty(p)) return LOP_OK;
+    if ((rc = program_launch(p, s)) != LOP_OK) return rc;
+    plans[0]->exec->launches++;
+    return LOP_OK;
+}
+
+int lop_run_chain_pipelined(lop_plan_t *const *plans, int n_plans, const void *host, void *staging, void *const *outs_dev,
+                            void *const *workspaces, void *stream)
+{
+    if (!host) { set_error("lop_run_chain_pipelined: host input is NULL"); return LOP_EINVAL; }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    std::vector<SegBind> segs;
+    int rc = chain_prepare(plans, n_plans, staging, outs_dev, workspaces, s, segs);
+    if (rc != LOP_OK) return rc;
+    ExecState *e = plans[0]->exec;
+    e->timing_valid = false;
+    LOP_CUDA(cudaEventRecord(e->ev_begin, s));
+    Program *p = nullptr;
+    if ((rc = get_program(segs, PROG_PIPELINED, &p)) != LOP_OK) return rc;
+    if ((rc = enqueue_pipelined(plans[0], p, host, staging, s)) != LOP_OK) return rc;
     LOP_CUDA(cudaEventRecord(e->ev_end, s));
     e->timing_valid = true;
     return LOP_OK;

@@ -6,6 +6,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <cmath>
 #include <vector>
 
 #include "lop_internal.h"
@@ -111,7 +112,7 @@ Geom choose_geom(const ConvArgs &a, int rows, bool even_tiles)
     return g;
 }
 
-struct MapSet { int layer, P, RI, TN, BN, BK, tb, base; };
+struct MapSet { int seg, layer, P, RI, TN, BN, BK, tb, base; };
 
 // Five tensor maps of a convolution stage: the activation seen through the (row parity, column parity)
 // classes of its stride, and the weights as [tap][cout][cin].
@@ -181,12 +182,151 @@ bool program_supported(const lop_plan_t *pl)
     return true;
 }
 
-int program_build(lop_plan_t *pl, const std::vector<StageReq> &reqs, const void *in, void *out, void *ws, Program **result)
+namespace {
+
+// What a request reads: rows of tensors produced inside the program, and whether it touches the raw chain input
+// (only plan 0 can: a later plan's "input" is the previous plan's last layer).
+struct Need { int tensor, lo, hi; bool same_seg; };
+struct Reads { Need need[3]; int n = 0; bool raw = false; };
+
+struct Ctx {
+    const std::vector<SegBind> &segs;
+    std::vector<int> base;              // first tensor id of each plan; id base+layer, base+L = the stem's patches
+    int tensor_id(int seg, int layer) const { return base[seg] + layer; }
+    int patches_id(int seg) const { return base[seg] + (int)segs[seg].pl->layers.size(); }
+    int input_id(int seg) const { return tensor_id(seg - 1, (int)segs[seg - 1].pl->layers.size() - 1); }
+};
+
+// Rows [o0, o1) of request rq: the tensors and rows they are computed from (Sec. IV-B: a dependency exists as soon as
+// any part of a producer's output is used).
+Reads reads_of(const Ctx &cx, const StageReq &rq, int o0, int o1)
+{
+    Reads r;
+    const lop_plan_t *pl = cx.segs[rq.seg].pl;
+    const LayerInfo &li = pl->layers[rq.layer];
+    const lop_layer &l = li.l;
+    auto window = [&](int &a_out, int &b_out) {
+        long long a = (long long)o0 * l.sh - l.ph, b = (long long)(o1 - 1) * l.sh - l.ph + (long long)(l.kh - 1) * l.dh;
+        a = std::max(a, 0LL); b = std::min(b, (long long)li.Hin - 1);
+        a_out = (int)a; b_out = (int)b + 1;
+        return a <= b;
+    };
+    int a = 0, b = 0;
+    if (rq.gather || (l.input_from == LOP_INPUT && !li.stem_gather)) {
+        if (rq.seg == 0) r.raw = true;
+        else if (window(a, b)) r.need[r.n++] = Need{cx.input_id(rq.seg), a, b, false};
+    } else if (li.stem_gather) {
+        r.need[r.n++] = Need{cx.patches_id(rq.seg), o0, o1, true};            // the patches of exactly these rows
+    } else if (window(a, b)) {
+        r.need[r.n++] = Need{cx.tensor_id(rq.seg, l.input_from), a, b, true};
+    }
+    if (!rq.gather && l.op == LOP_CONV2D && l.residual_from != LOP_NO_RESIDUAL) {
+        if (l.residual_from >= 0) r.need[r.n++] = Need{cx.tensor_id(rq.seg, l.residual_from), o0, o1, true};
+        else if (rq.seg == 0) r.raw = true;
+        else r.need[r.n++] = Need{cx.input_id(rq.seg), o0, o1, false};
+    }
+    return r;
+}
+
+// Rough time, in microseconds, one stage keeps the machine busy: its items over the SMs, an item costing a fixed part
+// plus its tensor-core instructions (about 0.06 us each, issued by one thread).  Only used to order stages.
+double stage_cost_us(const Ctx &cx, const StageReq &rq)
+{
+    const lop_plan_t *pl = cx.segs[rq.seg].pl;
+    const LayerInfo &li = pl->layers[rq.layer];
+    const double rows = rq.hi - rq.lo;
+    if (rq.gather || li.l.op == LOP_MAXPOOL2D) return 1.0 + 3.0 * std::ceil(rows * pl->N / 148.0);
+    const double tiles = std::ceil(rows * li.Wo * pl->N / 128.0) * std::max(1, li.l.cout / 128);
+    const double item = 1.5 + 0.06 * li.l.kh * li.l.kw * (li.cin_eff / 16.0);
+    return 1.0 + item * std::ceil(tiles / 148.0);
+}
+
+// Puts the requests into ascending priority as far as dependencies allow (a stable topological order).  With
+// arrival_us (when each band of plan 0 is expected on the device) the priorities are first replaced by each stage's
+// earliest possible start under that arrival schedule, so that stages of later plans fill the time in which the
+// first plan waits for its input.
+int order_requests(const Ctx &cx, std::vector<StageReq> &reqs, bool reuse, const std::vector<double> *arrival_us)
+{
+    const size_t n = reqs.size();
+    std::vector<int> produces(n);
+    for (size_t i = 0; i < n; ++i)
+        produces[i] = reqs[i].gather ? cx.patches_id(reqs[i].seg) : cx.tensor_id(reqs[i].seg, reqs[i].layer);
+    bool sorted_already = arrival_us == nullptr;
+    for (size_t i = 1; i < n; ++i)
+        if (reqs[i].prio < reqs[i - 1].prio) sorted_already = false;
+    std::vector<std::vector<int>> users(n), prods(n);
+    std::vector<char> raw(n, 0);
+    for (size_t i = 0; i < n; ++i) {
+        const Reads r = reads_of(cx, reqs[i], reqs[i].lo, reqs[i].hi);
+        raw[i] = r.raw;
+        for (int q = 0; q < r.n; ++q)
+            for (size_t j = 0; j < n; ++j) {
+                if (j == i || produces[j] != r.need[q].tensor) continue;
+                if (!reuse && r.need[q].same_seg && reqs[j].band != reqs[i].band) continue;
+                if (std::max(r.need[q].lo, reqs[j].lo) >= std::min(r.need[q].hi, reqs[j].hi)) continue;
+                users[j].push_back((int)i);
+                prods[i].push_back((int)j);
+                if (j > i) sorted_already = false;
+            }
+    }
+    if (sorted_already) return LOP_OK;
+    auto kahn = [&](std::vector<int> &order) {
+        auto later = [&](int x, int y) { return reqs[x].prio != reqs[y].prio ? reqs[x].prio > reqs[y].prio : x > y; };
+        std::vector<int> pending(n), heap;
+        for (size_t i = 0; i < n; ++i) {
+            pending[i] = (int)prods[i].size();
+            if (!pending[i]) heap.push_back((int)i);
+        }
+        std::make_heap(heap.begin(), heap.end(), later);
+        order.clear();
+        while (!heap.empty()) {
+            std::pop_heap(heap.begin(), heap.end(), later);
+            const int i = heap.back();
+            heap.pop_back();
+            order.push_back(i);
+            for (int u : users[i])
+                if (--pending[u] == 0) { heap.push_back(u); std::push_heap(heap.begin(), heap.end(), later); }
+        }
+        return order.size() == n;
+    };
+    std::vector<int> order;
+    if (!kahn(order)) { set_error("the stage requests depend on each other in a cycle"); return LOP_EINVAL; }
+    if (arrival_us) {
+        std::vector<double> end(n, 0.0);
+        for (int i : order) {
+            double start = 0.0;
+            if (raw[i] && reqs[i].wait_arrival && reqs[i].band < (int)arrival_us->size()) start = (*arrival_us)[reqs[i].band];
+            for (int j : prods[i]) start = std::max(start, end[j]);
+            end[i] = start + stage_cost_us(cx, reqs[i]);
+            reqs[i].prio = (long long)(start * 1000.0);
+        }
+        if (!kahn(order)) { set_error("the stage requests depend on each other in a cycle"); return LOP_EINVAL; }
+    }
+    std::vector<StageReq> out;
+    out.reserve(n);
+    for (int i : order) out.push_back(reqs[i]);
+    reqs.swap(out);
+    return LOP_OK;
+}
+
+}  // namespace
+
+int program_build(const std::vector<SegBind> &segs, std::vector<StageReq> reqs, Program **result, const std::vector<double> *arrival_us)
 {
     *result = nullptr;
-    const int L = (int)pl->layers.size();
-    const bool reuse = (pl->flags & LOP_FLAG_REUSE_HALO) != 0;
-    char *wsb = static_cast<char *>(ws);
+    if (segs.empty()) { set_error("program_build: no plan"); return LOP_EINVAL; }
+    const bool reuse = (segs[0].pl->flags & LOP_FLAG_REUSE_HALO) != 0;
+    Ctx cx{segs, {}};
+    int n_tensors = 0;
+    for (const SegBind &sb : segs) { cx.base.push_back(n_tensors); n_tensors += (int)sb.pl->layers.size() + 1; }
+    {
+        std::vector<StageReq> live;
+        for (const StageReq &rq : reqs)
+            if (rq.hi > rq.lo) live.push_back(rq);
+        reqs.swap(live);
+    }
+    int orc = order_requests(cx, reqs, reuse, arrival_us);
+    if (orc != LOP_OK) return orc;
 
     std::vector<WfStage> stages;
     std::vector<int> stage_band, stage_rows_per_group;
@@ -194,7 +334,7 @@ int program_build(lop_plan_t *pl, const std::vector<StageReq> &reqs, const void 
     std::vector<CUtensorMap> maps;
     std::vector<MapSet> mapsets;
     std::vector<int2> deps;
-    std::vector<std::vector<int>> by_tensor(L + 1);     // stage indices per produced tensor; index L: the stem's patches
+    std::vector<std::vector<int>> by_tensor(n_tensors);   // stage indices per produced tensor
     std::vector<int> expected;                         // completions per row group, per stage
     int n_ctr = WF_CTR_FIRST;
     bool uses_flags = false;
@@ -204,15 +344,19 @@ int program_build(lop_plan_t *pl, const std::vector<StageReq> &reqs, const void 
     std::vector<int> prod_lo, prod_hi;                     // per stage: rows of the tensor it produces
     for (size_t ri = 0; ri < reqs.size(); ++ri) {
         const StageReq &rq = reqs[ri];
-        if (rq.hi <= rq.lo || consumed[ri]) continue;
+        if (consumed[ri]) continue;
         if (stages.size() >= 65535) { set_error("program has too many stages"); return LOP_EUNSUPPORTED; }
+        lop_plan_t *pl = segs[rq.seg].pl;
+        const void *in = segs[rq.seg].in;
+        void *out = segs[rq.seg].out, *ws = segs[rq.seg].ws;
+        char *wsb = static_cast<char *>(ws);
         const LayerInfo &li = pl->layers[rq.layer];
         const lop_layer &l = li.l;
         WfStage st{};
         st.oh_lo = rq.lo; st.oh_hi = rq.hi;
         const int rows = rq.hi - rq.lo;
         int group_rows = 1, tiles_r = rows, tiles_w = 1, tiles_n = pl->N, cout_tiles = 1;
-        int produces = rq.gather ? L : rq.layer;
+        int produces = rq.gather ? cx.patches_id(rq.seg) : cx.tensor_id(rq.seg, rq.layer);
         int out_lo = rq.lo, out_hi = rq.hi;                    // rows of the produced tensor
         if (rq.gather) {
             st.kind = WF_GATHER;
@@ -236,8 +380,8 @@ int program_build(lop_plan_t *pl, const std::vector<StageReq> &reqs, const void 
             size_t rj = reqs.size();
             if (pool_fusable(pl, rq.layer))
                 for (size_t k = 0; k < reqs.size(); ++k)
-                    if (!consumed[k] && !reqs[k].gather && reqs[k].band == rq.band && reqs[k].layer == rq.layer + 1 &&
-                        reqs[k].hi > reqs[k].lo && rq.lo == 2 * reqs[k].lo && rq.hi == 2 * reqs[k].hi) { rj = k; break; }
+                    if (!consumed[k] && !reqs[k].gather && reqs[k].seg == rq.seg && reqs[k].band == rq.band &&
+                        reqs[k].layer == rq.layer + 1 && rq.lo == 2 * reqs[k].lo && rq.hi == 2 * reqs[k].hi) { rj = k; break; }
             const bool fuse = rj < reqs.size();
             const Geom g = choose_geom(a, rows, fuse);
             st.kind = WF_CONV;
@@ -248,7 +392,8 @@ int program_build(lop_plan_t *pl, const std::vector<StageReq> &reqs, const void 
             st.act = a.act; st.res_pos = a.res_pos;
             int base = -1;
             for (const MapSet &m : mapsets)
-                if (m.layer == rq.layer && m.P == g.P && m.RI == g.RI && m.TN == g.TN && m.BN == g.BN && m.BK == g.BK && m.tb == g.tb)
+                if (m.seg == rq.seg && m.layer == rq.layer && m.P == g.P && m.RI == g.RI && m.TN == g.TN && m.BN == g.BN && m.BK == g.BK &&
+                    m.tb == g.tb)
                     base = m.base;
             CUtensorMap cm[5];
             int mask = 0;
@@ -257,7 +402,7 @@ int program_build(lop_plan_t *pl, const std::vector<StageReq> &reqs, const void 
             if (base < 0) {
                 base = (int)maps.size();
                 for (int i = 0; i < 5; ++i) maps.push_back(cm[i]);
-                mapsets.push_back(MapSet{rq.layer, g.P, g.RI, g.TN, g.BN, g.BK, g.tb, base});
+                mapsets.push_back(MapSet{rq.seg, rq.layer, g.P, g.RI, g.TN, g.BN, g.BK, g.tb, base});
             }
             st.map_base = base;
             st.a_valid_mask = mask;
@@ -277,7 +422,7 @@ int program_build(lop_plan_t *pl, const std::vector<StageReq> &reqs, const void 
                 consumed[rj] = 1;
                 st.fuse_pool = 1; st.pool_Ho = pool.Ho; st.pool_Wo = pool.Wo;
                 st.y = const_cast<void *>(tensor_of(pl, rq.layer + 1, in, out, ws));
-                produces = rq.layer + 1;
+                produces = cx.tensor_id(rq.seg, rq.layer + 1);
                 out_lo = reqs[rj].lo; out_hi = reqs[rj].hi;
             }
             group_rows = g.TR;
@@ -296,27 +441,11 @@ int program_build(lop_plan_t *pl, const std::vector<StageReq> &reqs, const void 
         const int sidx = (int)stages.size();
 
         // ---- dependencies of every row group of this stage on earlier stages of this program
-        struct Need { int tensor, lo, hi; };
         for (int tr = 0; tr < tiles_r; ++tr) {
             const int o0 = rq.lo + tr * group_rows, o1 = std::min(o0 + group_rows, rq.hi);
-            Need needs[2];
-            int nn = 0;
-            bool raw = rq.gather;                                   // reads the chain input itself
-            if (!rq.gather) {
-                if (li.stem_gather) {
-                    needs[nn++] = Need{L, o0, o1};                  // the patches of exactly these rows
-                } else if (l.input_from == LOP_INPUT) {
-                    raw = true;
-                } else {
-                    long long a = (long long)o0 * l.sh - l.ph, b = (long long)(o1 - 1) * l.sh - l.ph + (long long)(l.kh - 1) * l.dh;
-                    a = std::max(a, 0LL); b = std::min(b, (long long)li.Hin - 1);
-                    if (a <= b) needs[nn++] = Need{l.input_from, (int)a, (int)b + 1};
-                }
-                if (l.op == LOP_CONV2D && l.residual_from >= 0) needs[nn++] = Need{l.residual_from, o0, o1};
-                if (l.op == LOP_CONV2D && l.residual_from == LOP_INPUT) raw = true;
-            }
+            const Reads rd = reads_of(cx, rq, o0, o1);
             const int first = (int)deps.size();
-            if (rq.wait_arrival && raw) {
+            if (rq.wait_arrival && rd.raw) {
                 // every band whose transfer brought rows this band reads (its own, and earlier ones for the halo); no
                 // assumption is made about the order in which arrivals become visible
                 const lop_range &mine = pl->in_need[rq.band];
@@ -327,11 +456,11 @@ int program_build(lop_plan_t *pl, const std::vector<StageReq> &reqs, const void 
                 }
                 uses_flags = true;
             }
-            for (int q = 0; q < nn; ++q)
-                for (int ps : by_tensor[needs[q].tensor]) {
-                    if (!reuse && stage_band[ps] != rq.band) continue;
+            for (int q = 0; q < rd.n; ++q)
+                for (int ps : by_tensor[rd.need[q].tensor]) {
+                    if (!reuse && rd.need[q].same_seg && stage_band[ps] != rq.band) continue;
                     const WfStage &p = stages[ps];
-                    const int lo = std::max(needs[q].lo, prod_lo[ps]), hi = std::min(needs[q].hi, prod_hi[ps]);
+                    const int lo = std::max(rd.need[q].lo, prod_lo[ps]), hi = std::min(rd.need[q].hi, prod_hi[ps]);
                     if (lo >= hi) continue;
                     const int gr = stage_rows_per_group[ps];
                     for (int g = (lo - prod_lo[ps]) / gr; g <= (hi - 1 - prod_lo[ps]) / gr; ++g)
@@ -353,11 +482,12 @@ int program_build(lop_plan_t *pl, const std::vector<StageReq> &reqs, const void 
         expected.push_back(exp_here);
     }
 
+    lop_plan_t *pl0 = segs[0].pl;
     Program *p = new (std::nothrow) Program();
     if (!p) { set_error("out of host memory"); return LOP_ENOMEM; }
     if (uses_flags) {                                        // arrival flags live after the row-group counters
         p->flag_base = n_ctr;
-        p->n_flags = pl->n_bands;
+        p->n_flags = pl0->n_bands;
         for (int2 &d : deps)
             if (d.x < 0) d.x = p->flag_base + (-1 - d.x);
         n_ctr += p->n_flags;
@@ -405,7 +535,7 @@ int program_build(lop_plan_t *pl, const std::vector<StageReq> &reqs, const void 
     P.maps = reinterpret_cast<const CUtensorMap *>(d + o_maps);
     P.deps = reinterpret_cast<const int2 *>(d + o_deps);
     P.counters = p->counters;
-    P.status = reinterpret_cast<unsigned *>(wsb + pl->status_off);
+    P.status = reinterpret_cast<unsigned *>(static_cast<char *>(segs[0].ws) + pl0->status_off);
     P.flag_base = p->flag_base; P.n_flags = p->n_flags;
     P.n_stages = (int)stages.size();
     P.n_items = n_items;

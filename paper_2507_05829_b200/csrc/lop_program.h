@@ -8,16 +8,24 @@
 
 namespace lop {
 
-// Rows [lo, hi) of a layer for one band.  gather: the patch-gather stage that precedes a gathered stem layer
-// (same rows).  wait_arrival: stages that read the raw chain input wait for their band's arrival flag
-// (single-launch pipelined programs).
-struct StageReq { int band, layer, lo, hi; bool wait_arrival; bool gather; };
+// One plan of a chain with its buffers bound: `in` is the plan's input tensor (for plan s > 0 the output of plan
+// s-1), `out` its last layer's output, `ws` its workspace.
+struct SegBind { lop_plan_t *pl; const void *in; void *out; void *ws; };
+
+// Rows [lo, hi) of a layer of plan `seg` for one band.  gather: the patch-gather stage that precedes a gathered stem
+// layer (same rows).  wait_arrival: stages of plan 0 that read the raw chain input wait for the arrival flags of the
+// bands that bring their rows (single-launch pipelined programs).  prio: stages are put into the program in
+// ascending priority, as far as their dependencies allow (a stage never precedes one it reads from).
+struct StageReq { int seg, band, layer, lo, hi; bool wait_arrival; bool gather; long long prio; };
 struct Program;
 
 bool program_supported(const lop_plan_t *pl);
-int program_build(lop_plan_t *pl, const std::vector<StageReq> &reqs, const void *in, void *out, void *ws, Program **result);
+// arrival_us (optional): expected arrival time of each band of plan 0; stages are then ordered by their earliest
+// possible start under that schedule instead of by prio.
+int program_build(const std::vector<SegBind> &segs, std::vector<StageReq> reqs, Program **result,
+                  const std::vector<double> *arrival_us = nullptr);
 int program_launch(Program *p, cudaStream_t s);
-// Device address of band b's arrival flag (a 4-byte word the copy stream sets non-zero), or nullptr.
+// Device address of band b's arrival flag (a 4-byte word a side stream sets non-zero), or nullptr.
 unsigned *program_arrival_flag(Program *p, int band);
 bool program_empty(const Program *p);
 void program_destroy(Program *p);

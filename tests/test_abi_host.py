@@ -95,6 +95,8 @@ def test_errors_are_reported_not_raised_in_c():
     assert L.lop_plan_num_bands(None) == -1 and L.lop_plan_get_range(None, 0, 0, None) == -1
     assert L.lop_strerror(-5) == b"CUDA error" and L.lop_strerror(0) == b"success"
     L.lop_plan_destroy(None)
+    assert L.lop_run_chain_banded(None, 0, None, None, None, None) == -1
+    assert L.lop_run_chain_pipelined(None, 1, None, None, None, None, None) == -1
     p = lop.Plan([good], 1, 8, 8, 4, lop.LOP_F32, 2)
     with pytest.raises(lop.LopError):
         p.get_range(2, 0)

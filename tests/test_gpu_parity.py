@@ -185,6 +185,57 @@ def test_tensor_core_and_cuda_core_paths_agree():
         assert rel_err(x, y) <= 2e-2
 
 
+# ------------------------------------------------------------------------------------ several plans, one launch
+def _chain_args(dc):
+    return [o.data_ptr() for o in dc.outs], [w.data_ptr() for w in dc.ws]
+
+
+@pytest.mark.parametrize("flags", [0, lop.LOP_FLAG_REUSE_HALO])
+def test_chain_entry_points_run_all_plans_in_one_launch(flags):
+    """lop_run_chain_*: one persistent launch for the whole multi-segment network, same bits as plan after plan."""
+    wl = li.build("resnet18", H=64, W=64)
+    ref = DeviceChain(wl, flags=flags)
+    ref.per_plan = True                                  # the plans one by one
+    ref.run_banded(ref.input_tensor())
+    torch.cuda.synchronize()
+    assert sum(p.last_launches() for p in ref.plans) >= len(ref.plans) > 1
+    s = torch.cuda.current_stream().cuda_stream
+    for mode in ("banded", "pipelined"):
+        dc = DeviceChain(wl, flags=flags)
+        outs, wss = _chain_args(dc)
+        x_dev, x_host = dc.input_tensor(), dc.pinned_input()
+        for call in range(2):                            # the first call also pads the stem's weights, once
+            if mode == "banded":
+                lop.run_chain_banded(dc.plans, x_dev.data_ptr(), outs, wss, s)
+            else:
+                lop.run_chain_pipelined(dc.plans, x_host.data_ptr(), dc.staging.data_ptr(), outs, wss, s)
+            torch.cuda.synchronize()
+        dc.check_device()
+        assert dc.plans[0].last_launches() == 1 and all(p.last_launches() == 0 for p in dc.plans[1:])
+        for a, b in zip(ref.outs, dc.outs):
+            assert torch.equal(a, b), mode
+
+
+def test_chain_entry_points_refuse_plans_that_do_not_follow_each_other():
+    wl = li.build("resnet18", H=64, W=64)
+    dc = DeviceChain(wl)
+    outs, wss = _chain_args(dc)
+    s = torch.cuda.current_stream().cuda_stream
+    x = dc.input_tensor()
+    with pytest.raises(lop.LopError) as e:                 # plan 3 does not take plan 0's output
+        lop.run_chain_banded([dc.plans[0], dc.plans[3]], x.data_ptr(), [outs[0], outs[3]], [wss[0], wss[3]], s)
+    assert e.value.status == -2
+    simt = DeviceChain(wl, flags=lop.LOP_FLAG_FORCE_SIMT)  # CUDA-core plans are not taken by the persistent kernel
+    o2, w2 = _chain_args(simt)
+    with pytest.raises(lop.LopError) as e:
+        lop.run_chain_banded(simt.plans, simt.input_tensor().data_ptr(), o2, w2, s)
+    assert e.value.status == -3
+    simt.run_banded(simt.input_tensor())                   # the wrapper falls back to plan after plan
+    torch.cuda.synchronize()
+    assert simt.per_plan
+    assert rel_err(to_host_f32(simt.outs[-1]), ochain.run_workload(wl)) <= TOL["bf16"]
+
+
 # ------------------------------------------------------------------------------------ edge cases
 def test_very_wide_image_gathers_patches_without_staging_rows():
     """Three rows of a 4200-pixel image do not fit the shared staging tile: the gather reads the image in place."""
