@@ -56,8 +56,10 @@ enum {
                                      independent of the others (operation replication, Sec. IV-C) */
     LOP_FLAG_TIME_LAYERS = 2u,    /* record a CUDA event pair around every (band, layer) launch    */
     LOP_FLAG_FORCE_SIMT = 4u,     /* never use the tensor-core convolution (second on-GPU opinion) */
-    LOP_FLAG_PER_LAYER = 8u       /* one kernel launch per (band, layer) instead of one persistent
+    LOP_FLAG_PER_LAYER = 8u,      /* one kernel launch per (band, layer) instead of one persistent
                                      wavefront launch per call / per band                          */
+    LOP_FLAG_COPY_ENGINE = 16u    /* pipelined runs always move the bands with copy-engine copies on
+                                     a side stream, also when the kernel could fetch them itself  */
 };
 
 /*
@@ -139,7 +141,11 @@ double lop_plan_flops(const lop_plan_t *plan);
  * address row ranges inside them.  stream is a cudaStream_t passed as void* (NULL = legacy
  * default stream).  The first execution call on a plan for a given (input, output, workspace)
  * triple creates the side stream, events and program tables (cudaMalloc + synchronous uploads):
- * make it outside any stream capture; later calls with the same buffers allocate nothing. */
+ * make it outside any stream capture; later calls with the same buffers allocate nothing.
+ * out_dev (the LAST plan's, for a chain) may also be page-locked host memory that the device can
+ * address (cudaHostAlloc / cudaHostRegister): nothing reads the output tensor back, so the last
+ * layer's kernels then store the result rows straight to host memory as they are finished --
+ * the result's transfer overlaps the computation and no device-to-host copy is needed. */
 
 /* Whole-tensor execution: every layer over all its rows (the unpartitioned reference order). */
 int lop_run_whole(lop_plan_t *plan, const void *in_dev, void *out_dev, void *workspace, void *stream);
@@ -155,11 +161,20 @@ int lop_run_banded(lop_plan_t *plan, const void *in_dev, void *out_dev, void *wo
  * the chain-input rows the band needs and no earlier band has brought, for all N images, from
  * in_host_pinned (PINNED HOST, full-size tensor) to the same rows of staging_dev. */
 int lop_copy_band(lop_plan_t *plan, int band, const void *in_host_pinned, void *staging_dev, void *stream);
-/* Band pipeline (Sec. IV-B computation/transmission overlap): band i+1's rows are copied on the
- * plan's side stream while band i is computed on the caller's stream.  CUDA events fork and join
- * the side stream; inside the run a band's arrival is a 4-byte stream-ordered write behind its
- * copy that the persistent kernel polls (per-layer launches wait on one event per band instead).
- * Returns after enqueueing.  staging_dev: lop_plan_staging_bytes() bytes. */
+/* Band pipeline (Sec. IV-B computation/transmission overlap): band i+1's rows come in while band i is
+ * computed.  Two transports:
+ *   - fetched (default when in_host_pinned is mapped into the device's address space, as cudaHostAlloc /
+ *     cudaHostRegister memory is): the persistent kernel itself reads each band's rows from host memory
+ *     and stores them to staging_dev -- fetch stages that precede the band's first operator in the
+ *     dependency graph, spread over the SMs -- so the whole request is ONE launch on the caller's stream
+ *     with no copy, event or flag command at all;
+ *   - copy engine (LOP_FLAG_COPY_ENGINE, unmapped host memory, or plans the persistent kernel does not
+ *     take): one asynchronous copy per band on the plan's side stream, forked and joined by CUDA events;
+ *     a band's arrival is a 4-byte stream-ordered write behind its copy that the persistent kernel polls
+ *     (per-layer launches wait on one event per band instead).
+ * Both leave the input in staging_dev and give the same output bits.  Returns after enqueueing; the
+ * host buffer must stay unchanged until the stream has passed the call.  staging_dev:
+ * lop_plan_staging_bytes() bytes. */
 int lop_run_pipelined(lop_plan_t *plan, const void *in_host_pinned, void *staging_dev, void *out_dev,
                       void *workspace, void *stream);
 /* ---- several plans as one chain (Sec. III-A: later operators start as soon as the rows they
@@ -183,7 +198,9 @@ int lop_run_chain_banded(lop_plan_t *const *plans, int n_plans, const void *in_d
 int lop_run_chain_pipelined(lop_plan_t *const *plans, int n_plans, const void *in_host_pinned, void *staging_dev,
                             void *const *outs_dev, void *const *workspaces, void *stream);
 
-/* Event times of the last lop_run_pipelined call.  SYNCHRONISES with that call's completion. */
+/* Event times of the last lop_run_pipelined call of a plan made with LOP_FLAG_TIME_LAYERS (other plans
+ * record no events -- each would be one more command on the stream -- and get LOP_EINVAL).
+ * SYNCHRONISES with that call's completion. */
 int lop_plan_last_timing(lop_plan_t *plan, lop_timing *out);
 /* With LOP_FLAG_TIME_LAYERS (implies per-layer launches): device time in ms of the (band, layer) launch of the last
  * lop_run_band / banded / pipelined call (band = -1: last lop_run_whole).  SYNCHRONISES.

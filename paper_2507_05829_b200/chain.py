@@ -119,25 +119,27 @@ class DeviceChain:
             x_dev = out
         return self.outs[-1]
 
-    def run_pipelined(self, x_pinned, stream=None):
-        """Segment 0 streams its input bands from pinned host memory; later segments run band-wise on the device."""
+    def run_pipelined(self, x_pinned, stream=None, out_pinned=None):
+        """Segment 0 streams its input bands from pinned host memory; later segments run band-wise on the device.
+
+        out_pinned: a pinned host tensor of the last output's shape; the last layer's kernels then store the result
+        straight into it (every execution call takes device-addressable host memory as its output tensor)."""
         s = self._stream(stream)
+        outs = [o.data_ptr() for o in self.outs]
+        if out_pinned is not None:
+            outs[-1] = out_pinned.data_ptr()
         if self._chain():
             try:
-                B.run_chain_pipelined(self.plans, x_pinned.data_ptr(), self.staging.data_ptr(), [o.data_ptr() for o in self.outs],
-                                      [w.data_ptr() for w in self.ws], s)
-                return self.outs[-1]
+                B.run_chain_pipelined(self.plans, x_pinned.data_ptr(), self.staging.data_ptr(), outs, [w.data_ptr() for w in self.ws], s)
+                return self.outs[-1] if out_pinned is None else out_pinned
             except B.LopError as e:
                 if e.status != -3:
                     raise
                 self.per_plan = True
-        self.plans[0].run_pipelined(x_pinned.data_ptr(), self.staging.data_ptr(), self.outs[0].data_ptr(),
-                                    self.ws[0].data_ptr(), s)
-        x_dev = self.outs[0]
-        for plan, ws, out in list(zip(self.plans, self.ws, self.outs))[1:]:
-            plan.run_banded(x_dev.data_ptr(), out.data_ptr(), ws.data_ptr(), s)
-            x_dev = out
-        return self.outs[-1]
+        self.plans[0].run_pipelined(x_pinned.data_ptr(), self.staging.data_ptr(), outs[0], self.ws[0].data_ptr(), s)
+        for i in range(1, len(self.plans)):
+            self.plans[i].run_banded(outs[i - 1], outs[i], self.ws[i].data_ptr(), s)
+        return self.outs[-1] if out_pinned is None else out_pinned
 
     def check_device(self):
         for plan, ws in zip(self.plans, self.ws):

@@ -32,10 +32,14 @@ struct MapKey {
 };
 
 struct ProgKey {
-    int kind;                        // -1 whole, -2 all bands, -3 pipelined, >= 0 one band
+    int kind;                        // -1 whole, -2 all bands, -3 pipelined, -4 pipelined with in-kernel fetch, >= 0 one band
     int n_plans;                     // plans of the chain the program spans
     const void *in, *out, *ws;       // first plan's input and workspace, last plan's output
-    bool operator<(const ProgKey &o) const { return std::tie(kind, n_plans, in, out, ws) < std::tie(o.kind, o.n_plans, o.in, o.out, o.ws); }
+    const void *src;                 // fetch source (host memory as the device addresses it) or nullptr
+    bool operator<(const ProgKey &o) const
+    {
+        return std::tie(kind, n_plans, in, out, ws, src) < std::tie(o.kind, o.n_plans, o.in, o.out, o.ws, o.src);
+    }
 };
 
 struct ExecState {
@@ -58,6 +62,7 @@ struct ExecState {
     int copies = 0;                                            // async copies enqueued by it
     bool timing_valid = false;
     bool copies_timed = false;                                 // per-band copy events were recorded by the last pipelined run
+    const void *mapped_host = nullptr, *mapped_dev = nullptr;  // last host buffer looked up and its device-side address (or nullptr)
     std::vector<char> copy_issued;
 };
 
@@ -255,15 +260,16 @@ void band_requests(const lop_plan_t *pl, int seg, int band, bool wait_arrival, s
     }
 }
 
-enum { PROG_WHOLE = -1, PROG_ALL_BANDS = -2, PROG_PIPELINED = -3 };
+enum { PROG_WHOLE = -1, PROG_ALL_BANDS = -2, PROG_PIPELINED = -3, PROG_FETCHED = -4 };
 
-// kind: PROG_WHOLE, PROG_ALL_BANDS, PROG_PIPELINED, or b >= 0 for band b alone (single plan only).  segs: the plans of
-// a chain with their buffers; the program is cached in the first plan.
-int get_program(const std::vector<SegBind> &segs, int kind, Program **prog)
+// kind: PROG_WHOLE, PROG_ALL_BANDS, PROG_PIPELINED, PROG_FETCHED (fetch_src: the host input as the device addresses
+// it), or b >= 0 for band b alone (single plan only).  segs: the plans of a chain with their buffers; the program is
+// cached in the first plan.
+int get_program(const std::vector<SegBind> &segs, int kind, Program **prog, const void *fetch_src = nullptr)
 {
     lop_plan_t *pl0 = segs[0].pl;
     ExecState *e = pl0->exec;
-    const ProgKey key{kind, (int)segs.size(), segs.front().in, segs.back().out, segs.front().ws};
+    const ProgKey key{kind, (int)segs.size(), segs.front().in, segs.back().out, segs.front().ws, fetch_src};
     auto it = e->programs.find(key);
     if (it == e->programs.end()) {
         if (e->programs.size() >= 64) {
@@ -282,7 +288,7 @@ int get_program(const std::vector<SegBind> &segs, int kind, Program **prog)
                     reqs.push_back(StageReq{sg, 0, i, 0, pl->layers[i].Ho, false, false, next++});
                 }
             }
-        } else if (kind == PROG_ALL_BANDS || kind == PROG_PIPELINED) {
+        } else if (kind == PROG_ALL_BANDS || kind == PROG_PIPELINED || kind == PROG_FETCHED) {
             // ALL_BANDS (input resident): the bands' operations of one layer do not depend on each other, so they are
             // batched layer by layer (operation batching, Sec. IV-C); dependencies stay per band row group.
             // PIPELINED: bands arrive one after the other and each band's stages form a dependency chain, so the
@@ -292,17 +298,25 @@ int get_program(const std::vector<SegBind> &segs, int kind, Program **prog)
             // lags by a band; the builder moves a stage back wherever its producers come later still).  Inside a
             // diagonal the deeper stages come first, so a CTA does not sit on a band that has not arrived while
             // older bands have work.
+            // FETCHED: the same, each band of plan 0 preceded by the fetch of its new input rows; the builder orders
+            // these programs by earliest start.
             long long joff = 0;
             for (int sg = 0; sg < (int)segs.size(); ++sg) {
                 const lop_plan_t *pl = segs[sg].pl;
                 size_t per = 0;
                 for (int b = 0; b < pl->n_bands; ++b) {
                     std::vector<StageReq> one;
+                    if (kind == PROG_FETCHED && sg == 0) {
+                        const lop_range &need = pl->in_need[b];
+                        StageReq f{0, b, 0, need.new_lo, need.out_hi, false, false, (long long)b * 65536 - 1};
+                        f.fetch = true;
+                        reqs.push_back(f);
+                    }
                     band_requests(pl, sg, b, kind == PROG_PIPELINED, one);
                     per = one.size();
                     for (size_t j = 0; j < one.size(); ++j) {
                         const long long depth = joff + (long long)j;
-                        one[j].prio = kind == PROG_ALL_BANDS ? depth * 65536 + b : (b + depth + sg) * 65536 + (65535 - depth);
+                        one[j].prio = kind == PROG_ALL_BANDS ? depth * 65536 + b : (b + depth + sg) * 65536 + (65534 - depth);
                         reqs.push_back(one[j]);
                     }
                 }
@@ -326,7 +340,7 @@ int get_program(const std::vector<SegBind> &segs, int kind, Program **prog)
             }
         }
         Program *p = nullptr;
-        int rc = program_build(segs, reqs, &p, kind == PROG_PIPELINED ? &arrival : nullptr);
+        int rc = program_build(segs, reqs, &p, kind == PROG_PIPELINED ? &arrival : nullptr, fetch_src);
         if (rc != LOP_OK) return rc;
         it = e->programs.emplace(key, p).first;
     }
@@ -334,9 +348,28 @@ int get_program(const std::vector<SegBind> &segs, int kind, Program **prog)
     return LOP_OK;
 }
 
-int get_program(lop_plan_t *pl, int kind, const void *in, void *out, void *ws, Program **prog)
+int get_program(lop_plan_t *pl, int kind, const void *in, void *out, void *ws, Program **prog, const void *fetch_src = nullptr)
 {
-    return get_program(std::vector<SegBind>{SegBind{pl, in, out, ws}}, kind, prog);
+    return get_program(std::vector<SegBind>{SegBind{pl, in, out, ws}}, kind, prog, fetch_src);
+}
+
+// The address under which the device reads the host buffer, when it can (page-locked memory is mapped into the
+// unified address space) and the plan does not insist on the copy engine; nullptr otherwise.
+const void *fetchable(lop_plan_t *pl, const void *host)
+{
+    if (pl->flags & LOP_FLAG_COPY_ENGINE) return nullptr;
+    ExecState *e = pl->exec;
+    if (e->mapped_host == host) return e->mapped_dev;
+    cudaPointerAttributes at{};
+    const void *dev = nullptr;
+    if (cudaPointerGetAttributes(&at, host) == cudaSuccess) {
+        if (at.type == cudaMemoryTypeHost && at.devicePointer) dev = at.devicePointer;
+    } else {
+        cudaGetLastError();                                  // an unknown pointer is no error here: it gets copies
+    }
+    e->mapped_host = host;
+    e->mapped_dev = dev;
+    return dev;
 }
 
 int run_program(lop_plan_t *pl, int kind, const void *in, void *out, void *ws, cudaStream_t s)
@@ -487,7 +520,9 @@ int lop_run_pipelined(lop_plan_t *pl, const void *host, void *staging, void *out
     e->last_stream = s;
     e->timing_valid = false;
     reset_layer_timing(pl);
-    LOP_CUDA(cudaEventRecord(e->ev_begin, s));
+    // an event record is a stream command of its own (microseconds): only plans that ask for timing pay for them
+    const bool timed = (pl->flags & LOP_FLAG_TIME_LAYERS) != 0;
+    if (timed) LOP_CUDA(cudaEventRecord(e->ev_begin, s));
     if ((rc = prepare_workspace(pl, ws, s)) != LOP_OK) return rc;
     if (e->wavefront) {
         // One persistent launch for the whole request: it starts at once and every band's first stage waits
@@ -496,10 +531,22 @@ int lop_run_pipelined(lop_plan_t *pl, const void *host, void *staging, void *out
         // microseconds with 32 bands of 196 KB), so no graph is built here; a caller whose stream is capturing
         // simply gets these operations into its own graph.
         Program *p = nullptr;
-        if ((rc = get_program(pl, PROG_PIPELINED, staging, out, ws, &p)) != LOP_OK) return rc;
-        if ((rc = enqueue_pipelined(pl, p, host, staging, s)) != LOP_OK) return rc;
-        LOP_CUDA(cudaEventRecord(e->ev_end, s));
-        e->timing_valid = true;
+        const void *src = fetchable(pl, host);
+        if (src && (reinterpret_cast<uintptr_t>(src) & 15) == (reinterpret_cast<uintptr_t>(staging) & 15)) {
+            // the kernel fetches the bands itself: nothing but the launch
+            if ((rc = get_program(pl, PROG_FETCHED, staging, out, ws, &p, src)) != LOP_OK) return rc;
+            for (int b = 0; b < pl->n_bands; ++b) e->copy_issued[b] = 0;
+            e->copies_timed = false;
+            if (!program_empty(p)) {
+                if ((rc = program_launch(p, s)) != LOP_OK) return rc;
+                e->launches++;
+            }
+        } else {
+            if ((rc = get_program(pl, PROG_PIPELINED, staging, out, ws, &p)) != LOP_OK) return rc;
+            if ((rc = enqueue_pipelined(pl, p, host, staging, s)) != LOP_OK) return rc;
+        }
+        if (timed) LOP_CUDA(cudaEventRecord(e->ev_end, s));
+        e->timing_valid = timed;
         return LOP_OK;
     }
     // the side stream starts after everything already queued on the caller's stream; all transfers are queued
@@ -524,8 +571,8 @@ int lop_run_pipelined(lop_plan_t *pl, const void *host, void *staging, void *out
         if ((rc = run_band_impl(pl, b, staging, out, ws, s)) != LOP_OK) return rc;
     }
     if (!joined) LOP_CUDA(cudaStreamWaitEvent(s, e->ev_fork, 0));
-    LOP_CUDA(cudaEventRecord(e->ev_end, s));
-    e->timing_valid = true;
+    if (timed) LOP_CUDA(cudaEventRecord(e->ev_end, s));
+    e->timing_valid = timed;
     return LOP_OK;
 }
 
@@ -587,19 +634,27 @@ int lop_run_chain_pipelined(lop_plan_t *const *plans, int n_plans, const void *h
     if (rc != LOP_OK) return rc;
     ExecState *e = plans[0]->exec;
     e->timing_valid = false;
-    LOP_CUDA(cudaEventRecord(e->ev_begin, s));
     Program *p = nullptr;
-    if ((rc = get_program(segs, PROG_PIPELINED, &p)) != LOP_OK) return rc;
-    if ((rc = enqueue_pipelined(plans[0], p, host, staging, s)) != LOP_OK) return rc;
-    LOP_CUDA(cudaEventRecord(e->ev_end, s));
-    e->timing_valid = true;
+    const void *src = fetchable(plans[0], host);
+    if (src && (reinterpret_cast<uintptr_t>(src) & 15) == (reinterpret_cast<uintptr_t>(staging) & 15)) {
+        if ((rc = get_program(segs, PROG_FETCHED, &p, src)) != LOP_OK) return rc;
+        for (int b = 0; b < plans[0]->n_bands; ++b) e->copy_issued[b] = 0;
+        e->copies_timed = false;
+        if (!program_empty(p)) {
+            if ((rc = program_launch(p, s)) != LOP_OK) return rc;
+            e->launches++;
+        }
+    } else {
+        if ((rc = get_program(segs, PROG_PIPELINED, &p)) != LOP_OK) return rc;
+        if ((rc = enqueue_pipelined(plans[0], p, host, staging, s)) != LOP_OK) return rc;
+    }
     return LOP_OK;
 }
 
 int lop_plan_last_timing(lop_plan_t *pl, lop_timing *out)
 {
     if (!pl || !out) { set_error("lop_plan_last_timing: NULL argument"); return LOP_EINVAL; }
-    if (!pl->exec || !pl->exec->timing_valid) { set_error("no pipelined run to report"); return LOP_EINVAL; }
+    if (!pl->exec || !pl->exec->timing_valid) { set_error("no timed pipelined run to report (the plan needs LOP_FLAG_TIME_LAYERS)"); return LOP_EINVAL; }
     ExecState *e = pl->exec;
     LOP_CUDA(cudaEventSynchronize(e->ev_end));
     lop_timing t = {0, 0, 0, 0, 0};

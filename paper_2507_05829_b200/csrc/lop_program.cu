@@ -34,6 +34,12 @@ void program_destroy(Program *p)
 
 namespace {
 
+#ifndef LOP_FETCH_ENTRY_BYTES
+#define LOP_FETCH_ENTRY_BYTES 3072
+#endif
+#ifndef LOP_FETCH_WINDOW_BYTES
+#define LOP_FETCH_WINDOW_BYTES (96 * 1024)
+#endif
 constexpr uint32_t A_BOX_MAX = 48u * 1024u;     // largest activation box a ring slot is sized for
 constexpr uint32_t B_BOX_MAX = 32u * 1024u;     // largest weight box
 
@@ -192,6 +198,7 @@ struct Reads { Need need[3]; int n = 0; bool raw = false; };
 struct Ctx {
     const std::vector<SegBind> &segs;
     std::vector<int> base;              // first tensor id of each plan; id base+layer, base+L = the stem's patches
+    int raw = -1;                       // tensor id of the chain input when the program fetches it itself, else -1
     int tensor_id(int seg, int layer) const { return base[seg] + layer; }
     int patches_id(int seg) const { return base[seg] + (int)segs[seg].pl->layers.size(); }
     int input_id(int seg) const { return tensor_id(seg - 1, (int)segs[seg - 1].pl->layers.size() - 1); }
@@ -212,9 +219,12 @@ Reads reads_of(const Ctx &cx, const StageReq &rq, int o0, int o1)
         return a <= b;
     };
     int a = 0, b = 0;
+    if (rq.fetch) return r;                                                   // reads host memory only
     if (rq.gather || (l.input_from == LOP_INPUT && !li.stem_gather)) {
-        if (rq.seg == 0) r.raw = true;
-        else if (window(a, b)) r.need[r.n++] = Need{cx.input_id(rq.seg), a, b, false};
+        if (rq.seg == 0) {
+            r.raw = true;
+            if (cx.raw >= 0 && window(a, b)) r.need[r.n++] = Need{cx.raw, a, b, false};     // whichever band fetched them
+        } else if (window(a, b)) r.need[r.n++] = Need{cx.input_id(rq.seg), a, b, false};
     } else if (li.stem_gather) {
         r.need[r.n++] = Need{cx.patches_id(rq.seg), o0, o1, true};            // the patches of exactly these rows
     } else if (window(a, b)) {
@@ -222,8 +232,10 @@ Reads reads_of(const Ctx &cx, const StageReq &rq, int o0, int o1)
     }
     if (!rq.gather && l.op == LOP_CONV2D && l.residual_from != LOP_NO_RESIDUAL) {
         if (l.residual_from >= 0) r.need[r.n++] = Need{cx.tensor_id(rq.seg, l.residual_from), o0, o1, true};
-        else if (rq.seg == 0) r.raw = true;
-        else r.need[r.n++] = Need{cx.input_id(rq.seg), o0, o1, false};
+        else if (rq.seg == 0) {
+            r.raw = true;
+            if (cx.raw >= 0) r.need[r.n++] = Need{cx.raw, o0, o1, false};
+        } else r.need[r.n++] = Need{cx.input_id(rq.seg), o0, o1, false};
     }
     return r;
 }
@@ -235,6 +247,7 @@ double stage_cost_us(const Ctx &cx, const StageReq &rq)
     const lop_plan_t *pl = cx.segs[rq.seg].pl;
     const LayerInfo &li = pl->layers[rq.layer];
     const double rows = rq.hi - rq.lo;
+    if (rq.fetch) return 3.0 + rows * pl->W * pl->C * 2.0 * pl->N / 24e3;       // link latency + bytes at the ~24 GB/s measured
     if (rq.gather || li.l.op == LOP_MAXPOOL2D) return 1.0 + 3.0 * std::ceil(rows * pl->N / 148.0);
     const double tiles = std::ceil(rows * li.Wo * pl->N / 128.0) * std::max(1, li.l.cout / 128);
     const double item = 1.5 + 0.06 * li.l.kh * li.l.kw * (li.cin_eff / 16.0);
@@ -250,8 +263,9 @@ int order_requests(const Ctx &cx, std::vector<StageReq> &reqs, bool reuse, const
     const size_t n = reqs.size();
     std::vector<int> produces(n);
     for (size_t i = 0; i < n; ++i)
-        produces[i] = reqs[i].gather ? cx.patches_id(reqs[i].seg) : cx.tensor_id(reqs[i].seg, reqs[i].layer);
-    bool sorted_already = arrival_us == nullptr;
+        produces[i] = reqs[i].fetch ? cx.raw : (reqs[i].gather ? cx.patches_id(reqs[i].seg) : cx.tensor_id(reqs[i].seg, reqs[i].layer));
+    const bool by_start = arrival_us != nullptr || cx.raw >= 0;
+    bool sorted_already = !by_start;
     for (size_t i = 1; i < n; ++i)
         if (reqs[i].prio < reqs[i - 1].prio) sorted_already = false;
     std::vector<std::vector<int>> users(n), prods(n);
@@ -291,12 +305,18 @@ int order_requests(const Ctx &cx, std::vector<StageReq> &reqs, bool reuse, const
     };
     std::vector<int> order;
     if (!kahn(order)) { set_error("the stage requests depend on each other in a cycle"); return LOP_EINVAL; }
-    if (arrival_us) {
+    if (by_start) {
         std::vector<double> end(n, 0.0);
+        double link_free = 0.0;                                   // fetches share the host link: one after the other
         for (int i : order) {
             double start = 0.0;
-            if (raw[i] && reqs[i].wait_arrival && reqs[i].band < (int)arrival_us->size()) start = (*arrival_us)[reqs[i].band];
+            if (arrival_us && raw[i] && reqs[i].wait_arrival && reqs[i].band < (int)arrival_us->size()) start = (*arrival_us)[reqs[i].band];
             for (int j : prods[i]) start = std::max(start, end[j]);
+            if (reqs[i].fetch) {
+                const double busy = stage_cost_us(cx, reqs[i]) - 3.0;
+                start = std::max(start, link_free);
+                link_free = start + busy;
+            }
             end[i] = start + stage_cost_us(cx, reqs[i]);
             reqs[i].prio = (long long)(start * 1000.0);
         }
@@ -311,7 +331,8 @@ int order_requests(const Ctx &cx, std::vector<StageReq> &reqs, bool reuse, const
 
 }  // namespace
 
-int program_build(const std::vector<SegBind> &segs, std::vector<StageReq> reqs, Program **result, const std::vector<double> *arrival_us)
+int program_build(const std::vector<SegBind> &segs, std::vector<StageReq> reqs, Program **result, const std::vector<double> *arrival_us,
+                  const void *fetch_src)
 {
     *result = nullptr;
     if (segs.empty()) { set_error("program_build: no plan"); return LOP_EINVAL; }
@@ -319,6 +340,17 @@ int program_build(const std::vector<SegBind> &segs, std::vector<StageReq> reqs, 
     Ctx cx{segs, {}};
     int n_tensors = 0;
     for (const SegBind &sb : segs) { cx.base.push_back(n_tensors); n_tensors += (int)sb.pl->layers.size() + 1; }
+    for (const StageReq &rq : reqs)
+        if (rq.fetch && rq.hi > rq.lo) cx.raw = n_tensors;
+    if (cx.raw >= 0) {
+        ++n_tensors;
+        if (!fetch_src) { set_error("program_build: fetch requests without a source"); return LOP_EINVAL; }
+        if ((reinterpret_cast<uintptr_t>(fetch_src) & 15) != (reinterpret_cast<uintptr_t>(segs[0].in) & 15) ||
+            (reinterpret_cast<uintptr_t>(fetch_src) & 1)) {
+            set_error("host input and staging tensor must agree in their address modulo 16");
+            return LOP_EUNSUPPORTED;
+        }
+    }
     {
         std::vector<StageReq> live;
         for (const StageReq &rq : reqs)
@@ -330,7 +362,7 @@ int program_build(const std::vector<SegBind> &segs, std::vector<StageReq> reqs, 
 
     std::vector<WfStage> stages;
     std::vector<int> stage_band, stage_rows_per_group;
-    std::vector<int4> items;
+    std::vector<int4> items, fetch_items;
     std::vector<CUtensorMap> maps;
     std::vector<MapSet> mapsets;
     std::vector<int2> deps;
@@ -356,9 +388,19 @@ int program_build(const std::vector<SegBind> &segs, std::vector<StageReq> reqs, 
         st.oh_lo = rq.lo; st.oh_hi = rq.hi;
         const int rows = rq.hi - rq.lo;
         int group_rows = 1, tiles_r = rows, tiles_w = 1, tiles_n = pl->N, cout_tiles = 1;
-        int produces = rq.gather ? cx.patches_id(rq.seg) : cx.tensor_id(rq.seg, rq.layer);
+        int produces = rq.fetch ? cx.raw : (rq.gather ? cx.patches_id(rq.seg) : cx.tensor_id(rq.seg, rq.layer));
         int out_lo = rq.lo, out_hi = rq.hi;                    // rows of the produced tensor
-        if (rq.gather) {
+        if (rq.fetch) {
+            // a stage only in the book-keeping sense (row-group counters its readers wait for): its work goes to the
+            // fetch list.  Entries of about 3 KB, whole rows: a warp has that much in flight at a time.
+            const long long row_b = (long long)pl->W * pl->C * 2;
+            st.kind = WF_FETCH;
+            st.x = fetch_src; st.y = const_cast<void *>(in);
+            st.N = pl->N; st.Hin = pl->H; st.Win = pl->W; st.Cin = pl->C;
+            group_rows = (int)std::max(1LL, std::min<long long>(rows, LOP_FETCH_ENTRY_BYTES / row_b));
+            tiles_r = (rows + group_rows - 1) / group_rows;
+            if (row_b * group_rows > 0x7fffffffLL) { set_error("input rows too long to fetch"); return LOP_EUNSUPPORTED; }
+        } else if (rq.gather) {
             st.kind = WF_GATHER;
             st.x = in; st.y = wsb + pl->col_off;
             st.N = pl->N; st.Hin = pl->H; st.Win = pl->W; st.Cin = pl->C; st.Ho = li.Ho; st.Wo = li.Wo; st.Cout = li.cin_eff;
@@ -468,6 +510,15 @@ int program_build(const std::vector<SegBind> &segs, std::vector<StageReq> reqs, 
                 }
             const int count = (int)deps.size() - first;
             if (count > WF_MAX_DEPS) { set_error("layer %d: a tile depends on too many row groups", rq.layer); return LOP_EUNSUPPORTED; }
+            if (rq.fetch) {
+                const long long row_b = (long long)pl->W * pl->C * 2;
+                for (int n = 0; n < pl->N; ++n) {
+                    const unsigned long long off = (unsigned long long)(((long long)n * pl->H + o0) * row_b);
+                    fetch_items.push_back(make_int4((int)(unsigned)(off & 0xffffffffu), (int)(unsigned)(off >> 32), (int)((o1 - o0) * row_b),
+                                                    st.ctr_base + tr));
+                }
+                continue;
+            }
             for (int tn = 0; tn < tiles_n; ++tn)
                 for (int tw = 0; tw < tiles_w; ++tw)
                     for (int ct = 0; ct < cout_tiles; ++ct)
@@ -512,7 +563,8 @@ int program_build(const std::vector<SegBind> &segs, std::vector<StageReq> reqs, 
     const size_t o_items = o_stages + al(stages.size() * sizeof(WfStage));
     const size_t o_maps = o_items + al(items.size() * sizeof(int4));
     const size_t o_deps = o_maps + al(std::max<size_t>(maps.size(), 1) * sizeof(CUtensorMap));
-    const size_t o_ctr = o_deps + al(std::max<size_t>(deps.size(), 1) * sizeof(int2));
+    const size_t o_fetch = o_deps + al(std::max<size_t>(deps.size(), 1) * sizeof(int2));
+    const size_t o_ctr = o_fetch + al(fetch_items.size() * sizeof(int4));
     const size_t total = o_ctr + al((size_t)n_ctr * sizeof(unsigned));
     cudaError_t e = cudaMalloc(&p->dev, total);
     if (e != cudaSuccess) { delete p; set_error("cudaMalloc(%zu) failed: %s", total, cudaGetErrorString(e)); return LOP_ECUDA; }
@@ -523,7 +575,8 @@ int program_build(const std::vector<SegBind> &segs, std::vector<StageReq> reqs, 
     if ((e = cudaMemset(d, 0, total)) != cudaSuccess || (e = up(o_stages, stages.data(), stages.size() * sizeof(WfStage))) != cudaSuccess ||
         (e = up(o_items, items.data(), items.size() * sizeof(int4))) != cudaSuccess ||
         (e = up(o_maps, maps.data(), maps.size() * sizeof(CUtensorMap))) != cudaSuccess ||
-        (e = up(o_deps, deps.data(), deps.size() * sizeof(int2))) != cudaSuccess) {
+        (e = up(o_deps, deps.data(), deps.size() * sizeof(int2))) != cudaSuccess ||
+        (e = up(o_fetch, fetch_items.data(), fetch_items.size() * sizeof(int4))) != cudaSuccess) {
         program_destroy(p);
         set_error("program upload failed: %s", cudaGetErrorString(e));
         return LOP_ECUDA;
@@ -541,6 +594,16 @@ int program_build(const std::vector<SegBind> &segs, std::vector<StageReq> reqs, 
     P.n_items = n_items;
     P.sa = sa; P.sb = sb;
     P.a_slot_bytes = a_slot; P.b_slot_bytes = b_slot; P.stg_bytes = stg_bytes;
+    P.fetch_items = reinterpret_cast<const int4 *>(d + o_fetch);
+    P.fetch_src = fetch_src;
+    P.fetch_dst = const_cast<void *>(segs[0].in);
+    P.n_fetch = (int)fetch_items.size();
+    // entries in flight: about the link's bandwidth-delay product (some 25 GB/s x 3 us), at least a few warps' worth
+    if (P.n_fetch > 0) {
+        long long bytes = 0;
+        for (const int4 &f : fetch_items) bytes += f.z;
+        P.fetch_window = (int)std::max(8LL, (long long)LOP_FETCH_WINDOW_BYTES * P.n_fetch / std::max(1LL, bytes));
+    }
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);

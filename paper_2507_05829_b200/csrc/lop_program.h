@@ -16,14 +16,18 @@ struct SegBind { lop_plan_t *pl; const void *in; void *out; void *ws; };
 // layer (same rows).  wait_arrival: stages of plan 0 that read the raw chain input wait for the arrival flags of the
 // bands that bring their rows (single-launch pipelined programs).  prio: stages are put into the program in
 // ascending priority, as far as their dependencies allow (a stage never precedes one it reads from).
-struct StageReq { int seg, band, layer, lo, hi; bool wait_arrival; bool gather; long long prio; };
+// fetch: not an operator but the transfer of rows [lo, hi) of the chain input from host memory, done by the kernel
+// itself (layer is ignored); the stages of plan 0 that read those rows then depend on it like on any producer.
+struct StageReq { int seg, band, layer, lo, hi; bool wait_arrival; bool gather; long long prio; bool fetch = false; };
 struct Program;
 
 bool program_supported(const lop_plan_t *pl);
 // arrival_us (optional): expected arrival time of each band of plan 0; stages are then ordered by their earliest
-// possible start under that schedule instead of by prio.
+// possible start under that schedule instead of by prio.  fetch_src: the chain input in host memory as the device
+// addresses it, source of the fetch requests (segs[0].in is their destination); programs with fetch requests are
+// ordered by earliest start as well, the host link taken as a serial resource.
 int program_build(const std::vector<SegBind> &segs, std::vector<StageReq> reqs, Program **result,
-                  const std::vector<double> *arrival_us = nullptr);
+                  const std::vector<double> *arrival_us = nullptr, const void *fetch_src = nullptr);
 int program_launch(Program *p, cudaStream_t s);
 // Device address of band b's arrival flag (a 4-byte word a side stream sets non-zero), or nullptr.
 unsigned *program_arrival_flag(Program *p, int band);

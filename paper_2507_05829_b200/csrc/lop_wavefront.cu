@@ -57,6 +57,7 @@ __device__ __forceinline__ unsigned ld_relaxed(const unsigned *p)
 #ifdef LOP_WF_TRACE
 // Developer build only: per-item time stamps (global timer, ns) of the three roles.
 constexpr int TRACE_ITEMS = 1 << 15;
+constexpr int TRACE_FETCH0 = 1 << 14;                       // fetch entry j is stamped at row TRACE_FETCH0 + j
 __device__ unsigned long long g_wf_trace[TRACE_ITEMS * 16];
 __device__ __forceinline__ void tr(int item, int slot)
 {
@@ -172,7 +173,42 @@ __device__ __forceinline__ T ldg_ptr(const void *const *p)
     return reinterpret_cast<T>(__ldg(reinterpret_cast<const unsigned long long *>(p)));
 }
 
-__global__ void __launch_bounds__(WF_THREADS, 1) wavefront_kernel(const WfParams P)
+// len bytes (a multiple of 2) from host memory the device can address to device memory, by the 32 lanes of a warp.
+// Host lines are read around the caches (they change between launches without the device knowing); eight 16-byte
+// loads per lane are in flight to cover the host link's latency.  src and dst agree modulo 16.
+#ifndef LOP_FETCH_DEPTH
+#define LOP_FETCH_DEPTH 8
+#endif
+constexpr int FETCH_DEPTH = LOP_FETCH_DEPTH;
+__device__ __forceinline__ void fetch_bytes(const uint8_t *src, uint8_t *dst, int len, int lane)
+{
+    int head = (16 - (int)(reinterpret_cast<uintptr_t>(src) & 15)) & 15;
+    if (head > len) head = len;
+    for (int i = 2 * lane; i < head; i += 64)
+        *reinterpret_cast<uint16_t *>(dst + i) = __ldcv(reinterpret_cast<const uint16_t *>(src + i));
+    const int nvec = (len - head) >> 4;
+    const uint4 *s4 = reinterpret_cast<const uint4 *>(src + head);
+    uint4 *d4 = reinterpret_cast<uint4 *>(dst + head);
+    for (int v0 = 0; v0 < nvec; v0 += FETCH_DEPTH * 32) {
+        uint4 q[FETCH_DEPTH];
+#pragma unroll
+        for (int u = 0; u < FETCH_DEPTH; ++u) {
+            const int v = v0 + u * 32 + lane;
+            if (v < nvec) q[u] = __ldcv(s4 + v);
+        }
+#pragma unroll
+        for (int u = 0; u < FETCH_DEPTH; ++u) {
+            const int v = v0 + u * 32 + lane;
+            if (v < nvec) d4[v] = q[u];
+        }
+    }
+    for (int i = head + (nvec << 4) + 2 * lane; i < len; i += 64)
+        *reinterpret_cast<uint16_t *>(dst + i) = __ldcv(reinterpret_cast<const uint16_t *>(src + i));
+}
+
+// FETCH: the program has a fetch list; the CTA then has one more warp, which walks it.
+template <bool FETCH>
+__global__ void __launch_bounds__(FETCH ? WF_THREADS + 32 : WF_THREADS, 1) wavefront_kernel(const WfParams P)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -194,6 +230,7 @@ __global__ void __launch_bounds__(WF_THREADS, 1) wavefront_kernel(const WfParams
     uint8_t *stg = smem + (stg0 - base);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0 && blockIdx.x < 4) tr(TRACE_ITEMS - 8 + (int)blockIdx.x, 0);
     if (threadIdx.x == 0) {
         for (int s = 0; s < SA; ++s) {
             mbar_init(full_a + 8u * s, 1);
@@ -225,6 +262,7 @@ __global__ void __launch_bounds__(WF_THREADS, 1) wavefront_kernel(const WfParams
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    if (threadIdx.x == 0 && blockIdx.x < 4) tr(TRACE_ITEMS - 8 + (int)blockIdx.x, 1);
     const uint32_t tmem_base = misc[0];
     const unsigned run = misc[2];
     volatile uint32_t *abort_flag = &misc[1];
@@ -445,6 +483,45 @@ __global__ void __launch_bounds__(WF_THREADS, 1) wavefront_kernel(const WfParams
                 atomicOr(P.status, 0x8u);
                 atomicExch(P.counters + 2, 1u);
                 *abort_flag = 1;
+            }
+        }
+    } else if (FETCH && warp == WF_FIRST_WORKER + WF_WORKER_WARPS) {
+        // ---------------- fetch warp: the chain input, host memory -> device, in list order ----------------
+        const unsigned done_before = (run - 1u) * (unsigned)P.n_fetch;          // counters[3] never resets
+        const uint8_t *src0 = static_cast<const uint8_t *>(P.fetch_src);
+        uint8_t *dst0 = static_cast<uint8_t *>(P.fetch_dst);
+        for (int j = blockIdx.x; j < P.n_fetch; j += G) {
+            const int4 rec = __ldg(&P.fetch_items[j]);
+            if (j >= P.fetch_window) {
+                // the window keeps the link's queue short, so that early rows are not stuck behind late ones
+                const unsigned target = done_before + (unsigned)(j - P.fetch_window + 1);
+                int ok = 1;
+                if (lane == 0) {
+                    for (uint32_t i = 0; (int)(ld_acquire(P.counters + 3) - target) < 0; ++i) {
+                        if (i >= SPIN_LIMIT) { ok = 0; atomicOr(P.status, 0x20u); break; }
+                        if ((i & 63u) == 63u && (ld_relaxed(P.counters + 2) != 0u || *abort_flag)) { ok = -1; break; }
+                        __nanosleep(64);
+                    }
+                }
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (ok <= 0) {
+                    if (ok == 0 && lane == 0) {
+                        atomicExch(P.counters + 2, 1u);
+                        *abort_flag = 1;
+                    }
+                    break;
+                }
+            }
+            const long long off = (long long)(((unsigned long long)(unsigned)rec.y << 32) | (unsigned)rec.x);
+            if (lane == 0) tr(TRACE_FETCH0 + j, 0);
+            fetch_bytes(src0 + off, dst0 + off, rec.z, lane);
+            __syncwarp();
+            if (lane == 0) {
+                tr(TRACE_FETCH0 + j, 1);
+                __threadfence();                                   // the warp's stores, then the release increments
+                atomicAdd(P.counters + rec.w, 1u);
+                atomicAdd(P.counters + 3, 1u);
+                tr(TRACE_FETCH0 + j, 2);
             }
         }
     } else {
@@ -794,6 +871,7 @@ __global__ void __launch_bounds__(WF_THREADS, 1) wavefront_kernel(const WfParams
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (warp == 1)
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+    if (threadIdx.x == 0 && blockIdx.x < 4) tr(TRACE_ITEMS - 8 + (int)blockIdx.x, 2);
     if (threadIdx.x == 0) {
         __threadfence();
         const unsigned done = atomicAdd(P.counters + 1, 1u);
@@ -852,7 +930,9 @@ cudaError_t launch_wavefront(const WfParams &p, int grid, cudaStream_t s)
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64 || !configured[dev]) {
-        e = cudaFuncSetAttribute(wavefront_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        e = cudaFuncSetAttribute(wavefront_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(wavefront_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
@@ -860,7 +940,8 @@ cudaError_t launch_wavefront(const WfParams &p, int grid, cudaStream_t s)
 #ifdef LOP_WF_TRACE
     g_last_params = p;
 #endif
-    wavefront_kernel<<<grid, WF_THREADS, smem, s>>>(p);
+    if (p.n_fetch > 0) wavefront_kernel<true><<<grid, WF_THREADS + 32, smem, s>>>(p);
+    else wavefront_kernel<false><<<grid, WF_THREADS, smem, s>>>(p);
     return cudaGetLastError();
 }
 

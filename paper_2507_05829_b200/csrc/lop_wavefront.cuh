@@ -13,7 +13,9 @@
 
 namespace lop {
 
-enum WfKind { WF_GATHER = 0, WF_CONV = 1, WF_POOL = 2 };
+// WF_FETCH: rows of the chain input brought from host memory by the CTAs' fetch warps.  Such a stage has row-group
+// counters like any producer but no items in the main list: its work is the program's fetch list.
+enum WfKind { WF_GATHER = 0, WF_CONV = 1, WF_POOL = 2, WF_FETCH = 3 };
 // How a convolution stage feeds the tensor cores.
 //   WF_SLAB  one activation box per channel chunk: the output tile's receptive window (tile plus halo),
 //            laid out in shared memory as rows of P pixels; every filter tap is the same box read at a
@@ -57,13 +59,21 @@ struct WfParams {
     const int4 *items;
     const CUtensorMap *maps;
     const int2 *deps;         // (counter index, completions expected per run); y < 0: an arrival flag, target -y
-    unsigned *counters;       // [0] runs completed, [1] CTAs finished, [2] abort, [4..] row-group counters,
+    unsigned *counters;       // [0] runs completed, [1] CTAs finished, [2] abort, [3] fetch entries finished, [4..] row-group counters,
                               // then n_flags band-arrival flags (set by the copy stream, cleared at run end)
     int flag_base, n_flags;
     unsigned *status;
     int n_stages, n_items;
     int sa, sb;               // slots of the activation / weight ring
     uint32_t a_slot_bytes, b_slot_bytes, stg_bytes;
+    // In-kernel input transfer (Sec. IV-B transmission, done by the kernel itself): every CTA has one more warp that
+    // walks this list round-robin; entry j copies z bytes at byte offset (x | y << 32) from fetch_src (host memory
+    // the device can address) to fetch_dst and then increments counters[w].  At most fetch_window entries are in
+    // flight at a time (counters[3] counts finished ones), so the rows arrive in list order at the link's rate.
+    const int4 *fetch_items;
+    const void *fetch_src;
+    void *fetch_dst;
+    int n_fetch, fetch_window;
 };
 
 #ifndef LOP_WF_WORKER_WARPS

@@ -19,14 +19,17 @@ def rel_err(got, want):
     return float(np.max(np.abs(got.astype(np.float64) - want.astype(np.float64)))) / (scale if scale > 0 else 1.0)
 
 
-def check_workload(wl, flags=0, modes=("whole", "banded", "pipelined"), n_bands=None, tol=None):
-    """Run every segment on the GPU in each mode and compare the segment outputs with the oracle."""
+def check_workload(wl, flags=0, modes=("whole", "banded", "pipelined", "pipelined_copy"), n_bands=None, tol=None):
+    """Run every segment on the GPU in each mode and compare the segment outputs with the oracle.
+
+    pipelined: the kernel fetches the bands from the pinned host tensor itself (where the plan runs on the persistent
+    kernel); pipelined_copy: the bands come by copy-engine copies on the side stream."""
     want = ochain.run_workload(wl, keep_segments=True)
     tol = TOL[wl.dtype] if tol is None else tol
     results = {}
     for mode in modes:
-        dc = DeviceChain(wl, flags=flags, n_bands=n_bands)
-        if mode == "pipelined":
+        dc = DeviceChain(wl, flags=flags | (lop.LOP_FLAG_COPY_ENGINE if mode == "pipelined_copy" else 0), n_bands=n_bands)
+        if mode in ("pipelined", "pipelined_copy"):
             dc.run_pipelined(dc.pinned_input())
         elif mode == "banded":
             dc.run_banded(dc.input_tensor())
@@ -274,7 +277,7 @@ def test_set_params_takes_effect_on_a_plan_that_has_already_run():
 def test_more_bands_than_rows_and_single_band():
     wl = li.build("vgg_block", H=12, W=20)
     for nb in (1, 6, 7, 13):                                     # 6 output rows: empty bands from 7 on
-        check_workload(wl, n_bands=nb, modes=("whole", "banded", "pipelined"))
+        check_workload(wl, n_bands=nb)
 
 
 def test_bands_in_any_order_without_reuse():
@@ -319,18 +322,21 @@ def test_pipelined_timing_and_launch_count():
     assert dc.plans[0].layer_time(0, 1) > 0 and dc.plans[0].layer_time(3, 2) > 0
 
 
-def test_wavefront_launch_counts_and_repeatability():
+@pytest.mark.parametrize("copy_engine", [False, True])
+def test_wavefront_launch_counts_and_repeatability(copy_engine):
     wl = li.build("vgg_block")
-    dc = DeviceChain(wl, flags=lop.LOP_FLAG_REUSE_HALO)
+    dc = DeviceChain(wl, flags=lop.LOP_FLAG_REUSE_HALO | (lop.LOP_FLAG_COPY_ENGINE if copy_engine else 0))
     x, xd = dc.pinned_input(), dc.input_tensor()
     first = None
     for i in range(5):                                           # run counters advance from launch to launch
+        dc.staging.zero_()
         dc.run_pipelined(x)
         torch.cuda.synchronize()
         if i == 0:
             assert dc.plans[0].last_launches() == 1 + 1          # one persistent launch (+ weight padding once)
-        else:
-            assert dc.plans[0].last_launches() == 1 and dc.plans[0].last_copies() == 8
+        else:                                                    # fetched: the launch is the only command of the call
+            assert dc.plans[0].last_launches() == 1 and dc.plans[0].last_copies() == (8 if copy_engine else 0)
+        assert torch.equal(dc.staging.view(-1), xd.view(-1)), "the input was not brought to the device in full"
         out = dc.outs[-1].clone()
         first = out if first is None else first
         assert torch.equal(out, first)
@@ -339,6 +345,79 @@ def test_wavefront_launch_counts_and_repeatability():
     torch.cuda.synchronize()
     assert dc.plans[0].last_launches() == 1 and torch.equal(dc.outs[-1], first)
     dc.check_device()
+
+
+def test_fetched_pipeline_reads_the_host_buffer_afresh_on_every_call():
+    """The kernel reads pinned host memory directly: a later call must see what the host wrote in between."""
+    wl = li.build("vgg_block", H=44, W=36)
+    dc = DeviceChain(wl, flags=lop.LOP_FLAG_REUSE_HALO)
+    x = dc.pinned_input()
+    dc.run_pipelined(x)
+    torch.cuda.synchronize()
+    first = dc.outs[-1].clone()
+    keep = x.clone()
+    x.mul_(-0.5)                                                 # the host changes its buffer in place
+    wl.x = -0.5 * wl.x
+    want = ochain.run_workload(wl)
+    for _ in range(2):
+        dc.run_pipelined(x)
+        torch.cuda.synchronize()
+        dc.check_device()
+        assert rel_err(to_host_f32(dc.outs[-1]), want) <= TOL["bf16"]
+        assert not torch.equal(dc.outs[-1], first)
+    x.copy_(keep)
+    dc.run_pipelined(x)
+    torch.cuda.synchronize()
+    assert torch.equal(dc.outs[-1], first)
+
+
+@pytest.mark.parametrize("name,kw", [("vgg_block", dict(H=44, W=36)), ("resnet18", dict(H=64, W=64)), ("single_conv", {})])
+def test_output_straight_into_pinned_host_memory(name, kw):
+    """The last layer may store into host memory the device can address: same bits as the device tensor."""
+    wl = li.build(name, **kw)
+    dc = DeviceChain(wl, flags=lop.LOP_FLAG_REUSE_HALO)
+    x = dc.pinned_input()
+    dc.run_pipelined(x)
+    torch.cuda.synchronize()
+    want = dc.outs[-1].clone()
+    dc.outs[-1].zero_()
+    host = torch.zeros(want.shape, dtype=want.dtype).pin_memory()
+    for _ in range(2):
+        host.zero_()
+        got = dc.run_pipelined(x, out_pinned=host)
+        torch.cuda.synchronize()
+        dc.check_device()
+        assert got is host and torch.equal(host, want.cpu())
+    assert not dc.outs[-1].any()                                 # the device output tensor was not touched
+    s = torch.cuda.current_stream().cuda_stream
+    host.zero_()
+    xd = dc.input_tensor() if len(dc.plans) == 1 else dc.outs[-2]
+    dc.plans[-1].run_whole(xd.data_ptr(), host.data_ptr(), dc.ws[-1].data_ptr(), s)
+    torch.cuda.synchronize()
+    assert torch.equal(host, want.cpu())
+
+
+def test_unaligned_and_unpinned_host_buffers_take_the_copy_path():
+    wl = li.build("vgg_block", H=44, W=36)
+    dc = DeviceChain(wl, flags=lop.LOP_FLAG_REUSE_HALO)
+    x = dc.pinned_input()
+    dc.run_pipelined(x)
+    torch.cuda.synchronize()
+    want = dc.outs[-1].clone()
+    assert dc.plans[0].last_copies() == 0
+    big = torch.empty(x.numel() + 8, dtype=x.dtype).pin_memory()
+    off = big[1:1 + x.numel()].view(x.shape)                     # 2 bytes off the staging tensor's alignment
+    off.copy_(x)
+    pageable = x.clone()                                         # ordinary host memory
+    assert not pageable.is_pinned()
+    s = torch.cuda.current_stream().cuda_stream
+    for host in (off, pageable):
+        dc.outs[-1].zero_()
+        dc.plans[0].run_pipelined(host.data_ptr(), dc.staging.data_ptr(), dc.outs[0].data_ptr(), dc.ws[0].data_ptr(), s)
+        torch.cuda.synchronize()
+        dc.check_device()
+        assert dc.plans[0].last_copies() == dc.plans[0].num_bands()
+        assert torch.equal(dc.outs[-1], want)
 
 
 def test_wavefront_and_per_layer_executors_agree_bit_for_bit():
@@ -356,8 +435,8 @@ def test_wavefront_and_per_layer_executors_agree_bit_for_bit():
 # ------------------------------------------------------------------------------------ the named configurations, full size
 @pytest.mark.parametrize("name", ["vgg_block", "resnet18", "csp_stack"])
 def test_named_configurations_full_size(name):
-    check_workload(li.build(name), flags=lop.LOP_FLAG_REUSE_HALO, modes=("whole", "pipelined"))
+    check_workload(li.build(name), flags=lop.LOP_FLAG_REUSE_HALO, modes=("whole", "pipelined", "pipelined_copy"))
 
 
 def test_resnet50_batch8_full_size():
-    check_workload(li.build("resnet50"), flags=lop.LOP_FLAG_REUSE_HALO, modes=("pipelined",))
+    check_workload(li.build("resnet50"), flags=lop.LOP_FLAG_REUSE_HALO, modes=("pipelined", "pipelined_copy"))
