@@ -7,6 +7,7 @@
 
 #include <algorithm>
 #include <cmath>
+#include <cstdio>
 #include <vector>
 
 #include "lop_internal.h"
@@ -240,24 +241,32 @@ Reads reads_of(const Ctx &cx, const StageReq &rq, int o0, int o1)
     return r;
 }
 
-// Rough time, in microseconds, one stage keeps the machine busy: its items over the SMs, an item costing a fixed part
-// plus its tensor-core instructions (about 0.06 us each, issued by one thread).  Only used to order stages.
-double stage_cost_us(const Ctx &cx, const StageReq &rq)
+// Rough shape of a stage for the ordering below: how many items it is cut into and how long one takes (microseconds;
+// measured: ~1.2 us fixed per convolution tile plus ~0.035 us per tensor-core instruction and ~0.2 us per operand box, each
+// issued by one thread; ~4 us more until the tile's epilogue has run and its rows are visible;
+// ~2.5 us per pooling / gather row).  A fetch is not run by the CTAs: items = 0, item_us = its time on the host link.
+struct StageShape { int items; double item_us; double tail_us; };   // tail_us: from an item's end on its CTA to its result being visible
+StageShape stage_shape(const Ctx &cx, const StageReq &rq)
 {
     const lop_plan_t *pl = cx.segs[rq.seg].pl;
     const LayerInfo &li = pl->layers[rq.layer];
     const double rows = rq.hi - rq.lo;
-    if (rq.fetch) return 3.0 + rows * pl->W * pl->C * 2.0 * pl->N / 24e3;       // link latency + bytes at the ~24 GB/s measured
-    if (rq.gather || li.l.op == LOP_MAXPOOL2D) return 1.0 + 3.0 * std::ceil(rows * pl->N / 148.0);
+    if (rq.fetch) return StageShape{0, rows * pl->W * pl->C * 2.0 * pl->N / 24e3, 0.0};      // ~24 GB/s measured for SM-issued reads
+    if (rq.gather || li.l.op == LOP_MAXPOOL2D) return StageShape{(int)rows * pl->N, 2.5, 0.5};
     const double tiles = std::ceil(rows * li.Wo * pl->N / 128.0) * std::max(1, li.l.cout / 128);
-    const double item = 1.5 + 0.06 * li.l.kh * li.l.kw * (li.cin_eff / 16.0);
-    return 1.0 + item * std::ceil(tiles / 148.0);
+    // operand boxes, ~0.2 us each (issue, and the wait for a free ring slot): one per (tap, 64-channel chunk) and operand for strided windows, one
+    // activation box and a few weight boxes per chunk otherwise
+    const int taps = li.stem_gather ? 1 : li.l.kh * li.l.kw;
+    const double chunks = std::ceil(li.cin_eff / 64.0);
+    const bool per_tap = taps > 1 && (li.l.sh != 1 || li.l.sw != 1 || li.cin_eff % 64 != 0);
+    const double boxes = per_tap ? 2.0 * taps * chunks : (1.0 + std::ceil(taps / 3.0)) * chunks;
+    // a CTA overlaps a tile's epilogue with the next tile's loads and MMAs: the epilogue is latency, not occupancy
+    return StageShape{(int)tiles, 1.2 + 0.2 * boxes + 0.035 * taps * (li.cin_eff / 16.0), 4.0};
 }
 
-// Puts the requests into ascending priority as far as dependencies allow (a stable topological order).  With
-// arrival_us (when each band of plan 0 is expected on the device) the priorities are first replaced by each stage's
-// earliest possible start under that arrival schedule, so that stages of later plans fill the time in which the
-// first plan waits for its input.
+// Puts the requests into program order.  Resident programs: ascending priority as far as dependencies allow (a
+// stable topological order).  Programs whose input arrives while they run (arrival_us: when each band of plan 0 is
+// expected on the device; or fetch requests): the order in which a model of the machine would start the stages.
 int order_requests(const Ctx &cx, std::vector<StageReq> &reqs, bool reuse, const std::vector<double> *arrival_us)
 {
     const size_t n = reqs.size();
@@ -304,23 +313,103 @@ int order_requests(const Ctx &cx, std::vector<StageReq> &reqs, bool reuse, const
         return order.size() == n;
     };
     std::vector<int> order;
-    if (!kahn(order)) { set_error("the stage requests depend on each other in a cycle"); return LOP_EINVAL; }
-    if (by_start) {
-        std::vector<double> end(n, 0.0);
-        double link_free = 0.0;                                   // fetches share the host link: one after the other
-        for (int i : order) {
-            double start = 0.0;
-            if (arrival_us && raw[i] && reqs[i].wait_arrival && reqs[i].band < (int)arrival_us->size()) start = (*arrival_us)[reqs[i].band];
-            for (int j : prods[i]) start = std::max(start, end[j]);
-            if (reqs[i].fetch) {
-                const double busy = stage_cost_us(cx, reqs[i]) - 3.0;
-                start = std::max(start, link_free);
-                link_free = start + busy;
-            }
-            end[i] = start + stage_cost_us(cx, reqs[i]);
-            reqs[i].prio = (long long)(start * 1000.0);
-        }
+    if (!by_start) {
         if (!kahn(order)) { set_error("the stage requests depend on each other in a cycle"); return LOP_EINVAL; }
+    } else {
+        // A model of the machine as it really runs: items go round-robin to n_cta CTAs in program order and each
+        // CTA takes its items in order, waiting for an item's stage to be ready; fetches queue on the host link.
+        struct Machine {
+            std::vector<double> cta_free;
+            double link_free = 0.0, makespan = 0.0;
+            long long rr = 0;                                   // items placed so far: the round-robin position
+            explicit Machine(int n_cta) : cta_free(n_cta, 0.0) {}
+            double run(const StageShape &sh, bool fetch, double ready)
+            {
+                double fin = ready;
+                if (fetch) {
+                    const double start = std::max(ready, link_free);
+                    link_free = start + sh.item_us;
+                    fin = link_free + 3.0;                      // + the link's latency
+                } else {
+                    for (int it = 0; it < sh.items; ++it, ++rr) {
+                        double &f = cta_free[rr % (long long)cta_free.size()];
+                        f = std::max(f, ready) + sh.item_us;
+                        fin = std::max(fin, f + sh.tail_us);
+                    }
+                }
+                makespan = std::max(makespan, fin);
+                return fin;
+            }
+        };
+        const int n_cta = 148;
+        const double hop_us = 1.0;                              // producer's last store -> consumer sees the counter
+        std::vector<StageShape> shape(n);
+        for (size_t i = 0; i < n; ++i) shape[i] = stage_shape(cx, reqs[i]);
+        auto arrival_of = [&](int i) {
+            return (arrival_us && raw[i] && reqs[i].wait_arrival && reqs[i].band < (int)arrival_us->size()) ? (*arrival_us)[reqs[i].band] : 0.0;
+        };
+        // Candidate 1, greedy list scheduling: repeatedly append, among the stages whose producers are all placed,
+        // the one that is ready first, and let the model run it.  While the machine waits for input this follows
+        // each band down its layers (the pipeline of Sec. IV-B); once the machine is saturated, finish times slip,
+        // stages of other bands become ready first and the order turns layer-major by itself.
+        double span_greedy = 0.0;
+        {
+            Machine mc(n_cta);
+            std::vector<double> ready(n, 0.0);
+            std::vector<int> pending(n), heap;
+            auto later = [&](int x, int y) {
+                if (ready[x] != ready[y]) return ready[x] > ready[y];
+                if (reqs[x].prio != reqs[y].prio) return reqs[x].prio > reqs[y].prio;
+                return x > y;
+            };
+            for (size_t i = 0; i < n; ++i) {
+                pending[i] = (int)prods[i].size();
+                if (!pending[i]) { ready[i] = arrival_of((int)i); heap.push_back((int)i); }
+            }
+            std::make_heap(heap.begin(), heap.end(), later);
+            while (!heap.empty()) {
+                std::pop_heap(heap.begin(), heap.end(), later);
+                const int i = heap.back();
+                heap.pop_back();
+                order.push_back(i);
+                const double fin = mc.run(shape[i], reqs[i].fetch, ready[i]);
+                for (int u : users[i]) {
+                    ready[u] = std::max(ready[u], fin + hop_us);
+                    if (--pending[u] == 0) {
+                        ready[u] = std::max(ready[u], arrival_of(u));
+                        heap.push_back(u);
+                        std::push_heap(heap.begin(), heap.end(), later);
+                    }
+                }
+            }
+            if (order.size() != n) { set_error("the stage requests depend on each other in a cycle"); return LOP_EINVAL; }
+            span_greedy = mc.makespan;
+        }
+        // Candidate 2, layer-major (operation batching, Sec. IV-C): all bands' stages of one depth together, the
+        // way resident programs run; the input's transfer is then hidden only behind the first layers.  Deep
+        // chains of many thin bands do better this way: their late stages have too few tiles to fill the machine
+        // band by band.  The model decides.
+        {
+            std::vector<int> depth(n, 0);
+            for (int i : order)
+                for (int j : prods[i]) depth[i] = std::max(depth[i], depth[j] + 1);
+            std::vector<long long> keep(n);
+            for (size_t i = 0; i < n; ++i) { keep[i] = reqs[i].prio; reqs[i].prio = (long long)depth[i] * 65536 + reqs[i].band; }
+            std::vector<int> batched;
+            kahn(batched);
+            for (size_t i = 0; i < n; ++i) reqs[i].prio = keep[i];
+            Machine mc(n_cta);
+            std::vector<double> fin(n, 0.0);
+            for (int i : batched) {
+                double ready = arrival_of(i);
+                for (int j : prods[i]) ready = std::max(ready, fin[j] + hop_us);
+                fin[i] = mc.run(shape[i], reqs[i].fetch, ready);
+            }
+#ifdef LOP_WF_TRACE
+            fprintf(stderr, "order model: greedy %.1f us, layer-major %.1f us (%zu stages)\n", span_greedy, mc.makespan, n);
+#endif
+            if (batched.size() == n && mc.makespan < span_greedy) order.swap(batched);
+        }
     }
     std::vector<StageReq> out;
     out.reserve(n);
