@@ -30,7 +30,7 @@ if ROOT not in sys.path:
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one wavefront_kernel launch (ncu --set full, see
 # profiles/wavefront_kernel_vgg_block.md); None for workloads not captured, or once the kernel has changed since
-TRAFFIC = {"vgg_block": 500.1e3}
+TRAFFIC = {"vgg_block": 499.7e3}
 
 METRIC = "band-pipelined conv-chain images/s"
 UNIT = "images/s"
@@ -362,6 +362,8 @@ def main():
         "vs_baseline": None, "dtype": "bf16" if wl.dtype == "bf16" else "f32", "data": "synthetic",
         "config": {"workload": WORKLOAD_NOTES[args.workload], "images_per_step_per_gpu": wl.N,
                    "mode": "reuse-halo bands", "launch": "eager" if args.no_graph else "value: cuda-graph replay of one step; e2e: eager calls",
+                   "e2e_transport": "input bands fetched from pinned host memory by the persistent kernel's fetch warps; result "
+                                    "stored by the last layer straight into pinned host memory; one launch, no copy commands",
                    "l2": "256 MiB buffer written between timed steps", "multi_gpu": "independent replicas"},
         "e2e": {"value": job_images_per_s(wl.N, world, ms_e2e), "unit": UNIT, "ms_per_step": ms_e2e,
                 "h2d_bytes_per_step": int(x_pin.numel() * x_pin.element_size()),
@@ -375,9 +377,11 @@ def main():
         "pipeline": {"t_copy_ms": t_copy, "t_compute_ms": t_comp, "t_pipelined_ms": t_pipe, "exposed_ms": exposed,
                      "hidden_pct": hidden, "hidden_pct_bound": bound, "first_copy_ms": t_first,
                      "n_bands": dc.plans[0].num_bands(),
-                     "note": "t_copy: the band copies alone, back to back on one stream; a pipelined run adds per band an "
-                             "event record and a 4-byte arrival write on a second stream, each a stream command of a few "
-                             "microseconds like the copy itself",
+                     "note": "t_copy / first_copy: the bands as copy-engine copies alone, back to back on one stream (the "
+                             "transmission the pipeline has to hide; the bound is computed from them). t_pipelined: one "
+                             "launch whose fetch warps read the bands from pinned host memory while the other warps compute, "
+                             "output left on the device; it can beat the bound because the kernel's fetch has no per-copy "
+                             "command cost",
                      "launch": "eager calls"},
     }
     if world == 1 and not args.no_cpu_baseline:
