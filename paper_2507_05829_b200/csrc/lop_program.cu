@@ -636,7 +636,7 @@ int program_build(const std::vector<SegBind> &segs, std::vector<StageReq> reqs, 
     if (n_items == 0) { *result = p; return LOP_OK; }          // nothing to do: an empty program
 
     // ---- shared-memory rings: as many slots as fit beside the staging tile, weights first
-    const size_t fixed = 1024 + stg_bytes + 8 * (2 * 8 + 2 * 8 + 4 + 2 * WF_PUBQ) + 64 + 2048 + 1280 + 64;
+    const size_t fixed = 1024 + stg_bytes + 8 * (2 * 8 + 2 * 8 + 4 + 2 * WF_PUBQ + 4) + 64 + 2048 + 1280 + 64;
     const size_t budget = 227 * 1024 - fixed;
     int sa = 2, sb = 2;
     if ((size_t)sa * a_slot + (size_t)sb * b_slot > budget) { delete p; set_error("tile buffers do not fit shared memory"); return LOP_EUNSUPPORTED; }

@@ -67,8 +67,13 @@ __device__ __forceinline__ void tr(int item, int slot)
         g_wf_trace[item * 16 + slot] = t;
     }
 }
+__device__ __forceinline__ void trv(int item, int slot, unsigned long long v)
+{
+    if (item < TRACE_ITEMS) g_wf_trace[item * 16 + slot] = v;
+}
 #else
 #define tr(item, slot) ((void)0)
+#define trv(item, slot, v) ((void)0)
 #endif
 
 // ---- item records -------------------------------------------------------------------------------
@@ -221,16 +226,20 @@ __global__ void __launch_bounds__(FETCH ? WF_THREADS + 32 : WF_THREADS, 1) wavef
     const uint32_t full_a = bars, empty_a = full_a + 8u * SA, full_b = empty_a + 8u * SA, empty_b = full_b + 8u * SB;
     const uint32_t accf0 = empty_b + 8u * SB, acce0 = accf0 + 16u;
     const uint32_t pubf0 = acce0 + 16u, pube0 = pubf0 + 8u * WF_PUBQ;
-    uint8_t *tail = smem + (pube0 + 8u * WF_PUBQ - base);
+    const uint32_t ssf0 = pube0 + 8u * WF_PUBQ, sse0 = ssf0 + 16u;      // scale/shift buffers of two tiles: full / empty
+    uint8_t *tail = smem + (sse0 + 16u - base);
     volatile uint32_t *misc = reinterpret_cast<volatile uint32_t *>(tail);      // [0] TMEM base, [1] abort, [2] run, [3] epilogue failure
-    float *s_scale = reinterpret_cast<float *>(tail + 64);                       // [256]
-    float *s_shift = s_scale + 256;                                              // [256]
+    float *s_scale = reinterpret_cast<float *>(tail + 64);                       // [2][128]: per-channel scale of this and the next tile
+    float *s_shift = s_scale + 256;                                              // [2][128]
     long long *row_pix = reinterpret_cast<long long *>(tail + 64 + 2048);        // [128]: element offset of anchor m's output, or -1
     long long *pool_pix = row_pix + 128;                                         // [32]: element offset of a 2x2 window's pooled output, or -1
     uint8_t *stg = smem + (stg0 - base);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (threadIdx.x == 0 && blockIdx.x < 4) tr(TRACE_ITEMS - 8 + (int)blockIdx.x, 0);
+    if (threadIdx.x == 0 && blockIdx.x < 4) {
+        tr(TRACE_ITEMS - 8 + (int)blockIdx.x, 0);
+        trv(TRACE_ITEMS - 8 + (int)blockIdx.x, 4, (unsigned long long)clock64());
+    }
     if (threadIdx.x == 0) {
         for (int s = 0; s < SA; ++s) {
             mbar_init(full_a + 8u * s, 1);
@@ -243,6 +252,8 @@ __global__ void __launch_bounds__(FETCH ? WF_THREADS + 32 : WF_THREADS, 1) wavef
         for (int b = 0; b < 2; ++b) {
             mbar_init(accf0 + 8u * b, 1);
             mbar_init(acce0 + 8u * b, 1);
+            mbar_init(ssf0 + 8u * b, 1);
+            mbar_init(sse0 + 8u * b, 1);
         }
         for (int q = 0; q < WF_PUBQ; ++q) {
             mbar_init(pubf0 + 8u * q, 1);
@@ -282,7 +293,12 @@ __global__ void __launch_bounds__(FETCH ? WF_THREADS + 32 : WF_THREADS, 1) wavef
             amask = 0, kh = 1, kw = 1, sh = 1, sw = 1, ph = 0, pw = 0, dh = 1, dw = 1;
         uint32_t a_bytes = 0, b_bytes = 0;
         const CUtensorMap *maps = nullptr;
-        uint32_t a_slot = 0, a_phase = 0, b_slot = 0, b_phase = 0;
+        const float *scale = nullptr, *shift = nullptr;
+        int slab_offh = 0, slab_offw = 0, slab_mi = 0, n_boxes = 1;
+        bool slab_have = true;
+        uint32_t a_slot = 0, a_phase = 0, b_slot = 0, b_phase = 0, pc = 0;
+        bool w_kept = false;                                   // (lane 0) the ring holds the weights of tile key w_key
+        long long w_key = -1;
         for (; item < NI; item += G) {
             // two items ahead: the record; one item ahead: this lane's dependency entry
             const int4 nn = item + 2 * G < NI ? __ldg(&P.items[item + 2 * G]) : zero4;
@@ -298,10 +314,32 @@ __global__ void __launch_bounds__(FETCH ? WF_THREADS + 32 : WF_THREADS, 1) wavef
                 maps = P.maps + __ldg(&sp->map_base);
                 kh = __ldg(&sp->kh); kw = __ldg(&sp->kw); sh = __ldg(&sp->sh); sw = __ldg(&sp->sw);
                 ph = __ldg(&sp->ph); pw = __ldg(&sp->pw); dh = __ldg(&sp->dh); dw = __ldg(&sp->dw);
+                scale = ldg_ptr<const float *>(reinterpret_cast<const void *const *>(&sp->scale));
+                shift = ldg_ptr<const float *>(reinterpret_cast<const void *const *>(&sp->shift));
+                // slab mode: the box starts at the first tap's offset; which parity map that is and how far in
+                const int offh = floor_div_i(-ph, sh), offw = floor_div_i(-pw, sw);
+                slab_offh = offh; slab_offw = offw;
+                slab_mi = (-ph - offh * sh) * sw + (-pw - offw * sw);
+                slab_have = (amask >> slab_mi) & 1;
+                n_boxes = n_chunks * ((n_taps + tbx - 1) / tbx);
             }
             if (kind == WF_CONV) {
                 if (lane == 0) tr(item, 0);
-                const bool ok = wait_deps_warp(P, rec_dep0(cur), rec_ndep(cur), dep_cur, run, lane);
+                // the tile's per-channel scale / shift go to shared memory from here, a tile ahead of the epilogue
+                // that uses them: their load latency is off the workers' path
+                bool ok = __all_sync(0xffffffffu, mbar_wait_abortable(sse0 + 8u * (pc & 1u), ((pc >> 1) & 1u) ^ 1u, abort_flag));
+                if (ok) {
+                    float *ds = s_scale + 128 * (pc & 1u), *dsh = s_shift + 128 * (pc & 1u);
+                    const int c0 = rec_cout(cur) * BN;
+                    for (int i = lane; i < BN; i += 32) {
+                        ds[i] = scale ? __ldg(scale + c0 + i) : 1.0f;
+                        dsh[i] = shift ? __ldg(shift + c0 + i) : 0.0f;
+                    }
+                    __syncwarp();
+                    if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(ssf0 + 8u * (pc & 1u)) : "memory");
+                    ++pc;
+                }
+                ok = ok && wait_deps_warp(P, rec_dep0(cur), rec_ndep(cur), dep_cur, run, lane);
                 int fail = 0;
                 if (!ok) {
                     if (lane == 0) atomicOr(P.status, 0x10u);
@@ -313,21 +351,27 @@ __global__ void __launch_bounds__(FETCH ? WF_THREADS + 32 : WF_THREADS, 1) wavef
                     const int oh0 = oh_lo + (rec_tr(cur) << tr_log);
                     const int n0 = rec_tn(cur) * (128 >> (p_log + tr_log));
                     const int co0 = rec_cout(cur) * BN;
+                    // Weights stay in their ring slots from one tile to the next while consecutive tiles of this CTA
+                    // use the same ones (same layer, same output channels) and all their boxes fit the ring: only the
+                    // first such tile loads them.  The MMA issuer takes the same decisions from the same records and
+                    // frees the slots when a tile with other weights comes up.
+                    const long long wkey = (long long)(maps - P.maps) * 65536 + rec_cout(cur);
+                    const bool can_keep = mode == WF_SLAB && n_boxes <= SB;
+                    const bool reuse_w = w_kept && can_keep && wkey == w_key;
+                    w_kept = reuse_w || can_keep;
+                    w_key = wkey;
                     for (int ch = 0; ch < n_chunks && !fail; ++ch) {
                         if (mode == WF_SLAB) {
                             // the whole receptive window of the tile in one box: its first tap's offset places it
-                            const int qh = -ph, qw = -pw;
-                            const int offh = floor_div_i(qh, sh), parh = qh - offh * sh;
-                            const int offw = floor_div_i(qw, sw), parw = qw - offw * sw;
-                            const int mi = parh * sw + parw;
-                            const bool have = (amask >> mi) & 1;
+                            const int mi = slab_mi, offh = slab_offh, offw = slab_offw;
+                            const bool have = slab_have;
                             if (!mbar_wait_abortable(empty_a + 8u * a_slot, a_phase ^ 1u, abort_flag)) { fail = 1; break; }
                             const uint32_t fa = full_a + 8u * a_slot;
                             mbar_expect_tx(fa, a_bytes);
                             tma_load_4d(a0 + a_slot * a_slot_bytes, maps + mi, fa, ch * BK, have ? ow0 + offw : -65536,
                                         have ? oh0 + offh : -65536, n0);
                             if (++a_slot == (uint32_t)SA) { a_slot = 0; a_phase ^= 1u; }
-                            for (int t0 = 0; t0 < n_taps; t0 += tbx) {
+                            for (int t0 = 0; t0 < n_taps && !reuse_w; t0 += tbx) {
                                 if (!mbar_wait_abortable(empty_b + 8u * b_slot, b_phase ^ 1u, abort_flag)) { fail = 1; break; }
                                 const uint32_t fb = full_b + 8u * b_slot;
                                 mbar_expect_tx(fb, b_bytes);
@@ -380,6 +424,13 @@ __global__ void __launch_bounds__(FETCH ? WF_THREADS + 32 : WF_THREADS, 1) wavef
             uint32_t idesc = 0, desc_hi = 0, row_bytes = 0, tap_bytes = 0;
             uint32_t a_slot = 0, a_phase = 0, b_slot = 0, b_phase = 0, cnt = 0;
             bool fail = false, row3x64 = false;
+            bool w_kept = false;                               // weights kept in ring slots w_first .. w_first + w_n - 1 for key w_key
+            long long w_key = -1;
+            uint32_t w_first = 0, w_n = 0;
+            int map_base = 0, nblk = 1;                        // nblk: weight boxes per channel chunk
+#ifdef LOP_WF_TRACE
+            long long dbg_c0 = 0, dbg_fence = 0, dbg_mma = 0;
+#endif
             for (; item < NI && !fail; item += G) {
                 const int4 nxt = item + G < NI ? __ldg(&P.items[item + G]) : zero4;
                 if (rec_stage(cur) != sidx) {
@@ -388,6 +439,8 @@ __global__ void __launch_bounds__(FETCH ? WF_THREADS + 32 : WF_THREADS, 1) wavef
                     kind = __ldg(&sp->kind); mode = __ldg(&sp->mode);
                     n_chunks = __ldg(&sp->n_chunks); n_taps = __ldg(&sp->n_taps); tbx = __ldg(&sp->tb);
                     kw = __ldg(&sp->kw); dh = __ldg(&sp->dh); dw = __ldg(&sp->dw); p_log = __ldg(&sp->p_log);
+                    map_base = __ldg(&sp->map_base);
+                    nblk = (n_taps + tbx - 1) / tbx;
                     ksteps = __ldg(&sp->BK) / 16;
                     idesc = __ldg(&sp->idesc);
                     desc_hi = ((__ldg(&sp->sbo_bytes) >> 4) & 0x3FFFu) | (1u << 14) | (__ldg(&sp->layout_code) << 29);
@@ -402,31 +455,69 @@ __global__ void __launch_bounds__(FETCH ? WF_THREADS + 32 : WF_THREADS, 1) wavef
                     tr(item, 3);
                     const uint32_t acc = tmem_base + buf * 256u;
                     uint32_t accumulate = 0;
+                    // kept weights (see the loader): used in place by tiles with the same key, freed -- once the MMAs
+                    // that read them are done -- when a tile with another key comes up
+                    // (this thread issues every MMA of the CTA and is bound by its own instruction latencies: no division
+                    // or modulo in these loops)
+                    const uint32_t n_boxes = (uint32_t)(n_chunks * nblk);
+                    const long long wkey = (long long)map_base * 65536 + rec_cout(cur);
+                    const bool can_keep = mode == WF_SLAB && n_boxes <= (uint32_t)SB;
+                    const bool reuse_w = w_kept && can_keep && wkey == w_key;
+                    if (w_kept && !reuse_w) {
+                        for (uint32_t i = 0, sl = w_first; i < w_n; ++i) {
+                            umma_commit(empty_b + 8u * sl);
+                            if (++sl == (uint32_t)SB) sl = 0;
+                        }
+                        w_kept = false;
+                    }
+                    if (!reuse_w && can_keep) { w_kept = true; w_key = wkey; w_first = b_slot; w_n = n_boxes; }
+                    uint32_t ws = w_first;                                  // kept box of the current (chunk, tap block)
                     for (int ch = 0; ch < n_chunks && !fail; ++ch) {
                         if (mode == WF_SLAB) {
                             if (!mbar_wait_abortable(full_a + 8u * a_slot, a_phase, abort_flag)) { fail = true; break; }
+                            if (ch == 0) tr(item, 13);
                             const uint32_t sa = a0 + a_slot * a_slot_bytes;
+                            int ta = 0, tb = 0;                             // filter position of tap t0
                             for (int t0 = 0; t0 < n_taps; t0 += tbx) {
-                                if (!mbar_wait_abortable(full_b + 8u * b_slot, b_phase, abort_flag)) { fail = true; break; }
+                                uint32_t bs = b_slot;
+                                if (reuse_w) {
+                                    bs = ws;
+                                    if (++ws == (uint32_t)SB) ws = 0;
+                                } else if (!mbar_wait_abortable(full_b + 8u * b_slot, b_phase, abort_flag)) { fail = true; break; }
+                                if (ch == 0 && t0 == 0) tr(item, 14);
+#ifdef LOP_WF_TRACE
+                                const long long c0 = clock64();
+                                if (t0 == 0) dbg_c0 = c0;
+#endif
                                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                                const uint32_t sb = b0 + b_slot * b_slot_bytes;
-                                const int t1 = min(t0 + tbx, n_taps);
-                                int ta = t0 / kw, tb = t0 - ta * kw;
+#ifdef LOP_WF_TRACE
+                                const long long c1 = clock64();
+                                dbg_fence += c1 - c0;
+#endif
+                                const uint32_t sb = b0 + bs * b_slot_bytes;
                                 if (row3x64) {
-                                    // box = filter row t0 / 3 of a 3x3 filter: the slab row it starts at, then constants
+                                    // box = one row of a 3x3 filter: the slab row it starts at, then constants
                                     const uint32_t pa = sa + (uint32_t)((ta * dh) << p_log) * 128u;
                                     mma_row3x64(acc, ((pa & 0x3FFFFu) >> 4) | (1u << 16), ((sb & 0x3FFFFu) >> 4) | (1u << 16), tap_bytes >> 4,
                                                 desc_hi, idesc, accumulate);
-                                } else
-                                for (int t = t0; t < t1; ++t) {
-                                    // tap (ta, tb): the same box, read (ta*dh*P + tb*dw) pixels further on
-                                    const uint32_t pa = sa + (uint32_t)(((ta * dh) << p_log) + tb * dw) * row_bytes;
-                                    const uint32_t pb = sb + (uint32_t)(t - t0) * tap_bytes;
-                                    mma_tap(acc, pa, pb, desc_hi, idesc, ksteps, accumulate);
-                                    if (++tb == kw) { tb = 0; ++ta; }
+#ifdef LOP_WF_TRACE
+                                    dbg_mma += clock64() - c1;
+#endif
+                                    ++ta;
+                                } else {
+                                    const int t1 = min(t0 + tbx, n_taps);
+                                    uint32_t pb = sb;
+                                    for (int t = t0; t < t1; ++t, pb += tap_bytes) {
+                                        // tap (ta, tb): the same box, read (ta*dh*P + tb*dw) pixels further on
+                                        const uint32_t pa = sa + (uint32_t)(((ta * dh) << p_log) + tb * dw) * row_bytes;
+                                        mma_tap(acc, pa, pb, desc_hi, idesc, ksteps, accumulate);
+                                        if (++tb == kw) { tb = 0; ++ta; }
+                                    }
                                 }
-                                umma_commit(empty_b + 8u * b_slot);
-                                if (++b_slot == (uint32_t)SB) { b_slot = 0; b_phase ^= 1u; }
+                                if (!reuse_w) {
+                                    if (!can_keep) umma_commit(empty_b + 8u * b_slot);
+                                    if (++b_slot == (uint32_t)SB) { b_slot = 0; b_phase ^= 1u; }
+                                }
                             }
                             umma_commit(empty_a + 8u * a_slot);
                             if (++a_slot == (uint32_t)SA) { a_slot = 0; a_phase ^= 1u; }
@@ -445,6 +536,13 @@ __global__ void __launch_bounds__(FETCH ? WF_THREADS + 32 : WF_THREADS, 1) wavef
                         }
                     }
                     if (fail) break;
+#ifdef LOP_WF_TRACE
+                    trv(item, 8, (unsigned long long)dbg_fence);
+                    trv(item, 9, (unsigned long long)dbg_mma);
+                    trv(item, 10, (unsigned long long)(clock64() - dbg_c0));
+                    dbg_fence = dbg_mma = 0;
+#endif
+                    tr(item, 15);
                     umma_commit(accf0 + 8u * buf);
                     tr(item, 4);
                     ++cnt;
@@ -582,16 +680,14 @@ __global__ void __launch_bounds__(FETCH ? WF_THREADS + 32 : WF_THREADS, 1) wavef
                     const bool ok = valid && c + 1 < tw_valid && ow + 1 < Wo && oh + 1 < oh_hi;
                     pool_pix[q] = ok ? (((long long)n * pool_Ho + (oh >> 1)) * pool_Wo + (ow >> 1)) * Cout + co0 : -1LL;
                 }
-                for (int i = tid; i < BN; i += EPI_THREADS) {          // this tile's scale/shift while the main loop runs
-                    s_scale[i] = scale ? __ldg(scale + co0 + i) : 1.0f;
-                    s_shift[i] = shift ? __ldg(shift + co0 + i) : 0.0f;
-                }
-                epi_bar();
+                if (resp) epi_bar();                                   // the residual copy-in below reads row_pix
+                const float *t_scale = s_scale + 128 * buf, *t_shift = s_shift + 128 * buf;   // filled by warp 0 a tile ahead
                 const int cpr = BN >> 3;                               // 16-byte chunks per staged row
                 const int cpr_log = (cpr & (cpr - 1)) == 0 ? 31 - __clz(cpr) : -1;
                 const uint32_t row_stride = (uint32_t)BN * 2u;
                 const int swz = (cpr & 7) == 0 ? 7 : 0;                // chunk position = chunk ^ (row & 7): conflict-free columns
                 __nv_bfloat16 *y = static_cast<__nv_bfloat16 *>(yout);
+                if (!mbar_wait_abortable(ssf0 + 8u * buf, (cnt >> 1) & 1u, abort_flag)) *epi_fail = 1;
                 if (!mbar_wait_abortable(accf0 + 8u * buf, (cnt >> 1) & 1u, abort_flag)) *epi_fail = 1;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 if (tid == 0) tr(item, 5);
@@ -616,14 +712,12 @@ __global__ void __launch_bounds__(FETCH ? WF_THREADS + 32 : WF_THREADS, 1) wavef
                         uint32_t rr[16];
                         tmem_ld16(acc + (uint32_t)j, rr);
                         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                        if (tid == 0 && j == 0) tr(item, 8);
-                        if (tid == 0 && j == 16 * COL_GROUPS) tr(item, 10);
                         if (!valid) continue;
                         float v[16];
 #pragma unroll
                         for (int i = 0; i < 16; i += 4) {                  // 16-byte broadcast reads of the tile's scale / shift
-                            const float4 sc = *reinterpret_cast<const float4 *>(s_scale + j + i);
-                            const float4 sf = *reinterpret_cast<const float4 *>(s_shift + j + i);
+                            const float4 sc = *reinterpret_cast<const float4 *>(t_scale + j + i);
+                            const float4 sf = *reinterpret_cast<const float4 *>(t_shift + j + i);
                             v[i] = fmaf(sc.x, __uint_as_float(rr[i]), sf.x);
                             v[i + 1] = fmaf(sc.y, __uint_as_float(rr[i + 1]), sf.y);
                             v[i + 2] = fmaf(sc.z, __uint_as_float(rr[i + 2]), sf.z);
@@ -650,13 +744,15 @@ __global__ void __launch_bounds__(FETCH ? WF_THREADS + 32 : WF_THREADS, 1) wavef
                         }
                         *c0p = make_uint4(o[0], o[1], o[2], o[3]);
                         *c1p = make_uint4(o[4], o[5], o[6], o[7]);
-                        if (tid == 0 && j == 0) tr(item, 9);
                     }
                 }
                 asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
                 if (tid == 0) tr(item, 11);
                 epi_bar();                                             // accumulator drained, staging tile complete
-                if (tid == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(acce0 + 8u * buf) : "memory");
+                if (tid == 0) {
+                    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(acce0 + 8u * buf) : "memory");
+                    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(sse0 + 8u * buf) : "memory");
+                }
                 ++cnt;
                 if (!*epi_fail && fuse_pool) {
                     // 2x2 windows of staged rows -> their maxima (exact in bf16) -> the pooled tensor, 16 bytes per thread
@@ -871,7 +967,10 @@ __global__ void __launch_bounds__(FETCH ? WF_THREADS + 32 : WF_THREADS, 1) wavef
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (warp == 1)
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
-    if (threadIdx.x == 0 && blockIdx.x < 4) tr(TRACE_ITEMS - 8 + (int)blockIdx.x, 2);
+    if (threadIdx.x == 0 && blockIdx.x < 4) {
+        tr(TRACE_ITEMS - 8 + (int)blockIdx.x, 2);
+        trv(TRACE_ITEMS - 8 + (int)blockIdx.x, 5, (unsigned long long)clock64());
+    }
     if (threadIdx.x == 0) {
         __threadfence();
         const unsigned done = atomicAdd(P.counters + 1, 1u);
@@ -917,7 +1016,7 @@ extern "C" int lop_debug_trace_copy(void *host, size_t bytes, int clear)
 
 size_t wavefront_smem_bytes(const WfParams &p)
 {
-    return 1024 + (size_t)p.sa * p.a_slot_bytes + (size_t)p.sb * p.b_slot_bytes + p.stg_bytes + 8 * (size_t)(2 * p.sa + 2 * p.sb + 4 + 2 * WF_PUBQ) + 64 +
+    return 1024 + (size_t)p.sa * p.a_slot_bytes + (size_t)p.sb * p.b_slot_bytes + p.stg_bytes + 8 * (size_t)(2 * p.sa + 2 * p.sb + 4 + 2 * WF_PUBQ + 4) + 64 +
            2 * 256 * sizeof(float) + (128 + 32) * sizeof(long long) + 64;
 }
 
