@@ -472,6 +472,21 @@ __global__ void __launch_bounds__(FETCH ? WF_THREADS + 32 : WF_THREADS, 1) wavef
                     }
                     if (!reuse_w && can_keep) { w_kept = true; w_key = wkey; w_first = b_slot; w_n = n_boxes; }
                     uint32_t ws = w_first;                                  // kept box of the current (chunk, tap block)
+                    if (reuse_w && row3x64 && n_chunks == 1) {
+                        // the common tile of a 3x3 / 64-channel layer with its weights in place: 36 MMAs, nothing between
+                        // them but the start addresses of the three filter rows
+                        if (!mbar_wait_abortable(full_a + 8u * a_slot, a_phase, abort_flag)) { fail = true; break; }
+                        tr(item, 13);
+                        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                        const uint32_t la = (((a0 + a_slot * a_slot_bytes) & 0x3FFFFu) >> 4) | (1u << 16);
+                        const uint32_t row16 = (uint32_t)(dh << p_log) * 8u;          // one filter row further down the slab, in 16-byte units
+                        const uint32_t s0 = w_first, s1 = s0 + 1 == (uint32_t)SB ? 0u : s0 + 1, s2 = s1 + 1 == (uint32_t)SB ? 0u : s1 + 1;
+                        mma_row3x64(acc, la, (((b0 + s0 * b_slot_bytes) & 0x3FFFFu) >> 4) | (1u << 16), tap_bytes >> 4, desc_hi, idesc, accumulate);
+                        mma_row3x64(acc, la + row16, (((b0 + s1 * b_slot_bytes) & 0x3FFFFu) >> 4) | (1u << 16), tap_bytes >> 4, desc_hi, idesc, accumulate);
+                        mma_row3x64(acc, la + 2u * row16, (((b0 + s2 * b_slot_bytes) & 0x3FFFFu) >> 4) | (1u << 16), tap_bytes >> 4, desc_hi, idesc, accumulate);
+                        umma_commit(empty_a + 8u * a_slot);
+                        if (++a_slot == (uint32_t)SA) { a_slot = 0; a_phase ^= 1u; }
+                    } else
                     for (int ch = 0; ch < n_chunks && !fail; ++ch) {
                         if (mode == WF_SLAB) {
                             if (!mbar_wait_abortable(full_a + 8u * a_slot, a_phase, abort_flag)) { fail = true; break; }
