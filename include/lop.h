@@ -214,7 +214,11 @@ int lop_plan_last_launches(const lop_plan_t *plan);
 int lop_plan_last_copies(const lop_plan_t *plan);
 /* Reads the plan's device status word (0 = no kernel gave up on a bounded wait).  SYNCHRONISES
  * the stream of the last execution call.  On LOP_EDEVICE the outputs of that call are invalid; the
- * library drops its cached device tables and clears the word, so the plan can be used again. */
+ * library drops its cached device tables and clears the word, so the plan can be used again.
+ * lop_last_error() then shows the word; its bits name the role of the persistent kernel whose wait
+ * ran out: 0x1 loader (ring slot), 0x2 MMA issuer (operands), 0x4 epilogue / pooling / gather
+ * (accumulator, dependencies), 0x8 publisher, 0x10 loader (dependencies of a tile), 0x20 fetch warp
+ * (window of the in-kernel input transfer). */
 int lop_plan_check_device(lop_plan_t *plan, void *workspace);
 
 /* ---- execution without any allocation --------------------------------------------------------
