@@ -161,6 +161,22 @@ int lop_run_banded(lop_plan_t *plan, const void *in_dev, void *out_dev, void *wo
  * the chain-input rows the band needs and no earlier band has brought, for all N images, from
  * in_host_pinned (PINNED HOST, full-size tensor) to the same rows of staging_dev. */
 int lop_copy_band(lop_plan_t *plan, int band, const void *in_host_pinned, void *staging_dev, void *stream);
+/* ---- band sharding over several devices (Sec. IV-C: operation replication) ---------------------
+ * Bands that carry their halo are independent units: device `rank` of `world` takes the contiguous
+ * block of bands  [floor(rank*B/world), floor((rank+1)*B/world)), runs it with lop_run_shard on its own
+ * copy of the parameters, and the devices exchange the produced output rows once per plan (an
+ * all-gather; the Python package's shard module does it with torch.distributed). */
+/* HOST ONLY.  The block of bands of device `rank`, the rows [row_lo,row_hi) of the LAST layer's output
+ * it produces and the rows [in_lo,in_hi) of the chain input it reads (empty ranges have lo == hi). */
+int lop_plan_shard(const lop_plan_t *plan, int rank, int world, int *band_lo, int *band_hi, int *row_lo,
+                   int *row_hi, int *in_lo, int *in_hi);
+/* Runs bands [band_lo, band_hi) in ascending order as one unit.  Only rows [in_lo,in_hi) of in_dev need
+ * to be present and only rows [row_lo,row_hi) of out_dev are written.  With LOP_FLAG_REUSE_HALO a
+ * band computes what the BLOCK has not produced yet (no earlier band has run on this device, so the
+ * block's first band computes its whole halo); the output rows are bit-identical to those of
+ * lop_run_banded on one device. */
+int lop_run_shard(lop_plan_t *plan, int band_lo, int band_hi, const void *in_dev, void *out_dev,
+                  void *workspace, void *stream);
 /* Band pipeline (Sec. IV-B computation/transmission overlap): band i+1's rows come in while band i is
  * computed.  Two transports:
  *   - fetched (default when in_host_pinned is mapped into the device's address space, as cudaHostAlloc /

@@ -77,6 +77,38 @@ def run_banded(layers, x, plan, round_bf16, reuse=False, band_order=None):
     return stitched
 
 
+def run_band_block(layers, x, plan, round_bf16, b0, b1, reuse=False):
+    """Bands [b0, b1) on a device that runs no other band (the paper's operation replication across devices,
+    Sec. IV-C): tensors start poisoned, only the chain-input rows those bands need are present, and -- in reuse mode -- a band computes only the rows the
+    block itself has not yet produced (so the block's first band computes every row it needs).  Returns the last layer's output with the block's rows filled in and poison elsewhere."""
+    N = x.shape[0]
+    L = len(layers)
+    t = {-1: np.full(x.shape, POISON, dtype=np.float32)}
+    for i, (h, w, c) in enumerate(plan.shapes):
+        t[i] = np.full((N, h, w, c), POISON, dtype=np.float32)
+    stitched = np.full((N,) + tuple(plan.shapes[-1]), POISON, dtype=np.float32)
+    done = [0] * L                                     # rows [.., done) of layer i this block has produced so far
+    for b in range(b0, b1):
+        lo, hi, _ = plan.input_need[b]
+        t[-1][:, lo:hi] = x[:, lo:hi]
+        if not reuse and b != b0:                      # independent bands never read another band's rows
+            for i in range(L):
+                t[i][...] = POISON
+        for i, l in enumerate(layers):
+            r = plan.ranges[b][i]
+            if r.out_lo >= r.out_hi:
+                continue
+            r0 = min(max(r.out_lo, done[i]), r.out_hi) if reuse else r.out_lo
+            done[i] = max(done[i], r.out_hi)
+            if r0 >= r.out_hi:
+                continue
+            res = t[l.residual_from] if l.residual_from != NO_RESIDUAL else None
+            run_layer(l, t[l.input_from], res, (r0, r.out_hi), round_bf16, t[i])
+        r = plan.ranges[b][L - 1]
+        stitched[:, r.out_lo:r.out_hi] = t[L - 1][:, r.out_lo:r.out_hi]
+    return stitched
+
+
 def run_workload(wl, banded=False, reuse=False, keep_segments=False):
     """Run every segment of a workload in order; each segment's output feeds the next."""
     rb = wl.dtype == "bf16"

@@ -20,7 +20,8 @@ EXPORTS = [
     "lop_plan_out_shape", "lop_plan_set_params", "lop_plan_workspace_bytes", "lop_plan_staging_bytes",
     "lop_plan_flops", "lop_run_whole", "lop_run_band", "lop_run_banded", "lop_copy_band", "lop_run_pipelined",
     "lop_plan_last_timing", "lop_plan_layer_time", "lop_plan_layer_kernel", "lop_plan_last_launches", "lop_plan_last_copies",
-    "lop_plan_check_device", "lop_run_whole_static", "lop_run_chain_banded", "lop_run_chain_pipelined", "lop_strerror", "lop_last_error",
+    "lop_plan_check_device", "lop_run_whole_static", "lop_run_chain_banded", "lop_run_chain_pipelined", "lop_plan_shard", "lop_run_shard",
+    "lop_strerror", "lop_last_error",
 ]
 LOP_STATIC_SCRATCH_BYTES = 16 << 20
 
@@ -93,6 +94,8 @@ def lib():
     L.lop_run_whole_static.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
     L.lop_run_chain_banded.argtypes = [POINTER(c_void_p), c_int, c_void_p, POINTER(c_void_p), POINTER(c_void_p), c_void_p]
     L.lop_run_chain_pipelined.argtypes = [POINTER(c_void_p), c_int, c_void_p, c_void_p, POINTER(c_void_p), POINTER(c_void_p), c_void_p]
+    L.lop_plan_shard.argtypes = [c_void_p, c_int, c_int] + [POINTER(c_int)] * 6
+    L.lop_run_shard.argtypes = [c_void_p, c_int, c_int, c_void_p, c_void_p, c_void_p, c_void_p]
     L.lop_strerror.argtypes = [c_int]
     L.lop_strerror.restype = c_char_p
     L.lop_last_error.restype = c_char_p
@@ -194,6 +197,15 @@ class Plan:
 
     def copy_band(self, band, in_host, staging_dev, stream):
         _check(lib().lop_copy_band(self._h, band, in_host, staging_dev, stream))
+
+    def shard(self, rank, world):
+        """(band_lo, band_hi, row_lo, row_hi, in_lo, in_hi) of device ``rank`` of ``world`` (host only)."""
+        v = [c_int(0) for _ in range(6)]
+        _check(lib().lop_plan_shard(self._h, rank, world, *[byref(x) for x in v]))
+        return tuple(x.value for x in v)
+
+    def run_shard(self, band_lo, band_hi, in_dev, out_dev, ws, stream):
+        _check(lib().lop_run_shard(self._h, band_lo, band_hi, in_dev, out_dev, ws, stream))
 
     def run_pipelined(self, in_host, staging_dev, out_dev, ws, stream):
         _check(lib().lop_run_pipelined(self._h, in_host, staging_dev, out_dev, ws, stream))

@@ -32,7 +32,8 @@ struct MapKey {
 };
 
 struct ProgKey {
-    int kind;                        // -1 whole, -2 all bands, -3 pipelined, -4 pipelined with in-kernel fetch, >= 0 one band
+    int kind;                        // -1 whole, -2 all bands, -3 pipelined, -4 pipelined with in-kernel fetch, >= 0 one band,
+                                     // <= -16: the block of bands [lo, hi) encoded as -16 - (lo * 65536 + hi)
     int n_plans;                     // plans of the chain the program spans
     const void *in, *out, *ws;       // first plan's input and workspace, last plan's output
     const void *src;                 // fetch source (host memory as the device addresses it) or nullptr
@@ -248,19 +249,35 @@ int run_band_impl(lop_plan_t *pl, int band, const void *in, void *out, void *ws,
 
 // Requests of one band of plan `seg` in dependency order; a gathered stem is preceded by its patch-gather stage over
 // the same rows.
-void band_requests(const lop_plan_t *pl, int seg, int band, bool wait_arrival, std::vector<StageReq> &reqs)
+// First row of layer i that band `band` computes when bands [block_lo, band) are the only ones that have run on this
+// device: in reuse mode what the block has not produced yet (for block_lo = 0 that is the plan's new_lo).
+int first_row(const lop_plan_t *pl, int block_lo, int band, int i)
 {
     const int L = (int)pl->layers.size();
-    const bool reuse = (pl->flags & LOP_FLAG_REUSE_HALO) != 0;
+    const lop_range &r = pl->ranges[(size_t)band * L + i];
+    if (!(pl->flags & LOP_FLAG_REUSE_HALO)) return r.out_lo;
+    if (block_lo == 0) return r.new_lo;
+    int done = 0;
+    for (int b = block_lo; b < band; ++b) {
+        const lop_range &q = pl->ranges[(size_t)b * L + i];
+        if (q.out_hi > q.out_lo) done = std::max(done, (int)q.out_hi);
+    }
+    return std::min(std::max((int)r.out_lo, done), (int)r.out_hi);
+}
+
+// block_lo: the first band that runs on this device (0 unless the bands are sharded over devices).
+void band_requests(const lop_plan_t *pl, int seg, int band, bool wait_arrival, std::vector<StageReq> &reqs, int block_lo = 0)
+{
+    const int L = (int)pl->layers.size();
     for (int i = 0; i < L; ++i) {
         const lop_range &r = pl->ranges[(size_t)band * L + i];
-        const int lo = reuse ? r.new_lo : r.out_lo;
+        const int lo = first_row(pl, block_lo, band, i);
         if (pl->layers[i].stem_gather) reqs.push_back(StageReq{seg, band, i, lo, r.out_hi, wait_arrival && seg == 0, true, 0});
         reqs.push_back(StageReq{seg, band, i, lo, r.out_hi, wait_arrival && seg == 0, false, 0});
     }
 }
 
-enum { PROG_WHOLE = -1, PROG_ALL_BANDS = -2, PROG_PIPELINED = -3, PROG_FETCHED = -4 };
+enum { PROG_WHOLE = -1, PROG_ALL_BANDS = -2, PROG_PIPELINED = -3, PROG_FETCHED = -4, PROG_BLOCK0 = -16 };
 
 // kind: PROG_WHOLE, PROG_ALL_BANDS, PROG_PIPELINED, PROG_FETCHED (fetch_src: the host input as the device addresses
 // it), or b >= 0 for band b alone (single plan only).  segs: the plans of a chain with their buffers; the program is
@@ -321,6 +338,18 @@ int get_program(const std::vector<SegBind> &segs, int kind, Program **prog, cons
                     }
                 }
                 joff += (long long)per;
+            }
+            std::stable_sort(reqs.begin(), reqs.end(), [](const StageReq &x, const StageReq &y) { return x.prio < y.prio; });
+        } else if (kind <= PROG_BLOCK0) {
+            // a block of bands on a device that runs no other band: layer-major like ALL_BANDS, the first band whole
+            const int code = PROG_BLOCK0 - kind, lo = code >> 16, hi = code & 0xFFFF;
+            for (int b = lo; b < hi; ++b) {
+                std::vector<StageReq> one;
+                band_requests(pl0, 0, b, false, one, lo);
+                for (size_t j = 0; j < one.size(); ++j) {
+                    one[j].prio = (long long)j * 65536 + b;
+                    reqs.push_back(one[j]);
+                }
             }
             std::stable_sort(reqs.begin(), reqs.end(), [](const StageReq &x, const StageReq &y) { return x.prio < y.prio; });
         } else {
@@ -496,6 +525,56 @@ int lop_run_banded(lop_plan_t *pl, const void *in, void *out, void *ws, void *st
     if (pl->exec->wavefront) return run_program(pl, PROG_ALL_BANDS, in, out, ws, s);
     for (int b = 0; b < pl->n_bands; ++b)
         if ((rc = run_band_impl(pl, b, in, out, ws, s)) != LOP_OK) return rc;
+    return LOP_OK;
+}
+
+int lop_plan_shard(const lop_plan_t *pl, int rank, int world, int *band_lo, int *band_hi, int *row_lo, int *row_hi, int *in_lo,
+                   int *in_hi)
+{
+    if (!pl || !band_lo || !band_hi || !row_lo || !row_hi || !in_lo || !in_hi) { set_error("lop_plan_shard: NULL argument"); return LOP_EINVAL; }
+    if (world < 1 || rank < 0 || rank >= world) { set_error("lop_plan_shard: rank %d of %d", rank, world); return LOP_EINVAL; }
+    const int B = pl->n_bands, L = (int)pl->layers.size();
+    const int b0 = (int)((long long)rank * B / world), b1 = (int)((long long)(rank + 1) * B / world);
+    *band_lo = b0; *band_hi = b1;
+    *row_lo = *row_hi = *in_lo = *in_hi = 0;
+    bool have_rows = false, have_in = false;
+    for (int b = b0; b < b1; ++b) {
+        const lop_range &r = pl->ranges[(size_t)b * L + (L - 1)];
+        if (r.out_hi > r.out_lo) {
+            if (!have_rows) { *row_lo = r.out_lo; have_rows = true; }
+            *row_hi = r.out_hi;
+        }
+        const lop_range &n = pl->in_need[b];
+        if (n.out_hi > n.out_lo) {
+            if (!have_in || n.out_lo < *in_lo) *in_lo = n.out_lo;
+            if (!have_in || n.out_hi > *in_hi) *in_hi = n.out_hi;
+            have_in = true;
+        }
+    }
+    return LOP_OK;
+}
+
+int lop_run_shard(lop_plan_t *pl, int band_lo, int band_hi, const void *in, void *out, void *ws, void *stream)
+{
+    int rc = check_common(pl, in, out, ws);
+    if (rc != LOP_OK) return rc;
+    if (band_lo < 0 || band_hi > pl->n_bands || band_lo > band_hi) { set_error("bands [%d,%d) out of range", band_lo, band_hi); return LOP_EINVAL; }
+    if (pl->n_bands > 65535) { set_error("lop_run_shard: more than 65535 bands"); return LOP_EUNSUPPORTED; }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    pl->exec->launches = pl->exec->copies = 0;
+    pl->exec->last_stream = s;
+    reset_layer_timing(pl);
+    if ((rc = prepare_workspace(pl, ws, s)) != LOP_OK) return rc;
+    if (band_lo == band_hi) return LOP_OK;
+    if (pl->exec->wavefront) return run_program(pl, PROG_BLOCK0 - (band_lo * 65536 + band_hi), in, out, ws, s);
+    // per-layer launches
+    const int L = (int)pl->layers.size();
+    for (int b = band_lo; b < band_hi; ++b)
+        for (int i = 0; i < L; ++i) {
+            const lop_range &r = pl->ranges[(size_t)b * L + i];
+            rc = run_layer(pl, i, first_row(pl, band_lo, b, i), r.out_hi, in, out, ws, s, (b + 1) * L + i);
+            if (rc != LOP_OK) return rc;
+        }
     return LOP_OK;
 }
 

@@ -239,6 +239,52 @@ def test_chain_entry_points_refuse_plans_that_do_not_follow_each_other():
     assert rel_err(to_host_f32(simt.outs[-1]), ochain.run_workload(wl)) <= TOL["bf16"]
 
 
+# ------------------------------------------------------------------------------------ band blocks (sharding over devices)
+@pytest.mark.parametrize("flags", [0, lop.LOP_FLAG_REUSE_HALO, lop.LOP_FLAG_REUSE_HALO | lop.LOP_FLAG_PER_LAYER])
+@pytest.mark.parametrize("name,kw", [("vgg_block", dict(H=44, W=36)), ("resnet18", dict(H=64, W=64))])
+def test_band_blocks_run_alone_give_their_rows_of_the_banded_result(name, kw, flags):
+    """lop_run_shard for every rank of 1, 2 and 3 devices, one after the other on this GPU, each on a workspace of
+    its own and with only its input rows present: the stitched rows equal lop_run_banded bit for bit."""
+    wl = li.build(name, **kw)
+    ref = DeviceChain(wl, flags=flags)
+    ref.per_plan = True
+    ref.run_banded(ref.input_tensor())
+    torch.cuda.synchronize()
+    s = torch.cuda.current_stream().cuda_stream
+    for world in (1, 2, 3):
+        x = ref.input_tensor()
+        for si, plan in enumerate(ref.plans):
+            stitched = torch.full_like(ref.outs[si], float("nan"))
+            for rank in range(world):
+                dc = DeviceChain(wl, flags=flags)                  # this rank's device: its own tensors
+                b0, b1, r0, r1, i0, i1 = dc.plans[si].shard(rank, world)
+                x_mine = torch.full_like(x, float("nan"))
+                x_mine[:, i0:i1] = x[:, i0:i1]
+                dc.outs[si].fill_(float("nan"))
+                dc.plans[si].run_shard(b0, b1, x_mine.data_ptr(), dc.outs[si].data_ptr(), dc.ws[si].data_ptr(), s)
+                torch.cuda.synchronize()
+                dc.plans[si].check_device(dc.ws[si].data_ptr())
+                got = dc.outs[si]
+                assert not torch.isnan(got[:, r0:r1]).any()
+                assert torch.isnan(got[:, :r0]).all() and torch.isnan(got[:, r1:]).all()      # nothing but its rows written
+                stitched[:, r0:r1] = got[:, r0:r1]
+            assert torch.equal(stitched, ref.outs[si]), (name, world, si)
+            x = ref.outs[si]
+    assert rel_err(to_host_f32(ref.outs[-1]), ochain.run_workload(wl)) <= TOL["bf16"]
+
+
+def test_sharded_chain_with_one_rank_is_the_banded_run():
+    from paper_2507_05829_b200.shard import ShardedChain
+    wl = li.build("resnet18", H=64, W=64)
+    ref = DeviceChain(wl, flags=lop.LOP_FLAG_REUSE_HALO)
+    ref.run_banded(ref.input_tensor())
+    dc = DeviceChain(wl, flags=lop.LOP_FLAG_REUSE_HALO)
+    out = ShardedChain(dc, 0, 1).run(dc.input_tensor())
+    torch.cuda.synchronize()
+    dc.check_device()
+    assert torch.equal(out, ref.outs[-1])
+
+
 # ------------------------------------------------------------------------------------ edge cases
 def test_very_wide_image_gathers_patches_without_staging_rows():
     """Three rows of a 4200-pixel image do not fit the shared staging tile: the gather reads the image in place."""

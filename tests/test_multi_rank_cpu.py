@@ -65,3 +65,83 @@ def test_reference_arm_under_torchrun_prints_one_line_from_rank_0():
     d = json.loads(lines[0])
     assert d["impl"] == "reference" and d["n_gpus"] == 2 and d["value"] > 0
     assert d["cpu_baseline"]["kind"] == "oracle" and d["e2e"]["h2d_bytes_per_step"] == 0
+
+
+# ------------------------------------------------------------------------------------ band sharding (gloo, CPU tensors)
+def _shard_rank(rank, world, port, out):
+    """One rank of a band-sharded run on CPU: the library's planner and shard table, the package's row all-gather
+    over gloo, and -- in place of the GPU kernels -- the oracle computing the rank's block of bands."""
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+    sys.path.insert(0, ROOT)
+    import lop_inputs as li
+    import paper_2507_05829_b200 as lop
+    from oracle import chain as ochain, planner as oplanner
+    from paper_2507_05829_b200.shard import all_gather_rows, shard_table
+    dist.init_process_group("gloo", init_method="tcp://127.0.0.1:%d" % port, rank=rank, world_size=world)
+    try:
+        wl = li.build("resnet18", H=48, W=16, width=8)
+        x = wl.x
+        for seg in wl.segments:
+            reuse = True
+            plan = lop.Plan(seg.layers, x.shape[0], x.shape[1], x.shape[2], x.shape[3], lop.LOP_BF16, seg.n_bands,
+                            lop.LOP_FLAG_REUSE_HALO)
+            table = shard_table(plan, world)
+            oplan = oplanner.make_plan(seg.layers, x.shape[1], x.shape[2], x.shape[3], seg.n_bands, reuse)
+            b0, b1, r0, r1, i0, i1 = table[rank]
+            x_mine = np.full_like(x, np.inf)
+            x_mine[:, i0:i1] = x[:, i0:i1]                           # the rank receives only the rows the table names
+            got = ochain.run_band_block(seg.layers, x_mine, oplan, True, b0, b1, reuse)
+            t = torch.from_numpy(np.where(np.isfinite(got), got, 0.0).astype(np.float32)).to(torch.bfloat16)
+            assert np.isfinite(got[:, r0:r1]).all() and not np.isfinite(got[:, :r0]).any() and not np.isfinite(got[:, r1:]).any()
+            all_gather_rows(t, table, rank)
+            whole = ochain.run_whole(seg.layers, x, True)
+            assert torch.equal(t, torch.from_numpy(whole).to(torch.bfloat16)), "rank %d: stitched rows differ" % rank
+            x = whole
+        out.put((rank, [list(r) for r in table]))
+        dist.barrier()
+    finally:
+        dist.destroy_process_group()
+
+
+def test_band_sharding_over_two_and_three_ranks_gives_the_whole_output_on_every_rank():
+    ctx = mp.get_context("spawn")
+    for world in (2, 3):
+        out = ctx.SimpleQueue()
+        port = _free_port()
+        procs = [ctx.Process(target=_shard_rank, args=(r, world, port, out)) for r in range(world)]
+        for p in procs:
+            p.start()
+        for p in procs:
+            p.join(300)
+            assert p.exitcode == 0
+        tables = [out.get()[1] for _ in range(world)]
+        assert all(t == tables[0] for t in tables)                 # every rank derives the same table
+
+
+def test_shard_table_is_the_floor_partition_of_the_bands():
+    sys.path.insert(0, ROOT)
+    import lop_inputs as li
+    import paper_2507_05829_b200 as lop
+    from oracle import planner as oplanner
+    wl = li.build("vgg_block", with_data=False)
+    seg = wl.segments[0]
+    B = 8
+    plan = lop.Plan(seg.layers, wl.N, wl.H, wl.W, wl.C, lop.LOP_BF16, B)
+    oplan = oplanner.make_plan(seg.layers, wl.H, wl.W, wl.C, B)
+    for world in (1, 2, 3, 5, 8, 11):
+        covered = 0
+        for rank in range(world):
+            b0, b1, r0, r1, i0, i1 = plan.shard(rank, world)
+            assert (b0, b1) == (rank * B // world, (rank + 1) * B // world)
+            if b1 > b0:
+                assert (r0, r1) == (oplan.ranges[b0][-1].out_lo, oplan.ranges[b1 - 1][-1].out_hi)
+                assert (i0, i1) == (min(oplan.input_need[b][0] for b in range(b0, b1)), max(oplan.input_need[b][1] for b in range(b0, b1)))
+                assert r0 == covered
+                covered = r1
+            else:
+                assert (r0, r1, i0, i1) == (0, 0, 0, 0)
+        assert covered == 112
+    with __import__("pytest").raises(lop.LopError):
+        plan.shard(2, 2)

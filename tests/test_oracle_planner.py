@@ -289,6 +289,31 @@ def test_stitched_bands_equal_whole_tensor_execution(name, kw, reuse):
     assert np.all(np.isfinite(x))
 
 
+@pytest.mark.parametrize("name,kw", SMALL)
+@pytest.mark.parametrize("reuse", [False, True])
+def test_band_blocks_on_separate_devices_tile_the_whole_output(name, kw, reuse):
+    """A block of bands run alone (poisoned tensors, only its own input rows) gives exactly its rows of the
+    whole-tensor result, whichever way the bands are dealt out to 1, 2, 3 or more devices."""
+    wl = li.build(name, **kw)
+    rb = wl.dtype == "bf16"
+    x = wl.x
+    for seg in wl.segments:
+        whole = chain.run_whole(seg.layers, x, rb)
+        for B in (min(6, whole.shape[1] + 1), 2 * whole.shape[1] + 3):       # the second: most bands are empty
+            plan = planner.make_plan(seg.layers, x.shape[1], x.shape[2], x.shape[3], B, reuse)
+            for world in (1, 2, 3, B + 1):
+                seen = np.zeros(whole.shape[1], dtype=bool)
+                for rank in range(world):
+                    b0, b1 = rank * B // world, (rank + 1) * B // world
+                    got = chain.run_band_block(seg.layers, x, plan, rb, b0, b1, reuse)
+                    rows = np.isfinite(got).all(axis=(0, 2, 3))
+                    assert not (rows & seen).any()
+                    assert np.array_equal(got[:, rows], whole[:, rows]), (name, B, world, rank, reuse)
+                    seen |= rows
+                assert seen.all()
+        x = whole
+
+
 def test_a_plan_one_row_short_is_caught():
     """Planting a mistake in the plan (one halo row dropped) must break stitched == whole."""
     wl = li.build("vgg_block", H=22, W=10, width=8)
