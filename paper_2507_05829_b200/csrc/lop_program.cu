@@ -408,7 +408,16 @@ int order_requests(const Ctx &cx, std::vector<StageReq> &reqs, bool reuse, const
 #ifdef LOP_WF_TRACE
             fprintf(stderr, "order model: greedy %.1f us, layer-major %.1f us (%zu stages)\n", span_greedy, mc.makespan, n);
 #endif
-            if (batched.size() == n && mc.makespan < span_greedy) order.swap(batched);
+            // The model is too coarse to separate the two when they come out close, and measurements did: where the
+            // input's transfer is a small part of the run (under a fifth), the layer-major order wins by running the
+            // bulk of the work the way resident programs do (cfg4: 836 vs 862 us); where the transfer is a large
+            // part, following the arrivals wins (cfg2: 38 vs 51 us).
+            double transfer = 0.0;
+            for (size_t i = 0; i < n; ++i)
+                if (reqs[i].fetch) transfer += shape[i].item_us;
+            if (arrival_us && !arrival_us->empty()) transfer = std::max(transfer, arrival_us->back());
+            const bool compute_bound = transfer < 0.2 * mc.makespan;
+            if (batched.size() == n && (mc.makespan < 0.95 * span_greedy || (compute_bound && mc.makespan < 1.05 * span_greedy))) order.swap(batched);
         }
     }
     std::vector<StageReq> out;
