@@ -10,6 +10,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <cmath>
 #include <cstdio>
 #include <map>
 #include <tuple>
@@ -277,6 +278,42 @@ void band_requests(const lop_plan_t *pl, int seg, int band, bool wait_arrival, s
     }
 }
 
+// Operation batching across thin bands (Sec. IV-C): deep in a network a band is a row or two of a small map, far less
+// than the rows one tile covers, so every band would pay for a mostly empty tile -- and stream the layer's weights once
+// more.  In reuse mode consecutive bands compute consecutive rows, so the requests of g neighbouring bands at a layer
+// are joined into one wherever their row ranges touch; g is chosen so that a group has about eight rows of the plan's
+// last layer (a tile of a 16-pixel-wide map has eight).  The rows computed, and their bits, stay the same.
+// keep_plan0: leave the first plan's bands alone (they are gated by the arrival of their input).
+void merge_thin_bands(const std::vector<SegBind> &segs, std::vector<StageReq> &reqs, bool keep_plan0)
+{
+    for (int sg = keep_plan0 ? 1 : 0; sg < (int)segs.size(); ++sg) {
+        const lop_plan_t *pl = segs[sg].pl;
+        if (!(pl->flags & LOP_FLAG_REUSE_HALO) || pl->n_bands < 2) continue;
+        const double rows_per_band = (double)pl->layers.back().Ho / pl->n_bands;
+        if (rows_per_band >= 8.0) continue;
+        const int g = std::min(pl->n_bands, (int)std::ceil(8.0 / std::max(rows_per_band, 1.0 / 64)));
+        const int L = (int)pl->layers.size();
+        for (int layer = 0; layer < L; ++layer)
+            for (int gather = 0; gather < 2; ++gather) {
+                int open = -1;                                        // request the following bands are joined into
+                for (int b = 0; b < pl->n_bands; ++b) {
+                    int found = -1;
+                    for (size_t i = 0; i < reqs.size(); ++i)
+                        if (reqs[i].seg == sg && reqs[i].layer == layer && (int)reqs[i].gather == gather && !reqs[i].fetch &&
+                            reqs[i].band == b && reqs[i].hi > reqs[i].lo) { found = (int)i; break; }
+                    if (b % g == 0) open = -1;
+                    if (found < 0) continue;
+                    if (open >= 0 && reqs[found].lo == reqs[open].hi) {
+                        reqs[open].hi = reqs[found].hi;
+                        reqs[found].hi = reqs[found].lo;                  // empty: dropped by the builder
+                    } else {
+                        open = found;
+                    }
+                }
+            }
+    }
+}
+
 enum { PROG_WHOLE = -1, PROG_ALL_BANDS = -2, PROG_PIPELINED = -3, PROG_FETCHED = -4, PROG_BLOCK0 = -16 };
 
 // kind: PROG_WHOLE, PROG_ALL_BANDS, PROG_PIPELINED, PROG_FETCHED (fetch_src: the host input as the device addresses
@@ -368,6 +405,8 @@ int get_program(const std::vector<SegBind> &segs, int kind, Program **prog, cons
                 arrival.push_back(t + 5.0);
             }
         }
+        if (kind == PROG_ALL_BANDS || kind <= PROG_BLOCK0) merge_thin_bands(segs, reqs, false);
+        else if (kind == PROG_PIPELINED || kind == PROG_FETCHED) merge_thin_bands(segs, reqs, true);
         Program *p = nullptr;
         int rc = program_build(segs, reqs, &p, kind == PROG_PIPELINED ? &arrival : nullptr, fetch_src);
         if (rc != LOP_OK) return rc;

@@ -66,6 +66,11 @@ Geom choose_geom(const ConvArgs &a, int rows, bool even_tiles)
     g.BN = 16;
     for (int bn = 128; bn >= 16; bn -= 16)
         if (a.Cout % bn == 0) { g.BN = bn; break; }
+    // A layer with few pixel tiles (a small map deep in the network) would occupy a handful of SMs, each streaming
+    // all of K for a wide slice of the weights at what one SM can pull from L2 (~40 GB/s measured): narrower
+    // output-channel tiles spread the same weight traffic over more SMs.
+    const long long layer_tiles = ((long long)a.N * a.Ho * a.Wo + 127) / 128;
+    while (g.BN > 32 && g.BN % 32 == 0 && layer_tiles * (a.Cout / g.BN) < 148) g.BN /= 2;
     g.n_taps = a.kh * a.kw;
     g.n_chunks = a.Cin / g.BK;
     const uint32_t row_bytes = (uint32_t)g.BK * 2u;
