@@ -68,9 +68,10 @@ Geom choose_geom(const ConvArgs &a, int rows, bool even_tiles)
         if (a.Cout % bn == 0) { g.BN = bn; break; }
     // A layer with few pixel tiles (a small map deep in the network) would occupy a handful of SMs, each streaming
     // all of K for a wide slice of the weights at what one SM can pull from L2 (~40 GB/s measured): narrower
-    // output-channel tiles spread the same weight traffic over more SMs.
+    // output-channel tiles spread the same weight traffic over more SMs.  Not below 64: an MMA with N = 32 costs the
+    // issuing thread as much as one with N = 64 (measured: cfg4 669 us with a floor of 64, 732 us with 32).
     const long long layer_tiles = ((long long)a.N * a.Ho * a.Wo + 127) / 128;
-    while (g.BN > 32 && g.BN % 32 == 0 && layer_tiles * (a.Cout / g.BN) < 148) g.BN /= 2;
+    while (g.BN > 64 && g.BN % 32 == 0 && layer_tiles * (a.Cout / g.BN) < 148) g.BN /= 2;
     g.n_taps = a.kh * a.kw;
     g.n_chunks = a.Cin / g.BK;
     const uint32_t row_bytes = (uint32_t)g.BK * 2u;
@@ -660,6 +661,9 @@ int program_build(const std::vector<SegBind> &segs, std::vector<StageReq> reqs, 
         if (sa < 4 && (size_t)(sa + 1) * a_slot + (size_t)sb * b_slot <= budget) { ++sa; grew = true; }
     }
 
+#ifdef LOP_WF_TRACE
+    fprintf(stderr, "program: %zu stages, %d items, rings: %d x %u B activations, %d x %u B weights, staging %u B\n", stages.size(), n_items, sa, a_slot, sb, b_slot, stg_bytes);
+#endif
     // ---- one device allocation for all tables
     auto al = [](size_t v) { return (v + 255) / 256 * 256; };
     const size_t o_stages = 0;

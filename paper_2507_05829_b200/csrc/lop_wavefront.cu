@@ -132,10 +132,10 @@ __device__ __forceinline__ bool mbar_wait_abortable(uint32_t bar, uint32_t parit
 
 // The 16-channel MMA steps of one (tap, channel chunk): descriptors differ only in their start-address field.
 // desc_hi: upper word of the operand descriptors (stride between 8-row groups, version, swizzle mode).
+// la, lb: low words of the two descriptors (address >> 4 in the start field, leading-offset field 1).
 template <int KSTEPS>
-__device__ __forceinline__ void mma_ksteps(uint32_t acc, uint32_t pa, uint32_t pb, uint32_t desc_hi, uint32_t idesc, uint32_t &accumulate)
+__device__ __forceinline__ void mma_ksteps_f(uint32_t acc, uint32_t la, uint32_t lb, uint32_t desc_hi, uint32_t idesc, uint32_t &accumulate)
 {
-    const uint32_t la = ((pa & 0x3FFFFu) >> 4) | (1u << 16), lb = ((pb & 0x3FFFFu) >> 4) | (1u << 16);
 #pragma unroll
     for (int kk = 0; kk < KSTEPS; ++kk) {
         const uint64_t ad = ((uint64_t)desc_hi << 32) | (uint64_t)(la + 2u * kk);
@@ -144,12 +144,17 @@ __device__ __forceinline__ void mma_ksteps(uint32_t acc, uint32_t pa, uint32_t p
         accumulate = 1u;
     }
 }
+__device__ __forceinline__ uint32_t desc_lo(uint32_t smem_addr) { return ((smem_addr & 0x3FFFFu) >> 4) | (1u << 16); }
+__device__ __forceinline__ void mma_tap_f(uint32_t acc, uint32_t la, uint32_t lb, uint32_t desc_hi, uint32_t idesc, int ksteps, uint32_t &accumulate)
+{
+    if (ksteps == 4) mma_ksteps_f<4>(acc, la, lb, desc_hi, idesc, accumulate);
+    else if (ksteps == 2) mma_ksteps_f<2>(acc, la, lb, desc_hi, idesc, accumulate);
+    else mma_ksteps_f<1>(acc, la, lb, desc_hi, idesc, accumulate);
+}
 __device__ __forceinline__ void mma_tap(uint32_t acc, uint32_t pa, uint32_t pb, uint32_t desc_hi, uint32_t idesc, int ksteps,
                                         uint32_t &accumulate)
 {
-    if (ksteps == 4) mma_ksteps<4>(acc, pa, pb, desc_hi, idesc, accumulate);
-    else if (ksteps == 2) mma_ksteps<2>(acc, pa, pb, desc_hi, idesc, accumulate);
-    else mma_ksteps<1>(acc, pa, pb, desc_hi, idesc, accumulate);
+    mma_tap_f(acc, desc_lo(pa), desc_lo(pb), desc_hi, idesc, ksteps, accumulate);
 }
 
 // One weight box of three taps of a 3x3 filter row over a 64-channel chunk: twelve MMAs whose descriptors differ
@@ -428,6 +433,7 @@ __global__ void __launch_bounds__(FETCH ? WF_THREADS + 32 : WF_THREADS, 1) wavef
             long long w_key = -1;
             uint32_t w_first = 0, w_n = 0;
             int map_base = 0, nblk = 1;                        // nblk: weight boxes per channel chunk
+            uint32_t tap16 = 0, step_w16 = 0, step_h16 = 0;    // descriptor start-field steps: next tap's weights, next filter column / row
 #ifdef LOP_WF_TRACE
             long long dbg_c0 = 0, dbg_fence = 0, dbg_mma = 0;
 #endif
@@ -446,6 +452,9 @@ __global__ void __launch_bounds__(FETCH ? WF_THREADS + 32 : WF_THREADS, 1) wavef
                     desc_hi = ((__ldg(&sp->sbo_bytes) >> 4) & 0x3FFFu) | (1u << 14) | (__ldg(&sp->layout_code) << 29);
                     row_bytes = __ldg(&sp->row_bytes);
                     tap_bytes = (uint32_t)__ldg(&sp->BN) * row_bytes;
+                    tap16 = tap_bytes >> 4;
+                    step_w16 = ((uint32_t)dw * row_bytes) >> 4;
+                    step_h16 = ((uint32_t)(dh << p_log) * row_bytes) >> 4;
                     row3x64 = mode == WF_SLAB && n_taps == 9 && kw == 3 && tbx == 3 && ksteps == 4 && dw == 1;
                 }
                 if (kind == WF_CONV) {
@@ -493,6 +502,9 @@ __global__ void __launch_bounds__(FETCH ? WF_THREADS + 32 : WF_THREADS, 1) wavef
                             if (ch == 0) tr(item, 13);
                             const uint32_t sa = a0 + a_slot * a_slot_bytes;
                             int ta = 0, tb = 0;                             // filter position of tap t0
+                            // start field of the tap's activation operand: one pixel further per filter column, one
+                            // slab row further per filter row (kept incrementally: this thread pays for every instruction)
+                            uint32_t la_row = desc_lo(sa), la = la_row;
                             for (int t0 = 0; t0 < n_taps; t0 += tbx) {
                                 uint32_t bs = b_slot;
                                 if (reuse_w) {
@@ -521,12 +533,12 @@ __global__ void __launch_bounds__(FETCH ? WF_THREADS + 32 : WF_THREADS, 1) wavef
                                     ++ta;
                                 } else {
                                     const int t1 = min(t0 + tbx, n_taps);
-                                    uint32_t pb = sb;
-                                    for (int t = t0; t < t1; ++t, pb += tap_bytes) {
+                                    uint32_t lb = desc_lo(sb);
+                                    for (int t = t0; t < t1; ++t, lb += tap16) {
                                         // tap (ta, tb): the same box, read (ta*dh*P + tb*dw) pixels further on
-                                        const uint32_t pa = sa + (uint32_t)(((ta * dh) << p_log) + tb * dw) * row_bytes;
-                                        mma_tap(acc, pa, pb, desc_hi, idesc, ksteps, accumulate);
-                                        if (++tb == kw) { tb = 0; ++ta; }
+                                        mma_tap_f(acc, la, lb, desc_hi, idesc, ksteps, accumulate);
+                                        la += step_w16;
+                                        if (++tb == kw) { tb = 0; la_row += step_h16; la = la_row; }
                                     }
                                 }
                                 if (!reuse_w) {
