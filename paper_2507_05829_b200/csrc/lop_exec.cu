@@ -280,20 +280,31 @@ void band_requests(const lop_plan_t *pl, int seg, int band, bool wait_arrival, s
 
 // Operation batching across thin bands (Sec. IV-C): deep in a network a band is a row or two of a small map, far less
 // than the rows one tile covers, so every band would pay for a mostly empty tile -- and stream the layer's weights once
-// more.  In reuse mode consecutive bands compute consecutive rows, so the requests of g neighbouring bands at a layer
-// are joined into one wherever their row ranges touch; g is chosen so that a group has about eight rows of the plan's
-// last layer (a tile of a 16-pixel-wide map has eight).  The rows computed, and their bits, stay the same.
-// keep_plan0: leave the first plan's bands alone (they are gated by the arrival of their input).
+// more.  In reuse mode consecutive bands compute consecutive rows, so at a layer whose bands have fewer than eight rows
+// the requests of g neighbouring bands are joined into one wherever their row ranges touch (g: about eight rows per
+// group; a tile of a 16-pixel-wide map has eight).  The rows computed, and their bits, stay the same.
+// keep_plan0: leave the first plan's bands alone -- they are gated by the arrival of their input, and joining them
+// (even only at the plan's deep layers) was measured slower on every pipelined configuration.
 void merge_thin_bands(const std::vector<SegBind> &segs, std::vector<StageReq> &reqs, bool keep_plan0)
 {
     for (int sg = keep_plan0 ? 1 : 0; sg < (int)segs.size(); ++sg) {
         const lop_plan_t *pl = segs[sg].pl;
         if (!(pl->flags & LOP_FLAG_REUSE_HALO) || pl->n_bands < 2) continue;
-        const double rows_per_band = (double)pl->layers.back().Ho / pl->n_bands;
-        if (rows_per_band >= 8.0) continue;
-        const int g = std::min(pl->n_bands, (int)std::ceil(8.0 / std::max(rows_per_band, 1.0 / 64)));
         const int L = (int)pl->layers.size();
-        for (int layer = 0; layer < L; ++layer)
+        std::vector<int> group(L, 1);
+        for (int i = 0; i < L; ++i) {
+            const double rows_per_band = (double)pl->layers[i].Ho / pl->n_bands;
+            if (rows_per_band < 8.0) group[i] = std::min(pl->n_bands, (int)std::ceil(8.0 / std::max(rows_per_band, 1.0 / 64)));
+        }
+        for (int i = 0; i + 1 < L; ++i) {
+            // a convolution whose 2x2 pooling is folded into its epilogue must be cut like the pooling
+            const lop_layer &q = pl->layers[i + 1].l;
+            if (pl->layers[i].l.op == LOP_CONV2D && q.op == LOP_MAXPOOL2D && q.input_from == i && q.kh == 2 && q.kw == 2 && q.sh == 2 && q.sw == 2)
+                group[i] = group[i + 1];
+        }
+        for (int layer = 0; layer < L; ++layer) {
+            const int g = group[layer];
+            if (g <= 1) continue;
             for (int gather = 0; gather < 2; ++gather) {
                 int open = -1;                                        // request the following bands are joined into
                 for (int b = 0; b < pl->n_bands; ++b) {
@@ -311,6 +322,7 @@ void merge_thin_bands(const std::vector<SegBind> &segs, std::vector<StageReq> &r
                     }
                 }
             }
+        }
     }
 }
 
