@@ -443,6 +443,22 @@ def test_output_straight_into_pinned_host_memory(name, kw):
     assert torch.equal(host, want.cpu())
 
 
+@pytest.mark.parametrize("N,H,W,C,cout", [(2, 21, 37, 3, 32), (3, 9, 21, 5, 32), (1, 33, 50, 64, 64), (2, 16, 9, 7, 64)])
+def test_fetched_rows_of_any_length_and_alignment(N, H, W, C, cout):
+    """Row lengths that are no multiple of 16 bytes: every fetch entry then starts and ends inside a 16-byte vector
+    (2-byte head and tail around the vector body); several images, several bands, both band modes."""
+    wl = one_layer(conv(C, cout, 3, act=li.ACT_RELU), N, H, W, n_bands=4)
+    for flags in (0, lop.LOP_FLAG_REUSE_HALO):
+        res = check_workload(wl, flags=flags, modes=("whole", "pipelined", "pipelined_copy"))
+    dc = DeviceChain(wl, flags=lop.LOP_FLAG_REUSE_HALO, n_bands=4)
+    x = dc.pinned_input()
+    dc.staging.fill_(float("nan"))
+    dc.run_pipelined(x)
+    torch.cuda.synchronize()
+    assert dc.plans[0].last_copies() == 0                       # the kernel brought the input itself ...
+    assert torch.equal(dc.staging.cpu().view(-1), x.view(-1))   # ... all of it, bit for bit
+
+
 def test_unaligned_and_unpinned_host_buffers_take_the_copy_path():
     wl = li.build("vgg_block", H=44, W=36)
     dc = DeviceChain(wl, flags=lop.LOP_FLAG_REUSE_HALO)
