@@ -29,8 +29,8 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one wavefront_kernel launch (ncu --set full, see
-# profiles/wavefront_kernel_vgg_block.md); None for workloads not captured, or once the kernel has changed since
-TRAFFIC = {"vgg_block": 509.2e3}
+# profiles/wavefront_kernel_vgg_block.md and profiles/wavefront_kernel_resnet18_resnet50_csp_stack.md); None for workloads not captured, or once the kernel has changed since
+TRAFFIC = {"vgg_block": 509.2e3, "resnet18": 22.8e6, "resnet50": 236.3e6, "csp_stack": 37.0e6}
 
 METRIC = "band-pipelined conv-chain images/s"
 UNIT = "images/s"
