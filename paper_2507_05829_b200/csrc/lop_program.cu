@@ -69,7 +69,7 @@ Geom choose_geom(const ConvArgs &a, int rows, bool even_tiles)
     // A layer with few pixel tiles (a small map deep in the network) would occupy a handful of SMs, each streaming
     // all of K for a wide slice of the weights at what one SM can pull from L2 (~40 GB/s measured): narrower
     // output-channel tiles spread the same weight traffic over more SMs.  Not below 64: an MMA with N = 32 costs the
-    // issuing thread as much as one with N = 64 (measured: cfg4 669 us with a floor of 64, 732 us with 32).
+    // issuing thread as much as one with N = 64 (measured on a ResNet-50 of batch 8: 669 us with a floor of 64, 732 us with 32).
     const long long layer_tiles = ((long long)a.N * a.Ho * a.Wo + 127) / 128;
     while (g.BN > 64 && g.BN % 32 == 0 && layer_tiles * (a.Cout / g.BN) < 148) g.BN /= 2;
     g.n_taps = a.kh * a.kw;
@@ -416,8 +416,8 @@ int order_requests(const Ctx &cx, std::vector<StageReq> &reqs, bool reuse, const
 #endif
             // The model is too coarse to separate the two when they come out close, and measurements did: where the
             // input's transfer is a small part of the run (under a fifth), the layer-major order wins by running the
-            // bulk of the work the way resident programs do (cfg4: 836 vs 862 us); where the transfer is a large
-            // part, following the arrivals wins (cfg2: 38 vs 51 us).
+            // bulk of the work the way resident programs do (a ResNet-50 of batch 8: 836 vs 862 us); where the transfer is a large
+            // part, following the arrivals wins (one 224x224 image through a VGG block: 38 vs 51 us).
             double transfer = 0.0;
             for (size_t i = 0; i < n; ++i)
                 if (reqs[i].fetch) transfer += shape[i].item_us;
