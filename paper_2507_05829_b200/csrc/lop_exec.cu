@@ -420,7 +420,7 @@ int get_program(const std::vector<SegBind> &segs, int kind, Program **prog, cons
         if (kind == PROG_ALL_BANDS || kind <= PROG_BLOCK0) merge_thin_bands(segs, reqs, false);
         else if (kind == PROG_PIPELINED || kind == PROG_FETCHED) merge_thin_bands(segs, reqs, true);
         Program *p = nullptr;
-        int rc = program_build(segs, reqs, &p, kind == PROG_PIPELINED ? &arrival : nullptr, fetch_src);
+        int rc = program_build(segs, reqs, &p, (kind == PROG_PIPELINED || kind == PROG_ALL_BANDS) ? &arrival : nullptr, fetch_src);
         if (rc != LOP_OK) return rc;
         it = e->programs.emplace(key, p).first;
     }

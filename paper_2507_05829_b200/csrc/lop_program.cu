@@ -423,7 +423,12 @@ int order_requests(const Ctx &cx, std::vector<StageReq> &reqs, bool reuse, const
                 if (reqs[i].fetch) transfer += shape[i].item_us;
             if (arrival_us && !arrival_us->empty()) transfer = std::max(transfer, arrival_us->back());
             const bool compute_bound = transfer < 0.2 * mc.makespan;
-            if (batched.size() == n && (mc.makespan < 0.95 * span_greedy || (compute_bound && mc.makespan < 1.05 * span_greedy))) order.swap(batched);
+            // (a resident program, nothing arriving: the greedy order unless the model clearly prefers layer-major --
+            // it moves late layers of early bands in front of early layers of late bands where that shortens waits)
+            const bool resident = transfer == 0.0;
+            if (batched.size() == n && (resident ? mc.makespan < 0.98 * span_greedy
+                                                 : (mc.makespan < 0.95 * span_greedy || (compute_bound && mc.makespan < 1.05 * span_greedy))))
+                order.swap(batched);
         }
     }
     std::vector<StageReq> out;
