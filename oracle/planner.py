@@ -82,38 +82,32 @@ def hull(a, b):
 
 
 def input_rows(o0, o1, k, s, p, d, h_in):
-    """Rows of the input that output rows [o0, o1) actually read.
+    """Rows of the input that output rows [o0, o1) actually read, by enumeration.
 
-    Output row o reads the rows  o*s - p + t*d,  t = 0..k-1,  that lie inside [0, h_in); rows
-    in the padding are nobody's output and create no dependency.  The range returned is the
-    smallest interval holding every row read ("a dependency exists if any part is used").
-    For tap t the first output row whose tap is not above the tensor is ceil((p - t*d)/s), the
-    last whose tap is not below it is floor((h_in-1 + p - t*d)/s); the extremes over the taps
-    give the interval.  With d == 1 and p <= k-1 this is the analytic receptive range
-    [o0*s - p, (o1-1)*s - p + (k-1)*d] clamped to the tensor.
+    Output row o reads, through tap t = 0..k-1, the row  o*s - p + t*d.  Every (output row, tap)
+    pair is visited; a row inside [0, h_in) is a dependency (Sec. IV-B: a dependency exists as
+    soon as any part of the producer's output is used), a row outside it lies in the padding,
+    is nobody's output and creates none.  The range returned is the smallest interval that
+    holds every dependency; pad_top / pad_bot are how far above / below the tensor the taps
+    reach.  With d == 1 and p <= k-1 the result is the analytic receptive range
+    [o0*s - p, (o1-1)*s - p + (k-1)*d] cut to the tensor.
 
-    Returns (in_lo, in_hi, pad_top, pad_bot); pad_* are how many rows above / below the tensor
-    the analytic range reaches.
+    Returns (in_lo, in_hi, pad_top, pad_bot).
     """
-    a = o0 * s - p
-    b = (o1 - 1) * s - p + (k - 1) * d          # inclusive
-    pad_top = max(0, -a)
-    pad_bot = max(0, b - (h_in - 1))
-    lo, hi = None, None
-    for t in range(k):
-        first = max(o0, -((t * d - p) // s))                 # ceil((p - t*d) / s)
-        if first < o1:
-            r = first * s - p + t * d
-            if r < h_in:
-                lo = r if lo is None else min(lo, r)
-        last = min(o1 - 1, (h_in - 1 + p - t * d) // s)      # floor
-        if last >= o0:
-            r = last * s - p + t * d
-            if r >= 0:
-                hi = r if hi is None else max(hi, r)
-    if lo is None or hi is None:
+    read = []
+    pad_top = pad_bot = 0
+    for o in range(o0, o1):
+        for t in range(k):
+            r = o * s - p + t * d
+            if r < 0:
+                pad_top = max(pad_top, -r)
+            elif r >= h_in:
+                pad_bot = max(pad_bot, r - (h_in - 1))
+            else:
+                read.append(r)
+    if not read:
         return 0, 0, pad_top, pad_bot
-    return lo, hi + 1, pad_top, pad_bot
+    return min(read), max(read) + 1, pad_top, pad_bot
 
 
 class Plan:

@@ -43,6 +43,37 @@ def test_single_layer_closed_form():
                 assert clamped[0] <= r.in_lo and r.in_hi <= clamped[1]
 
 
+def per_tap_interval(o0, o1, k, s, p, d, h_in):
+    """The same interval from index arithmetic instead of enumeration: for tap t the first output row whose tap is
+    not above the tensor is ceil((p - t*d)/s), the last whose tap is not below it is floor((h_in-1 + p - t*d)/s)."""
+    lo = hi = None
+    for t in range(k):
+        first = max(o0, -((t * d - p) // s))
+        if first < o1 and first * s - p + t * d < h_in:
+            r = first * s - p + t * d
+            lo = r if lo is None else min(lo, r)
+        last = min(o1 - 1, (h_in - 1 + p - t * d) // s)
+        if last >= o0 and last * s - p + t * d >= 0:
+            r = last * s - p + t * d
+            hi = r if hi is None else max(hi, r)
+    return (0, 0) if lo is None or hi is None else (lo, hi + 1)
+
+
+def test_enumerated_input_rows_equal_the_per_tap_closed_form():
+    rnd = random.Random(77)
+    for _ in range(20000):
+        k, s, p, d = rnd.randint(1, 7), rnd.randint(1, 4), rnd.randint(0, 9), rnd.randint(1, 4)
+        h_in = rnd.randint(1, 40)
+        ho = (h_in + 2 * p - d * (k - 1) - 1) // s + 1
+        if ho <= 0:
+            continue
+        o0 = rnd.randint(0, ho - 1)
+        o1 = rnd.randint(o0 + 1, ho)
+        lo, hi, pt, pb = planner.input_rows(o0, o1, k, s, p, d, h_in)
+        assert (lo, hi) == per_tap_interval(o0, o1, k, s, p, d, h_in)
+        assert pt == max(0, p - o0 * s) and pb == max(0, (o1 - 1) * s - p + (k - 1) * d - (h_in - 1))
+
+
 # ----------------------------------------------------------------------------- brute-force touch marking
 def random_stack(rnd):
     """A random layer list with optional residual edges; all H extents stay positive."""
