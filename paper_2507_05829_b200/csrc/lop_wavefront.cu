@@ -341,10 +341,14 @@ __global__ void __launch_bounds__(FETCH ? WF_THREADS + 32 : WF_THREADS, 1) wavef
                         dsh[i] = shift ? __ldg(shift + c0 + i) : 0.0f;
                     }
                     __syncwarp();
+                }
+                ok = ok && wait_deps_warp(P, rec_dep0(cur), rec_ndep(cur), dep_cur, run, lane);
+                if (ok) {
+                    // "scale / shift are in place AND the tile's producers (the residual's included) are done": the
+                    // workers fetch the residual tile behind this barrier, while the operands are still on their way
                     if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(ssf0 + 8u * (pc & 1u)) : "memory");
                     ++pc;
                 }
-                ok = ok && wait_deps_warp(P, rec_dep0(cur), rec_ndep(cur), dep_cur, run, lane);
                 int fail = 0;
                 if (!ok) {
                     if (lane == 0) atomicOr(P.status, 0x10u);
@@ -707,19 +711,17 @@ __global__ void __launch_bounds__(FETCH ? WF_THREADS + 32 : WF_THREADS, 1) wavef
                     const bool ok = valid && c + 1 < tw_valid && ow + 1 < Wo && oh + 1 < oh_hi;
                     pool_pix[q] = ok ? (((long long)n * pool_Ho + (oh >> 1)) * pool_Wo + (ow >> 1)) * Cout + co0 : -1LL;
                 }
-                if (resp) epi_bar();                                   // the residual copy-in below reads row_pix
                 const float *t_scale = s_scale + 128 * buf, *t_shift = s_shift + 128 * buf;   // filled by warp 0 a tile ahead
                 const int cpr = BN >> 3;                               // 16-byte chunks per staged row
                 const int cpr_log = (cpr & (cpr - 1)) == 0 ? 31 - __clz(cpr) : -1;
                 const uint32_t row_stride = (uint32_t)BN * 2u;
                 const int swz = (cpr & 7) == 0 ? 7 : 0;                // chunk position = chunk ^ (row & 7): conflict-free columns
                 __nv_bfloat16 *y = static_cast<__nv_bfloat16 *>(yout);
+                // the loader warp arrives here once it has seen the tile's producers (the residual's included): the residual
+                // tile is fetched now, under the operands' transfer and the main loop
                 if (!mbar_wait_abortable(ssf0 + 8u * buf, (cnt >> 1) & 1u, abort_flag)) *epi_fail = 1;
-                if (!mbar_wait_abortable(accf0 + 8u * buf, (cnt >> 1) & 1u, abort_flag)) *epi_fail = 1;
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                if (tid == 0) tr(item, 5);
-                // (only now: the finished accumulator implies that warp 0 saw this item's producers, the residual's included)
                 if (resp) {
+                    epi_bar();                                         // row_pix of every anchor is written
                     // residual tile -> staging, coalesced; produced inside this launch by other SMs: read through L2
                     const __nv_bfloat16 *res = static_cast<const __nv_bfloat16 *>(resp);
 #pragma unroll 4
@@ -730,8 +732,11 @@ __global__ void __launch_bounds__(FETCH ? WF_THREADS + 32 : WF_THREADS, 1) wavef
                             *reinterpret_cast<uint4 *>(stg + row * row_stride + ((j ^ (row & swz)) << 4)) =
                                 __ldcg(reinterpret_cast<const uint4 *>(res + rp) + j);
                     }
-                    epi_bar();
                 }
+                if (!mbar_wait_abortable(accf0 + 8u * buf, (cnt >> 1) & 1u, abort_flag)) *epi_fail = 1;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                if (tid == 0) tr(item, 5);
+                if (resp) epi_bar();                                   // the staged residual tile is complete
                 {
                     const uint32_t acc = tmem_base + buf * 256u + ((uint32_t)(g * 32) << 16);
                     uint8_t *my_row = stg + m * row_stride;
