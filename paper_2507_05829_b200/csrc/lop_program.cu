@@ -41,6 +41,9 @@ namespace {
 #ifndef LOP_FETCH_WINDOW_BYTES
 #define LOP_FETCH_WINDOW_BYTES (96 * 1024)
 #endif
+#ifndef LOP_CPS_MAX
+#define LOP_CPS_MAX 4
+#endif
 constexpr uint32_t A_BOX_MAX = 48u * 1024u;     // largest activation box a ring slot is sized for
 constexpr uint32_t B_BOX_MAX = 32u * 1024u;     // largest weight box
 
@@ -664,6 +667,13 @@ int program_build(const std::vector<SegBind> &segs, std::vector<StageReq> reqs, 
         grew = false;
         if (sb < 8 && (size_t)sa * a_slot + (size_t)(sb + 1) * b_slot <= budget) { ++sb; grew = true; }
         if (sa < 4 && (size_t)(sa + 1) * a_slot + (size_t)sb * b_slot <= budget) { ++sa; grew = true; }
+    }
+
+    // chunks per ring slot of the long pointwise stages (see WfStage::cps), now that the slot sizes are known
+    for (WfStage &st : stages) {
+        st.cps = 1;
+        if (st.kind != WF_CONV || st.mode != WF_SLAB || st.n_taps != 1 || st.BK != 64 || st.n_chunks <= sb) continue;
+        st.cps = std::max(1, std::min({(int)(a_slot / st.a_bytes), (int)(b_slot / st.b_bytes), LOP_CPS_MAX}));
     }
 
 #ifdef LOP_WF_TRACE

@@ -299,7 +299,7 @@ __global__ void __launch_bounds__(FETCH ? WF_THREADS + 32 : WF_THREADS, 1) wavef
         uint32_t a_bytes = 0, b_bytes = 0;
         const CUtensorMap *maps = nullptr;
         const float *scale = nullptr, *shift = nullptr;
-        int slab_offh = 0, slab_offw = 0, slab_mi = 0, n_boxes = 1;
+        int slab_offh = 0, slab_offw = 0, slab_mi = 0, n_boxes = 1, cps = 1;
         bool slab_have = true;
         uint32_t a_slot = 0, a_phase = 0, b_slot = 0, b_phase = 0, pc = 0;
         bool w_kept = false;                                   // (lane 0) the ring holds the weights of tile key w_key
@@ -327,6 +327,7 @@ __global__ void __launch_bounds__(FETCH ? WF_THREADS + 32 : WF_THREADS, 1) wavef
                 slab_mi = (-ph - offh * sh) * sw + (-pw - offw * sw);
                 slab_have = (amask >> slab_mi) & 1;
                 n_boxes = n_chunks * ((n_taps + tbx - 1) / tbx);
+                cps = __ldg(&sp->cps);
             }
             if (kind == WF_CONV) {
                 if (lane == 0) tr(item, 0);
@@ -369,6 +370,23 @@ __global__ void __launch_bounds__(FETCH ? WF_THREADS + 32 : WF_THREADS, 1) wavef
                     const bool reuse_w = w_kept && can_keep && wkey == w_key;
                     w_kept = reuse_w || can_keep;
                     w_key = wkey;
+                    if (cps > 1) {
+                        for (int ch = 0; ch < n_chunks && !fail; ch += cps) {
+                            const int g = min(cps, n_chunks - ch);
+                            if (!mbar_wait_abortable(empty_a + 8u * a_slot, a_phase ^ 1u, abort_flag) ||
+                                !mbar_wait_abortable(empty_b + 8u * b_slot, b_phase ^ 1u, abort_flag)) { fail = 1; break; }
+                            const uint32_t fa = full_a + 8u * a_slot, fb = full_b + 8u * b_slot;
+                            mbar_expect_tx(fa, (uint32_t)g * a_bytes);
+                            mbar_expect_tx(fb, (uint32_t)g * b_bytes);
+                            for (int u = 0; u < g; ++u) {
+                                tma_load_4d(a0 + a_slot * a_slot_bytes + (uint32_t)u * a_bytes, maps + slab_mi, fa, (ch + u) * BK,
+                                            slab_have ? ow0 + slab_offw : -65536, slab_have ? oh0 + slab_offh : -65536, n0);
+                                tma_load_3d(b0 + b_slot * b_slot_bytes + (uint32_t)u * b_bytes, maps + 4, fb, (ch + u) * BK, co0, 0);
+                            }
+                            if (++a_slot == (uint32_t)SA) { a_slot = 0; a_phase ^= 1u; }
+                            if (++b_slot == (uint32_t)SB) { b_slot = 0; b_phase ^= 1u; }
+                        }
+                    } else
                     for (int ch = 0; ch < n_chunks && !fail; ++ch) {
                         if (mode == WF_SLAB) {
                             // the whole receptive window of the tile in one box: its first tap's offset places it
@@ -436,7 +454,8 @@ __global__ void __launch_bounds__(FETCH ? WF_THREADS + 32 : WF_THREADS, 1) wavef
             bool w_kept = false;                               // weights kept in ring slots w_first .. w_first + w_n - 1 for key w_key
             long long w_key = -1;
             uint32_t w_first = 0, w_n = 0;
-            int map_base = 0, nblk = 1;                        // nblk: weight boxes per channel chunk
+            int map_base = 0, nblk = 1, cps = 1;               // nblk: weight boxes per channel chunk; cps: chunks per ring slot
+            uint32_t a_bytes = 0, b_bytes = 0;
             uint32_t tap16 = 0, step_w16 = 0, step_h16 = 0;    // descriptor start-field steps: next tap's weights, next filter column / row
 #ifdef LOP_WF_TRACE
             long long dbg_c0 = 0, dbg_fence = 0, dbg_mma = 0;
@@ -460,6 +479,8 @@ __global__ void __launch_bounds__(FETCH ? WF_THREADS + 32 : WF_THREADS, 1) wavef
                     step_w16 = ((uint32_t)dw * row_bytes) >> 4;
                     step_h16 = ((uint32_t)(dh << p_log) * row_bytes) >> 4;
                     row3x64 = mode == WF_SLAB && n_taps == 9 && kw == 3 && tbx == 3 && ksteps == 4 && dw == 1;
+                    a_bytes = __ldg(&sp->a_bytes); b_bytes = __ldg(&sp->b_bytes);
+                    cps = __ldg(&sp->cps);
                 }
                 if (kind == WF_CONV) {
                     const uint32_t buf = cnt & 1u;
@@ -499,6 +520,20 @@ __global__ void __launch_bounds__(FETCH ? WF_THREADS + 32 : WF_THREADS, 1) wavef
                         mma_row3x64(acc, la + 2u * row16, (((b0 + s2 * b_slot_bytes) & 0x3FFFFu) >> 4) | (1u << 16), tap_bytes >> 4, desc_hi, idesc, accumulate);
                         umma_commit(empty_a + 8u * a_slot);
                         if (++a_slot == (uint32_t)SA) { a_slot = 0; a_phase ^= 1u; }
+                    } else if (cps > 1) {
+                        for (int ch = 0; ch < n_chunks; ch += cps) {
+                            const int g = min(cps, n_chunks - ch);
+                            if (!mbar_wait_abortable(full_a + 8u * a_slot, a_phase, abort_flag) ||
+                                !mbar_wait_abortable(full_b + 8u * b_slot, b_phase, abort_flag)) { fail = true; break; }
+                            if (ch == 0) tr(item, 13);
+                            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                            uint32_t la = desc_lo(a0 + a_slot * a_slot_bytes), lb = desc_lo(b0 + b_slot * b_slot_bytes);
+                            for (int u = 0; u < g; ++u, la += a_bytes >> 4, lb += b_bytes >> 4) mma_ksteps_f<4>(acc, la, lb, desc_hi, idesc, accumulate);
+                            umma_commit(empty_a + 8u * a_slot);
+                            umma_commit(empty_b + 8u * b_slot);
+                            if (++a_slot == (uint32_t)SA) { a_slot = 0; a_phase ^= 1u; }
+                            if (++b_slot == (uint32_t)SB) { b_slot = 0; b_phase ^= 1u; }
+                        }
                     } else
                     for (int ch = 0; ch < n_chunks && !fail; ++ch) {
                         if (mode == WF_SLAB) {
