@@ -225,6 +225,15 @@ int lop_plan_layer_time(lop_plan_t *plan, int band, int layer, float *ms);
 /* Which kernel family serves a layer: 0 = pooling, 1 = CUDA-core convolution,
  * 2 = tcgen05 tensor-core convolution.  <0 on error. */
 int lop_plan_layer_kernel(const lop_plan_t *plan, int layer);
+/* Where the full-size output tensor of an intermediate layer (0 <= layer < n_layers - 1) lives: byte offset into the
+ * workspace given to the lop_run_* calls; its shape is lop_plan_out_shape(layer), NHWC in the storage dtype.  The rows a
+ * call has computed are there when the call's stream work is done (for inspection and tests; the last layer's tensor is
+ * the caller's out_dev). */
+int lop_plan_layer_offset(const lop_plan_t *plan, int layer, size_t *offset);
+/* 1 if executions of this plan write the layer's output tensor, 0 if they never do: the persistent kernel folds a 2x2
+ * stride-2 max pooling that is a convolution's only reader into that convolution's epilogue (Sec. IV-A: both are local
+ * operators), and only the pooled tensor exists.  <0 on error. */
+int lop_plan_layer_stored(const lop_plan_t *plan, int layer);
 /* Number of kernels (this library's own) and of async copies the last execution call enqueued. */
 int lop_plan_last_launches(const lop_plan_t *plan);
 int lop_plan_last_copies(const lop_plan_t *plan);

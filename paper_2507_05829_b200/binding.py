@@ -20,7 +20,7 @@ EXPORTS = [
     "lop_plan_out_shape", "lop_plan_set_params", "lop_plan_workspace_bytes", "lop_plan_staging_bytes",
     "lop_plan_flops", "lop_run_whole", "lop_run_band", "lop_run_banded", "lop_copy_band", "lop_run_pipelined",
     "lop_plan_last_timing", "lop_plan_layer_time", "lop_plan_layer_kernel", "lop_plan_last_launches", "lop_plan_last_copies",
-    "lop_plan_check_device", "lop_run_whole_static", "lop_run_chain_banded", "lop_run_chain_pipelined", "lop_plan_shard", "lop_run_shard",
+    "lop_plan_check_device", "lop_plan_layer_offset", "lop_plan_layer_stored", "lop_run_whole_static", "lop_run_chain_banded", "lop_run_chain_pipelined", "lop_plan_shard", "lop_run_shard",
     "lop_strerror", "lop_last_error",
 ]
 LOP_STATIC_SCRATCH_BYTES = 16 << 20
@@ -88,6 +88,8 @@ def lib():
     L.lop_plan_last_timing.argtypes = [c_void_p, POINTER(LopTiming)]
     L.lop_plan_layer_time.argtypes = [c_void_p, c_int, c_int, POINTER(c_float)]
     L.lop_plan_layer_kernel.argtypes = [c_void_p, c_int]
+    L.lop_plan_layer_offset.argtypes = [c_void_p, c_int, POINTER(c_size_t)]
+    L.lop_plan_layer_stored.argtypes = [c_void_p, c_int]
     L.lop_plan_last_launches.argtypes = [c_void_p]
     L.lop_plan_last_copies.argtypes = [c_void_p]
     L.lop_plan_check_device.argtypes = [c_void_p, c_void_p]
@@ -222,6 +224,14 @@ class Plan:
 
     def layer_kernel(self, layer):
         return _check(lib().lop_plan_layer_kernel(self._h, layer))
+
+    def layer_offset(self, layer):
+        off = c_size_t()
+        _check(lib().lop_plan_layer_offset(self._h, layer, byref(off)))
+        return off.value
+
+    def layer_stored(self, layer):
+        return bool(_check(lib().lop_plan_layer_stored(self._h, layer)))
 
     def last_launches(self):
         return _check(lib().lop_plan_last_launches(self._h))

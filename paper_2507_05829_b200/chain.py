@@ -78,11 +78,19 @@ class DeviceChain:
         return s.cuda_stream
 
     def layer_output(self, seg, layer):
-        """View of an intermediate full-size tensor inside a segment's workspace (tests only)."""
+        """The full-size output tensor of one layer of a segment: the segment's output tensor for its last layer, else a
+        view into the segment's workspace (lop_plan_layer_offset).  None when executions never write it (a convolution
+        whose pooling is folded into its epilogue, lop_plan_layer_stored)."""
         plan = self.plans[seg]
         if layer == plan.num_layers() - 1:
             return self.outs[seg]
-        raise NotImplementedError
+        if not plan.layer_stored(layer):
+            return None
+        h, w, c = plan.out_shape(layer)
+        n = self.wl.N * h * w * c
+        off = plan.layer_offset(layer)
+        es = 2 if self.wl.dtype == "bf16" else 4
+        return self.ws[seg][off:off + n * es].view(self.tdtype).view(self.wl.N, h, w, c)
 
     # -- execution -----------------------------------------------------------------------------
     def run_whole(self, x_dev, stream=None):

@@ -817,6 +817,24 @@ int lop_plan_layer_time(lop_plan_t *pl, int band, int layer, float *ms)
     return LOP_OK;
 }
 
+int lop_plan_layer_offset(const lop_plan_t *pl, int layer, size_t *offset)
+{
+    if (!pl || !offset) { set_error("lop_plan_layer_offset: NULL argument"); return LOP_EINVAL; }
+    const int L = (int)pl->layers.size();
+    if (layer < 0 || layer >= L - 1) { set_error("lop_plan_layer_offset: layer %d is not an intermediate layer", layer); return LOP_EINVAL; }
+    *offset = pl->layers[layer].out_off;
+    return LOP_OK;
+}
+
+int lop_plan_layer_stored(const lop_plan_t *pl, int layer)
+{
+    if (!pl) { set_error("plan is NULL"); return LOP_EINVAL; }
+    const int L = (int)pl->layers.size();
+    if (layer < 0 || layer >= L) { set_error("lop_plan_layer_stored: layer %d out of range", layer); return LOP_EINVAL; }
+    const bool persistent = program_supported(pl) && !(pl->flags & (LOP_FLAG_PER_LAYER | LOP_FLAG_TIME_LAYERS));
+    return (persistent && program_folds_pool(pl, layer)) ? 0 : 1;
+}
+
 int lop_plan_last_launches(const lop_plan_t *pl)
 {
     if (!pl) { set_error("plan is NULL"); return LOP_EINVAL; }

@@ -188,6 +188,8 @@ bool pool_fusable(const lop_plan_t *pl, int i)
 
 }  // namespace
 
+bool program_folds_pool(const lop_plan_t *pl, int layer) { return pool_fusable(pl, layer); }
+
 bool program_supported(const lop_plan_t *pl)
 {
     if (pl->dtype != LOP_BF16) return false;
@@ -672,7 +674,9 @@ int program_build(const std::vector<SegBind> &segs, std::vector<StageReq> reqs, 
     // chunks per ring slot of the long pointwise stages (see WfStage::cps), now that the slot sizes are known
     for (WfStage &st : stages) {
         st.cps = 1;
-        if (st.kind != WF_CONV || st.mode != WF_SLAB || st.n_taps != 1 || st.BK != 64 || st.n_chunks <= sb) continue;
+        if (st.kind != WF_CONV) continue;
+        const bool long_pointwise = st.mode == WF_SLAB && st.n_taps == 1 && st.BK == 64 && st.n_chunks > sb;
+        if (!long_pointwise && st.mode != WF_TAP) continue;            // per-tap windows: cps consecutive taps per slot
         st.cps = std::max(1, std::min({(int)(a_slot / st.a_bytes), (int)(b_slot / st.b_bytes), LOP_CPS_MAX}));
     }
 

@@ -22,6 +22,9 @@ struct StageReq { int seg, band, layer, lo, hi; bool wait_arrival; bool gather; 
 struct Program;
 
 bool program_supported(const lop_plan_t *pl);
+// The persistent kernel folds a 2x2 stride-2 pooling that is convolution `layer`'s only reader into that
+// convolution's epilogue (its own output tensor is then never written).
+bool program_folds_pool(const lop_plan_t *pl, int layer);
 // arrival_us (optional): expected arrival time of each band of plan 0; stages are then ordered by their earliest
 // possible start under that schedule instead of by prio.  fetch_src: the chain input in host memory as the device
 // addresses it, source of the fetch requests (segs[0].in is their destination); programs with fetch requests are

@@ -370,7 +370,7 @@ __global__ void __launch_bounds__(FETCH ? WF_THREADS + 32 : WF_THREADS, 1) wavef
                     const bool reuse_w = w_kept && can_keep && wkey == w_key;
                     w_kept = reuse_w || can_keep;
                     w_key = wkey;
-                    if (cps > 1) {
+                    if (cps > 1 && mode == WF_SLAB) {
                         for (int ch = 0; ch < n_chunks && !fail; ch += cps) {
                             const int g = min(cps, n_chunks - ch);
                             if (!mbar_wait_abortable(empty_a + 8u * a_slot, a_phase ^ 1u, abort_flag) ||
@@ -386,7 +386,8 @@ __global__ void __launch_bounds__(FETCH ? WF_THREADS + 32 : WF_THREADS, 1) wavef
                             if (++a_slot == (uint32_t)SA) { a_slot = 0; a_phase ^= 1u; }
                             if (++b_slot == (uint32_t)SB) { b_slot = 0; b_phase ^= 1u; }
                         }
-                    } else
+                    } else {
+                    int tap_u = 0, in_slot = 0;                        // per-tap mode: boxes issued so far, boxes in the open slot
                     for (int ch = 0; ch < n_chunks && !fail; ++ch) {
                         if (mode == WF_SLAB) {
                             // the whole receptive window of the tile in one box: its first tap's offset places it
@@ -406,27 +407,36 @@ __global__ void __launch_bounds__(FETCH ? WF_THREADS + 32 : WF_THREADS, 1) wavef
                                 if (++b_slot == (uint32_t)SB) { b_slot = 0; b_phase ^= 1u; }
                             }
                         } else {
+                            // one activation and one weight box per (channel chunk, tap); `cps` consecutive taps share a
+                            // slot of each ring and its barrier (strides are 1 or 2 almost always: no division then)
                             for (int a = 0; a < kh && !fail; ++a) {
                                 const int qh = a * dh - ph;
-                                const int offh = floor_div_i(qh, sh), parh = qh - offh * sh;
-                                for (int b = 0; b < kw; ++b) {
+                                const int offh = sh == 1 ? qh : (sh == 2 ? qh >> 1 : floor_div_i(qh, sh)), parh = qh - offh * sh;
+                                for (int b = 0; b < kw; ++b, ++tap_u) {
                                     const int qw = b * dw - pw;
-                                    const int offw = floor_div_i(qw, sw), parw = qw - offw * sw;
+                                    const int offw = sw == 1 ? qw : (sw == 2 ? qw >> 1 : floor_div_i(qw, sw)), parw = qw - offw * sw;
                                     const int mi = parh * sw + parw;
                                     const bool have = (amask >> mi) & 1;
-                                    if (!mbar_wait_abortable(empty_a + 8u * a_slot, a_phase ^ 1u, abort_flag) ||
-                                        !mbar_wait_abortable(empty_b + 8u * b_slot, b_phase ^ 1u, abort_flag)) { fail = 1; break; }
-                                    const uint32_t fa = full_a + 8u * a_slot, fb = full_b + 8u * b_slot;
-                                    mbar_expect_tx(fa, a_bytes);
-                                    tma_load_4d(a0 + a_slot * a_slot_bytes, maps + mi, fa, ch * BK, have ? ow0 + offw : -65536,
-                                                have ? oh0 + offh : -65536, n0);
-                                    mbar_expect_tx(fb, b_bytes);
-                                    tma_load_3d(b0 + b_slot * b_slot_bytes, maps + 4, fb, ch * BK, co0, a * kw + b);
-                                    if (++a_slot == (uint32_t)SA) { a_slot = 0; a_phase ^= 1u; }
-                                    if (++b_slot == (uint32_t)SB) { b_slot = 0; b_phase ^= 1u; }
+                                    if (in_slot == 0) {
+                                        const int g = min(cps, n_chunks * n_taps - tap_u);
+                                        if (!mbar_wait_abortable(empty_a + 8u * a_slot, a_phase ^ 1u, abort_flag) ||
+                                            !mbar_wait_abortable(empty_b + 8u * b_slot, b_phase ^ 1u, abort_flag)) { fail = 1; break; }
+                                        mbar_expect_tx(full_a + 8u * a_slot, (uint32_t)g * a_bytes);
+                                        mbar_expect_tx(full_b + 8u * b_slot, (uint32_t)g * b_bytes);
+                                    }
+                                    tma_load_4d(a0 + a_slot * a_slot_bytes + (uint32_t)in_slot * a_bytes, maps + mi, full_a + 8u * a_slot, ch * BK,
+                                                have ? ow0 + offw : -65536, have ? oh0 + offh : -65536, n0);
+                                    tma_load_3d(b0 + b_slot * b_slot_bytes + (uint32_t)in_slot * b_bytes, maps + 4, full_b + 8u * b_slot, ch * BK, co0,
+                                                a * kw + b);
+                                    if (++in_slot == cps || tap_u + 1 == n_chunks * n_taps) {
+                                        in_slot = 0;
+                                        if (++a_slot == (uint32_t)SA) { a_slot = 0; a_phase ^= 1u; }
+                                        if (++b_slot == (uint32_t)SB) { b_slot = 0; b_phase ^= 1u; }
+                                    }
                                 }
                             }
                         }
+                    }
                     }
                     if (fail) atomicOr(P.status, 0x1u);
                     tr(item, 2);
@@ -520,7 +530,7 @@ __global__ void __launch_bounds__(FETCH ? WF_THREADS + 32 : WF_THREADS, 1) wavef
                         mma_row3x64(acc, la + 2u * row16, (((b0 + s2 * b_slot_bytes) & 0x3FFFFu) >> 4) | (1u << 16), tap_bytes >> 4, desc_hi, idesc, accumulate);
                         umma_commit(empty_a + 8u * a_slot);
                         if (++a_slot == (uint32_t)SA) { a_slot = 0; a_phase ^= 1u; }
-                    } else if (cps > 1) {
+                    } else if (cps > 1 && mode == WF_SLAB) {
                         for (int ch = 0; ch < n_chunks; ch += cps) {
                             const int g = min(cps, n_chunks - ch);
                             if (!mbar_wait_abortable(full_a + 8u * a_slot, a_phase, abort_flag) ||
@@ -534,7 +544,8 @@ __global__ void __launch_bounds__(FETCH ? WF_THREADS + 32 : WF_THREADS, 1) wavef
                             if (++a_slot == (uint32_t)SA) { a_slot = 0; a_phase ^= 1u; }
                             if (++b_slot == (uint32_t)SB) { b_slot = 0; b_phase ^= 1u; }
                         }
-                    } else
+                    } else {
+                    int tap_u = 0, in_slot = 0;                        // per-tap mode: boxes consumed so far, boxes used of the open slot
                     for (int ch = 0; ch < n_chunks && !fail; ++ch) {
                         if (mode == WF_SLAB) {
                             if (!mbar_wait_abortable(full_a + 8u * a_slot, a_phase, abort_flag)) { fail = true; break; }
@@ -588,18 +599,24 @@ __global__ void __launch_bounds__(FETCH ? WF_THREADS + 32 : WF_THREADS, 1) wavef
                             umma_commit(empty_a + 8u * a_slot);
                             if (++a_slot == (uint32_t)SA) { a_slot = 0; a_phase ^= 1u; }
                         } else {
-                            for (int t = 0; t < n_taps; ++t) {
-                                if (!mbar_wait_abortable(full_a + 8u * a_slot, a_phase, abort_flag) ||
-                                    !mbar_wait_abortable(full_b + 8u * b_slot, b_phase, abort_flag)) { fail = true; break; }
-                                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                                const uint32_t sa = a0 + a_slot * a_slot_bytes, sb = b0 + b_slot * b_slot_bytes;
-                                mma_tap(acc, sa, sb, desc_hi, idesc, ksteps, accumulate);
-                                umma_commit(empty_a + 8u * a_slot);
-                                umma_commit(empty_b + 8u * b_slot);
-                                if (++a_slot == (uint32_t)SA) { a_slot = 0; a_phase ^= 1u; }
-                                if (++b_slot == (uint32_t)SB) { b_slot = 0; b_phase ^= 1u; }
+                            for (int t = 0; t < n_taps; ++t, ++tap_u) {
+                                if (in_slot == 0) {
+                                    if (!mbar_wait_abortable(full_a + 8u * a_slot, a_phase, abort_flag) ||
+                                        !mbar_wait_abortable(full_b + 8u * b_slot, b_phase, abort_flag)) { fail = true; break; }
+                                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                                }
+                                mma_tap(acc, a0 + a_slot * a_slot_bytes + (uint32_t)in_slot * a_bytes, b0 + b_slot * b_slot_bytes + (uint32_t)in_slot * b_bytes,
+                                        desc_hi, idesc, ksteps, accumulate);
+                                if (++in_slot == cps || tap_u + 1 == n_chunks * n_taps) {
+                                    in_slot = 0;
+                                    umma_commit(empty_a + 8u * a_slot);
+                                    umma_commit(empty_b + 8u * b_slot);
+                                    if (++a_slot == (uint32_t)SA) { a_slot = 0; a_phase ^= 1u; }
+                                    if (++b_slot == (uint32_t)SB) { b_slot = 0; b_phase ^= 1u; }
+                                }
                             }
                         }
+                    }
                     }
                     if (fail) break;
 #ifdef LOP_WF_TRACE

@@ -48,9 +48,10 @@ struct WfStage {
     // fuse_pool: the convolution's only consumer is a 2x2 stride-2 max pooling; the tile's epilogue takes the
     // maximum of each 2x2 window of staged rows and writes the pooled tensor [N, pool_Ho, pool_Wo, Cout] instead
     int fuse_pool, pool_Ho, pool_Wo;
-    // cps > 1: a pointwise stage with a long walk over K puts `cps` consecutive channel chunks into one ring slot behind
-    // one barrier pair (activation boxes in the activation ring, weight boxes in the weight ring), so that more bytes
-    // are on their way at a time: the walk is bound by the loads' latency, a few slots deep, not by their rate
+    // cps > 1: a pointwise stage with a long walk over K puts `cps` consecutive channel chunks, a per-tap stage `cps`
+    // consecutive taps, into one ring slot behind one barrier pair (activation boxes in the activation ring, weight
+    // boxes in the weight ring), so that more bytes are on their way at a time: such a walk is bound by the loads'
+    // latency, a few slots deep, not by their rate
     int cps;
     int pad_[12];
 };

@@ -19,12 +19,41 @@ def rel_err(got, want):
     return float(np.max(np.abs(got.astype(np.float64) - want.astype(np.float64)))) / (scale if scale > 0 else 1.0)
 
 
+def oracle_layers(wl):
+    """Every layer's output of every segment, whole-tensor execution on the CPU: [segment][layer] -> array."""
+    x, out = wl.x, []
+    for seg in wl.segments:
+        out.append(ochain.run_whole(seg.layers, x, wl.dtype == "bf16", keep_all=True))
+        x = out[-1][-1]
+    return out
+
+
+def check_layers(dc, want_layers, tol, what, independent_bands=False):
+    """Every layer output the GPU run has stored (workspace tensors and segment outputs) against the oracle.
+
+    In reuse-halo and whole-tensor runs every row of every layer has been computed; with independent bands (each band
+    recomputing its halo into the same full-size tensors) the rows are complete as well -- the last band to write a
+    row wrote the same bits."""
+    for s, layers in enumerate(want_layers):
+        for i, w in enumerate(layers):
+            t = dc.layer_output(s, i)
+            if t is None:                    # folded into the next layer's stage: that layer's tensor is checked instead
+                continue
+            g = to_host_f32(t)
+            assert g.shape == w.shape, (what, s, i)
+            assert np.all(np.isfinite(g)), (what, "segment", s, "layer", i)
+            e = rel_err(g, w)
+            assert e <= tol, (what, "segment", s, "layer", i, "rel err", e)
+
+
 def check_workload(wl, flags=0, modes=("whole", "banded", "pipelined", "pipelined_copy"), n_bands=None, tol=None):
-    """Run every segment on the GPU in each mode and compare the segment outputs with the oracle.
+    """Run every segment on the GPU in each mode and compare EVERY LAYER's output with the oracle (the intermediate
+    tensors are read out of the workspaces), then the modes with each other bit for bit.
 
     pipelined: the kernel fetches the bands from the pinned host tensor itself (where the plan runs on the persistent
     kernel); pipelined_copy: the bands come by copy-engine copies on the side stream."""
-    want = ochain.run_workload(wl, keep_segments=True)
+    want_layers = oracle_layers(wl)
+    want = [layers[-1] for layers in want_layers]
     tol = TOL[wl.dtype] if tol is None else tol
     results = {}
     for mode in modes:
@@ -37,12 +66,10 @@ def check_workload(wl, flags=0, modes=("whole", "banded", "pipelined", "pipeline
             dc.run_whole(dc.input_tensor())
         torch.cuda.synchronize()
         dc.check_device()
+        check_layers(dc, want_layers, tol, (wl.name, mode))
         outs = [to_host_f32(o) for o in dc.outs]
         for s, (g, w) in enumerate(zip(outs, want)):
             assert g.shape == w.shape
-            assert np.all(np.isfinite(g)), (wl.name, mode, s)
-            e = rel_err(g, w)
-            assert e <= tol, (wl.name, mode, "segment", s, "rel err", e)
         results[mode] = outs
     base = results[modes[0]]
     for mode in modes[1:]:                   # band-wise execution reproduces whole-tensor execution bit for bit
