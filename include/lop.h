@@ -51,8 +51,8 @@ enum { LOP_RES_NONE = 0, LOP_RES_PRE_ACT = 1, LOP_RES_POST_ACT = 2 };
 enum { LOP_INPUT = -1, LOP_NO_RESIDUAL = -2 };              /* special layer indices             */
 enum {
     LOP_FLAG_REUSE_HALO = 1u,     /* bands run in ascending order and compute only rows no earlier
-                                     band produced ("only what is missing", Sec. IV-C data
-                                     dependency); otherwise every band recomputes its halo and is
+                                     band produced (Sec. IV-C, data dependency: rows that are already
+                                     there are not moved again); otherwise every band recomputes its halo and is
                                      independent of the others (operation replication, Sec. IV-C) */
     LOP_FLAG_TIME_LAYERS = 2u,    /* record a CUDA event pair around every (band, layer) launch    */
     LOP_FLAG_FORCE_SIMT = 4u,     /* never use the tensor-core convolution (second on-GPU opinion) */
@@ -177,6 +177,12 @@ int lop_plan_shard(const lop_plan_t *plan, int rank, int world, int *band_lo, in
  * lop_run_banded on one device. */
 int lop_run_shard(lop_plan_t *plan, int band_lo, int band_hi, const void *in_dev, void *out_dev,
                   void *workspace, void *stream);
+/* The same transfer step done by the persistent kernel's fetch warps instead of the copy engine (see lop_run_pipelined:
+ * the "fetched" transport), by itself: band >= 0 brings that band's new rows, band == -1 every band's, from
+ * in_host_pinned -- which must be mapped into the device's address space and agree with staging_dev modulo 16 bytes,
+ * else LOP_EUNSUPPORTED -- to staging_dev.  One launch, no operator runs.  For timing the transmission a pipelined run
+ * has to hide; workspace as for the lop_run_* calls. */
+int lop_fetch_band(lop_plan_t *plan, int band, const void *in_host_pinned, void *staging_dev, void *workspace, void *stream);
 /* Band pipeline (Sec. IV-B computation/transmission overlap): band i+1's rows come in while band i is
  * computed.  Two transports:
  *   - fetched (default when in_host_pinned is mapped into the device's address space, as cudaHostAlloc /

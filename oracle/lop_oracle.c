@@ -2,8 +2,8 @@
  * CPU oracle for local-operator chains: TEST INFRASTRUCTURE, not part of the product.
  *
  * Plain direct-loop definitions of the block-wise local operators of Sec. IV-A of the
- * paper (convolution and max pooling; "the block size is determined by the operator's
- * parameters": kernel size, padding, dilation, and stride) with the element-wise local
+ * paper (convolution and max pooling: an output element reads a block of the input whose
+ * extent follows from kernel size, padding, dilation and stride) with the element-wise local
  * operators (ReLU, SiLU) and the residual addition applied per output element.
  * Nothing here is blocked, fused or reordered; nothing here is shared with the CUDA
  * library.  Only tests, the smoke check and the benchmark's CPU-baseline leg call it.

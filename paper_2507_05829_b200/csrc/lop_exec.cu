@@ -33,15 +33,14 @@ struct MapKey {
 };
 
 struct ProgKey {
-    int kind;                        // -1 whole, -2 all bands, -3 pipelined, -4 pipelined with in-kernel fetch, >= 0 one band,
-                                     // <= -16: the block of bands [lo, hi) encoded as -16 - (lo * 65536 + hi)
-    int n_plans;                     // plans of the chain the program spans
-    const void *in, *out, *ws;       // first plan's input and workspace, last plan's output
+    int kind;                        // -1 whole, -2 all bands, -3 pipelined, -4 pipelined with in-kernel fetch, -5 fetch alone,
+                                     // >= 0 one band, <= -16: the block of bands [lo, hi) encoded as -16 - (lo * 65536 + hi)
+    int sub;                         // fetch alone: the band, or -1 for all bands; 0 otherwise
     const void *src;                 // fetch source (host memory as the device addresses it) or nullptr
-    bool operator<(const ProgKey &o) const
-    {
-        return std::tie(kind, n_plans, in, out, ws, src) < std::tie(o.kind, o.n_plans, o.in, o.out, o.ws, o.src);
-    }
+    // every plan of the chain the program spans: its input / output / workspace and its uid (new at creation and at
+    // every lop_plan_set_params), so a program built from other plans, buffers or parameters is never reused
+    std::vector<const void *> bound;
+    bool operator<(const ProgKey &o) const { return std::tie(kind, sub, src, bound) < std::tie(o.kind, o.sub, o.src, o.bound); }
 };
 
 struct ExecState {
@@ -326,16 +325,22 @@ void merge_thin_bands(const std::vector<SegBind> &segs, std::vector<StageReq> &r
     }
 }
 
-enum { PROG_WHOLE = -1, PROG_ALL_BANDS = -2, PROG_PIPELINED = -3, PROG_FETCHED = -4, PROG_BLOCK0 = -16 };
+enum { PROG_WHOLE = -1, PROG_ALL_BANDS = -2, PROG_PIPELINED = -3, PROG_FETCHED = -4, PROG_FETCH_ALONE = -5, PROG_BLOCK0 = -16 };
 
 // kind: PROG_WHOLE, PROG_ALL_BANDS, PROG_PIPELINED, PROG_FETCHED (fetch_src: the host input as the device addresses
 // it), or b >= 0 for band b alone (single plan only).  segs: the plans of a chain with their buffers; the program is
 // cached in the first plan.
-int get_program(const std::vector<SegBind> &segs, int kind, Program **prog, const void *fetch_src = nullptr)
+int get_program(const std::vector<SegBind> &segs, int kind, Program **prog, const void *fetch_src = nullptr, int sub = 0)
 {
     lop_plan_t *pl0 = segs[0].pl;
     ExecState *e = pl0->exec;
-    const ProgKey key{kind, (int)segs.size(), segs.front().in, segs.back().out, segs.front().ws, fetch_src};
+    ProgKey key{kind, sub, fetch_src, {}};
+    for (const SegBind &sb : segs) {
+        key.bound.push_back(sb.in);
+        key.bound.push_back(sb.out);
+        key.bound.push_back(sb.ws);
+        key.bound.push_back(reinterpret_cast<const void *>(static_cast<uintptr_t>(sb.pl->uid)));
+    }
     auto it = e->programs.find(key);
     if (it == e->programs.end()) {
         if (e->programs.size() >= 64) {
@@ -389,6 +394,15 @@ int get_program(const std::vector<SegBind> &segs, int kind, Program **prog, cons
                 joff += (long long)per;
             }
             std::stable_sort(reqs.begin(), reqs.end(), [](const StageReq &x, const StageReq &y) { return x.prio < y.prio; });
+        } else if (kind == PROG_FETCH_ALONE) {
+            // the transfer step by itself: the fetch requests of one band (sub) or of all bands, no operator
+            for (int b = 0; b < pl0->n_bands; ++b) {
+                if (sub >= 0 && b != sub) continue;
+                const lop_range &need = pl0->in_need[b];
+                StageReq f{0, b, 0, need.new_lo, need.out_hi, false, false, (long long)b};
+                f.fetch = true;
+                reqs.push_back(f);
+            }
         } else if (kind <= PROG_BLOCK0) {
             // a block of bands on a device that runs no other band: layer-major like ALL_BANDS, the first band whole
             const int code = PROG_BLOCK0 - kind, lo = code >> 16, hi = code & 0xFFFF;
@@ -428,9 +442,9 @@ int get_program(const std::vector<SegBind> &segs, int kind, Program **prog, cons
     return LOP_OK;
 }
 
-int get_program(lop_plan_t *pl, int kind, const void *in, void *out, void *ws, Program **prog, const void *fetch_src = nullptr)
+int get_program(lop_plan_t *pl, int kind, const void *in, void *out, void *ws, Program **prog, const void *fetch_src = nullptr, int sub = 0)
 {
-    return get_program(std::vector<SegBind>{SegBind{pl, in, out, ws}}, kind, prog, fetch_src);
+    return get_program(std::vector<SegBind>{SegBind{pl, in, out, ws}}, kind, prog, fetch_src, sub);
 }
 
 // The address under which the device reads the host buffer, when it can (page-locked memory is mapped into the
@@ -637,6 +651,31 @@ int lop_copy_band(lop_plan_t *pl, int band, const void *host, void *staging, voi
     if (rc != LOP_OK) return rc;
     pl->exec->launches = pl->exec->copies = 0;
     return copy_band_impl(pl, band, host, staging, static_cast<cudaStream_t>(stream));
+}
+
+int lop_fetch_band(lop_plan_t *pl, int band, const void *host, void *staging, void *ws, void *stream)
+{
+    if (!pl || !host || !staging) { set_error("lop_fetch_band: NULL argument"); return LOP_EINVAL; }
+    if (band < -1 || band >= pl->n_bands) { set_error("band %d out of range", band); return LOP_EINVAL; }
+    int rc = check_common(pl, staging, staging, ws);
+    if (rc != LOP_OK) return rc;
+    ExecState *e = pl->exec;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    e->launches = e->copies = 0;
+    e->last_stream = s;
+    if (!e->wavefront) { set_error("lop_fetch_band: this plan does not run on the persistent kernel; use lop_copy_band"); return LOP_EUNSUPPORTED; }
+    const void *src = fetchable(pl, host);
+    if (!src || (reinterpret_cast<uintptr_t>(src) & 15) != (reinterpret_cast<uintptr_t>(staging) & 15)) {
+        set_error("lop_fetch_band: the host buffer is not mapped into the device's address space, or differs from the staging tensor modulo 16 bytes");
+        return LOP_EUNSUPPORTED;
+    }
+    if ((rc = prepare_workspace(pl, ws, s)) != LOP_OK) return rc;
+    Program *p = nullptr;
+    if ((rc = get_program(pl, PROG_FETCH_ALONE, staging, staging, ws, &p, src, band)) != LOP_OK) return rc;
+    if (program_empty(p)) return LOP_OK;
+    if ((rc = program_launch(p, s)) != LOP_OK) return rc;
+    e->launches++;
+    return LOP_OK;
 }
 
 int lop_run_pipelined(lop_plan_t *pl, const void *host, void *staging, void *out, void *ws, void *stream)

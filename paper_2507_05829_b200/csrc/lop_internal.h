@@ -36,12 +36,15 @@ struct lop_plan {
     std::vector<lop_range> in_need;    // [band]: chain-input rows (out_lo,out_hi,new_lo)
     size_t ws_bytes = 0, status_off = 0, col_off = 0;   // col_off: the gathered patch tensor
     double flops = 0.0;
+    unsigned long long uid = 0;        // unique per plan and per state of its parameters (a new one at creation and at every
+                                       // lop_plan_set_params): cached device programs name the plans they were built from by it
     lop::ExecState *exec = nullptr;
 };
 
 namespace lop {
 
 void set_error(const char *fmt, ...);
+unsigned long long next_plan_uid();
 inline size_t elem_size(int dtype) { return dtype == LOP_BF16 ? 2 : 4; }
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 

@@ -6,6 +6,7 @@
 // an output is used) and the contiguous-interval rule of Sec. IV-C ("Computational Efficiency"):
 // the operations one executor runs for an operator form one interval, so a band is one row
 // interval per layer and one kernel launch.
+#include <atomic>
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
@@ -16,6 +17,12 @@
 namespace lop {
 
 static thread_local char g_err[512] = "";
+
+unsigned long long next_plan_uid()
+{
+    static std::atomic<unsigned long long> counter{0};
+    return ++counter;
+}
 
 void set_error(const char *fmt, ...)
 {
@@ -237,6 +244,7 @@ int lop_plan(const lop_layer *layers, int n_layers, int N, int H, int W, int C, 
         return LOP_EINVAL;
     }
     lop_plan_t *pl = new (std::nothrow) lop_plan_t();
+    if (pl) pl->uid = next_plan_uid();
     if (!pl) { set_error("lop_plan: out of host memory"); return LOP_ENOMEM; }
     try {
         pl->N = N; pl->H = H; pl->W = W; pl->C = C; pl->dtype = dtype; pl->n_bands = n_bands; pl->flags = flags;
@@ -311,6 +319,7 @@ int lop_plan_set_params(lop_plan_t *plan, int layer, const void *weight, const f
     if (layer < 0 || layer >= (int)plan->layers.size()) { set_error("lop_plan_set_params: layer %d out of range", layer); return LOP_EINVAL; }
     lop_layer &l = plan->layers[layer].l;
     l.weight = weight; l.scale = scale; l.shift = shift;
+    plan->uid = next_plan_uid();           // chain programs cached in another plan were built from the old pointers too
     exec_invalidate(plan->exec);           // device tables and tensor maps were built from the old pointers
     return LOP_OK;
 }

@@ -41,6 +41,12 @@ namespace {
 #ifndef LOP_FETCH_WINDOW_BYTES
 #define LOP_FETCH_WINDOW_BYTES (96 * 1024)
 #endif
+#ifndef LOP_SA_MAX
+#define LOP_SA_MAX 4
+#endif
+#ifndef LOP_SB_MAX
+#define LOP_SB_MAX 8
+#endif
 #ifndef LOP_CPS_MAX
 #define LOP_CPS_MAX 4
 #endif
@@ -658,7 +664,7 @@ int program_build(const std::vector<SegBind> &segs, std::vector<StageReq> reqs, 
         n_ctr += p->n_flags;
     }
     const int n_items = (int)items.size();
-    if (n_items == 0) { *result = p; return LOP_OK; }          // nothing to do: an empty program
+    if (n_items == 0 && fetch_items.empty()) { *result = p; return LOP_OK; }          // nothing to do: an empty program
 
     // ---- shared-memory rings: as many slots as fit beside the staging tile, weights first
     const size_t fixed = 1024 + stg_bytes + 8 * (2 * 8 + 2 * 8 + 4 + 2 * WF_PUBQ + 4) + 64 + 2048 + 1280 + 64;
@@ -667,8 +673,8 @@ int program_build(const std::vector<SegBind> &segs, std::vector<StageReq> reqs, 
     if ((size_t)sa * a_slot + (size_t)sb * b_slot > budget) { delete p; set_error("tile buffers do not fit shared memory"); return LOP_EUNSUPPORTED; }
     for (bool grew = true; grew;) {
         grew = false;
-        if (sb < 8 && (size_t)sa * a_slot + (size_t)(sb + 1) * b_slot <= budget) { ++sb; grew = true; }
-        if (sa < 4 && (size_t)(sa + 1) * a_slot + (size_t)sb * b_slot <= budget) { ++sa; grew = true; }
+        if (sb < LOP_SB_MAX && (size_t)sa * a_slot + (size_t)(sb + 1) * b_slot <= budget) { ++sb; grew = true; }
+        if (sa < LOP_SA_MAX && (size_t)(sa + 1) * a_slot + (size_t)sb * b_slot <= budget) { ++sa; grew = true; }
     }
 
     // chunks per ring slot of the long pointwise stages (see WfStage::cps), now that the slot sizes are known
@@ -733,7 +739,7 @@ int program_build(const std::vector<SegBind> &segs, std::vector<StageReq> reqs, 
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    p->grid = std::min(n_items, sms);
+    p->grid = n_items > 0 ? std::min(n_items, sms) : std::min((int)fetch_items.size(), sms);   // (a fetch-only program: its fetch warps)
     *result = p;
     return LOP_OK;
 }

@@ -55,11 +55,17 @@ class ShardedChain:
         self.tables = [shard_table(p, world) for p in device_chain.plans]
 
     def run(self, x_dev, stream=None):
+        """Every plan's block of bands on ``stream`` (default: torch's current stream), each followed by the all-gather of
+        its output rows.  torch orders a collective, and the copies around it, against its CURRENT stream, so the whole
+        loop runs with ``stream`` made current: the gather then waits for this rank's launch, and the next plan's launch
+        for the gathered rows."""
         dc = self.dc
-        s = dc._stream(stream)
-        for plan, ws, out, table in zip(dc.plans, dc.ws, dc.outs, self.tables):
-            b_lo, b_hi = table[self.rank][0], table[self.rank][1]
-            plan.run_shard(b_lo, b_hi, x_dev.data_ptr(), out.data_ptr(), ws.data_ptr(), s)
-            all_gather_rows(out, table, self.rank, self.group)       # same stream: torch orders the collective behind the launch
-            x_dev = out
+        cur = torch.cuda.current_stream(dc.device) if stream is None else stream
+        with torch.cuda.stream(cur):
+            s = cur.cuda_stream
+            for plan, ws, out, table in zip(dc.plans, dc.ws, dc.outs, self.tables):
+                b_lo, b_hi = table[self.rank][0], table[self.rank][1]
+                plan.run_shard(b_lo, b_hi, x_dev.data_ptr(), out.data_ptr(), ws.data_ptr(), s)
+                all_gather_rows(out, table, self.rank, self.group)
+                x_dev = out
         return dc.outs[-1]

@@ -312,6 +312,107 @@ def test_sharded_chain_with_one_rank_is_the_banded_run():
     assert torch.equal(out, ref.outs[-1])
 
 
+def test_sharded_chain_on_a_stream_that_is_not_current():
+    """The launches and the row exchange are ordered on the stream that was passed, also when torch's current stream is
+    another one: the result equals the banded run and the current stream never sees half-written rows."""
+    from paper_2507_05829_b200 import shard
+    wl = li.build("resnet18", H=64, W=64)
+    ref = DeviceChain(wl, flags=lop.LOP_FLAG_REUSE_HALO)
+    ref.run_banded(ref.input_tensor())
+    torch.cuda.synchronize()
+    dc = DeviceChain(wl, flags=lop.LOP_FLAG_REUSE_HALO)
+    side = torch.cuda.Stream()
+    x = dc.input_tensor()
+    torch.cuda.synchronize()
+    out = shard.ShardedChain(dc, 0, 1).run(x, stream=side)
+    side.synchronize()
+    dc.check_device()
+    assert torch.equal(out, ref.outs[-1])
+    # the copy path of the exchange for two ranks, driven by hand on the side stream: rank 0's rows stay, rank 1's arrive
+    table = shard.shard_table(dc.plans[-1], 2)
+    full = ref.outs[-1]
+    mine = torch.zeros_like(full)
+    mine[:, table[0][2]:table[0][3]] = full[:, table[0][2]:table[0][3]]
+    torch.cuda.synchronize()
+
+    class FakeGroup:
+        pass
+
+    def fake_all_gather(parts, tensor, group=None):
+        n_max = tensor.shape[1]
+        for r, part in enumerate(parts):
+            lo, hi = table[r][2], table[r][3]
+            part.zero_()
+            part[:, :hi - lo].copy_(full[:, lo:hi])
+
+    import torch.distributed as dist
+    keep = dist.all_gather
+    dist.all_gather = fake_all_gather
+    try:
+        with torch.cuda.stream(side):
+            got = shard.all_gather_rows(mine, table, 0)
+        side.synchronize()
+    finally:
+        dist.all_gather = keep
+    assert torch.equal(got, full)
+
+
+def test_set_params_on_a_later_plan_of_a_chain_takes_effect():
+    """A chain program is cached in the first plan; re-pointing the parameters of a LATER plan must not leave it in use."""
+    wl = li.build("resnet18", H=64, W=64)
+    dc = DeviceChain(wl, flags=lop.LOP_FLAG_REUSE_HALO)
+    x = dc.input_tensor()
+    first = dc.run_banded(x).clone()
+    torch.cuda.synchronize()
+    assert not dc.per_plan                                  # the plans ran as one launch
+    seg_i = 2
+    seg = wl.segments[seg_i]
+    keep = []
+    for i, l in enumerate(seg.layers):
+        if l.weight is None:
+            continue
+        l.weight = -l.weight
+        w = torch.from_numpy(l.weight).to(torch.bfloat16).cuda().contiguous()
+        sc = torch.from_numpy(l.scale).cuda() if l.scale is not None else None
+        sh = torch.from_numpy(l.shift).cuda() if l.shift is not None else None
+        keep += [w, sc, sh]
+        dc.plans[seg_i].set_params(i, w.data_ptr(), sc.data_ptr() if sc is not None else None, sh.data_ptr() if sh is not None else None)
+    want = oracle_layers(wl)
+    for mode in ("banded", "pipelined"):
+        got = dc.run_banded(x) if mode == "banded" else dc.run_pipelined(dc.pinned_input())
+        torch.cuda.synchronize()
+        dc.check_device()
+        assert not dc.per_plan
+        check_layers(dc, want, TOL["bf16"], ("resnet18 re-pointed", mode))
+    assert not torch.equal(first, dc.outs[-1])
+
+
+def test_fetch_band_alone_brings_exactly_its_rows():
+    """lop_fetch_band: the transfer step of the fetched transport by itself (what a pipelined run has to hide)."""
+    wl = li.build("vgg_block", H=44, W=36)
+    dc = DeviceChain(wl, flags=lop.LOP_FLAG_REUSE_HALO)
+    plan = dc.plans[0]
+    x, xd = dc.pinned_input(), dc.input_tensor()
+    s = torch.cuda.current_stream().cuda_stream
+    dc.staging.fill_(float("nan"))
+    plan.fetch_band(-1, x.data_ptr(), dc.staging.data_ptr(), dc.ws[0].data_ptr(), s)
+    torch.cuda.synchronize()
+    plan.check_device(dc.ws[0].data_ptr())
+    assert plan.last_launches() >= 1 and plan.last_copies() == 0
+    assert torch.equal(dc.staging.view(-1), xd.view(-1))
+    for b in (0, 2):
+        r = plan.get_range(b, lop.LOP_INPUT)
+        dc.staging.fill_(float("nan"))
+        plan.fetch_band(b, x.data_ptr(), dc.staging.data_ptr(), dc.ws[0].data_ptr(), s)
+        torch.cuda.synchronize()
+        assert torch.equal(dc.staging[:, r.new_lo:r.out_hi], xd[:, r.new_lo:r.out_hi])
+        assert torch.isnan(dc.staging[:, :r.new_lo].float()).all() and torch.isnan(dc.staging[:, r.out_hi:].float()).all()
+    dc.run_pipelined(x)                                     # and the plan still runs
+    torch.cuda.synchronize()
+    dc.check_device()
+    assert rel_err(to_host_f32(dc.outs[-1]), ochain.run_workload(wl)) <= TOL["bf16"]
+
+
 # ------------------------------------------------------------------------------------ edge cases
 def test_very_wide_image_gathers_patches_without_staging_rows():
     """Three rows of a 4200-pixel image do not fit the shared staging tile: the gather reads the image in place."""

@@ -11,11 +11,13 @@ every other test.
 """
 import ctypes
 
+import numpy as np
 import pytest
 import torch
 
 import lop_inputs as li
 import paper_2507_05829_b200 as lop
+from oracle import chain as ochain
 from paper_2507_05829_b200.chain import DeviceChain
 
 
@@ -29,6 +31,15 @@ def test_plan_larger_than_the_built_in_scratch_is_refused():
     assert e.value.status == -3
     assert str(lop.LOP_STATIC_SCRATCH_BYTES) in str(e.value) and str(p.workspace_bytes()) in str(e.value)
     assert lop.lib().lop_run_whole_static(None, None, None, None, None) == -1
+
+
+TOL = {"f32": 1e-4, "bf16": 2e-2}       # max |gpu - oracle| / max |oracle|, the tolerances of the other GPU tests
+
+
+def _oracle_err(got, want):
+    """Distance of a device tensor from the CPU oracle's result, relative to the oracle's output scale."""
+    g = got.detach().to("cpu", torch.float32).numpy().astype(np.float64)
+    return float(np.max(np.abs(g - want))) / float(np.max(np.abs(want)))
 
 
 def _reference(wl):
@@ -61,6 +72,9 @@ def test_static_scratch_entry_point_matches_run_whole_on_two_calls_in_a_row():
     dcv.plans[0].run_whole_static(xv.data_ptr(), out_v.data_ptr(), status.data_ptr(), s)
     stream.synchronize()
     assert torch.equal(out_v, want_v) and int(status.item()) == 0
+    # the oracle's results: the whole VGG block, and the first segment (stem + pooling) of the residual network
+    oracle_v = ochain.run_workload(vgg)
+    oracle_r = ochain.run_whole(res.segments[0].layers, res.x, True)
     free_before = None
     for call in range(3):
         out_v.fill_(-5.0)
@@ -71,6 +85,8 @@ def test_static_scratch_entry_point_matches_run_whole_on_two_calls_in_a_row():
         stream.synchronize()
         assert torch.equal(out_v, want_v), "call %d differs from lop_run_whole" % call
         assert torch.equal(out_r, want_r), "call %d (second plan) differs from lop_run_whole" % call
+        assert _oracle_err(out_v, oracle_v) <= TOL["bf16"], "call %d differs from the oracle" % call
+        assert _oracle_err(out_r, oracle_r) <= TOL["bf16"], "call %d (second plan) differs from the oracle" % call
         assert int(status.item()) == 0
         if free_before is None:                 # torch's own caches for fill_/equal/item are warm from here on
             free_before, _ = torch.cuda.mem_get_info()
@@ -91,3 +107,4 @@ def test_static_scratch_entry_point_fp32_and_cuda_core_paths():
             dc.plans[0].run_whole_static(x.data_ptr(), got.data_ptr(), None, torch.cuda.current_stream().cuda_stream)
             torch.cuda.synchronize()
             assert torch.equal(got, want)
+            assert _oracle_err(got, ochain.run_workload(wl)) <= TOL[wl.dtype]
