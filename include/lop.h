@@ -252,6 +252,22 @@ int lop_plan_last_copies(const lop_plan_t *plan);
  * (window of the in-kernel input transfer). */
 int lop_plan_check_device(lop_plan_t *plan, void *workspace);
 
+/* ---- the device-side waits and their failure path ----------------------------------------------
+ * Every wait inside the persistent kernel (for a producer's rows, a band's arrival, a ring slot) is bounded: when it
+ * runs out the kernel raises the plan's status word, tells every CTA to stop and returns; the outputs of that call are
+ * invalid and lop_plan_check_device() reports LOP_EDEVICE and readies the plan for the next call.  The paper names the
+ * failure of one unit as a risk of fine-grained partitioning (Sec. I) and answers it by tracking dependencies; this is
+ * what happens here when a dependency is never satisfied.
+ * lop_plan_set_wait_limit: polls (of some tens of nanoseconds each) a wait for rows or for an arrival may take; 0
+ * restores the default (about four million).  Applies to the plan's later launches (for a chain: the first plan's). */
+int lop_plan_set_wait_limit(lop_plan_t *plan, unsigned polls);
+/* lop_run_pipelined with the copy-engine transport, except that band `band` never arrives: neither its copy nor its
+ * arrival write is enqueued.  Exists to exercise the failure path above without faulting anything: the kernel's wait
+ * for that band runs out after the plan's wait limit -- which must have been set, to at most 65536 polls, a few
+ * milliseconds -- and the call's stream work ends normally with the status word raised (bit 0x10). */
+int lop_run_pipelined_withheld(lop_plan_t *plan, int band, const void *in_host_pinned, void *staging_dev, void *out_dev,
+                               void *workspace, void *stream);
+
 /* ---- execution without any allocation --------------------------------------------------------
  * (The paper has no counterpart: this entry point exists for how the library is deployed.)
  * Some callers are not allowed to allocate: a plug-in running inside an application that forbids

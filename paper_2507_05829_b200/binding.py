@@ -20,7 +20,7 @@ EXPORTS = [
     "lop_plan_out_shape", "lop_plan_set_params", "lop_plan_workspace_bytes", "lop_plan_staging_bytes",
     "lop_plan_flops", "lop_run_whole", "lop_run_band", "lop_run_banded", "lop_copy_band", "lop_fetch_band", "lop_run_pipelined",
     "lop_plan_last_timing", "lop_plan_layer_time", "lop_plan_layer_kernel", "lop_plan_last_launches", "lop_plan_last_copies",
-    "lop_plan_check_device", "lop_plan_layer_offset", "lop_plan_layer_stored", "lop_run_whole_static", "lop_run_chain_banded", "lop_run_chain_pipelined", "lop_plan_shard", "lop_run_shard",
+    "lop_plan_check_device", "lop_plan_set_wait_limit", "lop_run_pipelined_withheld", "lop_plan_layer_offset", "lop_plan_layer_stored", "lop_run_whole_static", "lop_run_chain_banded", "lop_run_chain_pipelined", "lop_plan_shard", "lop_run_shard",
     "lop_strerror", "lop_last_error",
 ]
 LOP_STATIC_SCRATCH_BYTES = 16 << 20
@@ -94,6 +94,8 @@ def lib():
     L.lop_plan_last_launches.argtypes = [c_void_p]
     L.lop_plan_last_copies.argtypes = [c_void_p]
     L.lop_plan_check_device.argtypes = [c_void_p, c_void_p]
+    L.lop_plan_set_wait_limit.argtypes = [c_void_p, c_uint]
+    L.lop_run_pipelined_withheld.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
     L.lop_run_whole_static.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
     L.lop_run_chain_banded.argtypes = [POINTER(c_void_p), c_int, c_void_p, POINTER(c_void_p), POINTER(c_void_p), c_void_p]
     L.lop_run_chain_pipelined.argtypes = [POINTER(c_void_p), c_int, c_void_p, c_void_p, POINTER(c_void_p), POINTER(c_void_p), c_void_p]
@@ -247,6 +249,12 @@ class Plan:
     def run_whole_static(self, in_dev, out_dev, status_dev, stream):
         """lop_run_whole_static: no workspace argument, nothing is allocated (see include/lop.h)."""
         _check(lib().lop_run_whole_static(self._h, in_dev, out_dev, status_dev, stream))
+
+    def set_wait_limit(self, polls):
+        _check(lib().lop_plan_set_wait_limit(self._h, polls))
+
+    def run_pipelined_withheld(self, band, in_host, staging_dev, out_dev, ws, stream):
+        _check(lib().lop_run_pipelined_withheld(self._h, band, in_host, staging_dev, out_dev, ws, stream))
 
     def check_device(self, ws):
         _check(lib().lop_plan_check_device(self._h, ws))

@@ -502,7 +502,8 @@ int copy_band_impl(lop_plan_t *pl, int band, const void *host, void *staging, cu
 
 // The single-launch band pipeline on stream s (which may be capturing): fork the side streams, launch the
 // persistent kernel, enqueue every band's copy and arrival write, join.
-int enqueue_pipelined(lop_plan_t *pl, Program *p, const void *host, void *staging, cudaStream_t s)
+// withheld: a band whose copy and arrival write are left out (lop_run_pipelined_withheld), or -1.
+int enqueue_pipelined(lop_plan_t *pl, Program *p, const void *host, void *staging, cudaStream_t s, int withheld = -1)
 {
     ExecState *e = pl->exec;
     int rc = LOP_OK;
@@ -521,7 +522,8 @@ int enqueue_pipelined(lop_plan_t *pl, Program *p, const void *host, void *stagin
     LOP_CUDA(cudaStreamWaitEvent(e->signal_stream, e->ev_fork, 0));
     for (int b = 0; b < pl->n_bands; ++b) {
         const lop_range &need = pl->in_need[b];
-        e->copy_issued[b] = need.out_hi > need.new_lo;
+        e->copy_issued[b] = need.out_hi > need.new_lo && b != withheld;
+        if (b == withheld) continue;
         if (e->copy_issued[b] && (rc = copy_band_impl(pl, b, host, staging, e->copy_stream)) != LOP_OK) return rc;
         unsigned *flag = program_arrival_flag(p, b);
         if (!flag) continue;
@@ -744,6 +746,35 @@ int lop_run_pipelined(lop_plan_t *pl, const void *host, void *staging, void *out
     if (timed) LOP_CUDA(cudaEventRecord(e->ev_end, s));
     e->timing_valid = timed;
     return LOP_OK;
+}
+
+int lop_plan_set_wait_limit(lop_plan_t *pl, unsigned polls)
+{
+    if (!pl) { set_error("plan is NULL"); return LOP_EINVAL; }
+    pl->wait_limit = polls;
+    return LOP_OK;
+}
+
+int lop_run_pipelined_withheld(lop_plan_t *pl, int band, const void *host, void *staging, void *out, void *ws, void *stream)
+{
+    int rc = check_common(pl, staging, out, ws);
+    if (rc != LOP_OK) return rc;
+    if (!host) { set_error("lop_run_pipelined_withheld: host input is NULL"); return LOP_EINVAL; }
+    if (band < 0 || band >= pl->n_bands) { set_error("band %d out of range", band); return LOP_EINVAL; }
+    ExecState *e = pl->exec;
+    if (!e->wavefront) { set_error("lop_run_pipelined_withheld: this plan does not run on the persistent kernel"); return LOP_EUNSUPPORTED; }
+    if (pl->wait_limit == 0 || pl->wait_limit > (1u << 16)) {
+        set_error("lop_run_pipelined_withheld: set a wait limit of at most 65536 polls first (lop_plan_set_wait_limit)");
+        return LOP_EINVAL;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    e->launches = e->copies = 0;
+    e->last_stream = s;
+    e->timing_valid = false;
+    if ((rc = prepare_workspace(pl, ws, s)) != LOP_OK) return rc;
+    Program *p = nullptr;
+    if ((rc = get_program(pl, PROG_PIPELINED, staging, out, ws, &p)) != LOP_OK) return rc;
+    return enqueue_pipelined(pl, p, host, staging, s, band);
 }
 
 namespace {

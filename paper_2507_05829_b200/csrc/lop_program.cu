@@ -24,6 +24,7 @@ struct Program {
     WfParams params{};
     int grid = 0;
     int flag_base = 0, n_flags = 0;
+    const lop_plan_t *owner = nullptr;  // the first plan: its wait limit applies to the launches
 };
 
 void program_destroy(Program *p)
@@ -611,12 +612,16 @@ int program_build(const std::vector<SegBind> &segs, std::vector<StageReq> reqs, 
             const Reads rd = reads_of(cx, rq, o0, o1);
             const int first = (int)deps.size();
             if (rq.wait_arrival && rd.raw) {
-                // every band whose transfer brought rows this band reads (its own, and earlier ones for the halo); no
-                // assumption is made about the order in which arrivals become visible
-                const lop_range &mine = pl->in_need[rq.band];
-                for (int b2 = 0; b2 <= rq.band; ++b2) {
+                // every band whose transfer brings rows these output rows read (a request may span several bands where
+                // thin bands were joined); no assumption is made about the order in which arrivals become visible
+                long long a = (long long)o0 * l.sh - l.ph, b = (long long)(o1 - 1) * l.sh - l.ph + (long long)(l.kh - 1) * l.dh + 1;
+                const bool main_raw = rq.gather || (l.input_from == LOP_INPUT && !li.stem_gather);
+                if (!main_raw) { a = o0; b = o1; }                          // only the residual reads the chain input: its own rows
+                else if (!rq.gather && l.op == LOP_CONV2D && l.residual_from == LOP_INPUT) { a = std::min<long long>(a, o0); b = std::max<long long>(b, o1); }
+                a = std::max(a, 0LL); b = std::min<long long>(b, pl->H);
+                for (int b2 = 0; b2 < pl->n_bands; ++b2) {
                     const lop_range &o = pl->in_need[b2];
-                    if (b2 != rq.band && (o.out_hi <= o.new_lo || o.out_hi <= mine.out_lo || o.new_lo >= mine.out_hi)) continue;
+                    if (o.out_hi <= o.new_lo || o.out_hi <= a || o.new_lo >= b) continue;
                     deps.push_back(make_int2(-1 - b2, -1));             // patched below
                 }
                 uses_flags = true;
@@ -745,7 +750,19 @@ int program_build(const std::vector<SegBind> &segs, std::vector<StageReq> reqs, 
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    p->owner = pl0;
     p->grid = n_items > 0 ? std::min(n_items, sms) : std::min((int)fetch_items.size(), sms);   // (a fetch-only program: its fetch warps)
+    // every CTA of a launch must be resident (see the kernel's deadlock-freedom argument); what the device can hold
+    // with this kernel's shared memory and registers says whether that is possible at all -- whether the SMs are free
+    // at launch time is the caller's business: the stream must have the GPU to itself while the kernel runs
+    int resident = 0;
+    e = wavefront_resident_ctas(P, &resident);
+    if (e != cudaSuccess) { program_destroy(p); set_error("occupancy query failed: %s", cudaGetErrorString(e)); return LOP_ECUDA; }
+    if (resident < p->grid) {
+        program_destroy(p);
+        set_error("the device holds %d CTAs of the persistent kernel at a time, the program needs %d", resident, p->grid);
+        return LOP_EUNSUPPORTED;
+    }
     *result = p;
     return LOP_OK;
 }
@@ -753,6 +770,7 @@ int program_build(const std::vector<SegBind> &segs, std::vector<StageReq> reqs, 
 int program_launch(Program *p, cudaStream_t s)
 {
     if (!p || p->grid == 0) return LOP_OK;
+    p->params.spin_limit = (p->owner && p->owner->wait_limit) ? p->owner->wait_limit : WF_SPIN_LIMIT_DEFAULT;
     cudaError_t e = launch_wavefront(p->params, p->grid, s);
     if (e != cudaSuccess) { set_error("wavefront launch failed: %s", cudaGetErrorString(e)); return LOP_ECUDA; }
     return LOP_OK;

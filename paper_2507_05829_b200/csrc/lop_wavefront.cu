@@ -37,7 +37,6 @@ namespace {
 
 using namespace ptx;
 
-constexpr uint32_t SPIN_LIMIT = 1u << 22;
 constexpr int EPI_THREADS = 32 * WF_WORKER_WARPS;
 constexpr int COL_GROUPS = WF_WORKER_WARPS / 4;            // worker warps sharing a TMEM lane group split the columns
 
@@ -101,7 +100,7 @@ __device__ __forceinline__ bool wait_deps_warp(const WfParams &P, int first, int
         for (uint32_t i = 0;; ++i) {
             if (!done) done = (int)(ld_acquire(ctr) - target) >= 0;
             if (__all_sync(0xffffffffu, done)) break;
-            if (i >= SPIN_LIMIT) return false;
+            if (i >= P.spin_limit) return false;
             if ((i & 63u) == 63u && __any_sync(0xffffffffu, ld_relaxed(P.counters + 2) != 0u)) return false;
             __nanosleep(32);
         }
@@ -679,7 +678,7 @@ __global__ void __launch_bounds__(FETCH ? WF_THREADS + 32 : WF_THREADS, 1) wavef
                 int ok = 1;
                 if (lane == 0) {
                     for (uint32_t i = 0; (int)(ld_acquire(P.counters + 3) - target) < 0; ++i) {
-                        if (i >= SPIN_LIMIT) { ok = 0; atomicOr(P.status, 0x20u); break; }
+                        if (i >= P.spin_limit) { ok = 0; atomicOr(P.status, 0x20u); break; }
                         if ((i & 63u) == 63u && (ld_relaxed(P.counters + 2) != 0u || *abort_flag)) { ok = -1; break; }
                         __nanosleep(64);
                     }
@@ -1102,6 +1101,27 @@ size_t wavefront_smem_bytes(const WfParams &p)
 {
     return 1024 + (size_t)p.sa * p.a_slot_bytes + (size_t)p.sb * p.b_slot_bytes + p.stg_bytes + 8 * (size_t)(2 * p.sa + 2 * p.sb + 4 + 2 * WF_PUBQ + 4) + 64 +
            2 * 256 * sizeof(float) + (128 + 32) * sizeof(long long) + 64;
+}
+
+// How many CTAs of the kernel this device can hold at once (the kernel's dependency waits assume that every CTA of
+// a launch is resident: a CTA that has not started cannot produce what a running one waits for).
+cudaError_t wavefront_resident_ctas(const WfParams &p, int *ctas)
+{
+    int dev = 0, sms = 0, per_sm = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+    const size_t smem = wavefront_smem_bytes(p);
+    if (p.n_fetch > 0) {
+        if ((e = cudaFuncSetAttribute(wavefront_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024)) != cudaSuccess) return e;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, wavefront_kernel<true>, WF_THREADS + 32, smem);
+    } else {
+        if ((e = cudaFuncSetAttribute(wavefront_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024)) != cudaSuccess) return e;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, wavefront_kernel<false>, WF_THREADS, smem);
+    }
+    if (e != cudaSuccess) return e;
+    *ctas = per_sm * sms;
+    return cudaSuccess;
 }
 
 cudaError_t launch_wavefront(const WfParams &p, int grid, cudaStream_t s)

@@ -75,6 +75,7 @@ struct WfParams {
     // walks this list round-robin; entry j copies z bytes at byte offset (x | y << 32) from fetch_src (host memory
     // the device can address) to fetch_dst and then increments counters[w].  At most fetch_window entries are in
     // flight at a time (counters[3] counts finished ones), so the rows arrive in list order at the link's rate.
+    uint32_t spin_limit;      // polls of a row-group counter, an arrival flag or the fetch window before the kernel gives up
     const int4 *fetch_items;
     const void *fetch_src;
     void *fetch_dst;
@@ -93,5 +94,7 @@ constexpr int WF_MAX_DEPS = 4095;
 
 size_t wavefront_smem_bytes(const WfParams &p);
 cudaError_t launch_wavefront(const WfParams &p, int grid, cudaStream_t s);
+cudaError_t wavefront_resident_ctas(const WfParams &p, int *ctas);
+constexpr uint32_t WF_SPIN_LIMIT_DEFAULT = 1u << 22;
 
 }  // namespace lop

@@ -413,6 +413,48 @@ def test_fetch_band_alone_brings_exactly_its_rows():
     assert rel_err(to_host_f32(dc.outs[-1]), ochain.run_workload(wl)) <= TOL["bf16"]
 
 
+def test_a_band_that_never_arrives_ends_the_launch_with_a_status_not_a_hang():
+    """The bounded device-side wait, made to run out on purpose: band 1 is never copied and its arrival flag never
+    written; with a limit of a few thousand polls the kernel gives up within milliseconds, returns by itself, the status
+    word names the loader's dependency wait (0x10), and the plan works again afterwards."""
+    wl = li.build("vgg_block", H=44, W=36)
+    dc = DeviceChain(wl, flags=lop.LOP_FLAG_REUSE_HALO | lop.LOP_FLAG_COPY_ENGINE)
+    plan, ws = dc.plans[0], dc.ws[0]
+    x, xd = dc.pinned_input(), dc.input_tensor()
+    s = torch.cuda.current_stream().cuda_stream
+    dc.run_pipelined(x)
+    torch.cuda.synchronize()
+    dc.check_device()
+    good = dc.outs[-1].clone()
+    with pytest.raises(lop.LopError):                       # refuses to run without a short limit
+        plan.run_pipelined_withheld(1, x.data_ptr(), dc.staging.data_ptr(), dc.outs[0].data_ptr(), ws.data_ptr(), s)
+    plan.set_wait_limit(4000)
+    dc.outs[-1].zero_()
+    t0 = torch.cuda.Event(enable_timing=True)
+    t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    plan.run_pipelined_withheld(1, x.data_ptr(), dc.staging.data_ptr(), dc.outs[0].data_ptr(), ws.data_ptr(), s)
+    t1.record()
+    torch.cuda.synchronize()                                # returns: the kernel ended by itself
+    assert t0.elapsed_time(t1) < 2000.0
+    with pytest.raises(lop.LopError) as e:
+        plan.check_device(ws.data_ptr())
+    assert e.value.status == -7
+    word = int(str(e.value).split("0x")[1].split(":")[0].split()[0], 16)
+    assert word & 0x10
+    plan.check_device(ws.data_ptr())                        # the word was cleared, the device tables dropped
+    plan.set_wait_limit(0)
+    for mode in ("pipelined", "banded"):
+        dc.outs[-1].zero_()
+        if mode == "pipelined":
+            dc.run_pipelined(x)
+        else:
+            dc.run_banded(xd)
+        torch.cuda.synchronize()
+        dc.check_device()
+        assert torch.equal(dc.outs[-1], good), mode
+
+
 # ------------------------------------------------------------------------------------ edge cases
 def test_very_wide_image_gathers_patches_without_staging_rows():
     """Three rows of a 4200-pixel image do not fit the shared staging tile: the gather reads the image in place."""
