@@ -591,8 +591,36 @@ int lop_run_banded(lop_plan_t *pl, const void *in, void *out, void *ws, void *st
     reset_layer_timing(pl);
     if ((rc = prepare_workspace(pl, ws, s)) != LOP_OK) return rc;
     if (pl->exec->wavefront) return run_program(pl, PROG_ALL_BANDS, in, out, ws, s);
-    for (int b = 0; b < pl->n_bands; ++b)
-        if ((rc = run_band_impl(pl, b, in, out, ws, s)) != LOP_OK) return rc;
+    if (pl->flags & LOP_FLAG_TIME_LAYERS) {                       // timed plans keep one launch per (band, layer)
+        for (int b = 0; b < pl->n_bands; ++b)
+            if ((rc = run_band_impl(pl, b, in, out, ws, s)) != LOP_OK) return rc;
+        return LOP_OK;
+    }
+    // Operation batching (Sec. IV-C): with the whole input on the device, the bands' operations at a layer are one
+    // contiguous run of rows (neighbouring bands' ranges touch or overlap), so each layer is ONE launch over the hull of
+    // the bands' rows.  Every row is computed once, with the same bits as band by band.
+    const int L = (int)pl->layers.size();
+    for (int i = 0; i < L; ++i) {
+        int lo = 0, hi = 0;
+        bool any = false, contiguous = true;
+        for (int b = 0; b < pl->n_bands; ++b) {
+            const lop_range &r = pl->ranges[(size_t)b * L + i];
+            if (r.out_hi <= r.out_lo) continue;
+            if (any && r.out_lo > hi) contiguous = false;
+            lo = any ? std::min(lo, (int)r.out_lo) : (int)r.out_lo;
+            hi = any ? std::max(hi, (int)r.out_hi) : (int)r.out_hi;
+            any = true;
+        }
+        if (!any) continue;
+        if (contiguous) {
+            if ((rc = run_layer(pl, i, lo, hi, in, out, ws, s, -1)) != LOP_OK) return rc;
+        } else {
+            for (int b = 0; b < pl->n_bands; ++b) {
+                const lop_range &r = pl->ranges[(size_t)b * L + i];
+                if ((rc = run_layer(pl, i, first_row(pl, 0, b, i), r.out_hi, in, out, ws, s, -1)) != LOP_OK) return rc;
+            }
+        }
+    }
     return LOP_OK;
 }
 

@@ -32,31 +32,36 @@ __device__ __forceinline__ float activate(float t, int act)
 // 64x64 tile per 256-thread block, 16-wide K slabs staged through shared memory, 4x4 outputs per
 // thread.  K is walked in one fixed order, so a pixel's value does not depend on the band it is in.
 // ---------------------------------------------------------------------------------------------
-constexpr int SM_BM = 64, SM_BN = 64, SM_BK = 16;
+constexpr int SM_BK = 16;
 
-template <typename T>
+// TM: outputs per thread along each tile axis; the tile is (16*TM) pixels x (16*TM) output channels.  TM = 4 for
+// layers with enough tiles to fill the machine, TM = 2 (four times as many CTAs) for small ones.  The next K slab's
+// operands are loaded into registers while the current slab is multiplied, so a slab costs one barrier pair, not a
+// global-memory round trip.  K is walked in ascending order whatever the tile, so a pixel's bits do not depend on it.
+template <typename T, int TM>
 __global__ void __launch_bounds__(256) conv_simt_kernel(ConvArgs p)
 {
-    __shared__ float As[SM_BK][SM_BM + 4];
-    __shared__ float Bs[SM_BK][SM_BN + 4];
+    constexpr int BM = 16 * TM, BN = 16 * TM;
+    __shared__ float As[SM_BK][BM + 4];
+    __shared__ float Bs[SM_BK][BN + 4];
 
     const T *__restrict__ x = static_cast<const T *>(p.x);
     const T *__restrict__ w = static_cast<const T *>(p.w);
     const int rows = p.oh_hi - p.oh_lo;
     const long long M = (long long)p.N * rows * p.Wo;
     const int K = p.kh * p.kw * p.Cin;
-    const long long m0 = (long long)blockIdx.x * SM_BM;
-    const int n0 = blockIdx.y * SM_BN;
+    const long long m0 = (long long)blockIdx.x * BM;
+    const int n0 = blockIdx.y * BN;
     const int t = threadIdx.x;
     const int kk = t & 15;              // K index inside the slab this thread stages
-    const int lr = t >> 4;              // 0..15: first of the 4 tile rows (stride 16) this thread stages
+    const int lr = t >> 4;              // 0..15: first of the TM tile rows (stride 16) this thread stages
 
-    // the four pixels / four output channels whose operands this thread stages
-    long long xbase[4];
-    int ih0[4], iw0[4];
-    bool mvalid[4];
+    // the TM pixels / TM output channels whose operands this thread stages
+    long long xbase[TM];
+    int ih0[TM], iw0[TM];
+    bool mvalid[TM];
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
+    for (int e = 0; e < TM; ++e) {
         const long long m = m0 + lr + e * 16;
         mvalid[e] = m < M;
         const long long mm = mvalid[e] ? m : 0;
@@ -70,13 +75,15 @@ __global__ void __launch_bounds__(256) conv_simt_kernel(ConvArgs p)
     }
 
     const int tx = t & 15, ty = t >> 4;
-    float acc[4][4];
+    float acc[TM][TM];
 #pragma unroll
-    for (int i = 0; i < 4; ++i)
+    for (int i = 0; i < TM; ++i)
 #pragma unroll
-        for (int j = 0; j < 4; ++j) acc[i][j] = 0.0f;
+        for (int j = 0; j < TM; ++j) acc[i][j] = 0.0f;
 
-    for (int k0 = 0; k0 < K; k0 += SM_BK) {
+    // this thread's operand values of the K slab starting at k0
+    float av[TM], wv[TM];
+    auto load_slab = [&](int k0) {
         const int k = k0 + kk;
         const bool kvalid = k < K;
         int ci = 0, a = 0, b = 0;
@@ -87,31 +94,40 @@ __global__ void __launch_bounds__(256) conv_simt_kernel(ConvArgs p)
             a = tap / p.kw;
         }
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
+        for (int e = 0; e < TM; ++e) {
             float v = 0.0f;
             if (kvalid && mvalid[e]) {
                 const int ih = ih0[e] + a * p.dh, iw = iw0[e] + b * p.dw;
                 if (ih >= 0 && ih < p.Hin && iw >= 0 && iw < p.Win)
                     v = to_f32(x[xbase[e] + ((long long)ih * p.Win + iw) * p.Cin + ci]);
             }
-            As[kk][lr + e * 16] = v;
-            float wv = 0.0f;
+            av[e] = v;
+            float u = 0.0f;
             const int co = n0 + lr + e * 16;
-            if (kvalid && co < p.Cout) wv = to_f32(w[(long long)co * K + k]);
-            Bs[kk][lr + e * 16] = wv;
+            if (kvalid && co < p.Cout) u = to_f32(w[(long long)co * K + k]);
+            wv[e] = u;
+        }
+    };
+    load_slab(0);
+    for (int k0 = 0; k0 < K; k0 += SM_BK) {
+#pragma unroll
+        for (int e = 0; e < TM; ++e) {
+            As[kk][lr + e * 16] = av[e];
+            Bs[kk][lr + e * 16] = wv[e];
         }
         __syncthreads();
+        if (k0 + SM_BK < K) load_slab(k0 + SM_BK);          // in flight while this slab is multiplied
 #pragma unroll
         for (int q = 0; q < SM_BK; ++q) {
-            float av[4], bv[4];
+            float ar[TM], br[TM];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) av[i] = As[q][ty * 4 + i];
+            for (int i = 0; i < TM; ++i) ar[i] = As[q][ty * TM + i];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) bv[j] = Bs[q][tx * 4 + j];
+            for (int j = 0; j < TM; ++j) br[j] = Bs[q][tx * TM + j];
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
+            for (int i = 0; i < TM; ++i)
 #pragma unroll
-                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+                for (int j = 0; j < TM; ++j) acc[i][j] = fmaf(ar[i], br[j], acc[i][j]);
         }
         __syncthreads();
     }
@@ -119,8 +135,8 @@ __global__ void __launch_bounds__(256) conv_simt_kernel(ConvArgs p)
     T *__restrict__ y = static_cast<T *>(p.y);
     const T *__restrict__ res = static_cast<const T *>(p.res);
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const long long m = m0 + ty * 4 + i;
+    for (int i = 0; i < TM; ++i) {
+        const long long m = m0 + ty * TM + i;
         if (m >= M) continue;
         const int ow = (int)(m % p.Wo);
         const long long q = m / p.Wo;
@@ -128,8 +144,8 @@ __global__ void __launch_bounds__(256) conv_simt_kernel(ConvArgs p)
         const int n = (int)(q / rows);
         const long long o = (((long long)n * p.Ho + oh) * p.Wo + ow) * p.Cout;
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int co = n0 + tx * 4 + j;
+        for (int j = 0; j < TM; ++j) {
+            const int co = n0 + tx * TM + j;
             if (co >= p.Cout) continue;
             float v = acc[i][j];
             v = fmaf(p.scale ? p.scale[co] : 1.0f, v, p.shift ? p.shift[co] : 0.0f);
@@ -189,6 +205,56 @@ __global__ void __launch_bounds__(256) maxpool_kernel(PoolArgs p)
     }
 }
 
+// bf16, channels a multiple of 8, a KH x KW window known at compile time: every tap's 16-byte load is issued
+// before the first maximum is taken (four to nine independent loads in flight per thread), one thread per
+// (output pixel, 8-channel group), as many blocks as there is work.
+template <int KH, int KW>
+__global__ void __launch_bounds__(256) maxpool_bf16x8_kernel(PoolArgs p)
+{
+    const int rows = p.oh_hi - p.oh_lo;
+    const int cg = p.C >> 3;
+    const long long total = (long long)p.N * rows * p.Wo * cg;
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= total) return;
+    const uint4 *__restrict__ x = static_cast<const uint4 *>(p.x);
+    const int g = (int)(idx % cg);
+    long long q = idx / cg;
+    const int ow = (int)(q % p.Wo);
+    q /= p.Wo;
+    const int oh = p.oh_lo + (int)(q % rows);
+    const int n = (int)(q / rows);
+    uint4 v[KH * KW];
+    bool ok[KH * KW];
+#pragma unroll
+    for (int a = 0; a < KH; ++a) {
+        const int ih = oh * p.sh - p.ph + a * p.dh;
+#pragma unroll
+        for (int b = 0; b < KW; ++b) {
+            const int iw = ow * p.sw - p.pw + b * p.dw;
+            ok[a * KW + b] = ih >= 0 && ih < p.Hin && iw >= 0 && iw < p.Win;
+            if (ok[a * KW + b]) v[a * KW + b] = __ldg(x + (((long long)n * p.Hin + ih) * p.Win + iw) * cg + g);
+        }
+    }
+    float m[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) m[i] = -INFINITY;
+#pragma unroll
+    for (int tpos = 0; tpos < KH * KW; ++tpos)
+        if (ok[tpos]) {
+            const uint32_t w4[4] = {v[tpos].x, v[tpos].y, v[tpos].z, v[tpos].w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                m[2 * i] = fmaxf(m[2 * i], __uint_as_float(w4[i] << 16));
+                m[2 * i + 1] = fmaxf(m[2 * i + 1], __uint_as_float(w4[i] & 0xFFFF0000u));
+            }
+        }
+    uint32_t o[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)                      // the values are bf16 already: dropping the low half is exact
+        o[i] = (__float_as_uint(m[2 * i]) >> 16) | (__float_as_uint(m[2 * i + 1]) & 0xFFFF0000u);
+    static_cast<uint4 *>(p.y)[(((long long)n * p.Ho + oh) * p.Wo + ow) * cg + g] = make_uint4(o[0], o[1], o[2], o[3]);
+}
+
 // ---------------------------------------------------------------------------------------------
 // Patch gather for a thin chain input, rows [lo, hi) of the patch tensor (see lop_gather.cuh).
 // One thread per 16-byte group of eight patch elements: consecutive threads write consecutive
@@ -239,9 +305,16 @@ cudaError_t launch_conv_simt(const ConvArgs &a, int dtype, cudaStream_t s)
     const int rows = a.oh_hi - a.oh_lo;
     if (rows <= 0) return cudaSuccess;
     const long long M = (long long)a.N * rows * a.Wo;
-    dim3 grid((unsigned)((M + SM_BM - 1) / SM_BM), (unsigned)((a.Cout + SM_BN - 1) / SM_BN));
-    if (dtype == LOP_BF16) conv_simt_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>(a);
-    else conv_simt_kernel<float><<<grid, 256, 0, s>>>(a);
+    const long long big_tiles = ((M + 63) / 64) * ((a.Cout + 63) / 64);
+    if (big_tiles >= 2 * 148) {
+        dim3 grid((unsigned)((M + 63) / 64), (unsigned)((a.Cout + 63) / 64));
+        if (dtype == LOP_BF16) conv_simt_kernel<__nv_bfloat16, 4><<<grid, 256, 0, s>>>(a);
+        else conv_simt_kernel<float, 4><<<grid, 256, 0, s>>>(a);
+    } else {
+        dim3 grid((unsigned)((M + 31) / 32), (unsigned)((a.Cout + 31) / 32));
+        if (dtype == LOP_BF16) conv_simt_kernel<__nv_bfloat16, 2><<<grid, 256, 0, s>>>(a);
+        else conv_simt_kernel<float, 2><<<grid, 256, 0, s>>>(a);
+    }
     return cudaGetLastError();
 }
 
@@ -251,7 +324,12 @@ cudaError_t launch_maxpool(const PoolArgs &a, int dtype, cudaStream_t s)
     if (rows <= 0) return cudaSuccess;
     const long long pix = (long long)a.N * rows * a.Wo;
     if (dtype == LOP_BF16) {
-        if (a.C % 8 == 0) maxpool_kernel<__nv_bfloat16, 8><<<grid_for(pix * (a.C / 8), 256), 256, 0, s>>>(a);
+        const long long vecs = pix * (a.C / 8);
+        const bool aligned = (reinterpret_cast<uintptr_t>(a.x) & 15) == 0 && (reinterpret_cast<uintptr_t>(a.y) & 15) == 0;
+        const unsigned blocks = (unsigned)((vecs + 255) / 256);
+        if (a.C % 8 == 0 && aligned && vecs < (1LL << 38) && a.kh == 2 && a.kw == 2) maxpool_bf16x8_kernel<2, 2><<<blocks, 256, 0, s>>>(a);
+        else if (a.C % 8 == 0 && aligned && vecs < (1LL << 38) && a.kh == 3 && a.kw == 3) maxpool_bf16x8_kernel<3, 3><<<blocks, 256, 0, s>>>(a);
+        else if (a.C % 8 == 0) maxpool_kernel<__nv_bfloat16, 8><<<grid_for(pix * (a.C / 8), 256), 256, 0, s>>>(a);
         else maxpool_kernel<__nv_bfloat16, 1><<<grid_for(pix * a.C, 256), 256, 0, s>>>(a);
     } else {
         if (a.C % 4 == 0) maxpool_kernel<float, 4><<<grid_for(pix * (a.C / 4), 256), 256, 0, s>>>(a);

@@ -1,0 +1,62 @@
+"""Runs one named case of the library a few times, for captures under a profiler.
+
+    python -m paper_2507_05829_b200.profile_case <case> [launches]
+
+Cases: a named workload (``vgg_block``, ``resnet18``, ``resnet50``, ``csp_stack``: all bands from a device-resident
+input, one persistent launch per run; ``<name>:pipelined`` streams the bands from pinned host memory), ``pool`` (a
+3x3 stride-2 max pooling of an 8 x 224 x 224 x 64 bf16 tensor by the stand-alone kernel and, with ``pool:persistent``,
+by pooling items of the persistent kernel), ``gather`` (patch gather + 7x7 stride-2 stem convolution of 8 images by
+the stand-alone kernels; ``gather:persistent`` inside the persistent kernel).  The L2 is flushed before every run.
+"""
+import sys
+
+import torch
+
+import lop_inputs as li
+from lop_inputs.workloads import Segment, Workload, conv, pool
+
+from . import binding as B
+from .chain import DeviceChain
+
+
+def build_case(name):
+    base, _, mode = name.partition(":")
+    if base in ("vgg_block", "resnet18", "resnet50", "csp_stack", "single_conv"):
+        return li.build(base), (mode or "banded"), 0
+    if base == "pool":
+        l = pool(64, 3, 2, 1)
+        l.input_from = -1
+        wl = Workload("pool_only", "bf16", 8, 224, 224, 64, [Segment([l], 1)], seed=1)
+    elif base == "gather":
+        l = conv(3, 64, 7, s=2, p=3, act=li.ACT_RELU)
+        l.input_from = -1
+        wl = Workload("stem_only", "bf16", 8, 224, 224, 3, [Segment([l], 1)], seed=1)
+    else:
+        raise SystemExit("unknown case %r" % name)
+    li.fill_parameters(wl)
+    li.make_input(wl)
+    return wl, "whole", (0 if mode == "persistent" else B.LOP_FLAG_PER_LAYER)
+
+
+def main():
+    name = sys.argv[1] if len(sys.argv) > 1 else "resnet50"
+    launches = int(sys.argv[2]) if len(sys.argv) > 2 else 3
+    wl, mode, flags = build_case(name)
+    dc = DeviceChain(wl, flags=B.LOP_FLAG_REUSE_HALO | flags)
+    x_dev, x_pin = dc.input_tensor(), dc.pinned_input()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    for _ in range(launches):
+        flush.zero_()
+        if mode == "pipelined":
+            dc.run_pipelined(x_pin)
+        elif mode == "whole":
+            dc.run_whole(x_dev)
+        else:
+            dc.run_banded(x_dev)
+        torch.cuda.synchronize()
+    dc.check_device()
+    print("%s: %d run(s) of mode %s, %d launch(es) of the library's kernels per run" % (name, launches, mode, dc.launches()))
+
+
+if __name__ == "__main__":
+    main()
