@@ -45,7 +45,7 @@ typedef enum {
 } lop_status;
 
 enum { LOP_F32 = 0, LOP_BF16 = 1 };                         /* storage dtype                     */
-enum { LOP_CONV2D = 0, LOP_MAXPOOL2D = 1 };
+enum { LOP_CONV2D = 0, LOP_MAXPOOL2D = 1, LOP_LINEAR = 2 };
 enum { LOP_ACT_NONE = 0, LOP_ACT_RELU = 1, LOP_ACT_SILU = 2 };
 enum { LOP_RES_NONE = 0, LOP_RES_PRE_ACT = 1, LOP_RES_POST_ACT = 2 };
 enum { LOP_INPUT = -1, LOP_NO_RESIDUAL = -2 };              /* special layer indices             */
@@ -68,6 +68,10 @@ enum {
  *   t = scale[co]*acc + shift[co];  RES_PRE_ACT: t += r;  t = act(t);  RES_POST_ACT: t += r
  * with taps outside the input contributing zero.  Max pooling takes the maximum over the
  * in-bounds taps (padding never wins); cout must equal cin; act/residual are ignored.
+ * LOP_LINEAR is the row-wise operator of Sec. IV-A (Eq. 1): Y = X * W^T with the parameter matrix shared by every
+ * row; here every pixel's channel vector is a row of X, weight is [cout][cin], the epilogue is the convolution's,
+ * and a band's rows depend on the same rows of the input and on nothing else.  Its window fields must be
+ * kh = kw = sh = sw = dh = dw = 1, ph = pw = 0.
  * input_from / residual_from name an earlier layer of the same list, or LOP_INPUT for the
  * chain input; residual_from == LOP_NO_RESIDUAL means none.  The list order is topological.
  * The three pointers are DEVICE pointers; they are stored, never dereferenced on the host,

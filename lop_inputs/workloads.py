@@ -23,7 +23,7 @@ import numpy as np
 
 from . import rng
 
-CONV, POOL = 0, 1
+CONV, POOL, LINEAR = 0, 1, 2
 ACT_NONE, ACT_RELU, ACT_SILU = 0, 1, 2
 RES_NONE, RES_PRE_ACT, RES_POST_ACT = 0, 1, 2
 NO_RESIDUAL = -2
@@ -80,6 +80,11 @@ def conv(cin, cout, k, s=1, p=None, d=1, act=ACT_RELU, input_from=None, residual
     return Layer(CONV, cin, cout, k, k, s, s, p, p, d, d, act, input_from, residual_from, residual_pos)
 
 
+def linear(cin, cout, act=ACT_NONE, input_from=None, residual_from=NO_RESIDUAL, residual_pos=RES_NONE):
+    """The row-wise operator of Sec. IV-A (Eq. 1): every pixel's channel vector times a shared [cout, cin] matrix."""
+    return Layer(LINEAR, cin, cout, 1, 1, 1, 1, 0, 0, 1, 1, act, input_from, residual_from, residual_pos)
+
+
 def pool(c, k, s, p=0, input_from=None):
     return Layer(POOL, c, c, k, k, s, s, p, p, 1, 1, ACT_NONE, input_from)
 
@@ -98,7 +103,7 @@ def fill_parameters(wl: Workload):
     stream = 16
     for seg in wl.segments:
         for l in seg.layers:
-            if l.op == CONV:
+            if l.op in (CONV, LINEAR):
                 fan_in = l.kh * l.kw * l.cin
                 w = rng.normal(wl.seed, stream, (l.cout, l.kh, l.kw, l.cin), 0.0, float(np.sqrt(2.0 / fan_in)))
                 l.weight = rng.round_to_bf16(w) if bf16 else w
@@ -211,12 +216,21 @@ def csp_stack(N=1, H=1024, W=1024, n_bands=32, dtype="bf16", seed=505, base=32):
     return wl
 
 
+def pointwise_mlp(N=2, H=56, W=56, C=128, hidden=512, n_bands=8, dtype="bf16", seed=606):
+    """Row-wise local operators only (Sec. IV-A, Eq. 1), shaped like the point-wise MLP of a ConvNeXt block: every
+    pixel's channel vector through  linear(C -> hidden) + SiLU,  linear(hidden -> C) + shortcut.  Rows map one to one
+    through both layers, so bands need no halo at all."""
+    layers = [linear(C, hidden, act=ACT_SILU), linear(hidden, C, act=ACT_NONE, residual_from=-1, residual_pos=RES_POST_ACT)]
+    return Workload("pointwise_mlp", dtype, N, H, W, C, [Segment(_chain(layers), n_bands)], seed=seed)
+
+
 WORKLOADS = {
     "single_conv": single_conv,
     "vgg_block": vgg_block,
     "resnet18": resnet18,
     "resnet50": resnet50,
     "csp_stack": csp_stack,
+    "pointwise_mlp": pointwise_mlp,
 }
 
 

@@ -17,6 +17,8 @@ POISON = np.float32(np.inf)
 
 def run_layer(l, src, res, rows, round_bf16, out):
     """Rows ``rows`` of layer ``l`` applied to the full-size tensor ``src`` (residual ``res``) into ``out``."""
+    if l.op == 2:                       # row-wise operator (Sec. IV-A, Eq. 1): rows map one to one
+        return ops.linear(src, l.weight, l.scale, l.shift, res, l.residual_pos if res is not None else 0, l.act, round_bf16, rows, out)
     if l.op == 0:
         return ops.conv2d(src, l.weight, (l.sh, l.sw), (l.ph, l.pw), (l.dh, l.dw), l.scale, l.shift,
                           res, l.residual_pos if res is not None else 0, l.act, round_bf16, rows, out)
@@ -132,7 +134,7 @@ def flops(wl):
     for seg in wl.segments:
         shapes = planner.infer_shapes(seg.layers, H, W, C)
         for l, (h, w, c) in zip(seg.layers, shapes):
-            if l.op == 0:
+            if l.op in (0, 2):
                 total += 2 * wl.N * h * w * c * l.kh * l.kw * l.cin
         H, W, C = shapes[-1]
     return total

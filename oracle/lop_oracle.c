@@ -121,6 +121,33 @@ void lop_oracle_maxpool2d(const float *x, int N, int H, int W, int C,
                 }
 }
 
+/*
+ * Row-wise local operator (Sec. IV-A, Eq. 1 of the paper): Y = X * W^T, every row of X multiplied by the same
+ * parameter matrix W, so a block of rows of Y depends on the same block of rows of X and on nothing else.
+ * x: [M][K], w: [Cout][K], y: [M][Cout], all row-major; rows [r_lo, r_hi) of y are computed, the others left alone.
+ * Accumulation in double over k ascending; epilogue as for the convolution (res has y's shape).
+ */
+void lop_oracle_linear(const float *x, long long M, int K, const float *w, int Cout,
+                       const float *scale, const float *shift, const float *res, int res_pos, int act,
+                       int round_bf16, long long r_lo, long long r_hi, float *y)
+{
+    if (r_lo < 0) r_lo = 0;
+    if (r_hi > M) r_hi = M;
+#pragma omp parallel for schedule(dynamic, 16)
+    for (long long r = r_lo; r < r_hi; ++r)
+        for (int co = 0; co < Cout; ++co) {
+            double acc = 0.0;
+            for (int k = 0; k < K; ++k) acc += (double)x[(size_t)r * K + k] * (double)w[(size_t)co * K + k];
+            const size_t o = (size_t)r * Cout + co;
+            float t = (float)acc;
+            t = (scale ? scale[co] : 1.0f) * t + (shift ? shift[co] : 0.0f);
+            if (res && res_pos == 1) t += res[o];
+            t = activate(t, act);
+            if (res && res_pos == 2) t += res[o];
+            y[o] = round_bf16 ? lop_oracle_bf16_rne(t) : t;
+        }
+}
+
 int lop_oracle_num_threads(void)
 {
 #ifdef _OPENMP

@@ -17,6 +17,7 @@ def lib():
         _lib.lop_oracle_num_threads.restype = ctypes.c_int
         _lib.lop_oracle_conv2d.restype = None
         _lib.lop_oracle_maxpool2d.restype = None
+        _lib.lop_oracle_linear.restype = None
     return _lib
 
 
@@ -74,4 +75,29 @@ def maxpool2d(x, k, stride, pad=(0, 0), dil=(1, 1), rows=None, out=None):
     lo, hi = (0, Ho) if rows is None else rows
     lib().lop_oracle_maxpool2d(_fp(x), N, H, W, C, k[0], k[1], stride[0], stride[1], pad[0], pad[1],
                                dil[0], dil[1], int(lo), int(hi), _fp(out))
+    return out
+
+
+def linear(x, w, scale=None, shift=None, res=None, res_pos=0, act=0, round_bf16=False, rows=None, out=None):
+    """The row-wise operator Y = X W^T (Sec. IV-A, Eq. 1) on an NHWC tensor: every pixel's channel vector is a row of X.
+
+    ``w``: [Cout, K] (or [Cout, 1, 1, K]).  ``rows=(lo, hi)``: image rows of every image to compute (default all); the
+    matrix rows they stand for are  (n*H + h)*W .. for h in [lo, hi)."""
+    x, w = _f32(x), _f32(w)
+    N, H, W, K = x.shape
+    w2 = w.reshape(w.shape[0], -1)
+    Cout = w2.shape[0]
+    assert w2.shape[1] == K
+    if out is None:
+        out = np.zeros((N, H, W, Cout), dtype=np.float32)
+    assert out.shape == (N, H, W, Cout) and out.dtype == np.float32 and out.flags.c_contiguous
+    scale, shift, res = _f32(scale), _f32(shift), _f32(res)
+    if res is not None:
+        assert res.shape == out.shape
+    lo, hi = (0, H) if rows is None else rows
+    M = N * H * W
+    for n in range(N):
+        lib().lop_oracle_linear(_fp(x), ctypes.c_longlong(M), K, _fp(w2), Cout, _fp(scale), _fp(shift), _fp(res), int(res_pos),
+                                int(act), int(bool(round_bf16)), ctypes.c_longlong((n * H + lo) * W),
+                                ctypes.c_longlong((n * H + hi) * W), _fp(out))
     return out

@@ -51,6 +51,8 @@ def infer_shapes(layers, H, W, C):
         hin, win, cin = shape_of(l.input_from)
         if cin != l.cin:
             raise PlanError("layer %d: cin %d but its input has %d channels" % (i, l.cin, cin))
+        if l.op == 2 and (l.kh, l.kw, l.sh, l.sw, l.ph, l.pw, l.dh, l.dw) != (1, 1, 1, 1, 0, 0, 1, 1):
+            raise PlanError("layer %d: a row-wise operator has no window" % i)
         if l.op == 1 and l.cout != l.cin:
             raise PlanError("layer %d: pooling keeps the channel count" % i)
         ho = out_extent(hin, l.kh, l.sh, l.ph, l.dh)
@@ -60,7 +62,7 @@ def infer_shapes(layers, H, W, C):
         if l.residual_from != NO_RESIDUAL:
             if not (-1 <= l.residual_from < i):
                 raise PlanError("layer %d: residual_from must name the segment input or an earlier layer" % i)
-            if l.op != 0 or l.residual_pos not in (1, 2):
+            if l.op not in (0, 2) or l.residual_pos not in (1, 2):
                 raise PlanError("layer %d: a residual needs a convolution and a position" % i)
             if shape_of(l.residual_from) != (ho, wo, l.cout):
                 raise PlanError("layer %d: residual shape mismatch" % i)

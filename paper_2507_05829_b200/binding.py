@@ -8,7 +8,7 @@ from . import build as _build
 LIB_PATH = _build.LIB
 
 LOP_F32, LOP_BF16 = 0, 1
-LOP_CONV2D, LOP_MAXPOOL2D = 0, 1
+LOP_CONV2D, LOP_MAXPOOL2D, LOP_LINEAR = 0, 1, 2
 LOP_ACT_NONE, LOP_ACT_RELU, LOP_ACT_SILU = 0, 1, 2
 LOP_RES_NONE, LOP_RES_PRE_ACT, LOP_RES_POST_ACT = 0, 1, 2
 LOP_INPUT, LOP_NO_RESIDUAL = -1, -2

@@ -17,6 +17,7 @@ struct LayerInfo {
     int Ho = 0, Wo = 0, Co = 0;    // output shape
     int kernel = K_CONV_SIMT;
     int cin_eff = 0;               // channels the tensor-core kernel sees (= the patch length Kcol for a gathered stem)
+    bool linear = false;           // given as the row-wise operator LOP_LINEAR (runs as the pointwise convolution it is)
     bool stem_gather = false;      // thin chain input: the layer's receptive patches are gathered into a
                                    // [N, Ho, Wo, Kcol] tensor first and the convolution runs as 1x1 over it
     size_t out_off = 0;            // workspace offset of the full-size output (unused for the last layer)

@@ -93,8 +93,19 @@ static int check_layers(lop_plan_t &pl)
     const int L = (int)pl.layers.size();
     for (int i = 0; i < L; ++i) {
         LayerInfo &li = pl.layers[i];
+        if (li.l.op != LOP_CONV2D && li.l.op != LOP_MAXPOOL2D && li.l.op != LOP_LINEAR) { set_error("layer %d: unknown op %d", i, li.l.op); return LOP_EINVAL; }
+        if (li.l.op == LOP_LINEAR) {
+            const lop_layer &q = li.l;
+            if (q.kh != 1 || q.kw != 1 || q.sh != 1 || q.sw != 1 || q.dh != 1 || q.dw != 1 || q.ph != 0 || q.pw != 0) {
+                set_error("layer %d: a row-wise operator has no window (kh = kw = sh = sw = dh = dw = 1, ph = pw = 0)", i);
+                return LOP_EINVAL;
+            }
+            // Y = X * W^T over the channel vectors of the pixels is the pointwise convolution with the same [cout][cin]
+            // matrix: from here on the layer is planned and executed as one (rows map one to one, no halo)
+            li.linear = true;
+            li.l.op = LOP_CONV2D;
+        }
         const lop_layer &l = li.l;
-        if (l.op != LOP_CONV2D && l.op != LOP_MAXPOOL2D) { set_error("layer %d: unknown op %d", i, l.op); return LOP_EINVAL; }
         if (l.kh < 1 || l.kw < 1 || l.sh < 1 || l.sw < 1 || l.dh < 1 || l.dw < 1 || l.ph < 0 || l.pw < 0 ||
             l.cin < 1 || l.cout < 1) {
             set_error("layer %d: kernel/stride/dilation must be >= 1, padding >= 0, channels >= 1", i);

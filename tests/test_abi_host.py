@@ -106,3 +106,18 @@ def test_errors_are_reported_not_raised_in_c():
     assert L.lop_run_whole(p._h, None, None, None, None) == -1
     assert L.lop_run_band(p._h, 0, ctypes.c_void_p(16), ctypes.c_void_p(16), None, None) == -6
     assert L.lop_copy_band(p._h, 5, ctypes.c_void_p(16), ctypes.c_void_p(16), None) == -1
+
+
+def test_row_wise_operator_must_not_carry_a_window():
+    ok = li.linear(8, 16)
+    ok.input_from = -1
+    p = lop.Plan([ok], 1, 6, 5, 8, lop.LOP_BF16, 3)
+    assert p.out_shape(0) == (6, 5, 16) and p.layer_kernel(0) == 2         # runs on the tensor-core pointwise path
+    assert p.flops() == 2.0 * 6 * 5 * 16 * 8
+    for field, val in (("kh", 3), ("sw", 2), ("ph", 1), ("dh", 2)):
+        bad = li.linear(8, 16)
+        bad.input_from = -1
+        setattr(bad, field, val)
+        with pytest.raises(lop.LopError) as e:
+            lop.Plan([bad], 1, 6, 5, 8, lop.LOP_BF16, 3)
+        assert e.value.status == -1 and "row-wise" in str(e.value)

@@ -197,7 +197,8 @@ def test_maxpool(dtype, C, k, s, p):
 
 # ------------------------------------------------------------------------------------ chains, reduced sizes
 SMALL = [("vgg_block", dict(H=44, W=36)), ("resnet18", dict(H=64, W=64)),
-         ("resnet50", dict(N=2, H=64, W=64, depths=(2, 2, 2, 2))), ("csp_stack", dict(H=256, W=128))]
+         ("resnet50", dict(N=2, H=64, W=64, depths=(2, 2, 2, 2))), ("csp_stack", dict(H=256, W=128)),
+         ("pointwise_mlp", dict(H=21, W=19, C=64, hidden=192, n_bands=4))]      # row-wise operators (Sec. IV-A, Eq. 1)
 
 
 @pytest.mark.parametrize("name,kw", SMALL)
@@ -665,7 +666,7 @@ def test_wavefront_and_per_layer_executors_agree_bit_for_bit():
 
 
 # ------------------------------------------------------------------------------------ the named configurations, full size
-@pytest.mark.parametrize("name", ["vgg_block", "resnet18", "csp_stack"])
+@pytest.mark.parametrize("name", ["vgg_block", "resnet18", "csp_stack", "pointwise_mlp"])
 def test_named_configurations_full_size(name):
     check_workload(li.build(name), flags=lop.LOP_FLAG_REUSE_HALO, modes=("whole", "pipelined", "pipelined_copy"))
 

@@ -243,3 +243,51 @@ def test_pool_matches_naive_and_library(k, s, p, d):
     assert np.array_equal(y, want)
     t = F.max_pool2d(torch.from_numpy(x).permute(0, 3, 1, 2), k, s, p, d).permute(0, 2, 3, 1).numpy()
     assert np.array_equal(y, t)
+
+
+# ----------------------------------------------------------------------------- row-wise operator (Sec. IV-A, Eq. 1)
+def test_linear_equals_a_float64_matrix_product():
+    rnd = np.random.default_rng(21)
+    x = rnd.standard_normal((2, 5, 7, 19)).astype(np.float32)
+    w = rnd.standard_normal((11, 19)).astype(np.float32)
+    y = ops.linear(x, w)
+    want = (x.reshape(-1, 19).astype(np.float64) @ w.astype(np.float64).T).reshape(2, 5, 7, 11)
+    assert np.max(np.abs(y - want)) <= 1e-6 * np.max(np.abs(want))
+
+
+def test_linear_with_the_identity_matrix_returns_its_input_and_transposition_matters():
+    rnd = np.random.default_rng(22)
+    x = rnd.standard_normal((1, 3, 4, 6)).astype(np.float32)
+    assert np.array_equal(ops.linear(x, np.eye(6, dtype=np.float32)), x)
+    w = np.zeros((6, 6), dtype=np.float32)
+    w[2, 5] = 1.0                                    # output channel 2 reads input channel 5 (W is [cout][cin])
+    y = ops.linear(x, w)
+    assert np.array_equal(y[..., 2], x[..., 5]) and not y[..., [0, 1, 3, 4, 5]].any()
+
+
+def test_linear_row_blocks_computed_apart_stack_to_the_whole():
+    """Eq. 1: the rows of X may be partitioned freely, the parameter matrix is shared, nothing is summed across blocks."""
+    rnd = np.random.default_rng(23)
+    x = rnd.standard_normal((2, 9, 5, 8)).astype(np.float32)
+    w = rnd.standard_normal((4, 8)).astype(np.float32)
+    sc, sh = rnd.standard_normal(4).astype(np.float32), rnd.standard_normal(4).astype(np.float32)
+    whole = ops.linear(x, w, sc, sh, act=2)
+    parts = np.full_like(whole, np.inf)
+    for lo, hi in ((0, 2), (2, 3), (3, 9)):
+        ops.linear(x, w, sc, sh, act=2, rows=(lo, hi), out=parts)
+        assert np.all(np.isinf(parts[:, hi:]))       # rows outside the block are left alone
+    assert np.array_equal(parts, whole)
+
+
+def test_linear_is_the_pointwise_convolution_and_shares_its_epilogue():
+    rnd = np.random.default_rng(24)
+    x = rnd.standard_normal((2, 4, 6, 10)).astype(np.float32)
+    w = rnd.standard_normal((7, 10)).astype(np.float32)
+    sc, sh = rnd.standard_normal(7).astype(np.float32), rnd.standard_normal(7).astype(np.float32)
+    res = rnd.standard_normal((2, 4, 6, 7)).astype(np.float32)
+    for pos in (1, 2):
+        a = ops.linear(x, w, sc, sh, res, pos, act=1, round_bf16=True)
+        b = ops.conv2d(x, w.reshape(7, 1, 1, 10), scale=sc, shift=sh, res=res, res_pos=pos, act=1, round_bf16=True)
+        assert np.array_equal(a, b)
+    lin = ops.linear(x, w)                           # linear in x
+    assert np.allclose(ops.linear(2.0 * x, w), 2.0 * lin, rtol=1e-6, atol=1e-6)

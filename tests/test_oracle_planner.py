@@ -364,3 +364,20 @@ def test_flops_of_the_named_workloads():
     assert chain.flops(li.build("single_conv", with_data=False)) == 2 * 32 * 32 * 16 * 144
     v = chain.flops(li.build("vgg_block", with_data=False))
     assert v == 2 * 224 * 224 * 64 * (27 + 576)
+
+
+def test_row_wise_operators_need_no_halo():
+    """Sec. IV-A, Eq. 1: a block of output rows of a row-wise operator depends on the same rows of its input."""
+    wl = li.build("pointwise_mlp", with_data=False)
+    seg = wl.segments[0]
+    plan = planner.make_plan(seg.layers, wl.H, wl.W, wl.C, seg.n_bands)
+    for b in range(seg.n_bands):
+        band = ((b * wl.H) // seg.n_bands, ((b + 1) * wl.H) // seg.n_bands)
+        for i in range(len(seg.layers)):
+            r = plan.ranges[b][i]
+            assert (r.out_lo, r.out_hi) == band and rows_of(r) == band and r.pad_top == 0 and r.pad_bot == 0
+        assert plan.input_need[b][:2] == band
+    bad = li.linear(8, 8)
+    bad.input_from, bad.kh = -1, 3
+    with pytest.raises(planner.PlanError):
+        planner.make_plan([bad], 8, 8, 8, 2)
