@@ -165,6 +165,13 @@ int lop_run_banded(lop_plan_t *plan, const void *in_dev, void *out_dev, void *wo
  * the chain-input rows the band needs and no earlier band has brought, for all N images, from
  * in_host_pinned (PINNED HOST, full-size tensor) to the same rows of staging_dev. */
 int lop_copy_band(lop_plan_t *plan, int band, const void *in_host_pinned, void *staging_dev, void *stream);
+/* Rows [row_lo, row_hi) of ONE layer: the operator-level step of the paper's runtime loop (Sec. IV-D, Alg. 1 / 2: for
+ * each layer, compute its local operations, then send / receive rows along its edges).  One kernel launch of the
+ * per-layer kernels; the layer's input (and residual) rows it reads must be present in the tensors the other calls
+ * use (in_dev, the workspace, out_dev for the last layer).  The building block of the halo-exchange form of band
+ * sharding, where neighbouring devices trade halo rows between layers instead of recomputing them. */
+int lop_run_layer(lop_plan_t *plan, int layer, int row_lo, int row_hi, const void *in_dev, void *out_dev, void *workspace,
+                  void *stream);
 /* ---- band sharding over several devices (Sec. IV-C: operation replication) ---------------------
  * Bands that carry their halo are independent units: device `rank` of `world` takes the contiguous
  * block of bands  [floor(rank*B/world), floor((rank+1)*B/world)), runs it with lop_run_shard on its own

@@ -18,7 +18,7 @@ LOP_FLAG_REUSE_HALO, LOP_FLAG_TIME_LAYERS, LOP_FLAG_FORCE_SIMT, LOP_FLAG_PER_LAY
 EXPORTS = [
     "lop_plan", "lop_plan_destroy", "lop_plan_num_bands", "lop_plan_num_layers", "lop_plan_get_range",
     "lop_plan_out_shape", "lop_plan_set_params", "lop_plan_workspace_bytes", "lop_plan_staging_bytes",
-    "lop_plan_flops", "lop_run_whole", "lop_run_band", "lop_run_banded", "lop_copy_band", "lop_fetch_band", "lop_run_pipelined",
+    "lop_plan_flops", "lop_run_whole", "lop_run_band", "lop_run_layer", "lop_run_banded", "lop_copy_band", "lop_fetch_band", "lop_run_pipelined",
     "lop_plan_last_timing", "lop_plan_layer_time", "lop_plan_layer_kernel", "lop_plan_last_launches", "lop_plan_last_copies",
     "lop_plan_check_device", "lop_plan_set_wait_limit", "lop_run_pipelined_withheld", "lop_plan_layer_offset", "lop_plan_layer_stored", "lop_run_whole_static", "lop_run_chain_banded", "lop_run_chain_pipelined", "lop_plan_shard", "lop_run_shard",
     "lop_strerror", "lop_last_error",
@@ -82,6 +82,7 @@ def lib():
     L.lop_plan_flops.restype = c_double
     L.lop_run_whole.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
     L.lop_run_band.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_void_p]
+    L.lop_run_layer.argtypes = [c_void_p, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p, c_void_p]
     L.lop_run_banded.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
     L.lop_copy_band.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_void_p]
     L.lop_fetch_band.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_void_p]
@@ -196,6 +197,9 @@ class Plan:
 
     def run_band(self, band, in_dev, out_dev, ws, stream):
         _check(lib().lop_run_band(self._h, band, in_dev, out_dev, ws, stream))
+
+    def run_layer(self, layer, row_lo, row_hi, in_dev, out_dev, ws, stream):
+        _check(lib().lop_run_layer(self._h, layer, row_lo, row_hi, in_dev, out_dev, ws, stream))
 
     def run_banded(self, in_dev, out_dev, ws, stream):
         _check(lib().lop_run_banded(self._h, in_dev, out_dev, ws, stream))

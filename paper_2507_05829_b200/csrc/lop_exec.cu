@@ -624,6 +624,20 @@ int lop_run_banded(lop_plan_t *pl, const void *in, void *out, void *ws, void *st
     return LOP_OK;
 }
 
+int lop_run_layer(lop_plan_t *pl, int layer, int row_lo, int row_hi, const void *in, void *out, void *ws, void *stream)
+{
+    int rc = check_common(pl, in, out, ws);
+    if (rc != LOP_OK) return rc;
+    const int L = (int)pl->layers.size();
+    if (layer < 0 || layer >= L) { set_error("lop_run_layer: layer %d out of range", layer); return LOP_EINVAL; }
+    if (row_lo < 0 || row_hi > pl->layers[layer].Ho || row_lo > row_hi) { set_error("lop_run_layer: rows [%d,%d) out of range", row_lo, row_hi); return LOP_EINVAL; }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    pl->exec->launches = pl->exec->copies = 0;
+    pl->exec->last_stream = s;
+    if ((rc = prepare_workspace(pl, ws, s)) != LOP_OK) return rc;
+    return run_layer(pl, layer, row_lo, row_hi, in, out, ws, s, -1);
+}
+
 int lop_plan_shard(const lop_plan_t *pl, int rank, int world, int *band_lo, int *band_hi, int *row_lo, int *row_hi, int *in_lo,
                    int *in_hi)
 {

@@ -69,3 +69,137 @@ class ShardedChain:
                 all_gather_rows(out, table, self.rank, self.group)
                 x_dev = out
         return dc.outs[-1]
+
+
+# ---------------------------------------------------------------------------------------------------------------------
+# Halo exchange: the other side of the paper's trade between replication and transmission (Sec. IV-C).  Instead of
+# recomputing the halo rows of every intermediate tensor, each rank computes every row of every layer exactly ONCE and
+# the ranks trade the few rows a neighbour's receptive field reaches into, layer by layer -- the per-layer loop of the
+# paper's runtime (Sec. IV-D, Alg. 1 / 2: compute the layer's local operations, then Send / Receive along its edges).
+#
+# Who computes what: rank r owns the bands [b_lo, b_hi) of lop_plan_shard.  At layer i it computes the rows
+# [new_lo of its first band, out_hi of its last band) of a reuse-halo plan -- what its bands need and no lower rank has
+# produced -- so the ranks' rows tile every layer.  Its upper halo it computes itself (it is part of those rows); the
+# rows below its own that its taps reach were computed by lower ranks and are received from them before the layer runs.
+# ---------------------------------------------------------------------------------------------------------------------
+def owned_rows(plan, layer, table, rank):
+    """Rows [lo, hi) of ``layer``'s output (``-1``: the plan's input) that ``rank`` computes (for the input: holds)."""
+    b_lo, b_hi = table[rank][0], table[rank][1]
+    lo = hi = None
+    for b in range(b_lo, b_hi):
+        r = plan.get_range(b, layer)
+        if r.out_hi <= r.out_lo:
+            continue
+        first = r.out_lo if layer == -1 else r.new_lo          # the chain input comes from the host, halo included
+        lo = first if lo is None else min(lo, first)
+        hi = r.out_hi if hi is None else max(hi, r.out_hi)
+    return (0, 0) if lo is None else (lo, hi)
+
+
+def rows_read(layer_desc, lo, hi, h_in):
+    """Input rows the output rows [lo, hi) of a window operator reach (the analytic receptive range, cut to the tensor)."""
+    if hi <= lo:
+        return (0, 0)
+    a = lo * layer_desc.sh - layer_desc.ph
+    b = (hi - 1) * layer_desc.sh - layer_desc.ph + (layer_desc.kh - 1) * layer_desc.dh + 1
+    a, b = max(a, 0), min(b, h_in)
+    return (a, b) if a < b else (0, 0)
+
+
+class MailboxTransport:
+    """send / recv between ranks that live in one process and take turns (tests, one-GPU emulation)."""
+
+    def __init__(self):
+        self.box = {}
+        self.bytes_sent = 0
+
+    def send(self, src, dst, tag, tensor):
+        self.box[(src, dst, tag)] = tensor.clone()
+        self.bytes_sent += tensor.numel() * tensor.element_size()
+
+    def recv(self, src, dst, tag, out):
+        out.copy_(self.box.pop((src, dst, tag)))
+
+    def flush(self):
+        pass
+
+
+class DistTransport:
+    """send / recv over torch.distributed point-to-point calls (NCCL for CUDA tensors, gloo for CPU tensors)."""
+
+    def __init__(self, group=None):
+        self.group, self.pending, self.bytes_sent = group, [], 0
+
+    def send(self, src, dst, tag, tensor):
+        t = tensor.contiguous()
+        self.pending.append((dist.isend(t, dst, group=self.group, tag=tag), t))
+        self.bytes_sent += t.numel() * t.element_size()
+
+    def recv(self, src, dst, tag, out):
+        buf = torch.empty(out.shape, dtype=out.dtype, device=out.device)
+        dist.recv(buf, src, group=self.group, tag=tag)
+        out.copy_(buf)
+
+    def flush(self):
+        for work, _ in self.pending:
+            work.wait()
+        self.pending = []
+
+
+class HaloExchangeRank:
+    """One rank of the halo-exchange form of band sharding over one plan.
+
+    ``plan``: a reuse-halo plan (binding.Plan); ``layers``: the plan's layer descriptions (fields of lop_layer);
+    ``tensor(idx)``: the rank's full-size tensor of layer ``idx``'s output (``-1``: the plan's input) as a torch tensor
+    [N, H, W, C]; ``compute(layer, lo, hi)``: runs rows [lo, hi) of a layer on this rank's tensors (lop_run_layer on a
+    GPU; the oracle in CPU tests).  ``step(i)`` is split in two so that ranks sharing a process can take turns."""
+
+    def __init__(self, plan, layers, table, rank, tensor, compute, transport):
+        self.plan, self.layers, self.table, self.rank = plan, layers, table, rank
+        self.world = len(table)
+        self.tensor, self.compute, self.tr = tensor, compute, transport
+        self.rows_computed = 0
+
+    def _h_in(self, layer):
+        src = self.layers[layer].input_from
+        return self.tensor(src).shape[1]
+
+    def _wanted_from(self, layer, reader, owner):
+        """[(edge, source tensor, lo, hi)]: rows that rank ``reader`` reads at this layer -- through the layer's window from
+        its main input (edge 0), one to one from its residual tensor (edge 1) -- and that rank ``owner`` (< reader) computed."""
+        l = self.layers[layer]
+        lo, hi = owned_rows(self.plan, layer, self.table, reader)
+        out = []
+        edges = [(0, l.input_from, rows_read(l, lo, hi, self._h_in(layer)))]
+        if l.residual_from != -2:
+            edges.append((1, l.residual_from, (lo, hi)))
+        for edge, src, (a, b) in edges:
+            if src < 0 or b <= a:
+                continue                                       # the chain input arrives from the host with its halo
+            own_lo, _ = owned_rows(self.plan, src, self.table, reader)
+            o_lo, o_hi = owned_rows(self.plan, src, self.table, owner)
+            lo2, hi2 = max(a, o_lo), min(min(b, own_lo), o_hi)
+            if lo2 < hi2:
+                out.append((edge, src, lo2, hi2))
+        return out
+
+    def post_sends(self, layer):
+        for reader in range(self.rank + 1, self.world):
+            for edge, src, lo, hi in self._wanted_from(layer, reader, self.rank):
+                self.tr.send(self.rank, reader, 2 * layer + edge, self.tensor(src)[:, lo:hi])
+
+    def receive_and_compute(self, layer):
+        for owner in range(self.rank):
+            for edge, src, lo, hi in self._wanted_from(layer, self.rank, owner):
+                self.tr.recv(owner, self.rank, 2 * layer + edge, self.tensor(src)[:, lo:hi])
+        lo, hi = owned_rows(self.plan, layer, self.table, self.rank)
+        if hi > lo:
+            self.compute(layer, lo, hi)
+            self.rows_computed += hi - lo
+        self.tr.flush()
+
+    def run(self):
+        """All layers, for ranks that each live in a process of their own."""
+        for i in range(len(self.layers)):
+            self.post_sends(i)
+            self.receive_and_compute(i)

@@ -456,6 +456,55 @@ def test_a_band_that_never_arrives_ends_the_launch_with_a_status_not_a_hang():
         assert torch.equal(dc.outs[-1], good), mode
 
 
+@pytest.mark.parametrize("name,kw", [("vgg_block", dict(H=44, W=36)), ("resnet18", dict(H=64, W=64))])
+def test_halo_exchange_between_emulated_ranks_on_one_gpu(name, kw):
+    """The transmission form of band sharding (Sec. IV-C: trade halo rows instead of recomputing them), two and three
+    ranks taking turns on this GPU, each with tensors of its own: lop_run_layer computes every row of every layer once,
+    a mailbox carries the halo rows, and every rank's rows equal the whole-tensor run bit for bit."""
+    from paper_2507_05829_b200 import shard
+    wl = li.build(name, **kw)
+    flags = lop.LOP_FLAG_REUSE_HALO | lop.LOP_FLAG_PER_LAYER
+    ref = DeviceChain(wl, flags=flags)
+    ref.run_whole(ref.input_tensor())
+    torch.cuda.synchronize()
+    s = torch.cuda.current_stream().cuda_stream
+    for world in (2, 3):
+        x = ref.input_tensor()
+        for si, seg in enumerate(wl.segments):
+            box = shard.MailboxTransport()
+            ranks = []
+            for r in range(world):
+                dc = DeviceChain(wl, flags=flags)
+                plan = dc.plans[si]
+                table = shard.shard_table(plan, world)
+                xin = torch.full_like(x, float("nan"))
+                xin[:, table[r][4]:table[r][5]] = x[:, table[r][4]:table[r][5]]
+                dc.ws[si].view(torch.bfloat16).fill_(float("nan"))
+                dc.outs[si].fill_(float("nan"))
+
+                def tensor(idx, dc=dc, xin=xin):
+                    return xin if idx < 0 else dc.layer_output(si, idx)
+
+                def compute(layer, lo, hi, dc=dc, xin=xin, plan=plan):
+                    plan.run_layer(layer, lo, hi, xin.data_ptr(), dc.outs[si].data_ptr(), dc.ws[si].data_ptr(), s)
+
+                ranks.append((shard.HaloExchangeRank(plan, seg.layers, table, r, tensor, compute, box), dc, table))
+            for i in range(len(seg.layers)):
+                for hx, _, _ in ranks:
+                    hx.post_sends(i)
+                torch.cuda.synchronize()
+                for hx, _, _ in ranks:
+                    hx.receive_and_compute(i)
+                torch.cuda.synchronize()
+            for r, (hx, dc, table) in enumerate(ranks):
+                for i in range(len(seg.layers)):
+                    lo, hi = shard.owned_rows(dc.plans[si], i, table, r)
+                    want = ref.layer_output(si, i)
+                    assert torch.equal(dc.layer_output(si, i)[:, lo:hi], want[:, lo:hi]), (name, world, si, r, i)
+            assert sum(hx.rows_computed for hx, _, _ in ranks) == sum(ref.plans[si].out_shape(i)[0] for i in range(len(seg.layers)))
+            x = ref.outs[si]
+
+
 # ------------------------------------------------------------------------------------ edge cases
 def test_very_wide_image_gathers_patches_without_staging_rows():
     """Three rows of a 4200-pixel image do not fit the shared staging tile: the gather reads the image in place."""

@@ -145,3 +145,113 @@ def test_shard_table_is_the_floor_partition_of_the_bands():
         assert covered == 112
     with __import__("pytest").raises(lop.LopError):
         plan.shard(2, 2)
+
+
+# ------------------------------------------------------------------------------------ halo exchange (no recompute)
+def _halo_setup(wl_seg_layers, x, n_bands, world, transport_of):
+    """Per rank: poisoned tensors holding only the rank's input rows, the oracle as the compute step."""
+    import numpy as np
+    import torch
+    import paper_2507_05829_b200 as lop
+    from oracle import chain as ochain, planner as oplanner
+    from paper_2507_05829_b200 import shard
+    N, H, W, C = x.shape
+    plan = lop.Plan(wl_seg_layers, N, H, W, C, lop.LOP_BF16, n_bands, lop.LOP_FLAG_REUSE_HALO)
+    table = shard.shard_table(plan, world)
+    shapes = oplanner.infer_shapes(wl_seg_layers, H, W, C)
+    ranks = []
+    for r in range(world):
+        t = {-1: np.full(x.shape, np.inf, dtype=np.float32)}
+        i0, i1 = table[r][4], table[r][5]
+        t[-1][:, i0:i1] = x[:, i0:i1]
+        for i, (h, w, c) in enumerate(shapes):
+            t[i] = np.full((N, h, w, c), np.inf, dtype=np.float32)
+        views = {k: torch.from_numpy(v) for k, v in t.items()}
+
+        def compute(layer, lo, hi, t=t):
+            l = wl_seg_layers[layer]
+            res = t[l.residual_from] if l.residual_from != -2 else None
+            ochain.run_layer(l, t[l.input_from], res, (lo, hi), True, t[layer])
+
+        ranks.append((shard.HaloExchangeRank(plan, wl_seg_layers, table, r, lambda idx, v=views: v[idx], compute, transport_of(r)), t))
+    return plan, table, ranks
+
+
+def test_halo_exchange_computes_every_row_once_and_stitches_to_the_whole():
+    """Ranks taking turns in one process (a mailbox carries the rows): no row is computed twice, every rank's rows are
+    the whole-tensor result, and the rows traded are exactly the halo -- against the rows recomputed by the replication
+    form (lop_run_shard) of the same sharding."""
+    sys.path.insert(0, ROOT)
+    import numpy as np
+    import lop_inputs as li
+    from oracle import chain as ochain
+    from paper_2507_05829_b200 import shard
+    for name, kw in (("vgg_block", dict(H=44, W=12, width=8)), ("resnet18", dict(H=48, W=16, width=8)), ("csp_stack", dict(H=128, W=32, base=8))):
+        wl = li.build(name, **kw)
+        x = wl.x
+        for seg in wl.segments:
+            whole = ochain.run_whole(seg.layers, x, True, keep_all=True)
+            for world in (2, 3):
+                box = shard.MailboxTransport()
+                plan, table, ranks = _halo_setup(seg.layers, x, seg.n_bands, world, lambda r: box)
+                for i in range(len(seg.layers)):
+                    for hx, _ in ranks:
+                        hx.post_sends(i)
+                    for hx, _ in ranks:
+                        hx.receive_and_compute(i)
+                assert not box.box                                   # every row sent was wanted
+                for i, want in enumerate(whole):
+                    done = 0
+                    for r, (hx, t) in enumerate(ranks):
+                        lo, hi = shard.owned_rows(plan, i, table, r)
+                        if hi > lo:
+                            assert lo == done or done == 0           # the ranks' rows tile the layer
+                            assert np.array_equal(t[i][:, lo:hi], want[:, lo:hi]), (name, world, i, r)
+                            done = hi
+                    assert sum(hx.rows_computed for hx, _ in ranks) >= done
+                total = sum(hx.rows_computed for hx, _ in ranks)
+                assert total == sum(w.shape[1] for w in whole)        # every row of every layer exactly once
+            x = whole[-1]
+
+
+def _halo_rank(rank, world, port, out):
+    import numpy as np
+    import torch.distributed as dist
+    sys.path.insert(0, ROOT)
+    import lop_inputs as li
+    from oracle import chain as ochain
+    from paper_2507_05829_b200 import shard
+    dist.init_process_group("gloo", init_method="tcp://127.0.0.1:%d" % port, rank=rank, world_size=world)
+    try:
+        wl = li.build("resnet18", H=48, W=16, width=8)
+        x = wl.x
+        sent = 0
+        for seg in wl.segments:
+            tr = shard.DistTransport()
+            plan, table, ranks = _halo_setup(seg.layers, x, seg.n_bands, world, lambda r: tr)
+            hx, t = ranks[rank]
+            hx.run()
+            whole = ochain.run_whole(seg.layers, x, True, keep_all=True)
+            for i, want in enumerate(whole):
+                lo, hi = shard.owned_rows(plan, i, table, rank)
+                assert np.array_equal(t[i][:, lo:hi], want[:, lo:hi]), (rank, i)
+            sent += tr.bytes_sent
+            x = whole[-1]
+        out.put((rank, sent))
+        dist.barrier()
+    finally:
+        dist.destroy_process_group()
+
+
+def test_halo_exchange_over_two_gloo_ranks():
+    ctx = mp.get_context("spawn")
+    out = ctx.SimpleQueue()
+    port = _free_port()
+    procs = [ctx.Process(target=_halo_rank, args=(r, 2, port, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    for p in procs:
+        p.join(300)
+        assert p.exitcode == 0
+    got = dict(out.get() for _ in range(2))
+    assert got[0] > 0 and got[1] == 0                              # rows only travel upwards: rank 0 sends, rank 1 receives
