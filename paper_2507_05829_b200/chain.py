@@ -55,7 +55,12 @@ class DeviceChain:
                             self.keep.append(t)
                             setattr(d, name + "_ptr", t.data_ptr())
                     layers.append(d)
-                nb = seg.n_bands if n_bands is None else n_bands
+                if n_bands is None:
+                    nb = seg.n_bands
+                elif isinstance(n_bands, (list, tuple)):                 # one count per segment
+                    nb = n_bands[len(self.plans)]
+                else:
+                    nb = n_bands
                 plan = B.Plan(layers, wl.N, H, W, C, self.dtype, nb, flags)
                 self.plans.append(plan)
                 self.ws.append(torch.zeros(max(plan.workspace_bytes(), 256), dtype=torch.uint8, device=self.device))
