@@ -38,7 +38,40 @@ def build_case(name):
     return wl, "whole", (0 if mode == "persistent" else B.LOP_FLAG_PER_LAYER)
 
 
+def record_traffic(workload, ncu_csv):
+    """Reads dram__bytes_read.sum + dram__bytes_write.sum of the persistent kernel's captured launch from an ``ncu --csv``
+    log and stores their sum under ``workload`` in profiles/dram_traffic.json, together with the hash of the kernel's
+    sources (bench.py reports the figure only while that hash still matches)."""
+    import csv
+    import json
+    import os
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    sys.path.insert(0, root)
+    import bench
+    total, units = 0.0, {"byte": 1.0, "Kbyte": 1e3, "Mbyte": 1e6, "Gbyte": 1e9}
+    rows = [r for r in csv.reader(open(ncu_csv)) if len(r) > 10]
+    hdr = rows[0]
+    for r in rows[1:]:
+        d = dict(zip(hdr, r))
+        if "wavefront_kernel" in d.get("Kernel Name", "") and d.get("Metric Name") in ("dram__bytes_read.sum", "dram__bytes_write.sum"):
+            total += float(d["Metric Value"].replace(",", "")) * units[d["Metric Unit"]]
+    if total <= 0:
+        raise SystemExit("no DRAM counters of the persistent kernel in %s" % ncu_csv)
+    path = os.path.join(root, "profiles", "dram_traffic.json")
+    rec = {"kernel_hash": bench.kernel_hash(), "bytes_per_launch": {}}
+    if os.path.exists(path):
+        old = json.load(open(path))
+        if old.get("kernel_hash") == rec["kernel_hash"]:
+            rec = old
+    rec["bytes_per_launch"][workload] = total
+    rec["what"] = "dram__bytes_read.sum + dram__bytes_write.sum of one wavefront_kernel launch (all bands, device-resident input), ncu, L2 flushed before the launch"
+    json.dump(rec, open(path, "w"), indent=1, sort_keys=True)
+    print("%s: %.1f MB per launch (kernel %s)" % (workload, total / 1e6, rec["kernel_hash"]))
+
+
 def main():
+    if len(sys.argv) > 1 and sys.argv[1] == "--record-traffic":
+        return record_traffic(sys.argv[2], sys.argv[3])
     name = sys.argv[1] if len(sys.argv) > 1 else "resnet50"
     launches = int(sys.argv[2]) if len(sys.argv) > 2 else 3
     wl, mode, flags = build_case(name)

@@ -121,3 +121,19 @@ def test_row_wise_operator_must_not_carry_a_window():
         with pytest.raises(lop.LopError) as e:
             lop.Plan([bad], 1, 6, 5, 8, lop.LOP_BF16, 3)
         assert e.value.status == -1 and "row-wise" in str(e.value)
+
+
+def test_the_developer_trace_build_compiles(tmp_path):
+    """-DLOP_WF_TRACE adds per-item time stamps of the persistent kernel's roles and the lop_debug_* readers (a developer
+    build, never the shipped library): it must keep compiling for sm_100a as the kernel changes."""
+    import glob
+    import subprocess
+    csrc = os.path.join(ROOT, "paper_2507_05829_b200", "csrc")
+    out = str(tmp_path / "trace.o")
+    cmd = ["/usr/local/cuda/bin/nvcc", "-gencode", "arch=compute_100a,code=sm_100a", "-std=c++17", "-DLOP_WF_TRACE", "-I",
+           os.path.join(ROOT, "include"), "-I", csrc, "-c", os.path.join(csrc, "lop_wavefront.cu"), "-o", out]
+    r = subprocess.run(cmd, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0, r.stderr[-2000:]
+    syms = subprocess.run(["nm", "-g", out], capture_output=True, text=True).stdout
+    assert "lop_debug_trace_copy" in syms and "lop_debug_last_items" in syms
+    assert not any("lop_debug" in e for e in lop.EXPORTS)          # the shipped library exports none of them
