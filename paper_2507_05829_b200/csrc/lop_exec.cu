@@ -424,10 +424,17 @@ int get_program(const std::vector<SegBind> &segs, int kind, Program **prog, cons
         if (kind == PROG_PIPELINED) {
             const double row_bytes = (double)pl0->W * pl0->C * elem_size(pl0->dtype) * pl0->N;
             double t = 5.0;
+            std::vector<double> own(pl0->n_bands, 0.0);
             for (int b = 0; b < pl0->n_bands; ++b) {
                 const lop_range &need = pl0->in_need[b];
-                if (need.out_hi > need.new_lo) t += std::max(4.7, (need.out_hi - need.new_lo) * row_bytes / 64e3);
-                arrival.push_back(t + 5.0);
+                if (need.out_hi > need.new_lo) own[b] = (need.out_hi - need.new_lo) * row_bytes / 64e3;
+            }
+            for (int b0 = 0; b0 < pl0->n_bands; b0 += std::max(1, pl0->copy_group)) {
+                const int b1 = std::min(pl0->n_bands, b0 + std::max(1, pl0->copy_group));
+                double bytes_us = 0.0;
+                for (int b = b0; b < b1; ++b) bytes_us += own[b];
+                if (bytes_us > 0.0) t += std::max(4.7, bytes_us);
+                for (int b = b0; b < b1; ++b) arrival.push_back(t + 5.0);       // the bands of one copy arrive together
             }
         }
         if (kind == PROG_ALL_BANDS || kind <= PROG_BLOCK0) merge_thin_bands(segs, reqs, false);
@@ -483,10 +490,17 @@ void reset_layer_timing(lop_plan_t *pl)
     for (auto &c : pl->exec->layer_timed) c = 0;
 }
 
+int copy_rows_impl(lop_plan_t *pl, int lo, int hi, const void *host, void *staging, cudaStream_t s);
+
 int copy_band_impl(lop_plan_t *pl, int band, const void *host, void *staging, cudaStream_t s)
 {
     const lop_range &need = pl->in_need[band];
-    const int lo = need.new_lo, hi = need.out_hi;
+    return copy_rows_impl(pl, need.new_lo, need.out_hi, host, staging, s);
+}
+
+// Rows [lo, hi) of every image of the chain input, pinned host -> device, one asynchronous (2-D) copy.
+int copy_rows_impl(lop_plan_t *pl, int lo, int hi, const void *host, void *staging, cudaStream_t s)
+{
     if (hi <= lo) return LOP_OK;
     const size_t row = (size_t)pl->W * pl->C * elem_size(pl->dtype);
     const size_t img = row * pl->H;
@@ -520,11 +534,23 @@ int enqueue_pipelined(lop_plan_t *pl, Program *p, const void *host, void *stagin
     // event and performs the 4-byte arrival write the kernel polls: the write of band b overlaps the copy of band b+1.
     StreamWriteValue32Fn write32 = stream_write_fn();
     LOP_CUDA(cudaStreamWaitEvent(e->signal_stream, e->ev_fork, 0));
-    for (int b = 0; b < pl->n_bands; ++b) {
-        const lop_range &need = pl->in_need[b];
-        e->copy_issued[b] = need.out_hi > need.new_lo && b != withheld;
-        if (b == withheld) continue;
-        if (e->copy_issued[b] && (rc = copy_band_impl(pl, b, host, staging, e->copy_stream)) != LOP_OK) return rc;
+    const int G = std::max(1, pl->copy_group);
+    for (int b0 = 0; b0 < pl->n_bands; b0 += G) {
+        // one copy for the bands [b0, b1): their new rows are one contiguous run; the arrival is written for the last band
+        const int b1 = std::min(pl->n_bands, b0 + G), b = b1 - 1;
+        int lo = 0, hi = 0;
+        bool any = false;
+        for (int q = b0; q < b1; ++q) {
+            const lop_range &need = pl->in_need[q];
+            e->copy_issued[q] = 0;
+            if (need.out_hi <= need.new_lo) continue;
+            lo = any ? std::min(lo, (int)need.new_lo) : (int)need.new_lo;
+            hi = any ? std::max(hi, (int)need.out_hi) : (int)need.out_hi;
+            any = true;
+        }
+        if (withheld >= b0 && withheld < b1) continue;
+        e->copy_issued[b] = any;
+        if (any && (rc = copy_rows_impl(pl, lo, hi, host, staging, e->copy_stream)) != LOP_OK) return rc;
         unsigned *flag = program_arrival_flag(p, b);
         if (!flag) continue;
         LOP_CUDA(cudaEventRecord(e->ev_arrive[b], e->copy_stream));

@@ -37,6 +37,7 @@ struct lop_plan {
     std::vector<lop_range> in_need;    // [band]: chain-input rows (out_lo,out_hi,new_lo)
     size_t ws_bytes = 0, status_off = 0, col_off = 0;   // col_off: the gathered patch tensor
     double flops = 0.0;
+    int copy_group = 1;                // bands moved by one copy-engine copy in pipelined runs (see lop_plan.cpp)
     unsigned wait_limit = 0;           // polls a device-side wait may take before the kernel gives up (0: the default)
     unsigned long long uid = 0;        // unique per plan and per state of its parameters (a new one at creation and at every
                                        // lop_plan_set_params): cached device programs name the plans they were built from by it

@@ -18,6 +18,10 @@ namespace lop {
 
 static thread_local char g_err[512] = "";
 
+#ifndef LOP_MAX_BAND_COPIES
+#define LOP_MAX_BAND_COPIES 8
+#endif
+
 unsigned long long next_plan_uid()
 {
     static std::atomic<unsigned long long> counter{0};
@@ -213,6 +217,13 @@ static void choose_kernels(lop_plan_t &pl)
         li.kernel = K_CONV_TC;
     }
 
+    // Copy-engine band pipeline: every copy costs a few microseconds of stream commands whatever its size, so an input
+    // of megabytes cut into many bands is moved a few neighbouring bands per copy (at most LOP_MAX_BAND_COPIES copies);
+    // the bands of one copy arrive together.  Small inputs keep one copy per band.
+    {
+        const size_t in_bytes = (size_t)pl.N * pl.H * pl.W * pl.C * es;
+        pl.copy_group = (in_bytes >= (1u << 20) && pl.n_bands > LOP_MAX_BAND_COPIES) ? (pl.n_bands + LOP_MAX_BAND_COPIES - 1) / LOP_MAX_BAND_COPIES : 1;
+    }
     size_t off = 0;
     pl.status_off = off; off += 1024;
     for (int i = 0; i < L; ++i) {

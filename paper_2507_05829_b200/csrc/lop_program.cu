@@ -619,10 +619,15 @@ int program_build(const std::vector<SegBind> &segs, std::vector<StageReq> reqs, 
                 if (!main_raw) { a = o0; b = o1; }                          // only the residual reads the chain input: its own rows
                 else if (!rq.gather && l.op == LOP_CONV2D && l.residual_from == LOP_INPUT) { a = std::min<long long>(a, o0); b = std::max<long long>(b, o1); }
                 a = std::max(a, 0LL); b = std::min<long long>(b, pl->H);
+                int last_leader = -1;
                 for (int b2 = 0; b2 < pl->n_bands; ++b2) {
                     const lop_range &o = pl->in_need[b2];
                     if (o.out_hi <= o.new_lo || o.out_hi <= a || o.new_lo >= b) continue;
-                    deps.push_back(make_int2(-1 - b2, -1));             // patched below
+                    // the bands of one copy arrive together: the flag of the copy's last band stands for all of them
+                    const int leader = std::min(pl->n_bands - 1, (b2 / pl->copy_group) * pl->copy_group + pl->copy_group - 1);
+                    if (leader == last_leader) continue;
+                    last_leader = leader;
+                    deps.push_back(make_int2(-1 - leader, -1));         // patched below
                 }
                 uses_flags = true;
             }
