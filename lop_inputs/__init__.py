@@ -5,6 +5,6 @@ benchmark.  It only *describes* workloads and draws random numbers: it holds no
 convolution, pooling, planning or epilogue arithmetic of its own.
 """
 from .rng import uniform, normal, round_to_bf16, bf16_bits, from_bf16_bits
-from .workloads import (Layer, Segment, Workload, CONV, POOL, LINEAR, ACT_NONE, ACT_RELU, ACT_SILU,
-                        RES_NONE, RES_PRE_ACT, RES_POST_ACT, build, WORKLOADS, conv, pool, linear,
+from .workloads import (Layer, Segment, Workload, CONV, POOL, LINEAR, DWCONV, LAYERNORM, CONCAT, ACT_NONE, ACT_RELU, ACT_SILU, ACT_GELU,
+                        RES_NONE, RES_PRE_ACT, RES_POST_ACT, build, WORKLOADS, conv, pool, linear, dwconv, layernorm, concat,
                         fill_parameters, make_input)

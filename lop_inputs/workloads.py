@@ -23,8 +23,8 @@ import numpy as np
 
 from . import rng
 
-CONV, POOL, LINEAR = 0, 1, 2
-ACT_NONE, ACT_RELU, ACT_SILU = 0, 1, 2
+CONV, POOL, LINEAR, DWCONV, LAYERNORM, CONCAT = 0, 1, 2, 3, 4, 5
+ACT_NONE, ACT_RELU, ACT_SILU, ACT_GELU = 0, 1, 2, 3
 RES_NONE, RES_PRE_ACT, RES_POST_ACT = 0, 1, 2
 NO_RESIDUAL = -2
 
@@ -85,6 +85,23 @@ def linear(cin, cout, act=ACT_NONE, input_from=None, residual_from=NO_RESIDUAL, 
     return Layer(LINEAR, cin, cout, 1, 1, 1, 1, 0, 0, 1, 1, act, input_from, residual_from, residual_pos)
 
 
+def dwconv(c, k, s=1, p=None, d=1, act=ACT_NONE, input_from=None, residual_from=NO_RESIDUAL, residual_pos=RES_NONE):
+    """Depth-wise convolution: every channel filtered by its own k x k kernel (weight [c, k, k, 1])."""
+    if p is None:
+        p = d * (k - 1) // 2
+    return Layer(DWCONV, c, c, k, k, s, s, p, p, d, d, act, input_from, residual_from, residual_pos)
+
+
+def layernorm(c, input_from=None):
+    """Layer normalisation over the channels of every pixel (scale = gamma, shift = beta)."""
+    return Layer(LAYERNORM, c, c, 1, 1, 1, 1, 0, 0, 1, 1, ACT_NONE, input_from)
+
+
+def concat(c_main, c_second, input_from=None, second_from=NO_RESIDUAL):
+    """Channel concatenation (main input's channels first); the second input is named like a residual."""
+    return Layer(CONCAT, c_main, c_main + c_second, 1, 1, 1, 1, 0, 0, 1, 1, ACT_NONE, input_from, second_from, RES_NONE)
+
+
 def pool(c, k, s, p=0, input_from=None):
     return Layer(POOL, c, c, k, k, s, s, p, p, 1, 1, ACT_NONE, input_from)
 
@@ -103,13 +120,17 @@ def fill_parameters(wl: Workload):
     stream = 16
     for seg in wl.segments:
         for l in seg.layers:
-            if l.op in (CONV, LINEAR):
-                fan_in = l.kh * l.kw * l.cin
-                w = rng.normal(wl.seed, stream, (l.cout, l.kh, l.kw, l.cin), 0.0, float(np.sqrt(2.0 / fan_in)))
+            if l.op in (CONV, LINEAR, DWCONV):
+                cin_w = 1 if l.op == DWCONV else l.cin
+                fan_in = l.kh * l.kw * cin_w
+                w = rng.normal(wl.seed, stream, (l.cout, l.kh, l.kw, cin_w), 0.0, float(np.sqrt(2.0 / fan_in)))
                 l.weight = rng.round_to_bf16(w) if bf16 else w
                 if wl.affine:
                     l.scale = rng.normal(wl.seed, stream + 1, (l.cout,), 1.0, 0.1)
                     l.shift = rng.normal(wl.seed, stream + 2, (l.cout,), 0.0, 0.1)
+            elif l.op == LAYERNORM:
+                l.scale = rng.normal(wl.seed, stream + 1, (l.cout,), 1.0, 0.1)       # gamma
+                l.shift = rng.normal(wl.seed, stream + 2, (l.cout,), 0.0, 0.1)       # beta
             stream += 4
     return wl
 
@@ -224,6 +245,23 @@ def pointwise_mlp(N=2, H=56, W=56, C=128, hidden=512, n_bands=8, dtype="bf16", s
     return Workload("pointwise_mlp", dtype, N, H, W, C, [Segment(_chain(layers), n_bands)], seed=seed)
 
 
+def convnext_block(N=2, H=56, W=56, C=128, n_bands=8, dtype="bf16", seed=707):
+    """One ConvNeXt block (the paper evaluates ConvNeXt, Sec. V-B): depth-wise 7x7, layer normalisation over the
+    channels, point-wise MLP C -> 4C (GELU) -> C, shortcut.  A block-wise operator (3-row halo) followed by per-pixel and
+    row-wise ones."""
+    layers = [dwconv(C, 7), layernorm(C), linear(C, 4 * C, act=ACT_GELU),
+              linear(4 * C, C, act=ACT_NONE, residual_from=-1, residual_pos=RES_POST_ACT)]
+    return Workload("convnext_block", dtype, N, H, W, C, [Segment(_chain(layers), n_bands)], seed=seed)
+
+
+def dense_layer(N=2, H=28, W=28, C=64, growth=32, n_bands=4, dtype="bf16", seed=808):
+    """One DenseNet layer (Sec. V-B): 1x1 bottleneck to 4*growth, 3x3 to growth channels, concatenated behind the input."""
+    layers = [conv(C, 4 * growth, 1, p=0, act=ACT_RELU), conv(4 * growth, growth, 3, act=ACT_RELU),
+              concat(C, growth, input_from=-1, second_from=1)]
+    layers[0].input_from, layers[1].input_from = -1, 0
+    return Workload("dense_layer", dtype, N, H, W, C, [Segment(layers, n_bands)], seed=seed)
+
+
 WORKLOADS = {
     "single_conv": single_conv,
     "vgg_block": vgg_block,
@@ -231,6 +269,8 @@ WORKLOADS = {
     "resnet50": resnet50,
     "csp_stack": csp_stack,
     "pointwise_mlp": pointwise_mlp,
+    "convnext_block": convnext_block,
+    "dense_layer": dense_layer,
 }
 
 

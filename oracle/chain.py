@@ -17,6 +17,13 @@ POISON = np.float32(np.inf)
 
 def run_layer(l, src, res, rows, round_bf16, out):
     """Rows ``rows`` of layer ``l`` applied to the full-size tensor ``src`` (residual ``res``) into ``out``."""
+    if l.op == 3:                       # depth-wise convolution: a block-wise operator, every channel its own filter
+        return ops.dwconv2d(src, l.weight, (l.sh, l.sw), (l.ph, l.pw), (l.dh, l.dw), l.scale, l.shift, res,
+                            l.residual_pos if res is not None else 0, l.act, round_bf16, rows, out)
+    if l.op == 4:                       # layer normalisation over the channels of a pixel: rows map one to one
+        return ops.layernorm(src, l.scale, l.shift, ops.LAYERNORM_EPS, round_bf16, rows, out)
+    if l.op == 5:                       # channel concatenation of the main input and the second input
+        return ops.concat(src, res, rows, out)
     if l.op == 2:                       # row-wise operator (Sec. IV-A, Eq. 1): rows map one to one
         return ops.linear(src, l.weight, l.scale, l.shift, res, l.residual_pos if res is not None else 0, l.act, round_bf16, rows, out)
     if l.op == 0:
@@ -136,5 +143,7 @@ def flops(wl):
         for l, (h, w, c) in zip(seg.layers, shapes):
             if l.op in (0, 2):
                 total += 2 * wl.N * h * w * c * l.kh * l.kw * l.cin
+            elif l.op == 3:
+                total += 2 * wl.N * h * w * c * l.kh * l.kw
         H, W, C = shapes[-1]
     return total

@@ -42,6 +42,7 @@ static float activate(float t, int act)
 {
     if (act == 1) return t > 0.0f ? t : 0.0f;                /* ReLU */
     if (act == 2) return t / (1.0f + expf(-t));              /* SiLU */
+    if (act == 3) return 0.5f * t * (1.0f + erff(t * 0.70710678118654752f));   /* GELU, t * Phi(t) with the exact normal CDF */
     return t;
 }
 
@@ -146,6 +147,83 @@ void lop_oracle_linear(const float *x, long long M, int K, const float *w, int C
             if (res && res_pos == 2) t += res[o];
             y[o] = round_bf16 ? lop_oracle_bf16_rne(t) : t;
         }
+}
+
+/*
+ * Depth-wise convolution, a block-wise local operator like the convolution (Sec. IV-A): every channel is filtered by
+ * its own kh x kw kernel,  y[n,oh,ow,c] = epilogue( sum_{a,b} x[n, oh*sh-ph+a*dh, ow*sw-pw+b*dw, c] * w[c,a,b] ),
+ * taps outside the input contribute zero.  w: [C][kh][kw].  Accumulation in double over (a, b); epilogue as above.
+ */
+void lop_oracle_dwconv2d(const float *x, int N, int H, int W, int C, const float *w, int kh, int kw, int sh, int sw,
+                         int ph, int pw, int dh, int dw, const float *scale, const float *shift,
+                         const float *res, int res_pos, int act, int round_bf16, int oh_lo, int oh_hi, float *y)
+{
+    const int Ho = (H + 2 * ph - dh * (kh - 1) - 1) / sh + 1;
+    const int Wo = (W + 2 * pw - dw * (kw - 1) - 1) / sw + 1;
+    if (oh_lo < 0) oh_lo = 0;
+    if (oh_hi > Ho) oh_hi = Ho;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (int n = 0; n < N; ++n)
+        for (int oh = oh_lo; oh < oh_hi; ++oh)
+            for (int ow = 0; ow < Wo; ++ow)
+                for (int c = 0; c < C; ++c) {
+                    double acc = 0.0;
+                    for (int a = 0; a < kh; ++a) {
+                        const int ih = oh * sh - ph + a * dh;
+                        if (ih < 0 || ih >= H) continue;
+                        for (int b = 0; b < kw; ++b) {
+                            const int iw = ow * sw - pw + b * dw;
+                            if (iw < 0 || iw >= W) continue;
+                            acc += (double)x[(((size_t)n * H + ih) * W + iw) * C + c] * (double)w[((size_t)c * kh + a) * kw + b];
+                        }
+                    }
+                    const size_t o = (((size_t)n * Ho + oh) * Wo + ow) * C + c;
+                    float t = (float)acc;
+                    t = (scale ? scale[c] : 1.0f) * t + (shift ? shift[c] : 0.0f);
+                    if (res && res_pos == 1) t += res[o];
+                    t = activate(t, act);
+                    if (res && res_pos == 2) t += res[o];
+                    y[o] = round_bf16 ? lop_oracle_bf16_rne(t) : t;
+                }
+}
+
+/*
+ * Layer normalisation over the channels of every pixel (an element-wise-per-row local operator in the sense of
+ * Sec. IV-A: a row of the [pixels][C] matrix depends on that row alone):
+ *   y[r][c] = gamma[c] * (x[r][c] - mean_r) / sqrt(var_r + eps) + beta[c],  var_r the biased variance.
+ * Mean and variance in double; gamma / beta may be NULL (1 / 0).  Rows [r_lo, r_hi) of y are computed.
+ */
+void lop_oracle_layernorm(const float *x, long long M, int C, const float *gamma, const float *beta, float eps,
+                          int round_bf16, long long r_lo, long long r_hi, float *y)
+{
+    if (r_lo < 0) r_lo = 0;
+    if (r_hi > M) r_hi = M;
+#pragma omp parallel for schedule(dynamic, 16)
+    for (long long r = r_lo; r < r_hi; ++r) {
+        const float *xr = x + (size_t)r * C;
+        double mean = 0.0, var = 0.0;
+        for (int c = 0; c < C; ++c) mean += xr[c];
+        mean /= C;
+        for (int c = 0; c < C; ++c) var += ((double)xr[c] - mean) * ((double)xr[c] - mean);
+        var /= C;
+        const double rstd = 1.0 / sqrt(var + (double)eps);
+        for (int c = 0; c < C; ++c) {
+            float t = (float)(((double)xr[c] - mean) * rstd);
+            t = (gamma ? gamma[c] : 1.0f) * t + (beta ? beta[c] : 0.0f);
+            y[(size_t)r * C + c] = round_bf16 ? lop_oracle_bf16_rne(t) : t;
+        }
+    }
+}
+
+/* Channel concatenation: y[r] = (a[r][0..Ca), b[r][0..Cb)) for the rows [r_lo, r_hi) of the [pixels][C] matrices. */
+void lop_oracle_concat(const float *a, int Ca, const float *b, int Cb, long long M, long long r_lo, long long r_hi, float *y)
+{
+    if (r_lo < 0) r_lo = 0;
+    if (r_hi > M) r_hi = M;
+    for (long long r = r_lo; r < r_hi; ++r) {
+        memcpy(y + (size_t)r * (Ca + Cb), a + (size_t)r * Ca, sizeof(float) * (size_t)Ca);
+        memcpy(y + (size_t)r * (Ca + Cb) + Ca, b + (size_t)r * Cb, sizeof(float) * (size_t)Cb);
+    }
 }
 
 int lop_oracle_num_threads(void)

@@ -18,6 +18,9 @@ def lib():
         _lib.lop_oracle_conv2d.restype = None
         _lib.lop_oracle_maxpool2d.restype = None
         _lib.lop_oracle_linear.restype = None
+        _lib.lop_oracle_dwconv2d.restype = None
+        _lib.lop_oracle_layernorm.restype = None
+        _lib.lop_oracle_concat.restype = None
     return _lib
 
 
@@ -99,5 +102,60 @@ def linear(x, w, scale=None, shift=None, res=None, res_pos=0, act=0, round_bf16=
     for n in range(N):
         lib().lop_oracle_linear(_fp(x), ctypes.c_longlong(M), K, _fp(w2), Cout, _fp(scale), _fp(shift), _fp(res), int(res_pos),
                                 int(act), int(bool(round_bf16)), ctypes.c_longlong((n * H + lo) * W),
+                                ctypes.c_longlong((n * H + hi) * W), _fp(out))
+    return out
+
+
+LAYERNORM_EPS = 1e-6
+
+
+def dwconv2d(x, w, stride=(1, 1), pad=(0, 0), dil=(1, 1), scale=None, shift=None, res=None, res_pos=0, act=0,
+             round_bf16=False, rows=None, out=None):
+    """Rows ``rows`` of the depth-wise convolution (every channel its own kernel); ``w``: [C, kh, kw] (or [C, kh, kw, 1])."""
+    x, w = _f32(x), _f32(w)
+    N, H, W, C = x.shape
+    w3 = w.reshape(w.shape[0], w.shape[1], w.shape[2])
+    assert w3.shape[0] == C
+    kh, kw = w3.shape[1], w3.shape[2]
+    Ho, Wo = out_size(H, kh, stride[0], pad[0], dil[0]), out_size(W, kw, stride[1], pad[1], dil[1])
+    assert Ho > 0 and Wo > 0
+    if out is None:
+        out = np.zeros((N, Ho, Wo, C), dtype=np.float32)
+    assert out.shape == (N, Ho, Wo, C) and out.dtype == np.float32 and out.flags.c_contiguous
+    scale, shift, res = _f32(scale), _f32(shift), _f32(res)
+    lo, hi = (0, Ho) if rows is None else rows
+    lib().lop_oracle_dwconv2d(_fp(x), N, H, W, C, _fp(np.ascontiguousarray(w3)), kh, kw, stride[0], stride[1], pad[0], pad[1],
+                              dil[0], dil[1], _fp(scale), _fp(shift), _fp(res), int(res_pos), int(act), int(bool(round_bf16)),
+                              int(lo), int(hi), _fp(out))
+    return out
+
+
+def layernorm(x, gamma=None, beta=None, eps=LAYERNORM_EPS, round_bf16=False, rows=None, out=None):
+    """Layer normalisation over the channels of every pixel; ``rows``: image rows of every image (default all)."""
+    x = _f32(x)
+    N, H, W, C = x.shape
+    if out is None:
+        out = np.zeros((N, H, W, C), dtype=np.float32)
+    assert out.shape == x.shape and out.dtype == np.float32 and out.flags.c_contiguous
+    gamma, beta = _f32(gamma), _f32(beta)
+    lo, hi = (0, H) if rows is None else rows
+    for n in range(N):
+        lib().lop_oracle_layernorm(_fp(x), ctypes.c_longlong(N * H * W), C, _fp(gamma), _fp(beta), ctypes.c_float(eps),
+                                   int(bool(round_bf16)), ctypes.c_longlong((n * H + lo) * W), ctypes.c_longlong((n * H + hi) * W), _fp(out))
+    return out
+
+
+def concat(a, b, rows=None, out=None):
+    """Channel concatenation of two NHWC tensors of equal N, H, W."""
+    a, b = _f32(a), _f32(b)
+    N, H, W, Ca = a.shape
+    Cb = b.shape[3]
+    assert b.shape[:3] == (N, H, W)
+    if out is None:
+        out = np.zeros((N, H, W, Ca + Cb), dtype=np.float32)
+    assert out.shape == (N, H, W, Ca + Cb) and out.dtype == np.float32 and out.flags.c_contiguous
+    lo, hi = (0, H) if rows is None else rows
+    for n in range(N):
+        lib().lop_oracle_concat(_fp(a), Ca, _fp(b), Cb, ctypes.c_longlong(N * H * W), ctypes.c_longlong((n * H + lo) * W),
                                 ctypes.c_longlong((n * H + hi) * W), _fp(out))
     return out

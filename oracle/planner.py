@@ -53,8 +53,12 @@ def infer_shapes(layers, H, W, C):
             raise PlanError("layer %d: cin %d but its input has %d channels" % (i, l.cin, cin))
         if l.op == 2 and (l.kh, l.kw, l.sh, l.sw, l.ph, l.pw, l.dh, l.dw) != (1, 1, 1, 1, 0, 0, 1, 1):
             raise PlanError("layer %d: a row-wise operator has no window" % i)
-        if l.op == 1 and l.cout != l.cin:
-            raise PlanError("layer %d: pooling keeps the channel count" % i)
+        if l.op in (1, 3, 4) and l.cout != l.cin:
+            raise PlanError("layer %d: pooling, depth-wise convolution and layer normalisation keep the channel count" % i)
+        if l.op in (4, 5) and (l.kh, l.kw, l.sh, l.sw, l.ph, l.pw, l.dh, l.dw) != (1, 1, 1, 1, 0, 0, 1, 1):
+            raise PlanError("layer %d: a per-pixel operator has no window" % i)
+        if l.op == 5 and l.residual_from == NO_RESIDUAL:
+            raise PlanError("layer %d: a concatenation needs its second input (residual_from)" % i)
         ho = out_extent(hin, l.kh, l.sh, l.ph, l.dh)
         wo = out_extent(win, l.kw, l.sw, l.pw, l.dw)
         if ho <= 0 or wo <= 0:
@@ -62,10 +66,14 @@ def infer_shapes(layers, H, W, C):
         if l.residual_from != NO_RESIDUAL:
             if not (-1 <= l.residual_from < i):
                 raise PlanError("layer %d: residual_from must name the segment input or an earlier layer" % i)
-            if l.op not in (0, 2) or l.residual_pos not in (1, 2):
-                raise PlanError("layer %d: a residual needs a convolution and a position" % i)
-            if shape_of(l.residual_from) != (ho, wo, l.cout):
-                raise PlanError("layer %d: residual shape mismatch" % i)
+            if l.op == 5:
+                if shape_of(l.residual_from) != (ho, wo, l.cout - l.cin):
+                    raise PlanError("layer %d: the second input of a concatenation must bring cout - cin channels" % i)
+            else:
+                if l.op not in (0, 2, 3) or l.residual_pos not in (1, 2):
+                    raise PlanError("layer %d: a residual needs a convolution and a position" % i)
+                if shape_of(l.residual_from) != (ho, wo, l.cout):
+                    raise PlanError("layer %d: residual shape mismatch" % i)
         shapes.append((ho, wo, l.cout))
     return shapes
 

@@ -291,3 +291,76 @@ def test_linear_is_the_pointwise_convolution_and_shares_its_epilogue():
         assert np.array_equal(a, b)
     lin = ops.linear(x, w)                           # linear in x
     assert np.allclose(ops.linear(2.0 * x, w), 2.0 * lin, rtol=1e-6, atol=1e-6)
+
+
+# ----------------------------------------------------------------------------- depth-wise conv, layer norm, concat, GELU
+def test_depthwise_convolution_is_the_convolution_with_block_diagonal_weights():
+    rnd = np.random.default_rng(31)
+    for k, s_, p, d in ((7, 1, 3, 1), (3, 2, 1, 1), (3, 1, 2, 2)):
+        x = rnd.standard_normal((2, 11, 9, 5)).astype(np.float32)
+        w = rnd.standard_normal((5, k, k)).astype(np.float32)
+        full = np.zeros((5, k, k, 5), dtype=np.float32)
+        for c in range(5):
+            full[c, :, :, c] = w[c]
+        sc, sh = rnd.standard_normal(5).astype(np.float32), rnd.standard_normal(5).astype(np.float32)
+        a = ops.dwconv2d(x, w, (s_, s_), (p, p), (d, d), sc, sh, act=1)
+        b = ops.conv2d(x, full, (s_, s_), (p, p), (d, d), sc, sh, act=1)
+        assert a.shape == b.shape and np.max(np.abs(a - b)) <= 1e-6 * max(1.0, np.max(np.abs(b)))
+    delta = np.zeros((5, 3, 3), dtype=np.float32)
+    delta[:, 1, 1] = 1.0
+    x = rnd.standard_normal((1, 6, 7, 5)).astype(np.float32)
+    assert np.array_equal(ops.dwconv2d(x, delta, pad=(1, 1)), x)          # the centre tap alone returns the input
+
+
+def test_depthwise_convolution_matches_the_grouped_library_convolution():
+    import torch
+    import torch.nn.functional as F
+    rnd = np.random.default_rng(32)
+    x = rnd.standard_normal((2, 12, 10, 6)).astype(np.float32)
+    w = rnd.standard_normal((6, 7, 7)).astype(np.float32)
+    got = ops.dwconv2d(x, w, pad=(3, 3))
+    want = F.conv2d(torch.from_numpy(x).permute(0, 3, 1, 2).double(), torch.from_numpy(w).unsqueeze(1).double(), padding=3, groups=6)
+    assert np.max(np.abs(got - want.permute(0, 2, 3, 1).numpy())) <= 1e-5
+
+
+def test_layernorm_rows_have_zero_mean_unit_variance_and_ignore_shift_and_scale_of_their_input():
+    import torch
+    import torch.nn.functional as F
+    rnd = np.random.default_rng(33)
+    x = (3.0 * rnd.standard_normal((2, 4, 5, 32)) + 7.0).astype(np.float32)
+    y = ops.layernorm(x)
+    assert np.max(np.abs(y.mean(axis=-1))) < 1e-5 and np.max(np.abs(y.var(axis=-1) - 1.0)) < 1e-4
+    y2 = ops.layernorm((5.0 * x - 2.0).astype(np.float32))             # an affine map of the row changes nothing
+    assert np.max(np.abs(y2 - y)) < 1e-4
+    g, b = rnd.standard_normal(32).astype(np.float32), rnd.standard_normal(32).astype(np.float32)
+    want = F.layer_norm(torch.from_numpy(x).double(), (32,), torch.from_numpy(g).double(), torch.from_numpy(b).double(), eps=1e-6).numpy()
+    assert np.max(np.abs(ops.layernorm(x, g, b) - want)) < 1e-5
+    const = np.full((1, 2, 2, 8), 3.5, dtype=np.float32)
+    assert np.allclose(ops.layernorm(const, None, b[:8]), b[:8], atol=1e-6)    # no spread: only beta is left
+    part = np.full_like(y, np.inf)
+    ops.layernorm(x, rows=(1, 3), out=part)
+    assert np.array_equal(part[:, 1:3], y[:, 1:3]) and np.all(np.isinf(part[:, :1])) and np.all(np.isinf(part[:, 3:]))
+
+
+def test_concat_puts_the_main_input_first():
+    rnd = np.random.default_rng(34)
+    a, b = rnd.standard_normal((2, 3, 4, 5)).astype(np.float32), rnd.standard_normal((2, 3, 4, 2)).astype(np.float32)
+    y = ops.concat(a, b)
+    assert y.shape == (2, 3, 4, 7) and np.array_equal(y[..., :5], a) and np.array_equal(y[..., 5:], b)
+    part = np.full_like(y, np.inf)
+    ops.concat(a, b, rows=(2, 3), out=part)
+    assert np.array_equal(part[:, 2:3], y[:, 2:3]) and np.all(np.isinf(part[:, :2]))
+
+
+def test_gelu_identities():
+    import math
+    x = np.linspace(-6, 6, 97, dtype=np.float32).reshape(1, 1, 97, 1)
+    w = np.ones((1, 1, 1, 1), dtype=np.float32)
+    g = ops.conv2d(x, w, act=3).reshape(-1)
+    gm = ops.conv2d(-x, w, act=3).reshape(-1)
+    xs = x.reshape(-1)
+    assert np.max(np.abs((g - gm) - xs)) < 1e-6                         # x Phi(x) + x Phi(-x) = x
+    assert abs(g[48]) == 0.0 and abs(g[-1] - 6.0) < 1e-6 and abs(gm[-1]) < 1e-6
+    one = ops.conv2d(np.ones((1, 1, 1, 1), dtype=np.float32), w, act=3)[0, 0, 0, 0]
+    assert abs(one - 0.5 * (1.0 + math.erf(1.0 / math.sqrt(2.0)))) < 1e-7     # Phi(1) = 0.8413447...
+    assert abs(one - 0.8413447) < 1e-6

@@ -241,7 +241,8 @@ def test_csp_stack_one_row_bands():
 
 # ----------------------------------------------------------------------------- invariants
 @pytest.mark.parametrize("name,kw", [("vgg_block", dict(H=40, W=8)), ("resnet18", dict(H=64, W=8, width=8)),
-                                     ("resnet50", dict(H=64, W=8, width=8, N=1)), ("csp_stack", dict(H=256, W=32))])
+                                     ("resnet50", dict(H=64, W=8, width=8, N=1)), ("csp_stack", dict(H=256, W=32)),
+                                     ("convnext_block", dict(H=23, W=8, C=8)), ("dense_layer", dict(H=14, W=6, C=8, growth=4))])
 def test_invariants(name, kw):
     wl = li.build(name, with_data=False, **kw)
     H, W, C = wl.H, wl.W, wl.C
@@ -297,7 +298,8 @@ def test_invalid_layer_lists_are_rejected():
 # ----------------------------------------------------------------------------- stitched == whole
 SMALL = [("single_conv", dict(H=13, W=6, C=4)), ("vgg_block", dict(H=22, W=10, width=8)),
          ("resnet18", dict(H=48, W=16, width=8)), ("resnet50", dict(N=2, H=40, W=16, width=4, depths=(2, 1, 2, 1))),
-         ("csp_stack", dict(H=96, W=32, base=4))]
+         ("csp_stack", dict(H=96, W=32, base=4)), ("pointwise_mlp", dict(H=9, W=7, C=8, hidden=24)),
+         ("convnext_block", dict(H=17, W=9, C=8)), ("dense_layer", dict(H=11, W=6, C=8, growth=4))]
 
 
 @pytest.mark.parametrize("name,kw", SMALL)
@@ -379,5 +381,30 @@ def test_row_wise_operators_need_no_halo():
         assert plan.input_need[b][:2] == band
     bad = li.linear(8, 8)
     bad.input_from, bad.kh = -1, 3
+    with pytest.raises(planner.PlanError):
+        planner.make_plan([bad], 8, 8, 8, 2)
+
+
+def test_convnext_block_and_dense_layer_ranges():
+    """Depth-wise 7x7: three rows of halo at the block's first layer, none behind it; concatenation: both inputs 1:1."""
+    wl = li.build("convnext_block", with_data=False)
+    seg = wl.segments[0]
+    plan = planner.make_plan(seg.layers, wl.H, wl.W, wl.C, seg.n_bands)
+    for b in range(seg.n_bands):
+        lo, hi = (b * wl.H) // seg.n_bands, ((b + 1) * wl.H) // seg.n_bands
+        assert rows_of(plan.ranges[b][0]) == clamp(lo - 3, hi + 2, wl.H)
+        for i in (1, 2, 3):
+            assert rows_of(plan.ranges[b][i]) == (lo, hi)
+        assert plan.input_need[b][:2] == clamp(lo - 3, hi + 2, wl.H)      # hull of the halo and the shortcut's own rows
+    wl = li.build("dense_layer", with_data=False)
+    seg = wl.segments[0]
+    plan = planner.make_plan(seg.layers, wl.H, wl.W, wl.C, seg.n_bands)
+    assert plan.shapes[-1] == (wl.H, wl.W, wl.C + 32)
+    for b in range(seg.n_bands):
+        lo, hi = (b * wl.H) // seg.n_bands, ((b + 1) * wl.H) // seg.n_bands
+        assert (plan.ranges[b][2].out_lo, plan.ranges[b][2].out_hi) == (lo, hi)
+        assert (plan.ranges[b][1].out_lo, plan.ranges[b][1].out_hi) == (lo, hi)       # the concatenation's second input
+        assert plan.input_need[b][:2] == clamp(lo - 1, hi, wl.H)                      # 3x3 halo through the 1x1
+    bad = li.concat(8, 4, input_from=-1)
     with pytest.raises(planner.PlanError):
         planner.make_plan([bad], 8, 8, 8, 2)
