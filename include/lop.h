@@ -45,8 +45,8 @@ typedef enum {
 } lop_status;
 
 enum { LOP_F32 = 0, LOP_BF16 = 1 };                         /* storage dtype                     */
-enum { LOP_CONV2D = 0, LOP_MAXPOOL2D = 1, LOP_LINEAR = 2 };
-enum { LOP_ACT_NONE = 0, LOP_ACT_RELU = 1, LOP_ACT_SILU = 2 };
+enum { LOP_CONV2D = 0, LOP_MAXPOOL2D = 1, LOP_LINEAR = 2, LOP_DWCONV2D = 3, LOP_LAYERNORM = 4, LOP_CONCAT = 5 };
+enum { LOP_ACT_NONE = 0, LOP_ACT_RELU = 1, LOP_ACT_SILU = 2, LOP_ACT_GELU = 3 };   /* GELU: t * Phi(t), erf form */
 enum { LOP_RES_NONE = 0, LOP_RES_PRE_ACT = 1, LOP_RES_POST_ACT = 2 };
 enum { LOP_INPUT = -1, LOP_NO_RESIDUAL = -2 };              /* special layer indices             */
 enum {
@@ -72,6 +72,15 @@ enum {
  * row; here every pixel's channel vector is a row of X, weight is [cout][cin], the epilogue is the convolution's,
  * and a band's rows depend on the same rows of the input and on nothing else.  Its window fields must be
  * kh = kw = sh = sw = dh = dw = 1, ph = pw = 0.
+ * LOP_DWCONV2D is the depth-wise convolution (a block-wise operator, Sec. IV-A): channel c is filtered by its own
+ * kernel,  acc[n,oh,ow,c] = sum_{a,b} x[n, oh*sh-ph+a*dh, ow*sw-pw+b*dw, c] * weight[c,a,b]  (weight [cout][kh][kw][1],
+ * cout == cin), followed by the convolution's epilogue (scale, shift, residual, activation).
+ * LOP_LAYERNORM normalises every pixel's channel vector (row-wise: a row depends on that row alone):
+ *   y[c] = scale[c] * (x[c] - mean) / sqrt(var + 1e-6) + shift[c],  mean and biased variance over the cin channels,
+ * scale / shift the learned gain and offset (NULL => 1 / 0); no window, no weight, act and residual ignored.
+ * LOP_CONCAT joins two tensors of the same height and width along the channels: the main input's cin channels
+ * first, then the cout - cin channels of the tensor residual_from names (residual_pos is ignored); no window, no
+ * parameters.  A band's rows depend on the same rows of both inputs.
  * input_from / residual_from name an earlier layer of the same list, or LOP_INPUT for the
  * chain input; residual_from == LOP_NO_RESIDUAL means none.  The list order is topological.
  * The three pointers are DEVICE pointers; they are stored, never dereferenced on the host,

@@ -165,7 +165,7 @@ int check_common(lop_plan_t *pl, const void *in, const void *out, const void *ws
         return LOP_EINVAL;
     }
     for (size_t i = 0; i < pl->layers.size(); ++i)
-        if (pl->layers[i].l.op == LOP_CONV2D && !pl->layers[i].l.weight) {
+        if ((pl->layers[i].l.op == LOP_CONV2D || pl->layers[i].l.op == LOP_DWCONV2D) && !pl->layers[i].l.weight) {
             set_error("layer %zu has no weight pointer (lop_plan_set_params)", i);
             return LOP_EINVAL;
         }
@@ -207,6 +207,12 @@ int run_layer(lop_plan_t *pl, int i, int lo, int hi, const void *in, void *out, 
     }
     if (l.op == LOP_MAXPOOL2D) {
         LOP_CUDA(launch_maxpool(pool_args(pl, i, in, out, ws, lo, hi), pl->dtype, s));
+    } else if (li.kernel == K_DWCONV) {
+        LOP_CUDA(launch_dwconv(conv_args(pl, i, in, out, ws, lo, hi), pl->dtype, s));
+    } else if (li.kernel == K_LAYERNORM) {
+        LOP_CUDA(launch_layernorm(conv_args(pl, i, in, out, ws, lo, hi), pl->dtype, s));
+    } else if (li.kernel == K_CONCAT) {
+        LOP_CUDA(launch_concat(conv_args(pl, i, in, out, ws, lo, hi), pl->dtype, s));
     } else {
         const ConvArgs a = conv_args(pl, i, in, out, ws, lo, hi);
         if (li.kernel == K_CONV_TC) {

@@ -9,7 +9,7 @@
 
 namespace lop {
 
-enum KernelFamily { K_POOL = 0, K_CONV_SIMT = 1, K_CONV_TC = 2 };
+enum KernelFamily { K_POOL = 0, K_CONV_SIMT = 1, K_CONV_TC = 2, K_DWCONV = 3, K_LAYERNORM = 4, K_CONCAT = 5 };
 
 struct LayerInfo {
     lop_layer l;

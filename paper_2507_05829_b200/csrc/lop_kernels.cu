@@ -24,6 +24,7 @@ __device__ __forceinline__ float activate(float t, int act)
 {
     if (act == LOP_ACT_RELU) return fmaxf(t, 0.0f);
     if (act == LOP_ACT_SILU) return t / (1.0f + expf(-t));
+    if (act == LOP_ACT_GELU) return 0.5f * t * (1.0f + erff(t * 0.70710678f));
     return t;
 }
 

@@ -29,6 +29,11 @@ struct PoolArgs {
 // CUDA-core convolution (fp32 accumulate); dtype: LOP_F32 / LOP_BF16 storage.
 cudaError_t launch_conv_simt(const ConvArgs &a, int dtype, cudaStream_t s);
 cudaError_t launch_maxpool(const PoolArgs &a, int dtype, cudaStream_t s);
+// Depth-wise convolution (w: [C][kh][kw], Cout == Cin), layer normalisation over the channels (scale / shift = gain /
+// offset; the window fields are unused) and channel concatenation (x: Cin channels, res: Cout - Cin channels).
+cudaError_t launch_dwconv(const ConvArgs &a, int dtype, cudaStream_t s);
+cudaError_t launch_layernorm(const ConvArgs &a, int dtype, cudaStream_t s);
+cudaError_t launch_concat(const ConvArgs &a, int dtype, cudaStream_t s);
 // rows [lo,hi) of the patch tensor y[N,Ho,Wo,Kcol] of a thin chain input x[N,H,W,C] (bf16 only).
 struct GatherGeom;
 cudaError_t launch_stem_gather(const void *x, void *y, const GatherGeom &g, int lo, int hi, cudaStream_t s);

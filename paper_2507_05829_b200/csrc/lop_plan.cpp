@@ -97,13 +97,15 @@ static int check_layers(lop_plan_t &pl)
     const int L = (int)pl.layers.size();
     for (int i = 0; i < L; ++i) {
         LayerInfo &li = pl.layers[i];
-        if (li.l.op != LOP_CONV2D && li.l.op != LOP_MAXPOOL2D && li.l.op != LOP_LINEAR) { set_error("layer %d: unknown op %d", i, li.l.op); return LOP_EINVAL; }
-        if (li.l.op == LOP_LINEAR) {
+        if (li.l.op < LOP_CONV2D || li.l.op > LOP_CONCAT) { set_error("layer %d: unknown op %d", i, li.l.op); return LOP_EINVAL; }
+        if (li.l.op == LOP_LINEAR || li.l.op == LOP_LAYERNORM || li.l.op == LOP_CONCAT) {
             const lop_layer &q = li.l;
             if (q.kh != 1 || q.kw != 1 || q.sh != 1 || q.sw != 1 || q.dh != 1 || q.dw != 1 || q.ph != 0 || q.pw != 0) {
                 set_error("layer %d: a row-wise operator has no window (kh = kw = sh = sw = dh = dw = 1, ph = pw = 0)", i);
                 return LOP_EINVAL;
             }
+        }
+        if (li.l.op == LOP_LINEAR) {
             // Y = X * W^T over the channel vectors of the pixels is the pointwise convolution with the same [cout][cin]
             // matrix: from here on the layer is planned and executed as one (rows map one to one, no halo)
             li.linear = true;
@@ -115,7 +117,7 @@ static int check_layers(lop_plan_t &pl)
             set_error("layer %d: kernel/stride/dilation must be >= 1, padding >= 0, channels >= 1", i);
             return LOP_ESHAPE;
         }
-        if (l.act < LOP_ACT_NONE || l.act > LOP_ACT_SILU) { set_error("layer %d: unknown activation", i); return LOP_EINVAL; }
+        if (l.act < LOP_ACT_NONE || l.act > LOP_ACT_GELU) { set_error("layer %d: unknown activation", i); return LOP_EINVAL; }
         if (l.input_from < LOP_INPUT || l.input_from >= i) {
             set_error("layer %d: input_from=%d must be LOP_INPUT or an earlier layer", i, l.input_from);
             return LOP_ESHAPE;
@@ -124,25 +126,41 @@ static int check_layers(lop_plan_t &pl)
         if (l.input_from == LOP_INPUT) { hin = pl.H; win = pl.W; cin = pl.C; }
         else { const LayerInfo &s = pl.layers[l.input_from]; hin = s.Ho; win = s.Wo; cin = s.Co; }
         if (cin != l.cin) { set_error("layer %d: cin=%d but its input has %d channels", i, l.cin, cin); return LOP_ESHAPE; }
-        if (l.op == LOP_MAXPOOL2D && l.cout != l.cin) { set_error("layer %d: pooling keeps the channel count", i); return LOP_ESHAPE; }
+        if ((l.op == LOP_MAXPOOL2D || l.op == LOP_DWCONV2D || l.op == LOP_LAYERNORM) && l.cout != l.cin) {
+            set_error("layer %d: pooling, depth-wise convolution and layer normalisation keep the channel count", i);
+            return LOP_ESHAPE;
+        }
         li.Hin = hin; li.Win = win;
         li.Ho = window_out(hin, l.kh, l.sh, l.ph, l.dh);
         li.Wo = window_out(win, l.kw, l.sw, l.pw, l.dw);
         li.Co = l.cout;
         if (li.Ho <= 0 || li.Wo <= 0) { set_error("layer %d: empty output (%d x %d)", i, li.Ho, li.Wo); return LOP_ESHAPE; }
+        if (l.op == LOP_DWCONV2D && (long long)l.kh * l.kw > 1024) {
+            set_error("layer %d: a depth-wise filter of more than 1024 taps is not supported", i);
+            return LOP_EUNSUPPORTED;
+        }
         if (l.residual_from != LOP_NO_RESIDUAL) {
             if (l.residual_from < LOP_INPUT || l.residual_from >= i) {
                 set_error("layer %d: residual_from=%d must be LOP_INPUT or an earlier layer", i, l.residual_from);
                 return LOP_ESHAPE;
             }
-            if (l.op != LOP_CONV2D || (l.residual_pos != LOP_RES_PRE_ACT && l.residual_pos != LOP_RES_POST_ACT)) {
+            const bool conv_like = l.op == LOP_CONV2D || l.op == LOP_DWCONV2D;
+            if (l.op != LOP_CONCAT && (!conv_like || (l.residual_pos != LOP_RES_PRE_ACT && l.residual_pos != LOP_RES_POST_ACT))) {
                 set_error("layer %d: a residual needs a convolution and residual_pos PRE_ACT or POST_ACT", i);
                 return LOP_ESHAPE;
             }
             int rh, rw, rc;
             if (l.residual_from == LOP_INPUT) { rh = pl.H; rw = pl.W; rc = pl.C; }
             else { const LayerInfo &s = pl.layers[l.residual_from]; rh = s.Ho; rw = s.Wo; rc = s.Co; }
-            if (rh != li.Ho || rw != li.Wo || rc != li.Co) { set_error("layer %d: residual shape mismatch", i); return LOP_ESHAPE; }
+            const int want_c = l.op == LOP_CONCAT ? li.Co - l.cin : li.Co;
+            if (rh != li.Ho || rw != li.Wo || rc != want_c || want_c < 1) {
+                set_error(l.op == LOP_CONCAT ? "layer %d: the second input of a concatenation must have cout - cin channels and the main input's height and width"
+                                             : "layer %d: residual shape mismatch", i);
+                return LOP_ESHAPE;
+            }
+        } else if (l.op == LOP_CONCAT) {
+            set_error("layer %d: a concatenation names its second input in residual_from", i);
+            return LOP_ESHAPE;
         }
     }
     return LOP_OK;
@@ -199,6 +217,9 @@ static void choose_kernels(lop_plan_t &pl)
         li.cin_eff = l.cin;
         li.stem_gather = false;
         if (l.op == LOP_MAXPOOL2D) { li.kernel = K_POOL; continue; }
+        if (l.op == LOP_DWCONV2D) { li.kernel = K_DWCONV; continue; }
+        if (l.op == LOP_LAYERNORM) { li.kernel = K_LAYERNORM; continue; }
+        if (l.op == LOP_CONCAT) { li.kernel = K_CONCAT; continue; }
         li.kernel = K_CONV_SIMT;
         if (!tc_ok) continue;
         if (l.cout % 16 != 0 || l.sh * l.sw > 4) continue;
@@ -244,6 +265,8 @@ static void choose_kernels(lop_plan_t &pl)
     for (auto &li : pl.layers)
         if (li.l.op == LOP_CONV2D)
             pl.flops += 2.0 * pl.N * li.Ho * li.Wo * li.Co * (double)li.l.kh * li.l.kw * li.l.cin;
+        else if (li.l.op == LOP_DWCONV2D)
+            pl.flops += 2.0 * pl.N * li.Ho * li.Wo * li.Co * (double)li.l.kh * li.l.kw;
 }
 
 }  // namespace lop

@@ -205,6 +205,7 @@ bool program_supported(const lop_plan_t *pl)
     if (pl->dtype != LOP_BF16) return false;
     for (const auto &li : pl->layers) {
         if (li.l.op == LOP_CONV2D && li.kernel != K_CONV_TC) return false;
+        if (li.l.op != LOP_CONV2D && li.l.op != LOP_MAXPOOL2D) return false;      // depth-wise, layer norm, concat: per-layer kernels
         if (li.l.op == LOP_MAXPOOL2D && li.l.cin % 8 != 0) return false;
     }
     return true;

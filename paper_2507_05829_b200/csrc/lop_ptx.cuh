@@ -124,6 +124,7 @@ __device__ __forceinline__ float activate_t(float t)
 {
     if (ACT == LOP_ACT_RELU) return fmaxf(t, 0.0f);
     if (ACT == LOP_ACT_SILU) return __fdividef(t, 1.0f + __expf(-t));
+    if (ACT == LOP_ACT_GELU) return 0.5f * t * (1.0f + erff(t * 0.70710678f));     // t * Phi(t), the exact form
     return t;
 }
 
@@ -147,6 +148,7 @@ __device__ __forceinline__ void finish16(float (&v)[16], const float (&rv)[16], 
 {
     if (act == LOP_ACT_RELU) finish16_t<LOP_ACT_RELU>(v, rv, res_pos);
     else if (act == LOP_ACT_SILU) finish16_t<LOP_ACT_SILU>(v, rv, res_pos);
+    else if (act == LOP_ACT_GELU) finish16_t<LOP_ACT_GELU>(v, rv, res_pos);
     else finish16_t<LOP_ACT_NONE>(v, rv, res_pos);
 }
 

@@ -78,7 +78,7 @@ extern "C" int lop_run_whole_static(lop_plan_t *pl, const void *in, void *out, u
     }
     const int L = (int)pl->layers.size();
     for (int i = 0; i < L; ++i)
-        if (pl->layers[i].l.op == LOP_CONV2D && !pl->layers[i].l.weight) {
+        if ((pl->layers[i].l.op == LOP_CONV2D || pl->layers[i].l.op == LOP_DWCONV2D) && !pl->layers[i].l.weight) {
             set_error("layer %d has no weight pointer (lop_plan_set_params)", i);
             return LOP_EINVAL;
         }
@@ -98,6 +98,9 @@ extern "C" int lop_run_whole_static(lop_plan_t *pl, const void *in, void *out, u
             continue;
         }
         const ConvArgs a = conv_args(pl, i, in, out, ws, 0, li.Ho);
+        if (li.kernel == K_DWCONV) { ST_CUDA(launch_dwconv(a, pl->dtype, s)); continue; }
+        if (li.kernel == K_LAYERNORM) { ST_CUDA(launch_layernorm(a, pl->dtype, s)); continue; }
+        if (li.kernel == K_CONCAT) { ST_CUDA(launch_concat(a, pl->dtype, s)); continue; }
         if (li.kernel != K_CONV_TC) {
             ST_CUDA(launch_conv_simt(a, pl->dtype, s));
             continue;

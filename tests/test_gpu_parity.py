@@ -195,10 +195,57 @@ def test_maxpool(dtype, C, k, s, p):
     res = check_workload(wl, modes=("whole", "banded"), tol=0.0)   # pooling only selects: exact
 
 
+# ------------------------------------------------------------------------------------ depth-wise, layer norm, concat, GELU
+@pytest.mark.parametrize("dtype,C", [("bf16", 64), ("bf16", 40), ("bf16", 6), ("f32", 8), ("f32", 3)])
+@pytest.mark.parametrize("k,s,p,d", [(7, 1, 3, 1), (3, 2, 1, 1), (3, 1, 2, 2), (5, 1, 0, 1)])
+def test_depthwise_convolution(dtype, C, k, s, p, d):
+    l = li.dwconv(C, k, s=s, p=p, d=d, act=li.ACT_GELU)
+    check_workload(one_layer(l, 2, 23, 18, dtype=dtype, n_bands=4), modes=("whole", "banded", "pipelined"))
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("pos,act", [(li.RES_PRE_ACT, li.ACT_RELU), (li.RES_POST_ACT, li.ACT_SILU)])
+def test_depthwise_convolution_with_a_shortcut(dtype, pos, act):
+    l = li.dwconv(32, 3, act=act, residual_from=-1, residual_pos=pos)
+    check_workload(one_layer(l, 2, 14, 11, dtype=dtype), modes=("whole", "banded"))
+    check_workload(one_layer(l, 2, 14, 11, dtype=dtype), flags=lop.LOP_FLAG_REUSE_HALO, modes=("whole", "banded"))
+
+
+@pytest.mark.parametrize("dtype,C", [("bf16", 64), ("bf16", 520), ("bf16", 40), ("bf16", 7), ("f32", 12), ("f32", 5), ("f32", 260)])
+def test_layer_normalisation(dtype, C):
+    wl = one_layer(li.layernorm(C), 2, 13, 9, dtype=dtype)
+    wl.x = (wl.x * 3.0 + 1.5).astype(np.float32)               # a mean and a spread the normalisation has to remove
+    if dtype == "bf16":
+        wl.x = li.round_to_bf16(wl.x)
+    check_workload(wl, modes=("whole", "banded", "pipelined"))
+
+
+@pytest.mark.parametrize("dtype,ca,cb", [("bf16", 16, 8), ("bf16", 64, 32), ("bf16", 5, 3), ("f32", 8, 4), ("f32", 3, 2)])
+def test_concatenation(dtype, ca, cb):
+    layers = [conv(ca, cb, 3, act=li.ACT_RELU), li.concat(ca, cb, input_from=-1, second_from=0)]
+    layers[0].input_from = -1
+    wl = Workload("concat", dtype, 2, 12, 10, ca, [Segment(layers, 3)], seed=21)
+    li.fill_parameters(wl)
+    li.make_input(wl)
+    for flags in (0, lop.LOP_FLAG_REUSE_HALO):
+        res = check_workload(wl, flags=flags, modes=("whole", "banded", "pipelined"))
+        assert np.array_equal(res["whole"][0][..., :ca], wl.x)                 # the copied half is bit-exact
+
+
+@pytest.mark.parametrize("dtype,cin,cout,flags", [("bf16", 64, 64, 0), ("bf16", 64, 64, lop.LOP_FLAG_PER_LAYER),
+                                                  ("bf16", 64, 64, lop.LOP_FLAG_FORCE_SIMT), ("f32", 5, 9, 0)])
+def test_gelu_in_the_convolution_epilogue(dtype, cin, cout, flags):
+    """The persistent kernel's, the per-layer tensor-core kernel's and the CUDA-core kernel's epilogues."""
+    wl = one_layer(conv(cin, cout, 3, act=li.ACT_GELU), 2, 20, 16, dtype=dtype)
+    check_workload(wl, flags=flags, modes=("whole", "banded"))
+
+
 # ------------------------------------------------------------------------------------ chains, reduced sizes
 SMALL = [("vgg_block", dict(H=44, W=36)), ("resnet18", dict(H=64, W=64)),
          ("resnet50", dict(N=2, H=64, W=64, depths=(2, 2, 2, 2))), ("csp_stack", dict(H=256, W=128)),
-         ("pointwise_mlp", dict(H=21, W=19, C=64, hidden=192, n_bands=4))]      # row-wise operators (Sec. IV-A, Eq. 1)
+         ("pointwise_mlp", dict(H=21, W=19, C=64, hidden=192, n_bands=4)),      # row-wise operators (Sec. IV-A, Eq. 1)
+         ("convnext_block", dict(H=29, W=17, C=64, n_bands=5)), ("dense_layer", dict(H=19, W=14, n_bands=3)),
+         ("convnext_block", dict(H=15, W=9, C=12, n_bands=3, dtype="f32"))]
 
 
 @pytest.mark.parametrize("name,kw", SMALL)
@@ -715,7 +762,7 @@ def test_wavefront_and_per_layer_executors_agree_bit_for_bit():
 
 
 # ------------------------------------------------------------------------------------ the named configurations, full size
-@pytest.mark.parametrize("name", ["vgg_block", "resnet18", "csp_stack", "pointwise_mlp"])
+@pytest.mark.parametrize("name", ["vgg_block", "resnet18", "csp_stack", "pointwise_mlp", "convnext_block", "dense_layer"])
 def test_named_configurations_full_size(name):
     check_workload(li.build(name), flags=lop.LOP_FLAG_REUSE_HALO, modes=("whole", "pipelined", "pipelined_copy"))
 
