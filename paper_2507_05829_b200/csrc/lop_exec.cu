@@ -183,9 +183,10 @@ int prepare_workspace(lop_plan_t *pl, void *ws, cudaStream_t s)
     }
     for (size_t i = 0; i < pl->layers.size(); ++i) {
         LayerInfo &li = pl->layers[i];
-        if (!li.stem_gather) continue;
+        if (!li.stem_gather && !li.dw_transposed) continue;
         if (!fresh && e->prepared_w[i] == li.l.weight) continue;
-        LOP_CUDA(launch_pad_weights(li.l.weight, base + li.wpad_off, li.l.cout, li.l.kh * li.l.kw * li.l.cin, li.cin_eff, s));
+        if (li.stem_gather) LOP_CUDA(launch_pad_weights(li.l.weight, base + li.wpad_off, li.l.cout, li.l.kh * li.l.kw * li.l.cin, li.cin_eff, s));
+        else LOP_CUDA(launch_dw_transpose(li.l.weight, base + li.wpad_off, li.l.cin, li.l.kh * li.l.kw, s));
         e->prepared_w[i] = li.l.weight;
         e->launches++;
     }
@@ -208,7 +209,7 @@ int run_layer(lop_plan_t *pl, int i, int lo, int hi, const void *in, void *out, 
     if (l.op == LOP_MAXPOOL2D) {
         LOP_CUDA(launch_maxpool(pool_args(pl, i, in, out, ws, lo, hi), pl->dtype, s));
     } else if (li.kernel == K_DWCONV) {
-        LOP_CUDA(launch_dwconv(conv_args(pl, i, in, out, ws, lo, hi), pl->dtype, s));
+        LOP_CUDA(launch_dwconv(conv_args(pl, i, in, out, ws, lo, hi), pl->dtype, li.dw_transposed ? static_cast<char *>(ws) + li.wpad_off : nullptr, s));
     } else if (li.kernel == K_LAYERNORM) {
         LOP_CUDA(launch_layernorm(conv_args(pl, i, in, out, ws, lo, hi), pl->dtype, s));
     } else if (li.kernel == K_CONCAT) {

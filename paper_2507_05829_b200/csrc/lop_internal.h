@@ -21,7 +21,9 @@ struct LayerInfo {
     bool stem_gather = false;      // thin chain input: the layer's receptive patches are gathered into a
                                    // [N, Ho, Wo, Kcol] tensor first and the convolution runs as 1x1 over it
     size_t out_off = 0;            // workspace offset of the full-size output (unused for the last layer)
-    size_t wpad_off = 0;           // workspace offset of the [cout][Kcol] zero-padded weights (if stem_gather)
+    size_t wpad_off = 0;           // workspace offset of the [cout][Kcol] zero-padded weights (if stem_gather), of the
+                                   // [taps][C] transposed filters (if dw_transposed)
+    bool dw_transposed = false;    // bf16 depth-wise convolution with C % 8 == 0: the workspace keeps its filters tap-major
 };
 
 struct ExecState;                  // CUDA-side resources, defined in lop_exec.cu

@@ -31,9 +31,12 @@ cudaError_t launch_conv_simt(const ConvArgs &a, int dtype, cudaStream_t s);
 cudaError_t launch_maxpool(const PoolArgs &a, int dtype, cudaStream_t s);
 // Depth-wise convolution (w: [C][kh][kw], Cout == Cin), layer normalisation over the channels (scale / shift = gain /
 // offset; the window fields are unused) and channel concatenation (x: Cin channels, res: Cout - Cin channels).
-cudaError_t launch_dwconv(const ConvArgs &a, int dtype, cudaStream_t s);
+// w_taps: the filters as [tap][C] (launch_dw_transpose), or nullptr -- the tiled bf16 kernel needs them.
+cudaError_t launch_dwconv(const ConvArgs &a, int dtype, const void *w_taps, cudaStream_t s);
 cudaError_t launch_layernorm(const ConvArgs &a, int dtype, cudaStream_t s);
 cudaError_t launch_concat(const ConvArgs &a, int dtype, cudaStream_t s);
+// depth-wise filters w[C][taps] -> wt[taps][C] (bf16 only), the layout the persistent kernel reads
+cudaError_t launch_dw_transpose(const void *w, void *wt, int C, int taps, cudaStream_t s);
 // rows [lo,hi) of the patch tensor y[N,Ho,Wo,Kcol] of a thin chain input x[N,H,W,C] (bf16 only).
 struct GatherGeom;
 cudaError_t launch_stem_gather(const void *x, void *y, const GatherGeom &g, int lo, int hi, cudaStream_t s);

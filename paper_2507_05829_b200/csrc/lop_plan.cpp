@@ -217,7 +217,8 @@ static void choose_kernels(lop_plan_t &pl)
         li.cin_eff = l.cin;
         li.stem_gather = false;
         if (l.op == LOP_MAXPOOL2D) { li.kernel = K_POOL; continue; }
-        if (l.op == LOP_DWCONV2D) { li.kernel = K_DWCONV; continue; }
+        li.dw_transposed = false;
+        if (l.op == LOP_DWCONV2D) { li.kernel = K_DWCONV; li.dw_transposed = pl.dtype == LOP_BF16 && l.cin % 8 == 0; continue; }
         if (l.op == LOP_LAYERNORM) { li.kernel = K_LAYERNORM; continue; }
         if (l.op == LOP_CONCAT) { li.kernel = K_CONCAT; continue; }
         li.kernel = K_CONV_SIMT;
@@ -254,6 +255,10 @@ static void choose_kernels(lop_plan_t &pl)
             off += align_up((size_t)pl.N * li.Ho * li.Wo * li.cin_eff * es, 1024);
             li.wpad_off = off;
             off += align_up((size_t)li.l.cout * li.cin_eff * es, 1024);
+        }
+        if (li.dw_transposed) {
+            li.wpad_off = off;
+            off += align_up((size_t)li.l.kh * li.l.kw * li.l.cin * es, 1024);
         }
         if (i != L - 1) {
             li.out_off = off;

@@ -14,6 +14,7 @@
 #include "lop_kernels.cuh"
 #include "lop_layerargs.h"
 #include "lop_program.h"
+#include "lop_rowops.cuh"
 #include "lop_wavefront.cuh"
 
 namespace lop {
@@ -55,6 +56,7 @@ namespace {
 #define LOP_CPS_MAX 4
 #endif
 constexpr uint32_t A_BOX_MAX = 48u * 1024u;     // largest activation box a ring slot is sized for
+constexpr uint32_t LOP_ROWOP_STAGING_BYTES = 32u * 1024u;    // largest receptive window a depth-wise item stages
 constexpr uint32_t B_BOX_MAX = 32u * 1024u;     // largest weight box
 
 int ilog2i(int v) { int l = 0; while ((1 << l) < v) ++l; return l; }
@@ -198,6 +200,16 @@ bool pool_fusable(const lop_plan_t *pl, int i)
 
 }  // namespace
 
+// Item shape of a depth-wise stage in the persistent kernel (rows, columns and channels of one tile).
+static bool dw_tile(const lop_plan_t *pl, const LayerInfo &li, rowop::DwTile *t)
+{
+    const lop_layer &l = li.l;
+    rowop::DwTile tmp;
+    if (!li.dw_transposed) return false;
+    return rowop::dw_choose_tile(l.kh, l.kw, l.sh, l.sw, l.dh, l.dw, pl->N, li.Ho, li.Wo, l.cin, LOP_ROWOP_STAGING_BYTES, 32 * WF_WORKER_WARPS,
+                                 t ? t : &tmp);
+}
+
 bool program_folds_pool(const lop_plan_t *pl, int layer) { return pool_fusable(pl, layer); }
 
 bool program_supported(const lop_plan_t *pl)
@@ -205,7 +217,10 @@ bool program_supported(const lop_plan_t *pl)
     if (pl->dtype != LOP_BF16) return false;
     for (const auto &li : pl->layers) {
         if (li.l.op == LOP_CONV2D && li.kernel != K_CONV_TC) return false;
-        if (li.l.op != LOP_CONV2D && li.l.op != LOP_MAXPOOL2D) return false;      // depth-wise, layer norm, concat: per-layer kernels
+        // the worker warps move these in 16-byte vectors of eight channels
+        if (li.l.op == LOP_DWCONV2D && !dw_tile(pl, li, nullptr)) return false;
+        if (li.l.op == LOP_LAYERNORM && (li.l.cin % 8 != 0 || li.l.cin > 1024)) return false;     // a lane keeps at most four vectors
+        if (li.l.op == LOP_CONCAT && (li.l.cin % 8 != 0 || li.l.cout % 8 != 0)) return false;
         if (li.l.op == LOP_MAXPOOL2D && li.l.cin % 8 != 0) return false;
     }
     return true;
@@ -226,6 +241,12 @@ struct Ctx {
     int patches_id(int seg) const { return base[seg] + (int)segs[seg].pl->layers.size(); }
     int input_id(int seg) const { return tensor_id(seg - 1, (int)segs[seg - 1].pl->layers.size() - 1); }
 };
+
+// A convolution's shortcut, a concatenation's second tensor: read at the rows that are computed.
+bool has_second_input(const lop_layer &l)
+{
+    return (l.op == LOP_CONV2D || l.op == LOP_DWCONV2D || l.op == LOP_CONCAT) && l.residual_from != LOP_NO_RESIDUAL;
+}
 
 // Rows [o0, o1) of request rq: the tensors and rows they are computed from (Sec. IV-B: a dependency exists as soon as
 // any part of a producer's output is used).
@@ -253,7 +274,7 @@ Reads reads_of(const Ctx &cx, const StageReq &rq, int o0, int o1)
     } else if (window(a, b)) {
         r.need[r.n++] = Need{cx.tensor_id(rq.seg, l.input_from), a, b, true};
     }
-    if (!rq.gather && l.op == LOP_CONV2D && l.residual_from != LOP_NO_RESIDUAL) {
+    if (!rq.gather && has_second_input(l)) {
         if (l.residual_from >= 0) r.need[r.n++] = Need{cx.tensor_id(rq.seg, l.residual_from), o0, o1, true};
         else if (rq.seg == 0) {
             r.raw = true;
@@ -274,7 +295,13 @@ StageShape stage_shape(const Ctx &cx, const StageReq &rq)
     const LayerInfo &li = pl->layers[rq.layer];
     const double rows = rq.hi - rq.lo;
     if (rq.fetch) return StageShape{0, rows * pl->W * pl->C * 2.0 * pl->N / 24e3, 0.0};      // ~24 GB/s measured for SM-issued reads
-    if (rq.gather || li.l.op == LOP_MAXPOOL2D) return StageShape{(int)rows * pl->N, 2.5, 0.5};
+    if (rq.gather || li.l.op == LOP_MAXPOOL2D || li.l.op == LOP_CONCAT) return StageShape{(int)rows * pl->N, 2.5, 0.5};
+    if (li.l.op == LOP_LAYERNORM) return StageShape{(int)rows * pl->N, 4.0, 0.5};
+    if (li.l.op == LOP_DWCONV2D) {
+        rowop::DwTile t{1, 1, 8};
+        dw_tile(pl, li, &t);
+        return StageShape{(int)((rows + t.R - 1) / t.R) * pl->N * ((li.Wo + t.tw - 1) / t.tw) * (li.l.cin / t.cc), 4.0, 0.5};
+    }
     const double tiles = std::ceil(rows * li.Wo * pl->N / 128.0) * std::max(1, li.l.cout / 128);
     // operand boxes, ~0.2 us each (issue, and the wait for a free ring slot): one per (tap, 64-channel chunk) and operand for strided windows, one
     // activation box and a few weight boxes per chunk otherwise
@@ -541,6 +568,24 @@ int program_build(const std::vector<SegBind> &segs, std::vector<StageReq> reqs, 
             st.x = a.x; st.y = a.y;
             st.N = a.N; st.Hin = a.Hin; st.Win = a.Win; st.Cin = a.C; st.Ho = a.Ho; st.Wo = a.Wo; st.Cout = a.C;
             st.kh = a.kh; st.kw = a.kw; st.sh = a.sh; st.sw = a.sw; st.ph = a.ph; st.pw = a.pw; st.dh = a.dh; st.dw = a.dw;
+        } else if (l.op == LOP_DWCONV2D || l.op == LOP_LAYERNORM || l.op == LOP_CONCAT) {
+            const ConvArgs a = conv_args(pl, rq.layer, in, out, ws, rq.lo, rq.hi);
+            st.kind = l.op == LOP_DWCONV2D ? WF_DWCONV : (l.op == LOP_LAYERNORM ? WF_LAYERNORM : WF_CONCAT);
+            st.x = a.x; st.res = a.res; st.scale = a.scale; st.shift = a.shift; st.y = a.y;
+            st.N = a.N; st.Hin = a.Hin; st.Win = a.Win; st.Cin = a.Cin; st.Ho = a.Ho; st.Wo = a.Wo; st.Cout = a.Cout;
+            st.kh = a.kh; st.kw = a.kw; st.sh = a.sh; st.sw = a.sw; st.ph = a.ph; st.pw = a.pw; st.dh = a.dh; st.dw = a.dw;
+            st.act = a.act; st.res_pos = a.res_pos;
+            if (l.op == LOP_DWCONV2D) {
+                rowop::DwTile t{1, 1, 8};
+                if (!dw_tile(pl, li, &t)) { set_error("layer %d: depth-wise window does not fit the staging tile", rq.layer); return LOP_EUNSUPPORTED; }
+                st.BN = t.cc; st.tw_valid = t.tw; st.tr_log = ilog2i(t.R);
+                st.w_taps = wsb + li.wpad_off;
+                group_rows = t.R;
+                tiles_r = (rows + t.R - 1) / t.R;
+                tiles_w = (li.Wo + t.tw - 1) / t.tw;
+                cout_tiles = l.cin / t.cc;
+                stg_bytes = std::max(stg_bytes, round_up_u32((uint32_t)rowop::dw_tile_bytes(l.kh, l.kw, l.sh, l.sw, l.dh, l.dw, t), 1024u));
+            }
         } else {
             const ConvArgs a = conv_args(pl, rq.layer, in, out, ws, rq.lo, rq.hi);
             // a 2x2 pooling that is this convolution's only reader, asked for exactly the rows this stage feeds it
@@ -618,7 +663,7 @@ int program_build(const std::vector<SegBind> &segs, std::vector<StageReq> reqs, 
                 long long a = (long long)o0 * l.sh - l.ph, b = (long long)(o1 - 1) * l.sh - l.ph + (long long)(l.kh - 1) * l.dh + 1;
                 const bool main_raw = rq.gather || (l.input_from == LOP_INPUT && !li.stem_gather);
                 if (!main_raw) { a = o0; b = o1; }                          // only the residual reads the chain input: its own rows
-                else if (!rq.gather && l.op == LOP_CONV2D && l.residual_from == LOP_INPUT) { a = std::min<long long>(a, o0); b = std::max<long long>(b, o1); }
+                else if (!rq.gather && has_second_input(l) && l.residual_from == LOP_INPUT) { a = std::min<long long>(a, o0); b = std::max<long long>(b, o1); }
                 a = std::max(a, 0LL); b = std::min<long long>(b, pl->H);
                 int last_leader = -1;
                 for (int b2 = 0; b2 < pl->n_bands; ++b2) {
@@ -744,6 +789,9 @@ int program_build(const std::vector<SegBind> &segs, std::vector<StageReq> reqs, 
     P.fetch_src = fetch_src;
     P.fetch_dst = const_cast<void *>(segs[0].in);
     P.n_fetch = (int)fetch_items.size();
+    P.row_ops = 0;
+    for (const WfStage &st : stages)
+        if (st.kind == WF_DWCONV || st.kind == WF_LAYERNORM || st.kind == WF_CONCAT) P.row_ops = 1;
     // entries in flight: about the link's bandwidth-delay product (some 25 GB/s x 3 us), at least a few warps' worth
     if (P.n_fetch > 0) {
         long long bytes = 0;

@@ -10,6 +10,7 @@
 
 #include "lop.h"
 #include "lop_kernels.cuh"
+#include "lop_rowops.cuh"
 
 namespace lop {
 
@@ -19,14 +20,6 @@ __device__ __forceinline__ float to_f32(float v) { return v; }
 __device__ __forceinline__ float to_f32(__nv_bfloat16 v) { return __bfloat162float(v); }
 __device__ __forceinline__ void from_f32(float &d, float v) { d = v; }
 __device__ __forceinline__ void from_f32(__nv_bfloat16 &d, float v) { d = __float2bfloat16_rn(v); }
-
-__device__ __forceinline__ float activate(float t, int act)
-{
-    if (act == LOP_ACT_RELU) return fmaxf(t, 0.0f);
-    if (act == LOP_ACT_SILU) return t / (1.0f + expf(-t));
-    if (act == LOP_ACT_GELU) return 0.5f * t * (1.0f + erff(t * 0.70710678f));
-    return t;
-}
 
 template <typename T, int VEC>
 struct alignas(sizeof(T) * VEC) Vec {
@@ -94,76 +87,83 @@ __global__ void __launch_bounds__(DW_THREADS) dwconv_kernel(ConvArgs p, int CV, 
         const long long o = (((long long)n * p.Ho + oh) * p.Wo + ow) * p.Cout + c;
         V rv, out;
         if (res) rv = *reinterpret_cast<const V *>(res + o);
+        const int res_pos = res ? p.res_pos : LOP_RES_NONE;
 #pragma unroll
-        for (int j = 0; j < VEC; ++j) {
-            float v = fmaf(p.scale ? p.scale[c + j] : 1.0f, acc[j], p.shift ? p.shift[c + j] : 0.0f);
-            if (res && p.res_pos == LOP_RES_PRE_ACT) v += to_f32(rv.v[j]);
-            v = activate(v, p.act);
-            if (res && p.res_pos == LOP_RES_POST_ACT) v += to_f32(rv.v[j]);
-            from_f32(out.v[j], v);
-        }
+        for (int j = 0; j < VEC; ++j)
+            from_f32(out.v[j], rowop::epilogue(acc[j], p.scale ? p.scale[c + j] : 1.0f, p.shift ? p.shift[c + j] : 0.0f,
+                                               res ? to_f32(rv.v[j]) : 0.0f, res_pos, p.act));
         *reinterpret_cast<V *>(y + o) = out;
     }
 }
 
-// ---------------------------------------------------------------------------------------------
-// Layer normalisation: one warp per pixel.  Mean, then the biased variance of the centred values (two passes, the
-// numerically safe order), then the scaled and shifted result; the second and third pass re-read the pixel's
-// channel vector from L1.  Partial sums are combined lane-wise by a fixed butterfly, the same for every pixel.
-// ---------------------------------------------------------------------------------------------
-constexpr float LAYERNORM_EPS = 1e-6f;
+// bf16 with a multiple of eight channels: one block per tile, the same tile routine the persistent kernel runs
+// (rowop::dwconv_tile), so that both executors give the same bits.  w_taps: the filters as [tap][C].
+constexpr int DW_TILE_THREADS = 256;
+constexpr long long DW_TILE_SMEM = 40 * 1024;
 
-__device__ __forceinline__ float warp_sum(float v)
+__global__ void __launch_bounds__(DW_TILE_THREADS) dwconv_tile_kernel(rowop::DwGeom g, int oh_lo, int oh_hi, int tiles_w)
 {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-    return v;
+    extern __shared__ float dw_sm[];
+    const int tile_w = blockIdx.x % tiles_w, tile_c = blockIdx.x / tiles_w;
+    const int oh0 = oh_lo + blockIdx.y * g.t.R, ow0 = tile_w * g.t.tw;
+    rowop::dwconv_tile<false, 0, DW_TILE_THREADS>(g, blockIdx.z, oh0, min(g.t.R, oh_hi - oh0), ow0, min(g.t.tw, g.Wo - ow0), tile_c * g.t.cc,
+                                                  dw_sm, threadIdx.x);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Layer normalisation: a group of lanes per pixel (a whole warp from 32 vectors per pixel on, a power-of-two part of
+// it below), lane `sub` owning every lanes-th vector.  Mean, then the biased variance of the centred values (two
+// passes, the numerically safe order), then the scaled and shifted result; the second and third pass re-read the
+// pixel's channel vector from L1.  Partial sums are combined by a fixed butterfly, the same for every pixel.
+// ---------------------------------------------------------------------------------------------
 template <typename T, int VEC>
 __global__ void __launch_bounds__(256) layernorm_kernel(ConvArgs p)
 {
     const int rows = p.oh_hi - p.oh_lo;
     const long long M = (long long)p.N * rows * p.Wo;
-    const long long m = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (m >= M) return;
-    const int lane = threadIdx.x & 31;
-    const int C = p.Cin;
-    const int ow = (int)(m % p.Wo);
-    const long long q = m / p.Wo;
-    const int oh = p.oh_lo + (int)(q % rows);
-    const int n = (int)(q / rows);
-    const long long o = (((long long)n * p.Ho + oh) * p.Wo + ow) * C;
+    const int C = p.Cin, nvec = C / VEC;
+    const int lanes_log = rowop::ln_lanes_log(nvec), lanes = 1 << lanes_log;
+    const int sub = threadIdx.x & (lanes - 1);
+    const long long m = (long long)blockIdx.x * (blockDim.x >> lanes_log) + (threadIdx.x >> lanes_log);
+    const bool live = m < M;                               // dead lanes still take part in the group sums
+    long long o = 0;
+    if (live) {
+        const int ow = (int)(m % p.Wo);
+        const long long q = m / p.Wo;
+        const int oh = p.oh_lo + (int)(q % rows);
+        const int n = (int)(q / rows);
+        o = (((long long)n * p.Ho + oh) * p.Wo + ow) * C;
+    }
     const T *__restrict__ x = static_cast<const T *>(p.x) + o;
     T *__restrict__ y = static_cast<T *>(p.y) + o;
     using V = Vec<T, VEC>;
 
     float s = 0.0f;
-    for (int c = lane * VEC; c < C; c += 32 * VEC) {
-        const V xv = *reinterpret_cast<const V *>(x + c);
+    for (int v = sub; live && v < nvec; v += lanes) {
+        const V xv = *reinterpret_cast<const V *>(x + v * VEC);
 #pragma unroll
         for (int j = 0; j < VEC; ++j) s += to_f32(xv.v[j]);
     }
-    const float mean = warp_sum(s) / (float)C;
+    const float mean = rowop::group_sum(s, lanes_log) / (float)C;
     float s2 = 0.0f;
-    for (int c = lane * VEC; c < C; c += 32 * VEC) {
-        const V xv = *reinterpret_cast<const V *>(x + c);
+    for (int v = sub; live && v < nvec; v += lanes) {
+        const V xv = *reinterpret_cast<const V *>(x + v * VEC);
 #pragma unroll
         for (int j = 0; j < VEC; ++j) {
             const float d = to_f32(xv.v[j]) - mean;
             s2 = fmaf(d, d, s2);
         }
     }
-    const float inv = 1.0f / sqrtf(warp_sum(s2) / (float)C + LAYERNORM_EPS);
-    for (int c = lane * VEC; c < C; c += 32 * VEC) {
-        const V xv = *reinterpret_cast<const V *>(x + c);
+    const float inv = rowop::ln_inv_std(rowop::group_sum(s2, lanes_log), C);
+    for (int v = sub; live && v < nvec; v += lanes) {
+        const V xv = *reinterpret_cast<const V *>(x + v * VEC);
         V out;
 #pragma unroll
         for (int j = 0; j < VEC; ++j) {
-            const float g = p.scale ? p.scale[c + j] : 1.0f, b = p.shift ? p.shift[c + j] : 0.0f;
-            from_f32(out.v[j], fmaf((to_f32(xv.v[j]) - mean) * inv, g, b));
+            const int c = v * VEC + j;
+            from_f32(out.v[j], rowop::ln_value(to_f32(xv.v[j]), mean, inv, p.scale ? p.scale[c] : 1.0f, p.shift ? p.shift[c] : 0.0f));
         }
-        *reinterpret_cast<V *>(y + c) = out;
+        *reinterpret_cast<V *>(y + v * VEC) = out;
     }
 }
 
@@ -190,6 +190,15 @@ __global__ void __launch_bounds__(256) concat_kernel(ConvArgs p)
     const V val = v < va ? *reinterpret_cast<const V *>(static_cast<const T *>(p.x) + pix * Ca + (long long)v * VEC)
                          : *reinterpret_cast<const V *>(static_cast<const T *>(p.res) + pix * Cb + (long long)(v - va) * VEC);
     *reinterpret_cast<V *>(static_cast<T *>(p.y) + pix * p.Cout + (long long)v * VEC) = val;
+}
+
+// [C][taps] -> [taps][C] (16-bit elements): the persistent kernel reads a tap's weights of eight channels as one vector.
+__global__ void __launch_bounds__(256) dw_transpose_kernel(const uint16_t *__restrict__ w, uint16_t *__restrict__ wt, int C, int taps)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= C * taps) return;
+    const int t = i / C, c = i - t * C;
+    wt[i] = w[(long long)c * taps + t];
 }
 
 template <typename T>
@@ -222,14 +231,20 @@ cudaError_t dwconv_dispatch(const ConvArgs &a, cudaStream_t s)
     return dwconv_launch<T, 1>(a, s);
 }
 
+template <typename T, int VEC>
+cudaError_t layernorm_launch(const ConvArgs &a, cudaStream_t s)
+{
+    const long long M = (long long)a.N * (a.oh_hi - a.oh_lo) * a.Wo;
+    const int per_block = 256 >> rowop::ln_lanes_log(a.Cin / VEC);
+    layernorm_kernel<T, VEC><<<(unsigned)((M + per_block - 1) / per_block), 256, 0, s>>>(a);
+    return cudaGetLastError();
+}
+
 template <typename T>
 cudaError_t layernorm_dispatch(const ConvArgs &a, cudaStream_t s)
 {
-    const long long M = (long long)a.N * (a.oh_hi - a.oh_lo) * a.Wo;
-    const unsigned grid = (unsigned)((M + 7) / 8);
-    if (a.Cin % full_vec<T>() == 0) layernorm_kernel<T, full_vec<T>()><<<grid, 256, 0, s>>>(a);
-    else layernorm_kernel<T, 1><<<grid, 256, 0, s>>>(a);
-    return cudaGetLastError();
+    if (a.Cin % full_vec<T>() == 0) return layernorm_launch<T, full_vec<T>()>(a, s);
+    return layernorm_launch<T, 1>(a, s);
 }
 
 template <typename T, int VEC>
@@ -250,10 +265,34 @@ cudaError_t concat_dispatch(const ConvArgs &a, cudaStream_t s)
 
 }  // namespace
 
-cudaError_t launch_dwconv(const ConvArgs &a, int dtype, cudaStream_t s)
+cudaError_t launch_dwconv(const ConvArgs &a, int dtype, const void *w_taps, cudaStream_t s)
 {
     if (a.oh_hi <= a.oh_lo) return cudaSuccess;
+    rowop::DwTile t;
+    if (dtype == LOP_BF16 && w_taps && a.N <= 65535 &&
+        rowop::dw_choose_tile(a.kh, a.kw, a.sh, a.sw, a.dh, a.dw, a.N, a.oh_hi - a.oh_lo, a.Wo, a.Cin, DW_TILE_SMEM, DW_TILE_THREADS, &t)) {
+        rowop::DwGeom g;
+        g.Hin = a.Hin; g.Win = a.Win; g.C = a.Cin; g.Ho = a.Ho; g.Wo = a.Wo;
+        g.kh = a.kh; g.kw = a.kw; g.sh = a.sh; g.sw = a.sw; g.ph = a.ph; g.pw = a.pw; g.dh = a.dh; g.dw = a.dw;
+        g.act = a.act; g.res_pos = a.res ? a.res_pos : LOP_RES_NONE;
+        g.t = t;
+        g.x = static_cast<const uint16_t *>(a.x); g.res = static_cast<const uint16_t *>(a.res);
+        g.w_taps = static_cast<const uint16_t *>(w_taps);
+        g.scale = a.scale; g.shift = a.shift; g.y = static_cast<uint16_t *>(a.y);
+        const int tiles_w = (a.Wo + t.tw - 1) / t.tw, tiles_r = (a.oh_hi - a.oh_lo + t.R - 1) / t.R;
+        if (tiles_r <= 65535) {
+            dim3 grid((unsigned)(tiles_w * (a.Cin / t.cc)), (unsigned)tiles_r, (unsigned)a.N);
+            dwconv_tile_kernel<<<grid, DW_TILE_THREADS, (size_t)rowop::dw_tile_bytes(a.kh, a.kw, a.sh, a.sw, a.dh, a.dw, t), s>>>(g, a.oh_lo, a.oh_hi, tiles_w);
+            return cudaGetLastError();
+        }
+    }
     return dtype == LOP_BF16 ? dwconv_dispatch<__nv_bfloat16>(a, s) : dwconv_dispatch<float>(a, s);
+}
+
+cudaError_t launch_dw_transpose(const void *w, void *wt, int C, int taps, cudaStream_t s)
+{
+    dw_transpose_kernel<<<(unsigned)((C * taps + 255) / 256), 256, 0, s>>>(static_cast<const uint16_t *>(w), static_cast<uint16_t *>(wt), C, taps);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_layernorm(const ConvArgs &a, int dtype, cudaStream_t s)

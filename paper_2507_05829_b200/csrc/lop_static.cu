@@ -98,7 +98,15 @@ extern "C" int lop_run_whole_static(lop_plan_t *pl, const void *in, void *out, u
             continue;
         }
         const ConvArgs a = conv_args(pl, i, in, out, ws, 0, li.Ho);
-        if (li.kernel == K_DWCONV) { ST_CUDA(launch_dwconv(a, pl->dtype, s)); continue; }
+        if (li.kernel == K_DWCONV) {
+            const void *w_taps = nullptr;
+            if (li.dw_transposed) {                    // rebuilt by every call, like the padded stem weights
+                ST_CUDA(launch_dw_transpose(l.weight, ws + li.wpad_off, l.cin, l.kh * l.kw, s));
+                w_taps = ws + li.wpad_off;
+            }
+            ST_CUDA(launch_dwconv(a, pl->dtype, w_taps, s));
+            continue;
+        }
         if (li.kernel == K_LAYERNORM) { ST_CUDA(launch_layernorm(a, pl->dtype, s)); continue; }
         if (li.kernel == K_CONCAT) { ST_CUDA(launch_concat(a, pl->dtype, s)); continue; }
         if (li.kernel != K_CONV_TC) {

@@ -9,8 +9,8 @@
 //   warp 2      one lane publishes finished items: after the workers' barrier it fences and does the release
 //               increment of the item's row-group counter, so that memory-fence latency is off the workers' path
 //   workers     epilogue of convolution items: TMEM -> scale/shift/residual/activation -> bf16 rows in a
-//               shared staging tile -> coalesced 16-byte stores; and the whole of pooling / patch-gather
-//               items.
+//               shared staging tile -> coalesced 16-byte stores; and the whole of pooling, patch-gather,
+//               depth-wise convolution, layer-normalisation and concatenation items.
 //               Many of them because straight-line per-element code needs several warps per scheduler to
 //               hide its own latency; the four warps that share a TMEM lane group split a tile's columns.
 //
@@ -29,6 +29,7 @@
 
 #include "lop_gather.cuh"
 #include "lop_ptx.cuh"
+#include "lop_rowops.cuh"
 #include "lop_wavefront.cuh"
 
 namespace lop {
@@ -182,6 +183,112 @@ __device__ __forceinline__ T ldg_ptr(const void *const *p)
     return reinterpret_cast<T>(__ldg(reinterpret_cast<const unsigned long long *>(p)));
 }
 
+// ---- the memory-bound operators, run by all worker threads (tid = 0 .. EPI_THREADS-1) on one item.  Kept out of line:
+// they are rare and long, and inlined they cost the convolution roles registers.
+__device__ __forceinline__ uint4 pack_bf16x8(const float (&v)[8])
+{
+    uint32_t h[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) h[j] = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(v[j]));
+    return make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), h[4] | (h[5] << 16), h[6] | (h[7] << 16));
+}
+
+// Depth-wise convolution item: 2^tr_log output rows x tw_valid columns x BN channels of image n (see
+// rowop::dwconv_tile); the window is read through L2 -- other SMs produced it during this launch.
+__device__ __noinline__ void dwconv_item(const WfStage *sp, int n, int tile_r, int tile_w, int tile_c, int tid, uint8_t *stg)
+{
+    rowop::DwGeom g;
+    g.Hin = __ldg(&sp->Hin); g.Win = __ldg(&sp->Win); g.C = __ldg(&sp->Cin); g.Ho = __ldg(&sp->Ho); g.Wo = __ldg(&sp->Wo);
+    g.kh = __ldg(&sp->kh); g.kw = __ldg(&sp->kw); g.sh = __ldg(&sp->sh); g.sw = __ldg(&sp->sw);
+    g.ph = __ldg(&sp->ph); g.pw = __ldg(&sp->pw); g.dh = __ldg(&sp->dh); g.dw = __ldg(&sp->dw);
+    g.act = __ldg(&sp->act);
+    g.t.R = 1 << __ldg(&sp->tr_log); g.t.tw = __ldg(&sp->tw_valid); g.t.cc = __ldg(&sp->BN);
+    g.x = ldg_ptr<const uint16_t *>(&sp->x);
+    g.res = ldg_ptr<const uint16_t *>(&sp->res);
+    g.res_pos = g.res ? __ldg(&sp->res_pos) : LOP_RES_NONE;
+    g.w_taps = ldg_ptr<const uint16_t *>(&sp->w_taps);
+    g.scale = ldg_ptr<const float *>(reinterpret_cast<const void *const *>(&sp->scale));
+    g.shift = ldg_ptr<const float *>(reinterpret_cast<const void *const *>(&sp->shift));
+    g.y = ldg_ptr<uint16_t *>(reinterpret_cast<const void *const *>(&sp->y));
+    const int oh0 = __ldg(&sp->oh_lo) + tile_r * g.t.R, ow0 = tile_w * g.t.tw;
+    rowop::dwconv_tile<true, 1, EPI_THREADS>(g, n, oh0, min(g.t.R, __ldg(&sp->oh_hi) - oh0), ow0, min(g.t.tw, g.Wo - ow0), tile_c * g.t.cc,
+                                             reinterpret_cast<float *>(stg), tid);
+}
+
+// Layer normalisation over the channels of the pixels of output row oh of image n: a group of lanes per pixel, each
+// lane keeping its (at most four) vectors in registers between the three passes; sums in the stand-alone kernel's order.
+__device__ __noinline__ void layernorm_item(const WfStage *sp, int n, int oh, int tid)
+{
+    const int C = __ldg(&sp->Cin), Ho = __ldg(&sp->Ho), Wo = __ldg(&sp->Wo);
+    const __nv_bfloat16 *x = ldg_ptr<const __nv_bfloat16 *>(&sp->x);
+    __nv_bfloat16 *y = ldg_ptr<__nv_bfloat16 *>(reinterpret_cast<const void *const *>(&sp->y));
+    const float *gain = ldg_ptr<const float *>(reinterpret_cast<const void *const *>(&sp->scale));
+    const float *offset = ldg_ptr<const float *>(reinterpret_cast<const void *const *>(&sp->shift));
+    const int nv = C >> 3;
+    const int lanes_log = rowop::ln_lanes_log(nv), lanes = 1 << lanes_log;
+    const int sub = tid & (lanes - 1), slot = tid >> lanes_log, per_pass = EPI_THREADS >> lanes_log;
+    for (int w0 = 0; w0 < Wo; w0 += per_pass) {               // the same trip count for every lane
+        const int ow = w0 + slot;
+        const long long o = (((long long)n * Ho + oh) * Wo + ow) * C;
+        uint4 q[4];
+        bool have[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            have[k] = ow < Wo && sub + k * lanes < nv;
+            if (have[k]) q[k] = __ldcg(reinterpret_cast<const uint4 *>(x + o) + sub + k * lanes);
+        }
+        float s1 = 0.0f;
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+            if (have[k]) {
+                float f[8];
+                rowop::unpack_bf16x8(q[k], f);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) s1 += f[j];
+            }
+        const float mean = rowop::group_sum(s1, lanes_log) / (float)C;
+        float s2 = 0.0f;
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+            if (have[k]) {
+                float f[8];
+                rowop::unpack_bf16x8(q[k], f);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const float d = f[j] - mean;
+                    s2 = fmaf(d, d, s2);
+                }
+            }
+        const float inv = rowop::ln_inv_std(rowop::group_sum(s2, lanes_log), C);
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+            if (have[k]) {
+                float f[8], v[8];
+                rowop::unpack_bf16x8(q[k], f);
+                const int c = (sub + k * lanes) * 8;
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    v[j] = rowop::ln_value(f[j], mean, inv, gain ? __ldg(gain + c + j) : 1.0f, offset ? __ldg(offset + c + j) : 0.0f);
+                *(reinterpret_cast<uint4 *>(y + o) + sub + k * lanes) = pack_bf16x8(v);
+            }
+    }
+}
+
+// Channel concatenation of output row oh of image n: the main input's Cin channels, then the second input's Cout - Cin.
+__device__ __noinline__ void concat_item(const WfStage *sp, int n, int oh, int tid)
+{
+    const int Cin = __ldg(&sp->Cin), Cout = __ldg(&sp->Cout), Ho = __ldg(&sp->Ho), Wo = __ldg(&sp->Wo);
+    const int va = Cin >> 3, vo = Cout >> 3;
+    const long long row = ((long long)n * Ho + oh) * Wo;
+    const uint4 *xa = reinterpret_cast<const uint4 *>(ldg_ptr<const __nv_bfloat16 *>(&sp->x) + row * Cin);
+    const uint4 *xb = reinterpret_cast<const uint4 *>(ldg_ptr<const __nv_bfloat16 *>(&sp->res) + row * (Cout - Cin));
+    uint4 *y = reinterpret_cast<uint4 *>(ldg_ptr<__nv_bfloat16 *>(reinterpret_cast<const void *const *>(&sp->y)) + row * Cout);
+    for (int idx = tid; idx < Wo * vo; idx += EPI_THREADS) {
+        const int ow = idx / vo, v = idx - ow * vo;
+        y[idx] = v < va ? __ldcg(xa + (long long)ow * va + v) : __ldcg(xb + (long long)ow * (vo - va) + (v - va));
+    }
+}
+
 // len bytes (a multiple of 2) from host memory the device can address to device memory, by the 32 lanes of a warp.
 // Host lines are read around the caches (they change between launches without the device knowing); eight 16-byte
 // loads per lane are in flight to cover the host link's latency.  src and dst agree modulo 16.
@@ -216,7 +323,9 @@ __device__ __forceinline__ void fetch_bytes(const uint8_t *src, uint8_t *dst, in
 }
 
 // FETCH: the program has a fetch list; the CTA then has one more warp, which walks it.
-template <bool FETCH>
+// FETCH: one more warp per CTA brings the chain input from host memory.  ROWOPS: the program has depth-wise /
+// normalisation / concatenation stages; programs without them run an instantiation that does not carry their code.
+template <bool FETCH, bool ROWOPS>
 __global__ void __launch_bounds__(FETCH ? WF_THREADS + 32 : WF_THREADS, 1) wavefront_kernel(const WfParams P)
 {
     extern __shared__ uint8_t smem_raw[];
@@ -940,6 +1049,12 @@ __global__ void __launch_bounds__(FETCH ? WF_THREADS + 32 : WF_THREADS, 1) wavef
                                     make_uint4(o[0], o[1], o[2], o[3]);
                             }
                     }
+                } else if (ROWOPS && kind == WF_DWCONV) {
+                    dwconv_item(&P.stages[sidx], n, tile_r, rec_tw(cur), rec_cout(cur), tid, stg);
+                } else if (ROWOPS && kind == WF_LAYERNORM) {
+                    layernorm_item(&P.stages[sidx], n, oh, tid);
+                } else if (ROWOPS && kind == WF_CONCAT) {
+                    concat_item(&P.stages[sidx], n, oh, tid);
                 } else {
                     // patch gather: Cout holds the patch length Kcol; x is the chain input, possibly still arriving
                     GatherGeom gg;
@@ -1103,6 +1218,17 @@ size_t wavefront_smem_bytes(const WfParams &p)
            2 * 256 * sizeof(float) + (128 + 32) * sizeof(long long) + 64;
 }
 
+namespace {
+
+typedef void (*WfKernel)(const WfParams);
+WfKernel kernel_for(const WfParams &p)
+{
+    if (p.n_fetch > 0) return p.row_ops ? wavefront_kernel<true, true> : wavefront_kernel<true, false>;
+    return p.row_ops ? wavefront_kernel<false, true> : wavefront_kernel<false, false>;
+}
+
+}  // namespace
+
 // How many CTAs of the kernel this device can hold at once (the kernel's dependency waits assume that every CTA of
 // a launch is resident: a CTA that has not started cannot produce what a running one waits for).
 cudaError_t wavefront_resident_ctas(const WfParams &p, int *ctas)
@@ -1112,13 +1238,9 @@ cudaError_t wavefront_resident_ctas(const WfParams &p, int *ctas)
     if (e != cudaSuccess) return e;
     if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
     const size_t smem = wavefront_smem_bytes(p);
-    if (p.n_fetch > 0) {
-        if ((e = cudaFuncSetAttribute(wavefront_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024)) != cudaSuccess) return e;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, wavefront_kernel<true>, WF_THREADS + 32, smem);
-    } else {
-        if ((e = cudaFuncSetAttribute(wavefront_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024)) != cudaSuccess) return e;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, wavefront_kernel<false>, WF_THREADS, smem);
-    }
+    WfKernel k = kernel_for(p);
+    if ((e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024)) != cudaSuccess) return e;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, p.n_fetch > 0 ? WF_THREADS + 32 : WF_THREADS, smem);
     if (e != cudaSuccess) return e;
     *ctas = per_sm * sms;
     return cudaSuccess;
@@ -1133,18 +1255,18 @@ cudaError_t launch_wavefront(const WfParams &p, int grid, cudaStream_t s)
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64 || !configured[dev]) {
-        e = cudaFuncSetAttribute(wavefront_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-        if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(wavefront_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-        if (e != cudaSuccess) return e;
+        WfKernel all[4] = {wavefront_kernel<false, false>, wavefront_kernel<false, true>, wavefront_kernel<true, false>, wavefront_kernel<true, true>};
+        for (WfKernel k : all) {
+            e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+            if (e != cudaSuccess) return e;
+        }
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
     if (smem > 227 * 1024) return cudaErrorInvalidValue;
 #ifdef LOP_WF_TRACE
     g_last_params = p;
 #endif
-    if (p.n_fetch > 0) wavefront_kernel<true><<<grid, WF_THREADS + 32, smem, s>>>(p);
-    else wavefront_kernel<false><<<grid, WF_THREADS, smem, s>>>(p);
+    kernel_for(p)<<<grid, p.n_fetch > 0 ? WF_THREADS + 32 : WF_THREADS, smem, s>>>(p);
     return cudaGetLastError();
 }
 

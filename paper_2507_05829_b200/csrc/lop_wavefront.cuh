@@ -15,7 +15,10 @@ namespace lop {
 
 // WF_FETCH: rows of the chain input brought from host memory by the CTAs' fetch warps.  Such a stage has row-group
 // counters like any producer but no items in the main list: its work is the program's fetch list.
-enum WfKind { WF_GATHER = 0, WF_CONV = 1, WF_POOL = 2, WF_FETCH = 3 };
+// WF_DWCONV / WF_LAYERNORM / WF_CONCAT: the memory-bound operators, run by the worker warps like pooling.  A depth-wise
+// item is one output row of one image, tw_valid columns wide and BN channels deep (its receptive window is staged in
+// shared memory); a normalisation or concatenation item is one whole output row of one image.
+enum WfKind { WF_GATHER = 0, WF_CONV = 1, WF_POOL = 2, WF_FETCH = 3, WF_DWCONV = 4, WF_LAYERNORM = 5, WF_CONCAT = 6 };
 // How a convolution stage feeds the tensor cores.
 //   WF_SLAB  one activation box per channel chunk: the output tile's receptive window (tile plus halo),
 //            laid out in shared memory as rows of P pixels; every filter tap is the same box read at a
@@ -53,7 +56,8 @@ struct WfStage {
     // boxes in the weight ring), so that more bytes are on their way at a time: such a walk is bound by the loads'
     // latency, a few slots deep, not by their rate
     int cps;
-    int pad_[12];
+    const void *w_taps;       // depth-wise stage: the filters as [tap][channel] bf16
+    int pad_[10];
 };
 static_assert(sizeof(WfStage) == 256, "WfStage layout");
 
@@ -80,6 +84,7 @@ struct WfParams {
     const void *fetch_src;
     void *fetch_dst;
     int n_fetch, fetch_window;
+    int row_ops;              // the program has WF_DWCONV / WF_LAYERNORM / WF_CONCAT stages
 };
 
 #ifndef LOP_WF_WORKER_WARPS
