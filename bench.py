@@ -46,7 +46,7 @@ WORKLOAD_NOTES = {
     "csp_stack": "cfg5 CSP-style 12-layer stack 1x1024x1024x3 bf16, 32 bands, bands streamed from pinned host memory",
 }
 STEADY_REQUESTS = 8
-KERNEL_SOURCES = ("lop_wavefront.cu", "lop_wavefront.cuh", "lop_program.cu", "lop_ptx.cuh", "lop_gather.cuh")
+KERNEL_SOURCES = ("lop_wavefront.cu", "lop_wavefront.cuh", "lop_program.cu", "lop_ptx.cuh", "lop_gather.cuh", "lop_rowops.cuh")
 
 
 def kernel_hash():

@@ -56,7 +56,7 @@ namespace {
 #define LOP_CPS_MAX 4
 #endif
 constexpr uint32_t A_BOX_MAX = 48u * 1024u;     // largest activation box a ring slot is sized for
-constexpr uint32_t LOP_ROWOP_STAGING_BYTES = 32u * 1024u;    // largest receptive window a depth-wise item stages
+constexpr uint32_t LOP_ROWOP_STAGING_BYTES = 64u * 1024u;    // largest receptive window a depth-wise item stages
 constexpr uint32_t B_BOX_MAX = 32u * 1024u;     // largest weight box
 
 int ilog2i(int v) { int l = 0; while ((1 << l) < v) ++l; return l; }

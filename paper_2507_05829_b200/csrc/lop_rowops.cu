@@ -1,10 +1,12 @@
 // CUDA-core kernels of the local operators that are not dense contractions (Sec. IV-A of the paper): depth-wise
 // convolution (block-wise, one small filter per channel), layer normalisation over the channels of a pixel
-// (row-wise) and channel concatenation (row-wise, two inputs).  All three are bound by memory traffic -- a few
-// multiply-adds per byte at most -- so they run on plain loads: 16-byte vectors along the channels (the innermost,
-// contiguous axis of NHWC), consecutive lanes on consecutive vectors, every tensor element read from DRAM once
-// (neighbouring windows of the depth-wise filter overlap in L1/L2).  Each works on output rows [oh_lo, oh_hi) of
-// all N images, like every other layer kernel, and a pixel's arithmetic does not depend on the band it is in.
+// (row-wise) and channel concatenation (row-wise, two inputs).  None has more than a few multiply-adds per byte, so
+// they stay off the tensor cores: 16-byte vectors along the channels (the innermost, contiguous axis of NHWC),
+// consecutive lanes on consecutive vectors, every tensor element read from DRAM once.  The depth-wise convolution in
+// bf16 with a multiple of eight channels runs tile by tile out of shared memory (rowop::dwconv_tile, the routine the
+// persistent kernel's worker warps run as well); other dtypes and channel counts take the plain kernel below.  Each
+// kernel works on output rows [oh_lo, oh_hi) of all N images, like every other layer kernel, and a pixel's
+// arithmetic does not depend on the band it is in.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -99,7 +101,7 @@ __global__ void __launch_bounds__(DW_THREADS) dwconv_kernel(ConvArgs p, int CV, 
 // bf16 with a multiple of eight channels: one block per tile, the same tile routine the persistent kernel runs
 // (rowop::dwconv_tile), so that both executors give the same bits.  w_taps: the filters as [tap][C].
 constexpr int DW_TILE_THREADS = 256;
-constexpr long long DW_TILE_SMEM = 40 * 1024;
+constexpr long long DW_TILE_SMEM = 96 * 1024;          // two blocks per SM
 
 __global__ void __launch_bounds__(DW_TILE_THREADS) dwconv_tile_kernel(rowop::DwGeom g, int oh_lo, int oh_hi, int tiles_w)
 {
@@ -281,6 +283,15 @@ cudaError_t launch_dwconv(const ConvArgs &a, int dtype, const void *w_taps, cuda
         g.scale = a.scale; g.shift = a.shift; g.y = static_cast<uint16_t *>(a.y);
         const int tiles_w = (a.Wo + t.tw - 1) / t.tw, tiles_r = (a.oh_hi - a.oh_lo + t.R - 1) / t.R;
         if (tiles_r <= 65535) {
+            static bool configured[64] = {};                 // the shared-memory limit is an attribute per device
+            int dev = 0;
+            cudaError_t e = cudaGetDevice(&dev);
+            if (e != cudaSuccess) return e;
+            if (dev < 0 || dev >= 64 || !configured[dev]) {
+                e = cudaFuncSetAttribute(dwconv_tile_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DW_TILE_SMEM);
+                if (e != cudaSuccess) return e;
+                if (dev >= 0 && dev < 64) configured[dev] = true;
+            }
             dim3 grid((unsigned)(tiles_w * (a.Cin / t.cc)), (unsigned)tiles_r, (unsigned)a.N);
             dwconv_tile_kernel<<<grid, DW_TILE_THREADS, (size_t)rowop::dw_tile_bytes(a.kh, a.kw, a.sh, a.sw, a.dh, a.dw, t), s>>>(g, a.oh_lo, a.oh_hi, tiles_w);
             return cudaGetLastError();

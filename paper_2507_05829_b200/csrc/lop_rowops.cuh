@@ -15,19 +15,13 @@ namespace rowop {
 
 constexpr float LAYERNORM_EPS = 1e-6f;
 
-// Activation in its accurate form (library exp / erf): these operators are bound by memory, not by arithmetic.  The
-// transcendental kinds are kept out of line: the tile routines run their epilogue a few times per thread, so what
-// they cost is mostly the fetch of their instructions, and inlined copies of exp and erf multiply that.
-static __device__ __noinline__ float activate_smooth(float t, int act)
-{
-    if (act == LOP_ACT_SILU) return t / (1.0f + expf(-t));
-    return 0.5f * t * (1.0f + erff(t * 0.70710678f));       // GELU: t * Phi(t)
-}
+// Activation in its accurate form (library exp / erf): these operators are bound by memory, not by arithmetic.
 __device__ __forceinline__ float activate(float t, int act)
 {
-    if (act == LOP_ACT_NONE) return t;
     if (act == LOP_ACT_RELU) return fmaxf(t, 0.0f);
-    return activate_smooth(t, act);
+    if (act == LOP_ACT_SILU) return t / (1.0f + expf(-t));
+    if (act == LOP_ACT_GELU) return 0.5f * t * (1.0f + erff(t * 0.70710678f));      // t * Phi(t)
+    return t;
 }
 
 // scale * acc + shift, residual before or after the activation (res_pos is LOP_RES_NONE when there is none).
@@ -71,11 +65,13 @@ __device__ __forceinline__ void unpack_bf16x8(const uint4 &q, float (&f)[8])
 
 // ---------------------------------------------------------------------------------------------
 // Depth-wise convolution of one tile: R output rows x tw output columns x cc channels of one image, by `NTHREADS`
-// threads that share a barrier.  The tile's receptive window and the filters of its channels are put into shared
-// memory as fp32 first (every input value is used by up to kh*kw taps: converting it once, not per tap, and leaving
-// the bounds checks to the staging step -- taps outside the tensor read zeros -- more than halves the instructions
-// per multiply-add), then every thread walks the taps of one (pixel, four channels) at a time, a = 0..kh-1,
-// b = 0..kw-1, whatever the tile: a pixel's bits do not depend on the tile or the band it is computed in.
+// threads that share a barrier.  With kh*kw multiply-adds per output and two bytes of input and output each, a 7x7
+// filter is bound by the fp32 multiply-add rate, not by DRAM: what counts is the number of other instructions per
+// multiply-add.  So the tile's receptive window and the filters of its channels are put into shared memory as fp32
+// first (a value is widened once, not once per tap that reads it; taps outside the tensor read zeros, so the walk has
+// no bounds checks), and the walk keeps a filter row's run of inputs in registers for several adjacent outputs and
+// issues its multiply-adds two per instruction.  Every output sums its taps in the order a = 0..kh-1, b = 0..kw-1,
+// whatever the tile: a pixel's bits do not depend on the tile or the band it is computed in.
 // ---------------------------------------------------------------------------------------------
 struct DwTile { int R, tw, cc; };
 
@@ -91,7 +87,7 @@ struct DwGeom {
     uint16_t *y;
 };
 
-constexpr int DW_T = 4;               // adjacent output columns one thread computes on the sliding-window path
+constexpr int DW_T = 8;               // adjacent output columns one thread computes on the sliding-window path
 
 // The sliding-window path: stride 1 and dilation 1 along the width and a filter 3, 5 or 7 wide.  A thread then keeps a
 // filter row's run of DW_T + kw - 1 input values in registers and uses each for up to kw outputs.
@@ -105,16 +101,17 @@ __host__ __device__ inline int dw_cols_in(int ncol, int kw, int sw, int dw)
     return (nc - 1) * sw + (kw - 1) * dw + 1;
 }
 
-// Pixels between the starts of two rows of the staged window: the columns, padded so that a row's pitch in bytes is
-// cc * 4 more than a multiple of 128.  Threads that differ in the row then read different shared-memory banks (see
-// dw_walk_sliding).
+// Pixels between the starts of two rows of the staged window (a pixel is cc fp32 values): the columns, padded so that
+// a row's pitch in bytes is cc * 4 more than a multiple of 128.  The eight threads of one shared-memory access phase
+// (16 bytes each) are the cc / 4 channel quads of 32 / cc consecutive rows (see dw_walk_sliding): with this pitch they
+// read eight different groups of four banks.
 __host__ __device__ inline int dw_pitch(int cols_in, int cc)
 {
     const int m = 32 / cc;                                 // cc = 8, 16, 32: pitch = 1 modulo 4, 2, 1
     return m <= 1 ? cols_in : (cols_in + m - 2) / m * m + 1;
 }
 
-// Shared memory one tile needs (window + filters), in bytes.
+// Shared memory one tile needs (fp32 window + fp32 filters), in bytes.
 __host__ __device__ inline long long dw_tile_bytes(int kh, int kw, int sh, int sw, int dh, int dw, const DwTile &t)
 {
     const long long rows = (long long)(t.R - 1) * sh + (long long)(kh - 1) * dh + 1;
@@ -132,7 +129,7 @@ inline bool dw_choose_tile(int kh, int kw, int sh, int sw, int dh, int dw, int N
     bool found = false;
     double best = 0.0;
     for (int cc = (C % 32 == 0 ? 32 : (C % 16 == 0 ? 16 : 8)); cc >= 8; cc /= 2)
-        for (int R = 1; R <= 8; R *= 2)
+        for (int R = 1; R <= 16; R *= 2)
             for (int div = 1; div <= 64; div *= 2) {
                 const int tw = (Wo + div - 1) / div;
                 if (div > 1 && tw < 4) break;
@@ -155,11 +152,13 @@ __device__ __forceinline__ void tile_barrier()
     asm volatile("bar.sync %0, %1;" ::"n"(BAR_ID), "n"(NTHREADS) : "memory");
 }
 
-// Epilogue and store of four channels c .. c+3 of output pixel (n, oh, ow).
-template <bool THROUGH_L2>
-__device__ __forceinline__ void dw_store4(const DwGeom &g, int n, int oh, int ow, int c, const float (&acc)[4])
+// Epilogue and store of four channels at element offset o of the output (scale / shift of those channels in sc / sf).
+// SMOOTH: the activation is SiLU or GELU.  The caller picks the instantiation once per unit, so that the common
+// kinds (none, ReLU) run a few instructions per value with no exp / erf code in their way.
+template <bool THROUGH_L2, bool SMOOTH>
+__device__ __forceinline__ void dw_store4(const DwGeom &g, long long o, const float4 &sc, const float4 &sf, const float (&acc)[4])
 {
-    const long long o = (((long long)n * g.Ho + oh) * g.Wo + ow) * g.C + c;
+    float v[4] = {fmaf(sc.x, acc[0], sf.x), fmaf(sc.y, acc[1], sf.y), fmaf(sc.z, acc[2], sf.z), fmaf(sc.w, acc[3], sf.w)};
     float rf[4] = {0.0f, 0.0f, 0.0f, 0.0f};
     if (g.res) {
         const uint2 *src = reinterpret_cast<const uint2 *>(g.res + o);
@@ -167,65 +166,104 @@ __device__ __forceinline__ void dw_store4(const DwGeom &g, int n, int oh, int ow
         rf[0] = __uint_as_float(rq.x << 16); rf[1] = __uint_as_float(rq.x & 0xFFFF0000u);
         rf[2] = __uint_as_float(rq.y << 16); rf[3] = __uint_as_float(rq.y & 0xFFFF0000u);
     }
-    const float4 sc = g.scale ? __ldg(reinterpret_cast<const float4 *>(g.scale + c)) : make_float4(1.0f, 1.0f, 1.0f, 1.0f);
-    const float4 sf = g.shift ? __ldg(reinterpret_cast<const float4 *>(g.shift + c)) : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-    const float v0 = epilogue(acc[0], sc.x, sf.x, rf[0], g.res_pos, g.act), v1 = epilogue(acc[1], sc.y, sf.y, rf[1], g.res_pos, g.act);
-    const float v2 = epilogue(acc[2], sc.z, sf.z, rf[2], g.res_pos, g.act), v3 = epilogue(acc[3], sc.w, sf.w, rf[3], g.res_pos, g.act);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        if (g.res_pos == LOP_RES_PRE_ACT) v[j] += rf[j];
+        if (SMOOTH) v[j] = activate(v[j], g.act);
+        else if (g.act == LOP_ACT_RELU) v[j] = fmaxf(v[j], 0.0f);
+        if (g.res_pos == LOP_RES_POST_ACT) v[j] += rf[j];
+    }
     uint2 out;
-    out.x = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(v0)) | ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(v1)) << 16);
-    out.y = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(v2)) | ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(v3)) << 16);
+    out.x = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(v[0])) | ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(v[1])) << 16);
+    out.y = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(v[2])) | ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(v[3])) << 16);
     *reinterpret_cast<uint2 *>(g.y + o) = out;
 }
-
-// Sliding-window walk of a staged tile (stride 1, dilation 1 along the width, KW known at compile time): a thread owns
-// DW_T adjacent output columns of one row and four channels.  Per filter row it loads the DW_T + KW - 1 input values
-// those outputs read once, then one weight vector per tap.  Every output still sums its taps in the order a = 0..kh-1,
-// b = 0..KW-1, like the one-pixel walk.
-template <bool THROUGH_L2, int KW, int NTHREADS>
-__device__ __forceinline__ void dw_walk_sliding(const DwGeom &g, int n, int oh0, int nrow, int ow0, int ncol, int c0, const float *xs,
-                                                const float *wsm, int pitch, int cc_log, int tid)
+__device__ __forceinline__ float4 dw_load4(const float *p, int c, float dflt)
 {
-    const int q4_log = cc_log - 2, q4 = 1 << q4_log;
+    return p ? __ldg(reinterpret_cast<const float4 *>(p + c)) : make_float4(dflt, dflt, dflt, dflt);
+}
+
+// Two fp32 values in one 64-bit register pair, and the packed fused multiply-add of sm_100: d = a * b + d on both
+// halves, each rounded like a scalar fmaf (the results are the scalar ones; what is saved is issue slots).
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float lo, float hi)
+{
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 v, float &lo, float &hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
+__device__ __forceinline__ void fma2(f32x2 &d, f32x2 a, f32x2 b) { asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(d) : "l"(a), "l"(b)); }
+// Sliding-window walk of a staged tile (stride 1, dilation 1 along the width; KW and the tile's channel count 2^CC_LOG
+// known at compile time, so that every shared-memory offset is an immediate): a thread owns DW_T adjacent output
+// columns of one row and four channels.  Per filter row it loads the DW_T + KW - 1 input vectors those outputs read
+// once, then one weight vector per tap: DW_T + 2 * KW - 1 loads for 2 * DW_T * KW packed multiply-adds.  Every output
+// still sums its taps in the order a = 0..kh-1, b = 0..KW-1, like the one-pixel walk.
+// xs: the window, [row][pitch][cc] fp32; wsm: the filters, [tap][cc] fp32.
+template <bool THROUGH_L2, int KW, int CC_LOG, int NTHREADS>
+__device__ __forceinline__ void dw_walk_sliding(const DwGeom &g, int n, int oh0, int nrow, int ow0, int ncol, int c0, const float *xs,
+                                                const float *wsm, int pitch, int tid)
+{
+    constexpr int CC = 1 << CC_LOG, Q4_LOG = CC_LOG - 2, Q4 = 1 << Q4_LOG;
     const int groups = (ncol + DW_T - 1) / DW_T;
-    const int units = nrow * groups << q4_log;
-    // unit order: channel quad fastest, then the row, then the column group.  The eight threads of a quarter warp
-    // (one shared-memory access phase) are then the quads of 8 / q4 consecutive rows; with the padded row pitch their
-    // 16-byte reads fall into eight different bank groups for a row stride of one.
+    const int units = nrow * groups << Q4_LOG;
+    const int row_step = g.dh * pitch * CC;                        // floats between two filter rows
+    // unit order: channel quad fastest, then the row, then the column group.  The eight threads of a quarter warp (one
+    // shared-memory access phase of 16-byte reads) are then the quads of 8 / Q4 consecutive rows; with the padded row
+    // pitch they fall into eight different groups of four banks for a row stride of one.
     for (int i = tid; i < units; i += NTHREADS) {
-        const int c4 = i & (q4 - 1), gi = i >> q4_log;
+        const int c4 = i & (Q4 - 1), gi = i >> Q4_LOG;
         const int grp = gi / nrow, r = gi - grp * nrow, owl = grp * DW_T;
-        const float *xp = xs + (((size_t)(r * g.sh) * pitch + owl) << cc_log) + c4 * 4;
-        const float *wp = wsm + c4 * 4;
-        float4 acc[DW_T];
+        const float *xa = xs + ((size_t)(r * g.sh) * pitch + owl) * CC + c4 * 4;
+        const float *wa = wsm + c4 * 4;
+        f32x2 acc[DW_T][2];
 #pragma unroll
-        for (int t = 0; t < DW_T; ++t) acc[t] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-        for (int a = 0; a < g.kh; ++a) {
-            const float *xa = xp + (((size_t)a * g.dh * pitch) << cc_log);
-            const float *wa = wp + ((a * KW) << cc_log);
-            float4 xw[DW_T + KW - 1];
+        for (int t = 0; t < DW_T; ++t) acc[t][0] = acc[t][1] = 0ull;               // (+0, +0)
+        for (int a = 0; a < g.kh; ++a, xa += row_step, wa += KW * CC) {
+            f32x2 xw[DW_T + KW - 1][2];
 #pragma unroll
-            for (int j = 0; j < DW_T + KW - 1; ++j) xw[j] = *reinterpret_cast<const float4 *>(xa + ((size_t)j << cc_log));
+            for (int j = 0; j < DW_T + KW - 1; ++j) {
+                const float4 q = *reinterpret_cast<const float4 *>(xa + j * CC);
+                xw[j][0] = pack2(q.x, q.y); xw[j][1] = pack2(q.z, q.w);
+            }
 #pragma unroll
             for (int b = 0; b < KW; ++b) {
-                const float4 wv = *reinterpret_cast<const float4 *>(wa + (b << cc_log));
+                const float4 wv = *reinterpret_cast<const float4 *>(wa + b * CC);
+                const f32x2 w0 = pack2(wv.x, wv.y), w1 = pack2(wv.z, wv.w);
 #pragma unroll
                 for (int t = 0; t < DW_T; ++t) {
-                    acc[t].x = fmaf(xw[t + b].x, wv.x, acc[t].x); acc[t].y = fmaf(xw[t + b].y, wv.y, acc[t].y);
-                    acc[t].z = fmaf(xw[t + b].z, wv.z, acc[t].z); acc[t].w = fmaf(xw[t + b].w, wv.w, acc[t].w);
+                    fma2(acc[t][0], xw[t + b][0], w0);
+                    fma2(acc[t][1], xw[t + b][1], w1);
                 }
             }
         }
+        const int c = c0 + c4 * 4;
+        const float4 sc = dw_load4(g.scale, c, 1.0f), sf = dw_load4(g.shift, c, 0.0f);
+        const long long o = (((long long)n * g.Ho + oh0 + r) * g.Wo + ow0 + owl) * g.C + c;
+        const bool smooth = g.act > LOP_ACT_RELU;
 #pragma unroll
         for (int t = 0; t < DW_T; ++t)
             if (owl + t < ncol) {
-                const float a4[4] = {acc[t].x, acc[t].y, acc[t].z, acc[t].w};
-                dw_store4<THROUGH_L2>(g, n, oh0 + r, ow0 + owl + t, c0 + c4 * 4, a4);
+                float a4[4];
+                unpack2(acc[t][0], a4[0], a4[1]);
+                unpack2(acc[t][1], a4[2], a4[3]);
+                if (smooth) dw_store4<THROUGH_L2, true>(g, o + (long long)t * g.C, sc, sf, a4);
+                else dw_store4<THROUGH_L2, false>(g, o + (long long)t * g.C, sc, sf, a4);
             }
     }
 }
+template <bool THROUGH_L2, int KW, int NTHREADS>
+__device__ __forceinline__ void dw_walk_sliding_cc(const DwGeom &g, int n, int oh0, int nrow, int ow0, int ncol, int c0, const float *xs,
+                                                   const float *wsm, int pitch, int cc_log, int tid)
+{
+    if (cc_log == 3) dw_walk_sliding<THROUGH_L2, KW, 3, NTHREADS>(g, n, oh0, nrow, ow0, ncol, c0, xs, wsm, pitch, tid);
+    else if (cc_log == 4) dw_walk_sliding<THROUGH_L2, KW, 4, NTHREADS>(g, n, oh0, nrow, ow0, ncol, c0, xs, wsm, pitch, tid);
+    else dw_walk_sliding<THROUGH_L2, KW, 5, NTHREADS>(g, n, oh0, nrow, ow0, ncol, c0, xs, wsm, pitch, tid);
+}
 
-// THROUGH_L2: the input (and the residual) may have been written by other SMs during this launch: read around L1.
-// Rows [oh0, oh0 + nrow), columns [ow0, ow0 + ncol), channels [c0, c0 + cc) of image n.
+// Rows [oh0, oh0 + nrow), columns [ow0, ow0 + ncol), channels [c0, c0 + cc) of image n.  THROUGH_L2: the input and
+// the residual may have been written by other SMs during this launch: read around L1.  sm: dw_tile_bytes() bytes,
+// 16-byte aligned.
 template <bool THROUGH_L2, int BAR_ID, int NTHREADS>
 __device__ __forceinline__ void dwconv_tile(const DwGeom &g, int n, int oh0, int nrow, int ow0, int ncol, int c0, float *sm, int tid)
 {
@@ -245,18 +283,21 @@ __device__ __forceinline__ void dwconv_tile(const DwGeom &g, int n, int oh0, int
         d[0] = make_float4(f[0], f[1], f[2], f[3]);
         d[1] = make_float4(f[4], f[5], f[6], f[7]);
     }
-    // receptive window: [row][column][cc] fp32, zeros outside the tensor; four loads in flight per thread
+    // receptive window: [row][pitch][cc] fp32, zeros outside the tensor; four loads in flight per thread
     const int nvec = rows_in * cols_in << v8_log;
     for (int base = 0; base < nvec; base += 4 * NTHREADS) {
         uint4 q[4];
+        int dst[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
             const int i = base + u * NTHREADS + tid;
             q[u] = make_uint4(0u, 0u, 0u, 0u);
+            dst[u] = -1;
             if (i < nvec) {
                 const int v = i & (v8 - 1), pix = i >> v8_log;
                 const int r = pix / cols_in, col = pix - r * cols_in;
                 const int ih = ih0 + r, iw = iw0 + col;
+                dst[u] = ((r * pitch + col) << cc_log) + v * 8;
                 if (ih >= 0 && ih < g.Hin && iw >= 0 && iw < g.Win) {
                     const uint4 *src = reinterpret_cast<const uint4 *>(g.x + (((long long)n * g.Hin + ih) * g.Win + iw) * g.C + c0) + v;
                     q[u] = THROUGH_L2 ? __ldcg(src) : __ldg(src);
@@ -264,25 +305,21 @@ __device__ __forceinline__ void dwconv_tile(const DwGeom &g, int n, int oh0, int
             }
         }
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int i = base + u * NTHREADS + tid;
-            if (i < nvec) {
+        for (int u = 0; u < 4; ++u)
+            if (dst[u] >= 0) {
                 float f[8];
                 unpack_bf16x8(q[u], f);
-                const int v = i & (v8 - 1), pix = i >> v8_log;
-                const int r = pix / cols_in, col = pix - r * cols_in;
-                float4 *d = reinterpret_cast<float4 *>(xs + (((size_t)r * pitch + col) << cc_log) + v * 8);
+                float4 *d = reinterpret_cast<float4 *>(xs + dst[u]);
                 d[0] = make_float4(f[0], f[1], f[2], f[3]);
                 d[1] = make_float4(f[4], f[5], f[6], f[7]);
             }
-        }
     }
     tile_barrier<BAR_ID, NTHREADS>();
 
     if (dw_slides(g.kw, g.sw, g.dw)) {
-        if (g.kw == 3) dw_walk_sliding<THROUGH_L2, 3, NTHREADS>(g, n, oh0, nrow, ow0, ncol, c0, xs, wsm, pitch, cc_log, tid);
-        else if (g.kw == 5) dw_walk_sliding<THROUGH_L2, 5, NTHREADS>(g, n, oh0, nrow, ow0, ncol, c0, xs, wsm, pitch, cc_log, tid);
-        else dw_walk_sliding<THROUGH_L2, 7, NTHREADS>(g, n, oh0, nrow, ow0, ncol, c0, xs, wsm, pitch, cc_log, tid);
+        if (g.kw == 3) dw_walk_sliding_cc<THROUGH_L2, 3, NTHREADS>(g, n, oh0, nrow, ow0, ncol, c0, xs, wsm, pitch, cc_log, tid);
+        else if (g.kw == 5) dw_walk_sliding_cc<THROUGH_L2, 5, NTHREADS>(g, n, oh0, nrow, ow0, ncol, c0, xs, wsm, pitch, cc_log, tid);
+        else dw_walk_sliding_cc<THROUGH_L2, 7, NTHREADS>(g, n, oh0, nrow, ow0, ncol, c0, xs, wsm, pitch, cc_log, tid);
         return;
     }
     // any stride, dilation and filter width: one (pixel, four channels) at a time
@@ -305,7 +342,10 @@ __device__ __forceinline__ void dwconv_tile(const DwGeom &g, int n, int oh0, int
                 acc[2] = fmaf(xv.z, wv.z, acc[2]); acc[3] = fmaf(xv.w, wv.w, acc[3]);
             }
         }
-        dw_store4<THROUGH_L2>(g, n, oh0 + r, ow0 + owl, c0 + c4 * 4, acc);
+        const int c = c0 + c4 * 4;
+        const long long o = (((long long)n * g.Ho + oh0 + r) * g.Wo + ow0 + owl) * g.C + c;
+        if (g.act > LOP_ACT_RELU) dw_store4<THROUGH_L2, true>(g, o, dw_load4(g.scale, c, 1.0f), dw_load4(g.shift, c, 0.0f), acc);
+        else dw_store4<THROUGH_L2, false>(g, o, dw_load4(g.scale, c, 1.0f), dw_load4(g.shift, c, 0.0f), acc);
     }
 }
 

@@ -6,7 +6,10 @@ Cases: a named workload (``vgg_block``, ``resnet18``, ``resnet50``, ``csp_stack`
 input, one persistent launch per run; ``<name>:pipelined`` streams the bands from pinned host memory), ``pool`` (a
 3x3 stride-2 max pooling of an 8 x 224 x 224 x 64 bf16 tensor by the stand-alone kernel and, with ``pool:persistent``,
 by pooling items of the persistent kernel), ``gather`` (patch gather + 7x7 stride-2 stem convolution of 8 images by
-the stand-alone kernels; ``gather:persistent`` inside the persistent kernel).  The L2 is flushed before every run.
+the stand-alone kernels; ``gather:persistent`` inside the persistent kernel), ``convnext_block`` / ``dense_layer``
+(depth-wise convolution, layer normalisation, concatenation: items of the persistent kernel; ``<name>:per_layer``
+runs the stand-alone kernels, one launch per layer), ``dwconv`` / ``layernorm`` / ``concat`` (one such operator on an
+8 x 224 x 224 x 64 tensor, stand-alone kernel or ``:persistent``).  The L2 is flushed before every run.
 """
 import sys
 
@@ -21,12 +24,24 @@ from .chain import DeviceChain
 
 def build_case(name):
     base, _, mode = name.partition(":")
-    if base in ("vgg_block", "resnet18", "resnet50", "csp_stack", "single_conv"):
+    if base in ("vgg_block", "resnet18", "resnet50", "csp_stack", "single_conv", "pointwise_mlp", "convnext_block", "dense_layer"):
+        if mode == "per_layer":                                   # one stand-alone kernel per layer, whole tensors
+            return li.build(base), "whole", B.LOP_FLAG_PER_LAYER
         return li.build(base), (mode or "banded"), 0
     if base == "pool":
         l = pool(64, 3, 2, 1)
         l.input_from = -1
         wl = Workload("pool_only", "bf16", 8, 224, 224, 64, [Segment([l], 1)], seed=1)
+    elif base in ("dwconv", "layernorm", "concat"):
+        # the memory-bound operators on a tensor larger than the L2: 8 x 224 x 224 x 64 bf16 (51 MB)
+        if base == "dwconv":
+            layers = [li.dwconv(64, 7)]
+        elif base == "layernorm":
+            layers = [li.layernorm(64)]
+        else:
+            layers = [pool(64, 1, 1, 0), li.concat(64, 64, input_from=-1, second_from=0)]     # a copy, then input ++ copy
+        layers[0].input_from = -1
+        wl = Workload(base + "_only", "bf16", 8, 224, 224, 64, [Segment(layers, 1)], seed=1)
     elif base == "gather":
         l = conv(3, 64, 7, s=2, p=3, act=li.ACT_RELU)
         l.input_from = -1
