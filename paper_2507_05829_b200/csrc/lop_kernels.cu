@@ -20,6 +20,25 @@ __device__ __forceinline__ float to_f32(__nv_bfloat16 v) { return __bfloat162flo
 __device__ __forceinline__ void from_f32(float &d, float v) { d = v; }
 __device__ __forceinline__ void from_f32(__nv_bfloat16 &d, float v) { d = __float2bfloat16_rn(v); }
 
+// idx = ((n * rows + r) * Wo + ow) * inner + g, taken apart with 32-bit divisions where the count allows it (a 64-bit
+// division is a routine of several dozen instructions: four of them per thread outweigh a light kernel's real work).
+__device__ __forceinline__ void split_index(long long idx, long long total, int inner, int Wo, int rows, int &g, int &ow, int &r, int &n)
+{
+    if (total < (1LL << 31)) {
+        unsigned q = (unsigned)idx;
+        const unsigned q1 = q / (unsigned)inner; g = (int)(q - q1 * (unsigned)inner);
+        const unsigned q2 = q1 / (unsigned)Wo; ow = (int)(q1 - q2 * (unsigned)Wo);
+        const unsigned q3 = q2 / (unsigned)rows; r = (int)(q2 - q3 * (unsigned)rows);
+        n = (int)q3;
+    } else {
+        long long q = idx;
+        g = (int)(q % inner); q /= inner;
+        ow = (int)(q % Wo); q /= Wo;
+        r = (int)(q % rows);
+        n = (int)(q / rows);
+    }
+}
+
 __device__ __forceinline__ float activate(float t, int act)
 {
     if (act == LOP_ACT_RELU) return fmaxf(t, 0.0f);
@@ -178,12 +197,9 @@ __global__ void __launch_bounds__(256) maxpool_kernel(PoolArgs p)
     T *__restrict__ y = static_cast<T *>(p.y);
     for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
          idx += (long long)gridDim.x * blockDim.x) {
-        const int g = (int)(idx % cg);
-        long long q = idx / cg;
-        const int ow = (int)(q % p.Wo);
-        q /= p.Wo;
-        const int oh = p.oh_lo + (int)(q % rows);
-        const int n = (int)(q / rows);
+        int g, ow, r, n;
+        split_index(idx, total, cg, p.Wo, rows, g, ow, r, n);
+        const int oh = p.oh_lo + r;
         float m[VEC];
 #pragma unroll
         for (int i = 0; i < VEC; ++i) m[i] = -INFINITY;
@@ -218,12 +234,9 @@ __global__ void __launch_bounds__(256) maxpool_bf16x8_kernel(PoolArgs p)
     const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= total) return;
     const uint4 *__restrict__ x = static_cast<const uint4 *>(p.x);
-    const int g = (int)(idx % cg);
-    long long q = idx / cg;
-    const int ow = (int)(q % p.Wo);
-    q /= p.Wo;
-    const int oh = p.oh_lo + (int)(q % rows);
-    const int n = (int)(q / rows);
+    int g, ow, r, n;
+    split_index(idx, total, cg, p.Wo, rows, g, ow, r, n);
+    const int oh = p.oh_lo + r;
     uint4 v[KH * KW];
     bool ok[KH * KW];
 #pragma unroll

@@ -182,12 +182,20 @@ __global__ void __launch_bounds__(256) concat_kernel(ConvArgs p)
     const long long total = (long long)p.N * rows * p.Wo * vo;
     const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= total) return;
-    const int v = (int)(i % vo);
-    long long q = i / vo;
-    const int ow = (int)(q % p.Wo); q /= p.Wo;
-    const int oh = p.oh_lo + (int)(q % rows);
-    const int n = (int)(q / rows);
-    const long long pix = ((long long)n * p.Ho + oh) * p.Wo + ow;
+    // vector v of band pixel m; the band's rows * Wo pixels of an image are contiguous in the tensors.  Divisions
+    // in 32 bits where the counts are that small (64-bit division is a long routine).
+    const long long band = (long long)rows * p.Wo;
+    long long m, n, rem;
+    int v;
+    if (total < (1LL << 31)) {
+        const unsigned m32 = (unsigned)i / (unsigned)vo, n32 = m32 / (unsigned)band;
+        v = (int)((unsigned)i - m32 * (unsigned)vo);
+        m = m32; n = n32; rem = m32 - n32 * (unsigned)band;
+    } else {
+        m = i / vo; v = (int)(i - m * vo);
+        n = m / band; rem = m - n * band;
+    }
+    const long long pix = n * p.Ho * p.Wo + (long long)p.oh_lo * p.Wo + rem;
     using V = Vec<T, VEC>;
     const V val = v < va ? *reinterpret_cast<const V *>(static_cast<const T *>(p.x) + pix * Ca + (long long)v * VEC)
                          : *reinterpret_cast<const V *>(static_cast<const T *>(p.res) + pix * Cb + (long long)(v - va) * VEC);
@@ -231,6 +239,51 @@ cudaError_t dwconv_dispatch(const ConvArgs &a, cudaStream_t s)
 {
     if (a.Cin % full_vec<T>() == 0) return dwconv_launch<T, full_vec<T>()>(a, s);
     return dwconv_launch<T, 1>(a, s);
+}
+
+// bf16 with a multiple of eight channels, at most 1024: the routine the persistent kernel runs (rowop::ln_pixels),
+// 4 / VPL pixels per lane group.
+template <int VPL>
+__global__ void __launch_bounds__(256) layernorm_bf16_kernel(ConvArgs p)
+{
+    constexpr int PPG = 4 / VPL;
+    const int rows = p.oh_hi - p.oh_lo;
+    const long long M = (long long)p.N * rows * p.Wo;
+    const int C = p.Cin;
+    const int lanes_log = rowop::ln_lanes_log(C >> 3);
+    const int sub = threadIdx.x & ((1 << lanes_log) - 1);
+    const long long group = (long long)blockIdx.x * (256 >> lanes_log) + (threadIdx.x >> lanes_log);
+    long long o[PPG];
+    bool live[PPG];
+    // pixel m of the band is pixel (m mod band) of image m / band, band = rows * Wo pixels that are contiguous in the
+    // tensor: one division per pixel, in 32 bits where the band is that small (64-bit division is a long routine)
+    const long long band = (long long)rows * p.Wo, image = (long long)p.Ho * p.Wo, first = (long long)p.oh_lo * p.Wo;
+#pragma unroll
+    for (int q = 0; q < PPG; ++q) {
+        const long long m = group * PPG + q;
+        live[q] = m < M;
+        o[q] = 0;
+        if (live[q]) {
+            long long n, rem;
+            if (M < (1LL << 31)) {
+                const unsigned n32 = (unsigned)m / (unsigned)band;
+                n = n32; rem = (unsigned)m - n32 * (unsigned)band;
+            } else {
+                n = m / band; rem = m - n * band;
+            }
+            o[q] = (n * image + first + rem) * C;
+        }
+    }
+    rowop::ln_pixels<false, VPL>(static_cast<const uint16_t *>(p.x), static_cast<uint16_t *>(p.y), C, lanes_log, sub, o, live, p.scale, p.shift);
+}
+
+template <int VPL>
+cudaError_t layernorm_bf16_launch(const ConvArgs &a, cudaStream_t s)
+{
+    const long long M = (long long)a.N * (a.oh_hi - a.oh_lo) * a.Wo;
+    const long long per_block = (long long)(256 >> rowop::ln_lanes_log(a.Cin >> 3)) * (4 / VPL);
+    layernorm_bf16_kernel<VPL><<<(unsigned)((M + per_block - 1) / per_block), 256, 0, s>>>(a);
+    return cudaGetLastError();
 }
 
 template <typename T, int VEC>
@@ -309,6 +362,10 @@ cudaError_t launch_dw_transpose(const void *w, void *wt, int C, int taps, cudaSt
 cudaError_t launch_layernorm(const ConvArgs &a, int dtype, cudaStream_t s)
 {
     if (a.oh_hi <= a.oh_lo) return cudaSuccess;
+    if (dtype == LOP_BF16 && a.Cin % 8 == 0 && a.Cin <= 1024) {
+        const int vpl = rowop::ln_vpl(a.Cin >> 3);
+        return vpl == 1 ? layernorm_bf16_launch<1>(a, s) : (vpl == 2 ? layernorm_bf16_launch<2>(a, s) : layernorm_bf16_launch<4>(a, s));
+    }
     return dtype == LOP_BF16 ? layernorm_dispatch<__nv_bfloat16>(a, s) : layernorm_dispatch<float>(a, s);
 }
 

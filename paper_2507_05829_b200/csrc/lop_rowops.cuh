@@ -63,6 +63,105 @@ __device__ __forceinline__ void unpack_bf16x8(const uint4 &q, float (&f)[8])
     }
 }
 
+// Two fp32 values rounded to nearest-even bf16, lo in the low half of the word (one conversion instruction).
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
+{
+    const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t *>(&h);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Layer normalisation of bf16 pixels with a multiple of eight channels, at most 1024: a group of 2^lanes_log lanes
+// per pixel, lane `sub` owning vectors sub, sub + lanes, ... (VPL = 1, 2 or 4 of them, eight channels each).  A lane
+// keeps four vectors in registers: the 4 / VPL pixels its group normalises at a time, all loaded before the first
+// sum, so that a thread has 64 bytes on their way.  Per pixel: the lane's values summed in ascending order, the
+// butterfly over the group, the centred squares likewise; the same order as the plain kernel's, so the bits agree.
+// o[p]: element offset of pixel p, live[p]: whether the slot holds a pixel (dead slots still take part in the
+// shuffles).  gain / offset may be null.
+// ---------------------------------------------------------------------------------------------
+template <bool THROUGH_L2, int VPL>
+__device__ __forceinline__ void ln_pixels(const uint16_t *x, uint16_t *y, int C, int lanes_log, int sub, const long long (&o)[4 / VPL],
+                                          const bool (&live)[4 / VPL], const float *gain, const float *offset)
+{
+    constexpr int PPG = 4 / VPL;
+    const int nv = C >> 3, lanes = 1 << lanes_log;
+    uint4 q[PPG][VPL];
+    bool have[PPG][VPL];
+#pragma unroll
+    for (int p = 0; p < PPG; ++p)
+#pragma unroll
+        for (int k = 0; k < VPL; ++k) {
+            have[p][k] = live[p] && sub + k * lanes < nv;
+            if (have[p][k]) {
+                const uint4 *src = reinterpret_cast<const uint4 *>(x + o[p]) + sub + k * lanes;
+                q[p][k] = THROUGH_L2 ? __ldcg(src) : __ldg(src);
+            }
+        }
+    float mean[PPG], inv[PPG];
+#pragma unroll
+    for (int p = 0; p < PPG; ++p) {
+        float s1 = 0.0f;
+#pragma unroll
+        for (int k = 0; k < VPL; ++k)
+            if (have[p][k]) {
+                float f[8];
+                unpack_bf16x8(q[p][k], f);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) s1 += f[j];
+            }
+        mean[p] = group_sum(s1, lanes_log) / (float)C;
+    }
+#pragma unroll
+    for (int p = 0; p < PPG; ++p) {
+        float s2 = 0.0f;
+#pragma unroll
+        for (int k = 0; k < VPL; ++k)
+            if (have[p][k]) {
+                float f[8];
+                unpack_bf16x8(q[p][k], f);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const float d = f[j] - mean[p];
+                    s2 = fmaf(d, d, s2);
+                }
+            }
+        inv[p] = ln_inv_std(group_sum(s2, lanes_log), C);
+    }
+#pragma unroll
+    for (int k = 0; k < VPL; ++k) {
+        const int v = sub + k * lanes;
+        if (v >= nv) continue;
+        float gn[8], of[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { gn[j] = 1.0f; of[j] = 0.0f; }
+        if (gain) {
+            const float4 a = __ldg(reinterpret_cast<const float4 *>(gain + v * 8)), b = __ldg(reinterpret_cast<const float4 *>(gain + v * 8) + 1);
+            gn[0] = a.x; gn[1] = a.y; gn[2] = a.z; gn[3] = a.w; gn[4] = b.x; gn[5] = b.y; gn[6] = b.z; gn[7] = b.w;
+        }
+        if (offset) {
+            const float4 a = __ldg(reinterpret_cast<const float4 *>(offset + v * 8)), b = __ldg(reinterpret_cast<const float4 *>(offset + v * 8) + 1);
+            of[0] = a.x; of[1] = a.y; of[2] = a.z; of[3] = a.w; of[4] = b.x; of[5] = b.y; of[6] = b.z; of[7] = b.w;
+        }
+#pragma unroll
+        for (int p = 0; p < PPG; ++p)
+            if (have[p][k]) {
+                float f[8];
+                unpack_bf16x8(q[p][k], f);
+                float r[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) r[j] = ln_value(f[j], mean[p], inv[p], gn[j], of[j]);
+                *(reinterpret_cast<uint4 *>(y + o[p]) + v) =
+                    make_uint4(pack_bf16x2(r[0], r[1]), pack_bf16x2(r[2], r[3]), pack_bf16x2(r[4], r[5]), pack_bf16x2(r[6], r[7]));
+            }
+    }
+}
+// Vectors per lane for a pixel of nv vectors (1, 2 or 4; nv <= 128).
+__host__ __device__ inline int ln_vpl(int nv)
+{
+    const int lanes = 1 << ln_lanes_log(nv);
+    return nv <= lanes ? 1 : (nv <= 2 * lanes ? 2 : 4);
+}
+
 // ---------------------------------------------------------------------------------------------
 // Depth-wise convolution of one tile: R output rows x tw output columns x cc channels of one image, by `NTHREADS`
 // threads that share a barrier.  With kh*kw multiply-adds per output and two bytes of input and output each, a 7x7
@@ -173,10 +272,7 @@ __device__ __forceinline__ void dw_store4(const DwGeom &g, long long o, const fl
         else if (g.act == LOP_ACT_RELU) v[j] = fmaxf(v[j], 0.0f);
         if (g.res_pos == LOP_RES_POST_ACT) v[j] += rf[j];
     }
-    uint2 out;
-    out.x = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(v[0])) | ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(v[1])) << 16);
-    out.y = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(v[2])) | ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(v[3])) << 16);
-    *reinterpret_cast<uint2 *>(g.y + o) = out;
+    *reinterpret_cast<uint2 *>(g.y + o) = make_uint2(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]));
 }
 __device__ __forceinline__ float4 dw_load4(const float *p, int c, float dflt)
 {

@@ -185,14 +185,6 @@ __device__ __forceinline__ T ldg_ptr(const void *const *p)
 
 // ---- the memory-bound operators, run by all worker threads (tid = 0 .. EPI_THREADS-1) on one item.  Kept out of line:
 // they are rare and long, and inlined they cost the convolution roles registers.
-__device__ __forceinline__ uint4 pack_bf16x8(const float (&v)[8])
-{
-    uint32_t h[8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) h[j] = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(v[j]));
-    return make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), h[4] | (h[5] << 16), h[6] | (h[7] << 16));
-}
-
 // Depth-wise convolution item: 2^tr_log output rows x tw_valid columns x BN channels of image n (see
 // rowop::dwconv_tile); the window is read through L2 -- other SMs produced it during this launch.
 __device__ __noinline__ void dwconv_item(const WfStage *sp, int n, int tile_r, int tile_w, int tile_c, int tid, uint8_t *stg)
@@ -215,63 +207,39 @@ __device__ __noinline__ void dwconv_item(const WfStage *sp, int n, int tile_r, i
                                              reinterpret_cast<float *>(stg), tid);
 }
 
-// Layer normalisation over the channels of the pixels of output row oh of image n: a group of lanes per pixel, each
-// lane keeping its (at most four) vectors in registers between the three passes; sums in the stand-alone kernel's order.
+// Layer normalisation over the channels of the pixels of output row oh of image n (rowop::ln_pixels: a group of
+// lanes per pixel, four vectors in flight per lane).
+template <int VPL>
+__device__ __forceinline__ void layernorm_row(const uint16_t *x, uint16_t *y, const float *gain, const float *offset, int C, int Wo, long long row0,
+                                              int tid)
+{
+    constexpr int PPG = 4 / VPL;
+    const int lanes_log = rowop::ln_lanes_log(C >> 3);
+    const int sub = tid & ((1 << lanes_log) - 1), slot = tid >> lanes_log, per_pass = (EPI_THREADS >> lanes_log) * PPG;
+    for (int w0 = 0; w0 < Wo; w0 += per_pass) {               // the same trip count for every lane
+        long long o[PPG];
+        bool live[PPG];
+#pragma unroll
+        for (int q = 0; q < PPG; ++q) {
+            const int ow = w0 + slot * PPG + q;
+            live[q] = ow < Wo;
+            o[q] = (row0 + ow) * C;
+        }
+        rowop::ln_pixels<true, VPL>(x, y, C, lanes_log, sub, o, live, gain, offset);
+    }
+}
 __device__ __noinline__ void layernorm_item(const WfStage *sp, int n, int oh, int tid)
 {
     const int C = __ldg(&sp->Cin), Ho = __ldg(&sp->Ho), Wo = __ldg(&sp->Wo);
-    const __nv_bfloat16 *x = ldg_ptr<const __nv_bfloat16 *>(&sp->x);
-    __nv_bfloat16 *y = ldg_ptr<__nv_bfloat16 *>(reinterpret_cast<const void *const *>(&sp->y));
+    const uint16_t *x = ldg_ptr<const uint16_t *>(&sp->x);
+    uint16_t *y = ldg_ptr<uint16_t *>(reinterpret_cast<const void *const *>(&sp->y));
     const float *gain = ldg_ptr<const float *>(reinterpret_cast<const void *const *>(&sp->scale));
     const float *offset = ldg_ptr<const float *>(reinterpret_cast<const void *const *>(&sp->shift));
-    const int nv = C >> 3;
-    const int lanes_log = rowop::ln_lanes_log(nv), lanes = 1 << lanes_log;
-    const int sub = tid & (lanes - 1), slot = tid >> lanes_log, per_pass = EPI_THREADS >> lanes_log;
-    for (int w0 = 0; w0 < Wo; w0 += per_pass) {               // the same trip count for every lane
-        const int ow = w0 + slot;
-        const long long o = (((long long)n * Ho + oh) * Wo + ow) * C;
-        uint4 q[4];
-        bool have[4];
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            have[k] = ow < Wo && sub + k * lanes < nv;
-            if (have[k]) q[k] = __ldcg(reinterpret_cast<const uint4 *>(x + o) + sub + k * lanes);
-        }
-        float s1 = 0.0f;
-#pragma unroll
-        for (int k = 0; k < 4; ++k)
-            if (have[k]) {
-                float f[8];
-                rowop::unpack_bf16x8(q[k], f);
-#pragma unroll
-                for (int j = 0; j < 8; ++j) s1 += f[j];
-            }
-        const float mean = rowop::group_sum(s1, lanes_log) / (float)C;
-        float s2 = 0.0f;
-#pragma unroll
-        for (int k = 0; k < 4; ++k)
-            if (have[k]) {
-                float f[8];
-                rowop::unpack_bf16x8(q[k], f);
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const float d = f[j] - mean;
-                    s2 = fmaf(d, d, s2);
-                }
-            }
-        const float inv = rowop::ln_inv_std(rowop::group_sum(s2, lanes_log), C);
-#pragma unroll
-        for (int k = 0; k < 4; ++k)
-            if (have[k]) {
-                float f[8], v[8];
-                rowop::unpack_bf16x8(q[k], f);
-                const int c = (sub + k * lanes) * 8;
-#pragma unroll
-                for (int j = 0; j < 8; ++j)
-                    v[j] = rowop::ln_value(f[j], mean, inv, gain ? __ldg(gain + c + j) : 1.0f, offset ? __ldg(offset + c + j) : 0.0f);
-                *(reinterpret_cast<uint4 *>(y + o) + sub + k * lanes) = pack_bf16x8(v);
-            }
-    }
+    const long long row0 = ((long long)n * Ho + oh) * Wo;
+    const int vpl = rowop::ln_vpl(C >> 3);
+    if (vpl == 1) layernorm_row<1>(x, y, gain, offset, C, Wo, row0, tid);
+    else if (vpl == 2) layernorm_row<2>(x, y, gain, offset, C, Wo, row0, tid);
+    else layernorm_row<4>(x, y, gain, offset, C, Wo, row0, tid);
 }
 
 // Channel concatenation of output row oh of image n: the main input's Cin channels, then the second input's Cout - Cin.
