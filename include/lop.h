@@ -58,8 +58,16 @@ enum {
     LOP_FLAG_FORCE_SIMT = 4u,     /* never use the tensor-core convolution (second on-GPU opinion) */
     LOP_FLAG_PER_LAYER = 8u,      /* one kernel launch per (band, layer) instead of one persistent
                                      wavefront launch per call / per band                          */
-    LOP_FLAG_COPY_ENGINE = 16u    /* pipelined runs always move the bands with copy-engine copies on
+    LOP_FLAG_COPY_ENGINE = 16u,   /* pipelined runs always move the bands with copy-engine copies on
                                      a side stream, also when the kernel could fetch them itself  */
+    LOP_FLAG_DEBUG_BOUNDS = 32u   /* checked execution: every layer runs as a kernel of its own (as with
+                                     LOP_FLAG_PER_LAYER) and the CUDA-core kernels -- fp32 / fall-back convolution,
+                                     pooling, patch gather, depth-wise convolution, layer normalisation,
+                                     concatenation -- test every element offset they load from or store to
+                                     against the tensor it belongs to and every output row against the rows of the
+                                     launch.  A violation never traps: the access is skipped, bit 0x20 of the
+                                     plan's status word is set and lop_plan_check_device returns LOP_EDEVICE.  The
+                                     tensor-core kernel's operand loads are TMA copies, clipped by the hardware    */
 };
 
 /*

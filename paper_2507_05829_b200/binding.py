@@ -12,7 +12,7 @@ LOP_CONV2D, LOP_MAXPOOL2D, LOP_LINEAR = 0, 1, 2
 LOP_ACT_NONE, LOP_ACT_RELU, LOP_ACT_SILU = 0, 1, 2
 LOP_RES_NONE, LOP_RES_PRE_ACT, LOP_RES_POST_ACT = 0, 1, 2
 LOP_INPUT, LOP_NO_RESIDUAL = -1, -2
-LOP_FLAG_REUSE_HALO, LOP_FLAG_TIME_LAYERS, LOP_FLAG_FORCE_SIMT, LOP_FLAG_PER_LAYER, LOP_FLAG_COPY_ENGINE = 1, 2, 4, 8, 16
+LOP_FLAG_REUSE_HALO, LOP_FLAG_TIME_LAYERS, LOP_FLAG_FORCE_SIMT, LOP_FLAG_PER_LAYER, LOP_FLAG_COPY_ENGINE, LOP_FLAG_DEBUG_BOUNDS = 1, 2, 4, 8, 16, 32
 
 # every symbol include/lop.h declares
 EXPORTS = [

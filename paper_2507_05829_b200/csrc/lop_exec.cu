@@ -151,7 +151,7 @@ int ensure_exec(lop_plan_t *pl)
         for (auto &ev : e->ev_layer) LOP_CUDA(cudaEventCreate(&ev));
     }
     e->prepared_w.assign(L, nullptr);
-    e->wavefront = program_supported(pl) && !(pl->flags & (LOP_FLAG_PER_LAYER | LOP_FLAG_TIME_LAYERS));
+    e->wavefront = program_supported(pl) && !(pl->flags & (LOP_FLAG_PER_LAYER | LOP_FLAG_TIME_LAYERS | LOP_FLAG_DEBUG_BOUNDS));
     return LOP_OK;
 }
 
@@ -218,7 +218,7 @@ int run_layer(lop_plan_t *pl, int i, int lo, int hi, const void *in, void *out, 
         const ConvArgs a = conv_args(pl, i, in, out, ws, lo, hi);
         if (li.kernel == K_CONV_TC) {
             if (li.stem_gather) {                      // the band's patches first (the split step), same stream
-                LOP_CUDA(launch_stem_gather(in, static_cast<char *>(ws) + pl->col_off, gather_geom(pl, i), lo, hi, s));
+                LOP_CUDA(launch_stem_gather(in, static_cast<char *>(ws) + pl->col_off, gather_geom(pl, i), lo, hi, s, a.dbg));
                 e->launches++;
             }
             const ConvTcGeom g = conv_tc_geometry(a, hi - lo);
@@ -977,7 +977,7 @@ int lop_plan_layer_stored(const lop_plan_t *pl, int layer)
     if (!pl) { set_error("plan is NULL"); return LOP_EINVAL; }
     const int L = (int)pl->layers.size();
     if (layer < 0 || layer >= L) { set_error("lop_plan_layer_stored: layer %d out of range", layer); return LOP_EINVAL; }
-    const bool persistent = program_supported(pl) && !(pl->flags & (LOP_FLAG_PER_LAYER | LOP_FLAG_TIME_LAYERS));
+    const bool persistent = program_supported(pl) && !(pl->flags & (LOP_FLAG_PER_LAYER | LOP_FLAG_TIME_LAYERS | LOP_FLAG_DEBUG_BOUNDS));
     return (persistent && program_folds_pool(pl, layer)) ? 0 : 1;
 }
 
@@ -1006,7 +1006,8 @@ int lop_plan_check_device(lop_plan_t *pl, void *ws)
         for (auto &kv : pl->exec->programs) program_destroy(kv.second);
         pl->exec->programs.clear();
         cudaMemset(static_cast<char *>(ws) + pl->status_off, 0, sizeof(status));
-        set_error("device status word 0x%x: a bounded wait ran out", status);
+        set_error(status & 0x20u ? "device status word 0x%x: a checked kernel computed an address outside its tensor (the access was skipped)"
+                                 : "device status word 0x%x: a bounded wait ran out", status);
         return LOP_EDEVICE;
     }
     return LOP_OK;

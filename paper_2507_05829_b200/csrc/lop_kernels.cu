@@ -73,6 +73,7 @@ __global__ void __launch_bounds__(256) conv_simt_kernel(ConvArgs p)
     const long long m0 = (long long)blockIdx.x * BM;
     const int n0 = blockIdx.y * BN;
     const int t = threadIdx.x;
+    const long long x_elems = (long long)p.N * p.Hin * p.Win * p.Cin, y_elems = (long long)p.N * p.Ho * p.Wo * p.Cout;
     const int kk = t & 15;              // K index inside the slab this thread stages
     const int lr = t >> 4;              // 0..15: first of the TM tile rows (stride 16) this thread stages
 
@@ -118,13 +119,15 @@ __global__ void __launch_bounds__(256) conv_simt_kernel(ConvArgs p)
             float v = 0.0f;
             if (kvalid && mvalid[e]) {
                 const int ih = ih0[e] + a * p.dh, iw = iw0[e] + b * p.dw;
-                if (ih >= 0 && ih < p.Hin && iw >= 0 && iw < p.Win)
-                    v = to_f32(x[xbase[e] + ((long long)ih * p.Win + iw) * p.Cin + ci]);
+                if (ih >= 0 && ih < p.Hin && iw >= 0 && iw < p.Win) {
+                    const long long xo = xbase[e] + ((long long)ih * p.Win + iw) * p.Cin + ci;
+                    if (dbg_in_bounds(p.dbg, xo, 1, x_elems)) v = to_f32(x[xo]);
+                }
             }
             av[e] = v;
             float u = 0.0f;
             const int co = n0 + lr + e * 16;
-            if (kvalid && co < p.Cout) u = to_f32(w[(long long)co * K + k]);
+            if (kvalid && co < p.Cout && dbg_in_bounds(p.dbg, (long long)co * K + k, 1, (long long)p.Cout * K)) u = to_f32(w[(long long)co * K + k]);
             wv[e] = u;
         }
     };
@@ -167,6 +170,8 @@ __global__ void __launch_bounds__(256) conv_simt_kernel(ConvArgs p)
         for (int j = 0; j < TM; ++j) {
             const int co = n0 + tx * TM + j;
             if (co >= p.Cout) continue;
+            // the element inside the tensor, the row inside the rows of this launch (tested as a one-row "tensor")
+            if (!dbg_in_bounds(p.dbg, o + co, 1, y_elems) || !dbg_in_bounds(p.dbg, oh - p.oh_lo, 1, rows)) continue;
             float v = acc[i][j];
             v = fmaf(p.scale ? p.scale[co] : 1.0f, v, p.shift ? p.shift[co] : 0.0f);
             if (res && p.res_pos == LOP_RES_PRE_ACT) v += to_f32(res[o + co]);
@@ -209,8 +214,9 @@ __global__ void __launch_bounds__(256) maxpool_kernel(PoolArgs p)
             for (int b = 0; b < p.kw; ++b) {
                 const int iw = ow * p.sw - p.pw + b * p.dw;
                 if (iw < 0 || iw >= p.Win) continue;
-                const Pack<T, VEC> v = *reinterpret_cast<const Pack<T, VEC> *>(
-                    x + (((long long)n * p.Hin + ih) * p.Win + iw) * p.C + (long long)g * VEC);
+                const long long xo = (((long long)n * p.Hin + ih) * p.Win + iw) * p.C + (long long)g * VEC;
+                if (!dbg_in_bounds(p.dbg, xo, VEC, (long long)p.N * p.Hin * p.Win * p.C)) continue;
+                const Pack<T, VEC> v = *reinterpret_cast<const Pack<T, VEC> *>(x + xo);
 #pragma unroll
                 for (int i = 0; i < VEC; ++i) m[i] = fmaxf(m[i], to_f32(v.v[i]));
             }
@@ -218,7 +224,8 @@ __global__ void __launch_bounds__(256) maxpool_kernel(PoolArgs p)
         Pack<T, VEC> o;
 #pragma unroll
         for (int i = 0; i < VEC; ++i) from_f32(o.v[i], m[i]);
-        *reinterpret_cast<Pack<T, VEC> *>(y + (((long long)n * p.Ho + oh) * p.Wo + ow) * p.C + (long long)g * VEC) = o;
+        const long long yo = (((long long)n * p.Ho + oh) * p.Wo + ow) * p.C + (long long)g * VEC;
+        if (dbg_in_bounds(p.dbg, yo, VEC, (long long)p.N * p.Ho * p.Wo * p.C)) *reinterpret_cast<Pack<T, VEC> *>(y + yo) = o;
     }
 }
 
@@ -246,7 +253,9 @@ __global__ void __launch_bounds__(256) maxpool_bf16x8_kernel(PoolArgs p)
         for (int b = 0; b < KW; ++b) {
             const int iw = ow * p.sw - p.pw + b * p.dw;
             ok[a * KW + b] = ih >= 0 && ih < p.Hin && iw >= 0 && iw < p.Win;
-            if (ok[a * KW + b]) v[a * KW + b] = __ldg(x + (((long long)n * p.Hin + ih) * p.Win + iw) * cg + g);
+            const long long xo = (((long long)n * p.Hin + ih) * p.Win + iw) * cg + g;           // in 16-byte vectors
+            ok[a * KW + b] = ok[a * KW + b] && dbg_in_bounds(p.dbg, xo, 1, (long long)p.N * p.Hin * p.Win * cg);
+            if (ok[a * KW + b]) v[a * KW + b] = __ldg(x + xo);
         }
     }
     float m[8];
@@ -266,7 +275,8 @@ __global__ void __launch_bounds__(256) maxpool_bf16x8_kernel(PoolArgs p)
 #pragma unroll
     for (int i = 0; i < 4; ++i)                      // the values are bf16 already: dropping the low half is exact
         o[i] = (__float_as_uint(m[2 * i]) >> 16) | (__float_as_uint(m[2 * i + 1]) & 0xFFFF0000u);
-    static_cast<uint4 *>(p.y)[(((long long)n * p.Ho + oh) * p.Wo + ow) * cg + g] = make_uint4(o[0], o[1], o[2], o[3]);
+    const long long yo = (((long long)n * p.Ho + oh) * p.Wo + ow) * cg + g;
+    if (dbg_in_bounds(p.dbg, yo, 1, (long long)p.N * p.Ho * p.Wo * cg)) static_cast<uint4 *>(p.y)[yo] = make_uint4(o[0], o[1], o[2], o[3]);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -275,7 +285,7 @@ __global__ void __launch_bounds__(256) maxpool_bf16x8_kernel(PoolArgs p)
 // 16 bytes, reads hit the few image rows of the band in L1/L2.  HBM-bound on the write.
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) stem_gather_kernel(const uint16_t *__restrict__ x, uint16_t *__restrict__ y,
-                                                          GatherGeom g, int lo, int hi)
+                                                          GatherGeom g, int lo, int hi, unsigned *dbg)
 {
     const int k8n = g.Kcol >> 3;
     const long long total = (long long)g.N * (hi - lo) * g.Wo * k8n;
@@ -287,8 +297,9 @@ __global__ void __launch_bounds__(256) stem_gather_kernel(const uint16_t *__rest
         q /= g.Wo;
         const int oh = lo + (int)(q % (hi - lo));
         const int n = (int)(q / (hi - lo));
-        const uint4 v = gather8<false>(x, g, n, oh, ow, k8);
-        *reinterpret_cast<uint4 *>(y + (((long long)n * g.Ho + oh) * g.Wo + ow) * g.Kcol + k8 * 8) = v;
+        const uint4 v = gather8<false>(x, g, n, oh, ow, k8);        // reads in-bounds taps only, by construction of the patch
+        const long long yo = (((long long)n * g.Ho + oh) * g.Wo + ow) * g.Kcol + k8 * 8;
+        if (dbg_in_bounds(dbg, yo, 8, (long long)g.N * g.Ho * g.Wo * g.Kcol)) *reinterpret_cast<uint4 *>(y + yo) = v;
     }
 }
 
@@ -352,12 +363,12 @@ cudaError_t launch_maxpool(const PoolArgs &a, int dtype, cudaStream_t s)
     return cudaGetLastError();
 }
 
-cudaError_t launch_stem_gather(const void *x, void *y, const GatherGeom &g, int lo, int hi, cudaStream_t s)
+cudaError_t launch_stem_gather(const void *x, void *y, const GatherGeom &g, int lo, int hi, cudaStream_t s, unsigned *dbg)
 {
     if (hi <= lo) return cudaSuccess;
     if (g.Kcol % 8 != 0) return cudaErrorInvalidValue;
     const long long work = (long long)g.N * (hi - lo) * g.Wo * (g.Kcol / 8);
-    stem_gather_kernel<<<grid_for(work, 256), 256, 0, s>>>(static_cast<const uint16_t *>(x), static_cast<uint16_t *>(y), g, lo, hi);
+    stem_gather_kernel<<<grid_for(work, 256), 256, 0, s>>>(static_cast<const uint16_t *>(x), static_cast<uint16_t *>(y), g, lo, hi, dbg);
     return cudaGetLastError();
 }
 

@@ -16,6 +16,7 @@ struct ConvArgs {
     int kh, kw, sh, sw, ph, pw, dh, dw;
     int act, res_pos;
     int oh_lo, oh_hi;       // rows to compute
+    unsigned *dbg;          // checked execution: the status word that takes bit 0x20 on a violation, else nullptr
 };
 
 struct PoolArgs {
@@ -24,7 +25,19 @@ struct PoolArgs {
     int N, Hin, Win, C, Ho, Wo;
     int kh, kw, sh, sw, ph, pw, dh, dw;
     int oh_lo, oh_hi;
+    unsigned *dbg;          // as in ConvArgs
 };
+
+// Checked execution (LOP_FLAG_DEBUG_BOUNDS): elements [first, first + count) must lie inside a tensor of `limit`
+// elements.  Without a status word the test costs one predictable branch.
+#ifdef __CUDACC__
+__device__ __forceinline__ bool dbg_in_bounds(unsigned *dbg, long long first, long long count, long long limit)
+{
+    if (!dbg || (first >= 0 && first + count <= limit)) return true;
+    atomicOr(dbg, 0x20u);
+    return false;
+}
+#endif
 
 // CUDA-core convolution (fp32 accumulate); dtype: LOP_F32 / LOP_BF16 storage.
 cudaError_t launch_conv_simt(const ConvArgs &a, int dtype, cudaStream_t s);
@@ -39,7 +52,8 @@ cudaError_t launch_concat(const ConvArgs &a, int dtype, cudaStream_t s);
 cudaError_t launch_dw_transpose(const void *w, void *wt, int C, int taps, cudaStream_t s);
 // rows [lo,hi) of the patch tensor y[N,Ho,Wo,Kcol] of a thin chain input x[N,H,W,C] (bf16 only).
 struct GatherGeom;
-cudaError_t launch_stem_gather(const void *x, void *y, const GatherGeom &g, int lo, int hi, cudaStream_t s);
+// dbg: checked execution's status word (see ConvArgs), or nullptr
+cudaError_t launch_stem_gather(const void *x, void *y, const GatherGeom &g, int lo, int hi, cudaStream_t s, unsigned *dbg = nullptr);
 // w[rows][C] -> wp[rows][Cpad] zero-padded (bf16 only).
 cudaError_t launch_pad_weights(const void *w, void *wp, long long rows, int C, int Cpad, cudaStream_t s);
 

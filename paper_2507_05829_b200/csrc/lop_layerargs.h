@@ -41,6 +41,7 @@ inline ConvArgs conv_args(const lop_plan_t *pl, int i, const void *in, void *out
     a.kh = l.kh; a.kw = l.kw; a.sh = l.sh; a.sw = l.sw; a.ph = l.ph; a.pw = l.pw; a.dh = l.dh; a.dw = l.dw;
     a.act = l.act; a.res_pos = a.res ? l.residual_pos : LOP_RES_NONE;
     a.oh_lo = lo; a.oh_hi = hi;
+    a.dbg = (pl->flags & LOP_FLAG_DEBUG_BOUNDS) ? reinterpret_cast<unsigned *>(static_cast<char *>(ws) + pl->status_off) : nullptr;
     if (li.kernel == K_CONV_TC) {
         a.Cin = li.cin_eff;
         if (li.stem_gather) {
@@ -64,6 +65,7 @@ inline PoolArgs pool_args(const lop_plan_t *pl, int i, const void *in, void *out
     a.N = pl->N; a.Hin = li.Hin; a.Win = li.Win; a.C = l.cin; a.Ho = li.Ho; a.Wo = li.Wo;
     a.kh = l.kh; a.kw = l.kw; a.sh = l.sh; a.sw = l.sw; a.ph = l.ph; a.pw = l.pw; a.dh = l.dh; a.dw = l.dw;
     a.oh_lo = lo; a.oh_hi = hi;
+    a.dbg = (pl->flags & LOP_FLAG_DEBUG_BOUNDS) ? reinterpret_cast<unsigned *>(static_cast<char *>(ws) + pl->status_off) : nullptr;
     return a;
 }
 

@@ -289,7 +289,7 @@ int lop_plan(const lop_layer *layers, int n_layers, int N, int H, int W, int C, 
     if (N < 1 || H < 1 || W < 1 || C < 1) { set_error("lop_plan: N, H, W, C must be >= 1"); return LOP_ESHAPE; }
     if (n_bands < 1) { set_error("lop_plan: n_bands must be >= 1"); return LOP_EINVAL; }
     if (dtype != LOP_F32 && dtype != LOP_BF16) { set_error("lop_plan: unknown dtype %d", dtype); return LOP_EINVAL; }
-    if (flags & ~(LOP_FLAG_REUSE_HALO | LOP_FLAG_TIME_LAYERS | LOP_FLAG_FORCE_SIMT | LOP_FLAG_PER_LAYER | LOP_FLAG_COPY_ENGINE)) {
+    if (flags & ~(LOP_FLAG_REUSE_HALO | LOP_FLAG_TIME_LAYERS | LOP_FLAG_FORCE_SIMT | LOP_FLAG_PER_LAYER | LOP_FLAG_COPY_ENGINE | LOP_FLAG_DEBUG_BOUNDS)) {
         set_error("lop_plan: unknown flag bits 0x%x", flags);
         return LOP_EINVAL;
     }

@@ -81,12 +81,14 @@ __global__ void __launch_bounds__(DW_THREADS) dwconv_kernel(ConvArgs p, int CV, 
             for (int b = 0; b < p.kw; ++b) {
                 const int iw = iw0 + b * p.dw;
                 if (iw < 0 || iw >= p.Win) continue;
+                if (!dbg_in_bounds(p.dbg, (xr - x) + (long long)iw * p.Cin, VEC, (long long)p.N * p.Hin * p.Win * p.Cin)) continue;
                 const V xv = *reinterpret_cast<const V *>(xr + (long long)iw * p.Cin);
 #pragma unroll
                 for (int j = 0; j < VEC; ++j) acc[j] = fmaf(to_f32(xv.v[j]), wr[b * CB + j], acc[j]);
             }
         }
         const long long o = (((long long)n * p.Ho + oh) * p.Wo + ow) * p.Cout + c;
+        if (!dbg_in_bounds(p.dbg, o, VEC, (long long)p.N * p.Ho * p.Wo * p.Cout)) continue;
         V rv, out;
         if (res) rv = *reinterpret_cast<const V *>(res + o);
         const int res_pos = res ? p.res_pos : LOP_RES_NONE;
@@ -127,15 +129,16 @@ __global__ void __launch_bounds__(256) layernorm_kernel(ConvArgs p)
     const int lanes_log = rowop::ln_lanes_log(nvec), lanes = 1 << lanes_log;
     const int sub = threadIdx.x & (lanes - 1);
     const long long m = (long long)blockIdx.x * (blockDim.x >> lanes_log) + (threadIdx.x >> lanes_log);
-    const bool live = m < M;                               // dead lanes still take part in the group sums
+    const bool live0 = m < M;                              // dead lanes still take part in the group sums
     long long o = 0;
-    if (live) {
+    if (live0) {
         const int ow = (int)(m % p.Wo);
         const long long q = m / p.Wo;
         const int oh = p.oh_lo + (int)(q % rows);
         const int n = (int)(q / rows);
         o = (((long long)n * p.Ho + oh) * p.Wo + ow) * C;
     }
+    const bool live = live0 && dbg_in_bounds(p.dbg, o, C, (long long)p.N * p.Ho * p.Wo * C);
     const T *__restrict__ x = static_cast<const T *>(p.x) + o;
     T *__restrict__ y = static_cast<T *>(p.y) + o;
     using V = Vec<T, VEC>;
@@ -196,6 +199,8 @@ __global__ void __launch_bounds__(256) concat_kernel(ConvArgs p)
         n = m / band; rem = m - n * band;
     }
     const long long pix = n * p.Ho * p.Wo + (long long)p.oh_lo * p.Wo + rem;
+    const long long pixels = (long long)p.N * p.Ho * p.Wo;
+    if (!dbg_in_bounds(p.dbg, pix, 1, pixels) || v < 0 || v >= vo) return;       // every offset below is pix * channels + v * VEC
     using V = Vec<T, VEC>;
     const V val = v < va ? *reinterpret_cast<const V *>(static_cast<const T *>(p.x) + pix * Ca + (long long)v * VEC)
                          : *reinterpret_cast<const V *>(static_cast<const T *>(p.res) + pix * Cb + (long long)(v - va) * VEC);
@@ -272,6 +277,7 @@ __global__ void __launch_bounds__(256) layernorm_bf16_kernel(ConvArgs p)
                 n = m / band; rem = m - n * band;
             }
             o[q] = (n * image + first + rem) * C;
+            live[q] = dbg_in_bounds(p.dbg, o[q], C, (long long)p.N * image * C);
         }
     }
     rowop::ln_pixels<false, VPL>(static_cast<const uint16_t *>(p.x), static_cast<uint16_t *>(p.y), C, lanes_log, sub, o, live, p.scale, p.shift);
@@ -334,6 +340,7 @@ cudaError_t launch_dwconv(const ConvArgs &a, int dtype, const void *w_taps, cuda
         g.x = static_cast<const uint16_t *>(a.x); g.res = static_cast<const uint16_t *>(a.res);
         g.w_taps = static_cast<const uint16_t *>(w_taps);
         g.scale = a.scale; g.shift = a.shift; g.y = static_cast<uint16_t *>(a.y);
+        g.dbg = a.dbg; g.N = a.N;
         const int tiles_w = (a.Wo + t.tw - 1) / t.tw, tiles_r = (a.oh_hi - a.oh_lo + t.R - 1) / t.R;
         if (tiles_r <= 65535) {
             static bool configured[64] = {};                 // the shared-memory limit is an attribute per device

@@ -184,7 +184,17 @@ struct DwGeom {
     const uint16_t *w_taps;           // [kh*kw][C] bf16
     const float *scale, *shift;
     uint16_t *y;
+    unsigned *dbg;                    // checked execution: status word that takes bit 0x20 on an address outside a tensor, else nullptr
+    int N;                            // images (for the checks only)
 };
+// (the persistent kernel, THROUGH_L2, never runs checked: checked execution takes the stand-alone kernels)
+template <bool THROUGH_L2>
+__device__ __forceinline__ bool dw_in_bounds(const DwGeom &g, long long first, long long count, long long limit)
+{
+    if (THROUGH_L2 || !g.dbg || (first >= 0 && first + count <= limit)) return true;
+    atomicOr(g.dbg, 0x20u);
+    return false;
+}
 
 constexpr int DW_T = 8;               // adjacent output columns one thread computes on the sliding-window path
 
@@ -257,6 +267,7 @@ __device__ __forceinline__ void tile_barrier()
 template <bool THROUGH_L2, bool SMOOTH>
 __device__ __forceinline__ void dw_store4(const DwGeom &g, long long o, const float4 &sc, const float4 &sf, const float (&acc)[4])
 {
+    if (!dw_in_bounds<THROUGH_L2>(g, o, 4, (long long)g.N * g.Ho * g.Wo * g.C)) return;
     float v[4] = {fmaf(sc.x, acc[0], sf.x), fmaf(sc.y, acc[1], sf.y), fmaf(sc.z, acc[2], sf.z), fmaf(sc.w, acc[3], sf.w)};
     float rf[4] = {0.0f, 0.0f, 0.0f, 0.0f};
     if (g.res) {
@@ -394,7 +405,8 @@ __device__ __forceinline__ void dwconv_tile(const DwGeom &g, int n, int oh0, int
                 const int r = pix / cols_in, col = pix - r * cols_in;
                 const int ih = ih0 + r, iw = iw0 + col;
                 dst[u] = ((r * pitch + col) << cc_log) + v * 8;
-                if (ih >= 0 && ih < g.Hin && iw >= 0 && iw < g.Win) {
+                const long long xo = (((long long)n * g.Hin + ih) * g.Win + iw) * g.C + c0 + v * 8;
+                if (ih >= 0 && ih < g.Hin && iw >= 0 && iw < g.Win && dw_in_bounds<THROUGH_L2>(g, xo, 8, (long long)g.N * g.Hin * g.Win * g.C)) {
                     const uint4 *src = reinterpret_cast<const uint4 *>(g.x + (((long long)n * g.Hin + ih) * g.Win + iw) * g.C + c0) + v;
                     q[u] = THROUGH_L2 ? __ldcg(src) : __ldg(src);
                 }

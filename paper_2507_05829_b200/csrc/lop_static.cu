@@ -94,10 +94,13 @@ extern "C" int lop_run_whole_static(lop_plan_t *pl, const void *in, void *out, u
         const LayerInfo &li = pl->layers[i];
         const lop_layer &l = li.l;
         if (l.op == LOP_MAXPOOL2D) {
-            ST_CUDA(launch_maxpool(pool_args(pl, i, in, out, ws, 0, li.Ho), pl->dtype, s));
+            PoolArgs pa = pool_args(pl, i, in, out, ws, 0, li.Ho);
+            if (pa.dbg) pa.dbg = status;                   // checked execution reports into the word this call was given
+            ST_CUDA(launch_maxpool(pa, pl->dtype, s));
             continue;
         }
-        const ConvArgs a = conv_args(pl, i, in, out, ws, 0, li.Ho);
+        ConvArgs a = conv_args(pl, i, in, out, ws, 0, li.Ho);
+        if (a.dbg) a.dbg = status;
         if (li.kernel == K_DWCONV) {
             const void *w_taps = nullptr;
             if (li.dw_transposed) {                    // rebuilt by every call, like the padded stem weights
@@ -116,7 +119,7 @@ extern "C" int lop_run_whole_static(lop_plan_t *pl, const void *in, void *out, u
         if (li.stem_gather) {
             // another plan may have used the array since: padded weights and patches are rebuilt by every call
             ST_CUDA(launch_pad_weights(l.weight, ws + li.wpad_off, l.cout, l.kh * l.kw * l.cin, li.cin_eff, s));
-            ST_CUDA(launch_stem_gather(in, ws + pl->col_off, gather_geom(pl, i), 0, li.Ho, s));
+            ST_CUDA(launch_stem_gather(in, ws + pl->col_off, gather_geom(pl, i), 0, li.Ho, s, a.dbg));
         }
         const ConvTcGeom g = conv_tc_geometry(a, li.Ho);
         ConvTcMaps maps;                                   // encoded on the stack: nothing is cached between calls

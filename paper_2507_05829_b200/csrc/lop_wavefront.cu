@@ -202,6 +202,7 @@ __device__ __noinline__ void dwconv_item(const WfStage *sp, int n, int tile_r, i
     g.scale = ldg_ptr<const float *>(reinterpret_cast<const void *const *>(&sp->scale));
     g.shift = ldg_ptr<const float *>(reinterpret_cast<const void *const *>(&sp->shift));
     g.y = ldg_ptr<uint16_t *>(reinterpret_cast<const void *const *>(&sp->y));
+    g.dbg = nullptr; g.N = __ldg(&sp->N);                     // checked execution runs the stand-alone kernels
     const int oh0 = __ldg(&sp->oh_lo) + tile_r * g.t.R, ow0 = tile_w * g.t.tw;
     rowop::dwconv_tile<true, 1, EPI_THREADS>(g, n, oh0, min(g.t.R, __ldg(&sp->oh_hi) - oh0), ow0, min(g.t.tw, g.Wo - ow0), tile_c * g.t.cc,
                                              reinterpret_cast<float *>(stg), tid);

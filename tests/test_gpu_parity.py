@@ -255,6 +255,21 @@ def test_chains_small(name, kw, flags):
     check_workload(li.build(name, **kw), flags=flags)
 
 
+@pytest.mark.parametrize("name,kw", [("single_conv", {}), ("vgg_block", dict(H=30, W=22, dtype="f32", width=16, n_bands=4)),
+                                     ("resnet18", dict(H=64, W=64)), ("convnext_block", dict(H=29, W=17, C=64, n_bands=5)),
+                                     ("convnext_block", dict(H=15, W=9, C=12, n_bands=3, dtype="f32")), ("dense_layer", dict(H=19, W=14, n_bands=3))])
+def test_checked_execution_finds_nothing_and_changes_nothing(name, kw):
+    """LOP_FLAG_DEBUG_BOUNDS: the kernels test every address they compute.  On a correct library the status word stays
+    clear (check_device inside check_workload raises otherwise) and the results are those of the unchecked per-layer
+    kernels, bit for bit."""
+    wl = li.build(name, **kw)
+    for reuse in (0, lop.LOP_FLAG_REUSE_HALO):
+        a = check_workload(wl, flags=reuse | lop.LOP_FLAG_DEBUG_BOUNDS, modes=("whole", "banded", "pipelined_copy"))
+        b = check_workload(wl, flags=reuse | lop.LOP_FLAG_PER_LAYER, modes=("banded",))
+        for x, y in zip(a["banded"], b["banded"]):
+            assert np.array_equal(x, y)
+
+
 def test_tensor_core_and_cuda_core_paths_agree():
     wl = li.build("resnet18", H=64, W=64)
     a = check_workload(wl, modes=("whole",))["whole"]
