@@ -65,7 +65,7 @@ enum {
                                      pooling, patch gather, depth-wise convolution, layer normalisation,
                                      concatenation -- test every element offset they load from or store to
                                      against the tensor it belongs to and every output row against the rows of the
-                                     launch.  A violation never traps: the access is skipped, bit 0x20 of the
+                                     launch.  A violation never traps: the access is skipped, bit 0x100 of the
                                      plan's status word is set and lop_plan_check_device returns LOP_EDEVICE.  The
                                      tensor-core kernel's operand loads are TMA copies, clipped by the hardware    */
 };

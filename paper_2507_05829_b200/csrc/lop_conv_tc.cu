@@ -19,6 +19,8 @@
 // (channel slab, kh, kw), whatever the tile position, so a pixel's value does not depend on the
 // band that computes it.  Every wait is bounded; a wait that runs out sets the status word.
 #include <cuda.h>
+#include <atomic>
+
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -333,14 +335,14 @@ cudaError_t launch_conv_tc(const ConvArgs &a, const ConvTcGeom &g, const ConvTcM
     p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(g.BN >> 3) << 17) | ((128u >> 4) << 24);
     const size_t smem = 1024 + (size_t)g.stages * (p.a_stage_bytes + p.b_stage_bytes) + 16 * g.stages + 32;
     // the attribute is per device: set it once on each device a launch is made from
-    static bool configured[64] = {};
+    static std::atomic<bool> configured[64];            // set after the (idempotent) attribute call: plans on several host threads may race here
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
-    if (dev < 0 || dev >= 64 || !configured[dev]) {
+    if (dev < 0 || dev >= 64 || !configured[dev].load(std::memory_order_acquire)) {
         e = cudaFuncSetAttribute(conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(200 * 1024));
         if (e != cudaSuccess) return e;
-        if (dev >= 0 && dev < 64) configured[dev] = true;
+        if (dev >= 0 && dev < 64) configured[dev].store(true, std::memory_order_release);
     }
     dim3 grid((unsigned)(p.tiles_w * p.tiles_r * tiles_n), (unsigned)(a.Cout / g.BN));
     conv_tc_kernel<<<grid, TC_THREADS, smem, s>>>(maps, p);

@@ -1006,7 +1006,7 @@ int lop_plan_check_device(lop_plan_t *pl, void *ws)
         for (auto &kv : pl->exec->programs) program_destroy(kv.second);
         pl->exec->programs.clear();
         cudaMemset(static_cast<char *>(ws) + pl->status_off, 0, sizeof(status));
-        set_error(status & 0x20u ? "device status word 0x%x: a checked kernel computed an address outside its tensor (the access was skipped)"
+        set_error(status & 0x100u ? "device status word 0x%x: a checked kernel computed an address outside its tensor (the access was skipped)"
                                  : "device status word 0x%x: a bounded wait ran out", status);
         return LOP_EDEVICE;
     }

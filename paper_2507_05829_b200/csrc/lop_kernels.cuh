@@ -16,7 +16,7 @@ struct ConvArgs {
     int kh, kw, sh, sw, ph, pw, dh, dw;
     int act, res_pos;
     int oh_lo, oh_hi;       // rows to compute
-    unsigned *dbg;          // checked execution: the status word that takes bit 0x20 on a violation, else nullptr
+    unsigned *dbg;          // checked execution: the status word that takes bit 0x100 on a violation, else nullptr
 };
 
 struct PoolArgs {
@@ -34,7 +34,7 @@ struct PoolArgs {
 __device__ __forceinline__ bool dbg_in_bounds(unsigned *dbg, long long first, long long count, long long limit)
 {
     if (!dbg || (first >= 0 && first + count <= limit)) return true;
-    atomicOr(dbg, 0x20u);
+    atomicOr(dbg, 0x100u);
     return false;
 }
 #endif

@@ -7,6 +7,8 @@
 // persistent kernel's worker warps run as well); other dtypes and channel counts take the plain kernel below.  Each
 // kernel works on output rows [oh_lo, oh_hi) of all N images, like every other layer kernel, and a pixel's
 // arithmetic does not depend on the band it is in.
+#include <atomic>
+
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -343,14 +345,14 @@ cudaError_t launch_dwconv(const ConvArgs &a, int dtype, const void *w_taps, cuda
         g.dbg = a.dbg; g.N = a.N;
         const int tiles_w = (a.Wo + t.tw - 1) / t.tw, tiles_r = (a.oh_hi - a.oh_lo + t.R - 1) / t.R;
         if (tiles_r <= 65535) {
-            static bool configured[64] = {};                 // the shared-memory limit is an attribute per device
+            static std::atomic<bool> configured[64];     // the shared-memory limit is an attribute per device (set once; idempotent)
             int dev = 0;
             cudaError_t e = cudaGetDevice(&dev);
             if (e != cudaSuccess) return e;
-            if (dev < 0 || dev >= 64 || !configured[dev]) {
+            if (dev < 0 || dev >= 64 || !configured[dev].load(std::memory_order_acquire)) {
                 e = cudaFuncSetAttribute(dwconv_tile_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DW_TILE_SMEM);
                 if (e != cudaSuccess) return e;
-                if (dev >= 0 && dev < 64) configured[dev] = true;
+                if (dev >= 0 && dev < 64) configured[dev].store(true, std::memory_order_release);
             }
             dim3 grid((unsigned)(tiles_w * (a.Cin / t.cc)), (unsigned)tiles_r, (unsigned)a.N);
             dwconv_tile_kernel<<<grid, DW_TILE_THREADS, (size_t)rowop::dw_tile_bytes(a.kh, a.kw, a.sh, a.sw, a.dh, a.dw, t), s>>>(g, a.oh_lo, a.oh_hi, tiles_w);

@@ -184,7 +184,7 @@ struct DwGeom {
     const uint16_t *w_taps;           // [kh*kw][C] bf16
     const float *scale, *shift;
     uint16_t *y;
-    unsigned *dbg;                    // checked execution: status word that takes bit 0x20 on an address outside a tensor, else nullptr
+    unsigned *dbg;                    // checked execution: status word that takes bit 0x100 on an address outside a tensor, else nullptr
     int N;                            // images (for the checks only)
 };
 // (the persistent kernel, THROUGH_L2, never runs checked: checked execution takes the stand-alone kernels)
@@ -192,7 +192,7 @@ template <bool THROUGH_L2>
 __device__ __forceinline__ bool dw_in_bounds(const DwGeom &g, long long first, long long count, long long limit)
 {
     if (THROUGH_L2 || !g.dbg || (first >= 0 && first + count <= limit)) return true;
-    atomicOr(g.dbg, 0x20u);
+    atomicOr(g.dbg, 0x100u);
     return false;
 }
 

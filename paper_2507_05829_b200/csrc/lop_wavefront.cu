@@ -25,6 +25,8 @@
 // Deadlock freedom: items are numbered in a topological order, every CTA is resident and takes its
 // items in increasing order, so the lowest unfinished item never waits on an unstarted one.  All
 // waits are bounded all the same; one that runs out raises the status word and the abort flag.
+#include <atomic>
+
 #include <cuda_bf16.h>
 
 #include "lop_gather.cuh"
@@ -1219,17 +1221,17 @@ cudaError_t launch_wavefront(const WfParams &p, int grid, cudaStream_t s)
 {
     const size_t smem = wavefront_smem_bytes(p);
     // the attribute is per device: set it once on each device a launch is made from
-    static bool configured[64] = {};
+    static std::atomic<bool> configured[64];            // set after the (idempotent) attribute call: plans on several host threads may race here
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
-    if (dev < 0 || dev >= 64 || !configured[dev]) {
+    if (dev < 0 || dev >= 64 || !configured[dev].load(std::memory_order_acquire)) {
         WfKernel all[4] = {wavefront_kernel<false, false>, wavefront_kernel<false, true>, wavefront_kernel<true, false>, wavefront_kernel<true, true>};
         for (WfKernel k : all) {
             e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
             if (e != cudaSuccess) return e;
         }
-        if (dev >= 0 && dev < 64) configured[dev] = true;
+        if (dev >= 0 && dev < 64) configured[dev].store(true, std::memory_order_release);
     }
     if (smem > 227 * 1024) return cudaErrorInvalidValue;
 #ifdef LOP_WF_TRACE
