@@ -518,7 +518,8 @@ def test_a_band_that_never_arrives_ends_the_launch_with_a_status_not_a_hang():
         assert torch.equal(dc.outs[-1], good), mode
 
 
-@pytest.mark.parametrize("name,kw", [("vgg_block", dict(H=44, W=36)), ("resnet18", dict(H=64, W=64))])
+@pytest.mark.parametrize("name,kw", [("vgg_block", dict(H=44, W=36)), ("resnet18", dict(H=64, W=64)),
+                                     ("convnext_block", dict(H=29, W=17, C=64, n_bands=6)), ("dense_layer", dict(H=19, W=14, n_bands=6))])
 def test_halo_exchange_between_emulated_ranks_on_one_gpu(name, kw):
     """The transmission form of band sharding (Sec. IV-C: trade halo rows instead of recomputing them), two and three
     ranks taking turns on this GPU, each with tensors of its own: lop_run_layer computes every row of every layer once,
@@ -606,6 +607,10 @@ def test_more_bands_than_rows_and_single_band():
     wl = li.build("vgg_block", H=12, W=20)
     for nb in (1, 6, 7, 13):                                     # 6 output rows: empty bands from 7 on
         check_workload(wl, n_bands=nb)
+    for wl in (li.build("convnext_block", H=9, W=12, C=32), li.build("dense_layer", H=9, W=10)):
+        for nb in (1, 9, 10, 19):                                # 9 output rows
+            check_workload(wl, n_bands=nb)
+            check_workload(wl, n_bands=nb, flags=lop.LOP_FLAG_REUSE_HALO, modes=("whole", "banded"))
 
 
 def test_bands_in_any_order_without_reuse():
@@ -765,7 +770,8 @@ def test_unaligned_and_unpinned_host_buffers_take_the_copy_path():
 
 
 def test_wavefront_and_per_layer_executors_agree_bit_for_bit():
-    for name, kw in (("resnet18", dict(H=96, W=96)), ("csp_stack", dict(H=256, W=256))):
+    for name, kw in (("resnet18", dict(H=96, W=96)), ("csp_stack", dict(H=256, W=256)), ("convnext_block", dict(H=40, W=24, C=96)),
+                     ("dense_layer", {})):
         wl = li.build(name, **kw)
         a = DeviceChain(wl, flags=lop.LOP_FLAG_REUSE_HALO)
         b = DeviceChain(wl, flags=lop.LOP_FLAG_REUSE_HALO | lop.LOP_FLAG_PER_LAYER)
