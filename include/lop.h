@@ -271,13 +271,14 @@ int lop_plan_layer_stored(const lop_plan_t *plan, int layer);
 /* Number of kernels (this library's own) and of async copies the last execution call enqueued. */
 int lop_plan_last_launches(const lop_plan_t *plan);
 int lop_plan_last_copies(const lop_plan_t *plan);
-/* Reads the plan's device status word (0 = no kernel gave up on a bounded wait).  SYNCHRONISES
+/* Reads the plan's device status word (0 = no kernel gave up on a bounded wait or failed a bounds check).  SYNCHRONISES
  * the stream of the last execution call.  On LOP_EDEVICE the outputs of that call are invalid; the
  * library drops its cached device tables and clears the word, so the plan can be used again.
  * lop_last_error() then shows the word; its bits name the role of the persistent kernel whose wait
  * ran out: 0x1 loader (ring slot), 0x2 MMA issuer (operands), 0x4 epilogue / pooling / gather
  * (accumulator, dependencies), 0x8 publisher, 0x10 loader (dependencies of a tile), 0x20 fetch warp
- * (window of the in-kernel input transfer). */
+ * (window of the in-kernel input transfer).  0x100: a kernel of a LOP_FLAG_DEBUG_BOUNDS plan computed an
+ * address outside its tensor (the access was skipped). */
 int lop_plan_check_device(lop_plan_t *plan, void *workspace);
 
 /* ---- the device-side waits and their failure path ----------------------------------------------

@@ -282,7 +282,7 @@ __global__ void __launch_bounds__(256) layernorm_bf16_kernel(ConvArgs p)
             live[q] = dbg_in_bounds(p.dbg, o[q], C, (long long)p.N * image * C);
         }
     }
-    rowop::ln_pixels<false, VPL>(static_cast<const uint16_t *>(p.x), static_cast<uint16_t *>(p.y), C, lanes_log, sub, o, live, p.scale, p.shift);
+    rowop::ln_pixels<false, VPL, PPG>(static_cast<const uint16_t *>(p.x), static_cast<uint16_t *>(p.y), C, lanes_log, sub, o, live, p.scale, p.shift);
 }
 
 template <int VPL>

@@ -79,11 +79,10 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
 // o[p]: element offset of pixel p, live[p]: whether the slot holds a pixel (dead slots still take part in the
 // shuffles).  gain / offset may be null.
 // ---------------------------------------------------------------------------------------------
-template <bool THROUGH_L2, int VPL>
-__device__ __forceinline__ void ln_pixels(const uint16_t *x, uint16_t *y, int C, int lanes_log, int sub, const long long (&o)[4 / VPL],
-                                          const bool (&live)[4 / VPL], const float *gain, const float *offset)
+template <bool THROUGH_L2, int VPL, int PPG>
+__device__ __forceinline__ void ln_pixels(const uint16_t *x, uint16_t *y, int C, int lanes_log, int sub, const long long (&o)[PPG],
+                                          const bool (&live)[PPG], const float *gain, const float *offset)
 {
-    constexpr int PPG = 4 / VPL;
     const int nv = C >> 3, lanes = 1 << lanes_log;
     uint4 q[PPG][VPL];
     bool have[PPG][VPL];
@@ -92,23 +91,25 @@ __device__ __forceinline__ void ln_pixels(const uint16_t *x, uint16_t *y, int C,
 #pragma unroll
         for (int k = 0; k < VPL; ++k) {
             have[p][k] = live[p] && sub + k * lanes < nv;
+            q[p][k] = make_uint4(0u, 0u, 0u, 0u);
             if (have[p][k]) {
                 const uint4 *src = reinterpret_cast<const uint4 *>(x + o[p]) + sub + k * lanes;
                 q[p][k] = THROUGH_L2 ? __ldcg(src) : __ldg(src);
             }
         }
-    float mean[PPG], inv[PPG];
+    // widened once; from the second pass on f holds the centred values
+    float f[PPG][VPL][8], mean[PPG], inv[PPG];
 #pragma unroll
     for (int p = 0; p < PPG; ++p) {
         float s1 = 0.0f;
 #pragma unroll
-        for (int k = 0; k < VPL; ++k)
+        for (int k = 0; k < VPL; ++k) {
+            unpack_bf16x8(q[p][k], f[p][k]);
             if (have[p][k]) {
-                float f[8];
-                unpack_bf16x8(q[p][k], f);
 #pragma unroll
-                for (int j = 0; j < 8; ++j) s1 += f[j];
+                for (int j = 0; j < 8; ++j) s1 += f[p][k][j];
             }
+        }
         mean[p] = group_sum(s1, lanes_log) / (float)C;
     }
 #pragma unroll
@@ -117,12 +118,10 @@ __device__ __forceinline__ void ln_pixels(const uint16_t *x, uint16_t *y, int C,
 #pragma unroll
         for (int k = 0; k < VPL; ++k)
             if (have[p][k]) {
-                float f[8];
-                unpack_bf16x8(q[p][k], f);
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
-                    const float d = f[j] - mean[p];
-                    s2 = fmaf(d, d, s2);
+                    f[p][k][j] -= mean[p];
+                    s2 = fmaf(f[p][k][j], f[p][k][j], s2);
                 }
             }
         inv[p] = ln_inv_std(group_sum(s2, lanes_log), C);
@@ -145,11 +144,9 @@ __device__ __forceinline__ void ln_pixels(const uint16_t *x, uint16_t *y, int C,
 #pragma unroll
         for (int p = 0; p < PPG; ++p)
             if (have[p][k]) {
-                float f[8];
-                unpack_bf16x8(q[p][k], f);
                 float r[8];
 #pragma unroll
-                for (int j = 0; j < 8; ++j) r[j] = ln_value(f[j], mean[p], inv[p], gn[j], of[j]);
+                for (int j = 0; j < 8; ++j) r[j] = fmaf(f[p][k][j] * inv[p], gn[j], of[j]);       // ln_value on the centred value
                 *(reinterpret_cast<uint4 *>(y + o[p]) + v) =
                     make_uint4(pack_bf16x2(r[0], r[1]), pack_bf16x2(r[2], r[3]), pack_bf16x2(r[4], r[5]), pack_bf16x2(r[6], r[7]));
             }

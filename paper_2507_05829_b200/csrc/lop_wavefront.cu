@@ -228,7 +228,7 @@ __device__ __forceinline__ void layernorm_row(const uint16_t *x, uint16_t *y, co
             live[q] = ow < Wo;
             o[q] = (row0 + ow) * C;
         }
-        rowop::ln_pixels<true, VPL>(x, y, C, lanes_log, sub, o, live, gain, offset);
+        rowop::ln_pixels<true, VPL, PPG>(x, y, C, lanes_log, sub, o, live, gain, offset);
     }
 }
 __device__ __noinline__ void layernorm_item(const WfStage *sp, int n, int oh, int tid)
