@@ -68,9 +68,9 @@ def cost_model(wl, bands, machine=MACHINE):
                 if rows == 0:
                     continue
                 ho, wo, co = shapes[i]
-                if l.op == 1:
+                if l.op in (1, 3, 4, 5):      # pooling, depth-wise convolution, layer normalisation, concatenation: row items of the worker warps
                     items = rows * N
-                    per_item = machine["row_item_us"]
+                    per_item = machine["row_item_us"] * (2.0 if l.op == 3 else 1.0)
                     work = math.ceil(items / machine["ctas"]) * per_item
                 else:
                     chunks = math.ceil(l.cin / 64.0) if l.cin >= 16 else 1

@@ -1,4 +1,5 @@
 """The band-count search (the paper's scheduling optimisation re-targeted to one GPU behind a host link)."""
+import numpy as np
 import pytest
 
 import lop_inputs as li
@@ -65,3 +66,13 @@ def test_search_with_the_measured_objective_on_the_device():
     want = ochain.run_workload(wl)
     got = to_host_f32(dc.outs[-1])
     assert float(np.max(np.abs(got - want))) / float(np.max(np.abs(want))) <= 2e-2
+
+
+def test_model_covers_every_operator_kind():
+    """Depth-wise convolution, layer normalisation and concatenation are costed as row items: the model returns a
+    finite latency for the ConvNeXt block and the DenseNet layer, and more bands never cost less than the launch."""
+    for name in ("convnext_block", "dense_layer", "pointwise_mlp"):
+        wl = li.build(name, with_data=False)
+        for nb in (1, 4, 8):
+            t = ss.cost_model(wl, [nb])
+            assert np.isfinite(t) and t > ss.MACHINE["launch_us"]
